@@ -1,0 +1,173 @@
+/*
+ * videoscan.h -- C ABI of the B200 (sm_100a) streaming attention path of VideoScan
+ * (arXiv 2503.09387): one semantic-carrier token per frame, a bounded bank of carrier
+ * K/V, visual tokens discarded after their own prefill.
+ *
+ * Conventions
+ *  - Every call returns an int status: VS_OK (0) or a negative VS_ERR_* code.  Nothing
+ *    throws, aborts or sets errno.  vs_status_string() names a code.
+ *  - Pointers marked DEVICE are CUDA device pointers on `vs_config.device`; pointers
+ *    marked HOST are ordinary host memory.  All tensors are bf16 (2 bytes, upper half of
+ *    an IEEE fp32), row-major, densely packed.
+ *  - The library borrows memory, it owns none on the device: weights, the workspace,
+ *    inputs and outputs are allocated and freed by the caller, and weights and workspace
+ *    must outlive the handle.  No call allocates device memory.
+ *  - vs_frame_prefill / vs_decode_step only enqueue work on `cuda_stream` (a
+ *    cudaStream_t passed as void*; NULL is the default stream) and return without
+ *    synchronising.  vs_bank_state synchronises that stream.  All calls on one handle
+ *    must use the same CUDA stream (or be ordered by the caller).
+ *  - A handle is not thread safe.  Distinct handles are independent.
+ *  - Device-side waits are bounded; if one ever expires the kernel records
+ *    VS_ERR_DEVICE_TIMEOUT in a device status word that vs_bank_state reports.
+ */
+#ifndef VIDEOSCAN_H_
+#define VIDEOSCAN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define VS_OK                   0
+#define VS_ERR_INVALID_ARG     -1   /* NULL pointer, bad size, bad stream id, duplicate id   */
+#define VS_ERR_STATE           -2   /* call not legal in the stream's current phase         */
+#define VS_ERR_CAPACITY        -3   /* prefix / text tail / workspace too small             */
+#define VS_ERR_CUDA            -4   /* a CUDA runtime or driver call failed                 */
+#define VS_ERR_DEVICE_TIMEOUT  -5   /* a bounded device-side wait expired                   */
+#define VS_ERR_UNSUPPORTED     -6   /* shape outside what the kernels are built for         */
+
+#define VS_MAX_BATCH           64   /* most streams one call may list                       */
+
+typedef struct vs_stream vs_stream;   /* opaque handle: a batch of n_streams independent video streams */
+
+/* Model shape and stream limits.  Multi-head attention with grouped KV heads and rotary
+ * position embedding is the Qwen2 backbone the paper builds on (Section 4.1); Eq. (1) is
+ * applied per head with d_k = head_dim. */
+typedef struct {
+  int32_t n_layers;              /* attention layers chained through a residual stream (>= 1)      */
+  int32_t d_model;               /* hidden size d; multiple of 64                                    */
+  int32_t n_q_heads;             /* query heads Hq                                                   */
+  int32_t n_kv_heads;            /* KV heads Hkv; Hq % Hkv == 0, Hq / Hkv <= 8                       */
+  int32_t head_dim;              /* D: 64 or 128                                                     */
+  int32_t max_tokens_per_frame;  /* largest N one frame may bring (N + 1 <= 256)                     */
+  int32_t max_prefix;            /* prompt-prefix capacity in tokens                                 */
+  int32_t max_text;              /* question + answer tail capacity in tokens, per turn              */
+  int32_t max_step_tokens;       /* largest T of one vs_decode_step call (per stream)                */
+  int32_t bank_capacity;         /* M of Section 3.3 (memory mechanism); 0 = keep no carriers        */
+  int32_t n_streams;             /* independent streams held by the handle (1 .. VS_MAX_BATCH)       */
+  int32_t agg_mode;              /* 0: carrier = mean of the frame's tokens (Section 3.3);
+                                    1: carrier = last visual token (ablation "w/o emb", Table 4)     */
+  int32_t evict_policy;          /* 0: discard the stored carrier most cosine-similar to the incoming
+                                       one; 1: discard the older member of the most similar adjacent
+                                       pair (both readings of Section 3.3); 2: FIFO (test aid)       */
+  int32_t use_rmsnorm;           /* 1: QKV = RMSNorm(h) W (pre-attention norm); 0: QKV = h W         */
+  int32_t residual;              /* 1: h <- h + O between layers (needs Hq*D == d_model); required
+                                       when n_layers > 1                                             */
+  float   rope_theta;            /* rotary base (Qwen2: 1e6)                                         */
+  float   rms_eps;               /* RMSNorm epsilon                                                  */
+  int32_t device;                /* CUDA device ordinal                                              */
+  int32_t evict_log_capacity;    /* eviction-log entries kept per stream (most recent); may be 0     */
+} vs_config;
+
+/* DEVICE pointers to bf16 weights, one entry per layer.  The arrays of pointers themselves
+ * are HOST arrays of length n_layers and are copied at create. */
+typedef struct {
+  const void* const* w_qkv;      /* [n_layers] each [E_out, d_model] row-major ("out x in"),
+                                    E_out = (Hq + 2*Hkv) * D, rows ordered Q heads, K heads, V heads;
+                                    16-byte aligned                                                  */
+  const void* const* b_qkv;      /* [n_layers] each [E_out], or NULL (whole array or any entry)      */
+  const void* const* norm_w;     /* [n_layers] each [d_model] RMSNorm gain, or NULL = all ones       */
+} vs_weights;
+
+/* Filled by vs_bank_state (HOST). */
+typedef struct {
+  int32_t count;                 /* carriers in the bank == min(frames_seen, capacity)               */
+  int32_t capacity;
+  int64_t frames_seen;
+  int64_t evictions;
+  int64_t next_pos;              /* position id the next frame (or prefix token) starts at           */
+  int64_t prefix_len;
+  int64_t text_len;
+  int32_t last_victim_frame;     /* frame id discarded by the last frame step, -1 if none            */
+  int32_t device_status;         /* 0, or VS_ERR_DEVICE_TIMEOUT                                      */
+  uint64_t persistent_bytes;     /* bytes of the workspace that hold stream state; constant          */
+  uint64_t workspace_bytes;      /* whole workspace; constant for the life of the handle             */
+} vs_bank_info;
+
+/* Bytes of DEVICE workspace vs_create_stream needs for `cfg` (256-byte aligned base). */
+int vs_workspace_bytes(const vs_config* cfg, size_t* out_bytes);
+
+/* Builds a handle over caller memory: carves `workspace` (DEVICE, >= vs_workspace_bytes,
+ * 256-byte aligned) into bank, prefix, tail, metadata and per-step scratch, clears the
+ * metadata (synchronously) and encodes the TMA descriptors of the weights.  Nothing is
+ * allocated on the device, so memory use does not depend on stream length (the paper's
+ * "stable GPU memory consumption", Section 3.3). */
+int vs_create_stream(const vs_config* cfg, const vs_weights* weights,
+                     void* workspace, size_t workspace_bytes, vs_stream** out);
+
+/* One frame per listed stream -- the prefilling phase of Section 3.3:
+ *   carrier C = (1/N) sum_i E_i appended after the N visual tokens (Sections 3.2, 3.3);
+ *   per layer: Q,K,V projection, RoPE, softmax attention (Eq. 1) of the N+1 tokens over
+ *   [prompt prefix | carriers in the bank | own frame, causal];
+ *   then the carrier's K/V of every layer enters the bank (evicting first when the bank is
+ *   full) and everything else of the frame is dropped.
+ * stream_ids: HOST [n_active], distinct ids in [0, n_streams).
+ * hidden:     DEVICE bf16 [n_active][N][d_model].
+ * carrier_override: DEVICE bf16 [n_active][d_model] used as the carrier token instead of
+ *             the mean (e.g. projector(mean) computed by the caller), or NULL.
+ * out:        DEVICE bf16 [n_active][N+1][Hq*D], last layer's attention output, row N being
+ *             the carrier's; may be NULL.
+ * Errors: VS_ERR_STATE if a listed stream has an open text turn (call vs_end_turn first);
+ *         VS_ERR_CAPACITY if N > max_tokens_per_frame. */
+int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
+                     const void* hidden, int32_t N, const void* carrier_override,
+                     void* out, void* cuda_stream);
+
+/* T text tokens per listed stream -- the decoding phase of Section 3.3 (T = 1) and the
+ * text part of prefilling (T > 1).  Token i attends to [prefix | bank | tail tokens up to
+ * itself]; no visual-token K/V exists any more.  Before a stream's first frame the tokens
+ * extend the prompt prefix instead (the system instruction comes first, Section 3.3) and
+ * stay for the life of the stream.
+ * hidden: DEVICE bf16 [n_active][T][d_model];  out: DEVICE bf16 [n_active][T][Hq*D].
+ * All listed streams must be in the same phase (all before or all after their first frame).
+ * Errors: VS_ERR_CAPACITY on prefix / tail overflow or T > max_step_tokens. */
+int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
+                   const void* hidden, int32_t T, void* out, void* cuda_stream);
+
+/* Ends a question/answer turn: the text tail is dropped, prefix and bank stay, frame
+ * positions do not move.  Host-only bookkeeping. */
+int vs_end_turn(vs_stream* h, const int32_t* stream_ids, int32_t n_active);
+
+/* Synchronises the handle's CUDA stream and reports one stream's bank (Section 3.3,
+ * memory mechanism) in temporal order (oldest carrier first).  All outputs are HOST and
+ * optional (NULL skips them):
+ *   frame_ids, positions, slots : [capacity] -- first `count` entries valid; `slots` are the
+ *                                 physical slot numbers (implementation defined);
+ *   evict_log : [evict_log_cap][2] int32 (frame step, victim frame id), oldest kept first;
+ *               *evict_log_n receives the number written;
+ *   emb_out   : bf16 [count][d_model] carrier embeddings;
+ *   k_out, v_out : bf16 [count][Hkv][D] of `layer`. */
+int vs_bank_state(vs_stream* h, int32_t stream_id, vs_bank_info* info,
+                  int32_t* frame_ids, int64_t* positions, int32_t* slots,
+                  int32_t* evict_log, int32_t evict_log_cap, int32_t* evict_log_n,
+                  void* emb_out, int32_t layer, void* k_out, void* v_out);
+
+/* Test aids.  vs_last_step_kv copies the rotated K and V rows that the most recent
+ * vs_frame_prefill / vs_decode_step left in scratch for the LAST layer to HOST buffers
+ * bf16 [rows][Hkv*D] (rows = n_active*(N+1) or n_active*T), synchronising first; it lets a
+ * test check that the bank append is a pure copy.  vs_poison_scratch overwrites every
+ * per-step scratch region with NaN patterns (asynchronously on cuda_stream): later steps
+ * must not change, which shows that no visual-token state survives a step. */
+int vs_last_step_kv(vs_stream* h, void* k_out, void* v_out, int32_t rows);
+int vs_poison_scratch(vs_stream* h, void* cuda_stream);
+
+int vs_destroy_stream(vs_stream* h);
+
+const char* vs_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* VIDEOSCAN_H_ */
