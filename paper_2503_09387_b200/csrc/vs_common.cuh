@@ -1,0 +1,193 @@
+// Shared declarations of the CUDA path: workspace carve-up, per-call batch parameters,
+// launch wrappers.  Nothing here is shared with the CPU oracle.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda.h>
+#include <stdint.h>
+
+#include "../../include/videoscan.h"
+
+namespace vs {
+
+typedef __nv_bfloat16 bf16;
+
+// ---- device-resident metadata of one stream (Section 3.3, memory mechanism) ------------
+// `slots` = bank_capacity + 1 physical slots, so the incoming carrier can be written while
+// the victim is still readable.
+struct StreamMeta {
+  int32_t count;              // carriers currently in the bank
+  int32_t free_slot;          // physical slot the next carrier is written to
+  int32_t victim_logical;     // temporal index chosen by the scoring kernel, -1 = none
+  int32_t last_victim_frame;  // frame id discarded by the last step, -1 = none
+  int64_t frames_seen;
+  int64_t evictions;
+  int32_t log_count;          // evictions ever logged (ring position = log_count % cap)
+  int32_t score_ticket;       // blocks of the scoring kernel that have finished
+  int32_t pad[4];
+};
+
+// ---- per-call description of the listed streams (passed by value to kernels) -----------
+struct BatchParams {
+  int32_t n_active;
+  int32_t rows_per_stream;             // N + 1 for a frame step, T for a text step
+  int32_t stream_id[VS_MAX_BATCH];
+  int32_t count[VS_MAX_BATCH];         // carriers in the bank before this step (host mirror)
+  int32_t prefix_len[VS_MAX_BATCH];
+  int32_t text_len[VS_MAX_BATCH];      // tail length before this step
+  int64_t pos_base[VS_MAX_BATCH];      // position id of the step's first token
+  int64_t frame_id[VS_MAX_BATCH];      // frames_seen before this step
+};
+
+// ---- shapes ----------------------------------------------------------------------------
+struct Dims {
+  int L, d, Hq, Hkv, D, G, E_out;
+  int maxN, maxP, maxT, maxStepT, M, slots, S;
+  int rows_per_stream_max, R_max;
+  int log_cap;
+  int agg_mode, evict_policy, use_rmsnorm, residual;
+  float rope_theta, rms_eps;
+};
+
+constexpr int KSPLIT_MAX = 8;
+constexpr int DEC_SPLIT_MAX = 16;
+constexpr int GEMM_BLOCK_M = 128;
+constexpr int GEMM_BLOCK_K = 64;
+
+// ---- workspace layout (byte offsets from the workspace base) ----------------------------
+struct Layout {
+  // persistent: stream state
+  size_t bank_k, bank_v;        // bf16 [L][S][Hkv][slots][D]
+  size_t prefix_k, prefix_v;    // bf16 [L][S][Hkv][maxP][D]
+  size_t tail_k, tail_v;        // bf16 [L][S][Hkv][maxT][D]
+  size_t emb;                   // bf16 [S][slots][d]
+  size_t meta;                  // StreamMeta [S]
+  size_t order;                 // int32 [S][slots]  temporal index -> physical slot
+  size_t slot_frame;            // int32 [S][slots]  frame id held by a slot, -1 = free
+  size_t slot_pos;              // int64 [S][slots]  position id of the carrier
+  size_t evict_log;             // int32 [S][log_cap][2]
+  size_t scores;                // f64   [S][slots]
+  size_t inv_freq;              // f64   [D/2]
+  size_t status;                // int32 [8]
+  size_t tickets;               // int32 [S*Hkv]
+  size_t persistent_end;
+  // per-step scratch
+  size_t hbuf[2];               // bf16 [R_max][d]  residual ping-pong; hbuf[0] holds [E; carrier]
+  size_t xn;                    // bf16 [R_max][d]  normalised layer input
+  size_t partials;              // f32  [KSPLIT_MAX][R_max][E_out]
+  size_t q;                     // bf16 [R_max][Hq*D]
+  size_t kf, vf;                // bf16 [R_max][Hkv*D]
+  size_t rope;                  // float2 [R_max][D/2]
+  size_t obuf;                  // bf16 [R_max][Hq*D]
+  size_t dec_part;              // f32  [DEC_SPLIT_MAX][S][Hq][D+2]
+  size_t scratch_begin, scratch_end;
+  size_t total;
+};
+
+// ---- launch wrappers (each returns the cudaError_t of the launch) -----------------------
+struct PoolArgs {
+  const bf16* hidden;            // [n_active][N][d]
+  const bf16* carrier_override;  // [n_active][d] or null
+  bf16* x;                       // [n_active][N+1][d]
+  bf16* emb;                     // [S][slots][d]
+  const StreamMeta* meta;        // [S]
+  const double* inv_freq;        // [D/2]
+  float2* rope;                  // [n_active][N+1][D/2]
+  int N, d, D, slots, M, agg_mode;
+};
+cudaError_t launch_pool(const PoolArgs& a, const BatchParams& bp, cudaStream_t st);
+
+struct RopeArgs {
+  const double* inv_freq;
+  float2* rope;                  // [n_active][T][D/2]
+  int D;
+};
+cudaError_t launch_rope_table(const RopeArgs& a, const BatchParams& bp, cudaStream_t st);
+
+cudaError_t launch_rmsnorm(const bf16* h, const bf16* gain, bf16* xn, int rows, int d, float eps,
+                           cudaStream_t st);
+
+struct GemmArgs {
+  CUtensorMap tm_w;              // [E_out, d] bf16, box 64 x 128, 128-byte swizzle
+  CUtensorMap tm_x;              // [rows, d] bf16, box 64 x tile_n, 128-byte swizzle
+  float* partials;               // [ksplit][rows][E_out]
+  int rows, E_out, d;
+  int tile_n, n_tiles, ksplit;
+  int* status;
+};
+cudaError_t launch_qkv_gemm(const GemmArgs& a, cudaStream_t st);
+cudaError_t qkv_gemm_init();     // opt-in shared memory attribute, once per process/device
+
+struct FinalizeArgs {
+  const float* partials;         // [ksplit][rows][E_out]
+  const bf16* bias;              // [E_out] or null
+  const float2* rope;            // [rows][D/2]
+  bf16* q;                       // [rows][Hq*D]
+  bf16* kf;                      // [rows][Hkv*D]
+  bf16* vf;
+  bf16* bank_k; bf16* bank_v;    // layer base [S][Hkv][slots][D]
+  bf16* text_k; bf16* text_v;    // layer base [S][Hkv][text_cap][D]: prefix or tail
+  const StreamMeta* meta;
+  int rows, ksplit, E_out, Hq, Hkv, D, slots, text_cap;
+  int mode;                      // 0 frame step (carrier row -> bank), 1 text -> prefix, 2 text -> tail
+  int M;
+};
+cudaError_t launch_finalize(const FinalizeArgs& a, const BatchParams& bp, cudaStream_t st);
+
+struct AttnSegment {
+  const bf16* k; const bf16* v;
+  long long stream_stride;       // elements between streams (by stream id, or by batch slot when by_batch)
+  long long head_stride;         // elements between KV heads
+  long long row_stride;          // elements between keys
+  int kind;                      // 0 prefix, 1 bank, 2 tail (earlier tokens of the turn), 3 this step's rows (causal)
+  int by_batch;
+};
+struct AttnArgs {
+  const bf16* q;                 // [rows][Hq*D]
+  AttnSegment seg[4];
+  int n_seg;
+  bf16* out;                     // [rows][Hq*D]
+  const bf16* h_in;              // residual input [rows][d] or null
+  bf16* h_out;                   // residual output or null
+  const StreamMeta* meta;
+  int Hq, Hkv, D, slots, M;
+  float scale_log2e;
+};
+cudaError_t launch_prefill_attention(const AttnArgs& a, const BatchParams& bp, cudaStream_t st);
+cudaError_t prefill_attention_init();
+
+struct DecodeArgs {
+  const bf16* q;                 // [n_active][Hq*D]
+  const bf16* prefix_k; const bf16* prefix_v;  // layer base [S][Hkv][maxP][D]
+  const bf16* bank_k;   const bf16* bank_v;    // [S][Hkv][slots][D]
+  const bf16* tail_k;   const bf16* tail_v;    // [S][Hkv][maxT][D]
+  float* partials;               // [nsplit][n_active][Hq][D+2]
+  int* tickets;                  // [S*Hkv]
+  bf16* out;                     // [n_active][Hq*D]
+  const bf16* h_in; bf16* h_out;
+  const StreamMeta* meta;
+  int Hq, Hkv, D, slots, M, maxP, maxT, nsplit;
+  int to_prefix;                 // 1: the keys are the prefix alone (incl. the new token)
+  float scale_log2e;
+};
+cudaError_t launch_decode_attention(const DecodeArgs& a, const BatchParams& bp, cudaStream_t st);
+
+struct EvictArgs {
+  const bf16* emb;               // [S][slots][d]
+  StreamMeta* meta;
+  const int32_t* order; double* scores;  // per-stream arrays, stride `slots`
+  int d, slots, M, policy;
+};
+cudaError_t launch_evict_score(const EvictArgs& a, const BatchParams& bp, cudaStream_t st);
+
+struct CommitArgs {
+  StreamMeta* meta;
+  int32_t* order; int32_t* slot_frame; int64_t* slot_pos; int32_t* evict_log;
+  int slots, M, log_cap;
+};
+cudaError_t launch_commit(const CommitArgs& a, const BatchParams& bp, cudaStream_t st);
+
+cudaError_t launch_poison(void* p, size_t bytes, cudaStream_t st);
+
+}  // namespace vs

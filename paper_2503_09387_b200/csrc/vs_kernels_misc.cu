@@ -1,0 +1,367 @@
+// Memory-bound and bookkeeping kernels of the frame / text step:
+//   carrier aggregation (Section 3.3: C = (1/N) sum_i E_i), RoPE table, RMSNorm,
+//   split-K reduction + RoPE + K/V persistence, eviction scoring and bank commit
+//   (Section 3.3, memory mechanism).
+#include "vs_common.cuh"
+
+namespace vs {
+
+// fp64 -> bf16, round to nearest even, with no intermediate rounding: first to fp32 with
+// round-to-odd (keeps a sticky bit), then fp32 -> bf16 RNE; 24 bits >= 8 + 2 makes the
+// second rounding see exactly the information of the original value.
+__device__ __forceinline__ bf16 f64_to_bf16_rne(double x) {
+  float f = __double2float_rz(x);
+  if ((double)f != x) f = __uint_as_float(__float_as_uint(f) | 1u);
+  return __float2bfloat16_rn(f);
+}
+
+// ------------------------------------------------------------------------------------------
+// Carrier aggregation + layer-0 input assembly + RoPE table.
+// grid = (pool_blocks + rope_blocks, n_active); block = 256 = 8 row groups x 32 lanes, each
+// lane owns 2 adjacent channels, so one block covers 64 channels of every row.  The sum of
+// <= 256 bf16 values in fp64 is exact, hence independent of the order used here.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, int pool_blocks) {
+  const int b = blockIdx.y;
+  const int sid = bp.stream_id[b];
+  const int N = a.N, d = a.d;
+  if ((int)blockIdx.x >= pool_blocks) {
+    // RoPE table of this step's N + 1 positions: angle = pos * theta^(-2k/D), in fp64
+    const int half = a.D / 2;
+    const int idx = (blockIdx.x - pool_blocks) * blockDim.x + threadIdx.x;
+    if (idx < (N + 1) * half) {
+      const int r = idx / half, k = idx - r * half;
+      const double ang = (double)(bp.pos_base[b] + r) * a.inv_freq[k];
+      double s, c;
+      sincos(ang, &s, &c);
+      a.rope[((size_t)b * (N + 1) + r) * half + k] = make_float2((float)c, (float)s);
+    }
+    return;
+  }
+  __shared__ double red[8][64];
+  const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+  const int ch = blockIdx.x * 64 + lane * 2;
+  const bf16* src = a.hidden + (size_t)b * N * d;
+  bf16* dst = a.x + (size_t)b * (N + 1) * d;
+  double s0 = 0.0, s1 = 0.0;
+  if (ch < d) {
+    for (int r = grp; r < N; r += 8) {
+      const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(src + (size_t)r * d + ch);
+      *reinterpret_cast<__nv_bfloat162*>(dst + (size_t)r * d + ch) = v;
+      s0 += (double)__bfloat162float(v.x);
+      s1 += (double)__bfloat162float(v.y);
+    }
+  }
+  red[grp][lane * 2] = s0;
+  red[grp][lane * 2 + 1] = s1;
+  __syncthreads();
+  if (grp == 0 && ch < d) {
+    __nv_bfloat162 c;
+    if (a.carrier_override != nullptr) {
+      c = *reinterpret_cast<const __nv_bfloat162*>(a.carrier_override + (size_t)b * d + ch);
+    } else if (a.agg_mode == 1) {
+      c = *reinterpret_cast<const __nv_bfloat162*>(src + (size_t)(N - 1) * d + ch);
+    } else {
+      double t0 = 0.0, t1 = 0.0;
+#pragma unroll
+      for (int g = 0; g < 8; ++g) { t0 += red[g][lane * 2]; t1 += red[g][lane * 2 + 1]; }
+      c.x = f64_to_bf16_rne(t0 / (double)N);
+      c.y = f64_to_bf16_rne(t1 / (double)N);
+    }
+    *reinterpret_cast<__nv_bfloat162*>(dst + (size_t)N * d + ch) = c;   // carrier = last token of the frame
+    if (a.M > 0) {
+      const int slot = a.meta[sid].free_slot;
+      *reinterpret_cast<__nv_bfloat162*>(a.emb + ((size_t)sid * a.slots + slot) * d + ch) = c;
+    }
+  }
+}
+
+cudaError_t launch_pool(const PoolArgs& a, const BatchParams& bp, cudaStream_t st) {
+  const int pool_blocks = (a.d + 63) / 64;
+  const int rope_blocks = ((a.N + 1) * (a.D / 2) + 255) / 256;
+  dim3 grid(pool_blocks + rope_blocks, bp.n_active);
+  pool_kernel<<<grid, 256, 0, st>>>(a, bp, pool_blocks);
+  return cudaGetLastError();
+}
+
+__global__ void __launch_bounds__(256) rope_table_kernel(RopeArgs a, BatchParams bp) {
+  const int b = blockIdx.y;
+  const int half = a.D / 2, T = bp.rows_per_stream;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= T * half) return;
+  const int r = idx / half, k = idx - r * half;
+  const double ang = (double)(bp.pos_base[b] + r) * a.inv_freq[k];
+  double s, c;
+  sincos(ang, &s, &c);
+  a.rope[((size_t)b * T + r) * half + k] = make_float2((float)c, (float)s);
+}
+
+cudaError_t launch_rope_table(const RopeArgs& a, const BatchParams& bp, cudaStream_t st) {
+  dim3 grid((bp.rows_per_stream * (a.D / 2) + 255) / 256, bp.n_active);
+  rope_table_kernel<<<grid, 256, 0, st>>>(a, bp);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// RMSNorm of the layer input: xn = h / sqrt(mean(h^2) + eps) * gain.  One block per row.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const bf16* __restrict__ h, const bf16* __restrict__ gain,
+                                                      bf16* __restrict__ xn, int d, float eps) {
+  const size_t row = blockIdx.x;
+  const bf16* src = h + row * d;
+  float ss = 0.f;
+  for (int c = threadIdx.x * 2; c < d; c += 512) {
+    const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(src + c));
+    ss += v.x * v.x + v.y * v.y;
+  }
+  __shared__ float red[8];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tot += red[i];
+  const float r = rsqrtf(tot / (float)d + eps);
+  for (int c = threadIdx.x * 2; c < d; c += 512) {
+    float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(src + c));
+    v.x *= r; v.y *= r;
+    if (gain != nullptr) {
+      const float2 g = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(gain + c));
+      v.x *= g.x; v.y *= g.y;
+    }
+    *reinterpret_cast<__nv_bfloat162*>(xn + row * d + c) = __floats2bfloat162_rn(v.x, v.y);
+  }
+}
+
+cudaError_t launch_rmsnorm(const bf16* h, const bf16* gain, bf16* xn, int rows, int d, float eps,
+                           cudaStream_t st) {
+  rmsnorm_kernel<<<rows, 256, 0, st>>>(h, gain, xn, d, eps);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Split-K reduction + bias + RoPE + bf16 + persistence of K/V rows.
+// One thread per (row, head slot, rotation pair k): elements k and k + D/2 of one head.
+// Frame step: the carrier row's K/V (last token of each stream's N+1 rows) goes straight
+// into the bank's free slot (Section 3.2: only the carrier keeps its K/V in the cache).
+// Text step: every row's K/V is appended to the prefix or to the turn's tail.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) finalize_kernel(FinalizeArgs a, BatchParams bp) {
+  const int row = blockIdx.y;
+  const int half = a.D / 2;
+  const int pair = blockIdx.x * blockDim.x + threadIdx.x;
+  const int n_pairs = (a.Hq + 2 * a.Hkv) * half;
+  if (pair >= n_pairs) return;
+  const int hs = pair / half, k = pair - hs * half;
+  const int e1 = hs * a.D + k, e2 = e1 + half;
+  float x1 = 0.f, x2 = 0.f;
+  for (int s = 0; s < a.ksplit; ++s) {
+    const float* p = a.partials + ((size_t)s * a.rows + row) * a.E_out;
+    x1 += p[e1];
+    x2 += p[e2];
+  }
+  if (a.bias != nullptr) {
+    x1 += __bfloat162float(a.bias[e1]);
+    x2 += __bfloat162float(a.bias[e2]);
+  }
+  if (hs < a.Hq + a.Hkv) {
+    const float2 cs = a.rope[(size_t)row * half + k];
+    const float y1 = x1 * cs.x - x2 * cs.y;
+    const float y2 = x2 * cs.x + x1 * cs.y;
+    x1 = y1; x2 = y2;
+  }
+  const bf16 o1 = __float2bfloat16_rn(x1), o2 = __float2bfloat16_rn(x2);
+  if (hs < a.Hq) {
+    bf16* q = a.q + (size_t)row * a.Hq * a.D + hs * a.D;
+    q[k] = o1; q[k + half] = o2;
+    return;
+  }
+  const bool is_k = hs < a.Hq + a.Hkv;
+  const int hkv = is_k ? hs - a.Hq : hs - a.Hq - a.Hkv;
+  bf16* f = (is_k ? a.kf : a.vf) + (size_t)row * a.Hkv * a.D + hkv * a.D;
+  f[k] = o1; f[k + half] = o2;
+  const int rps = bp.rows_per_stream;
+  const int b = row / rps, t = row - b * rps;
+  const int sid = bp.stream_id[b];
+  if (a.mode == 0) {
+    if (t == rps - 1 && a.M > 0) {
+      const int slot = a.meta[sid].free_slot;
+      bf16* dst = (is_k ? a.bank_k : a.bank_v) + (((size_t)sid * a.Hkv + hkv) * a.slots + slot) * a.D;
+      dst[k] = o1; dst[k + half] = o2;
+    }
+  } else {
+    const int base = (a.mode == 1) ? bp.prefix_len[b] : bp.text_len[b];
+    bf16* dst = (is_k ? a.text_k : a.text_v) + (((size_t)sid * a.Hkv + hkv) * a.text_cap + base + t) * a.D;
+    dst[k] = o1; dst[k + half] = o2;
+  }
+}
+
+cudaError_t launch_finalize(const FinalizeArgs& a, const BatchParams& bp, cudaStream_t st) {
+  const int n_pairs = (a.Hq + 2 * a.Hkv) * (a.D / 2);
+  dim3 grid((n_pairs + 255) / 256, a.rows);
+  finalize_kernel<<<grid, 256, 0, st>>>(a, bp);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Eviction scoring (Section 3.3: discard the older carrier with the largest cosine
+// similarity).  One warp per temporal index j.  Dot products are accumulated in fp64 in a
+// fixed order -- lane p sums elements k = p (mod 32) in ascending k, then a butterfly
+// 16, 8, 4, 2, 1 -- so that the score, and with it the argmax, is reproducible bit for bit.
+// Products of two bf16 values are exact in fp64, so fused and unfused accumulation agree.
+// The last block to finish picks the victim: largest score, oldest on ties.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ double warp_tree_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = __dadd_rn(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+__global__ void __launch_bounds__(256) evict_score_kernel(EvictArgs a, BatchParams bp) {
+  const int b = blockIdx.y;
+  const int sid = bp.stream_id[b];
+  const int count = bp.count[b];
+  if (count < a.M || a.M == 0) return;             // bank not full: nothing to score
+  StreamMeta* meta = a.meta + sid;
+  const int32_t* order = a.order + (size_t)sid * a.slots;
+  double* scores = a.scores + (size_t)sid * a.slots;
+  const int lane = threadIdx.x & 31;
+  const int j = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int incoming = meta->free_slot;
+  if (j < count) {
+    const int sa = order[j];
+    const int sb = (a.policy == 1 && j + 1 < count) ? order[j + 1] : incoming;
+    const bf16* va = a.emb + ((size_t)sid * a.slots + sa) * a.d;
+    const bf16* vb = a.emb + ((size_t)sid * a.slots + sb) * a.d;
+    double dot = 0.0, na = 0.0, nb = 0.0;
+    for (int k = lane; k < a.d; k += 32) {
+      const double x = (double)__bfloat162float(va[k]);
+      const double y = (double)__bfloat162float(vb[k]);
+      dot = __dadd_rn(dot, __dmul_rn(x, y));
+      na = __dadd_rn(na, __dmul_rn(x, x));
+      nb = __dadd_rn(nb, __dmul_rn(y, y));
+    }
+    dot = warp_tree_sum(dot); na = warp_tree_sum(na); nb = warp_tree_sum(nb);
+    if (lane == 0) {
+      double s = 0.0;
+      if (na != 0.0 && nb != 0.0) s = __ddiv_rn(dot, __dmul_rn(__dsqrt_rn(na), __dsqrt_rn(nb)));
+      scores[j] = s;
+    }
+  }
+  // the last block of this stream to finish does the argmax
+  __shared__ int is_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int done = atomicAdd(&meta->score_ticket, 1);
+    is_last = (done == (int)gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  __shared__ double best_s[256];
+  __shared__ int best_j[256];
+  double bs = -2.0; int bj = 0x7fffffff;
+  for (int i = threadIdx.x; i < count; i += blockDim.x) {
+    const double s = __ldcg(scores + i);
+    if (s > bs) { bs = s; bj = i; }                 // ascending i: first maximum kept
+  }
+  best_s[threadIdx.x] = bs; best_j[threadIdx.x] = bj;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if ((int)threadIdx.x < o) {
+      const double s2 = best_s[threadIdx.x + o]; const int j2 = best_j[threadIdx.x + o];
+      if (s2 > best_s[threadIdx.x] || (s2 == best_s[threadIdx.x] && j2 < best_j[threadIdx.x])) {
+        best_s[threadIdx.x] = s2; best_j[threadIdx.x] = j2;
+      }
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    meta->victim_logical = (a.policy == 2) ? 0 : best_j[0];
+    meta->score_ticket = 0;
+  }
+}
+
+cudaError_t launch_evict_score(const EvictArgs& a, const BatchParams& bp, cudaStream_t st) {
+  dim3 grid((a.M + 7) / 8, bp.n_active);
+  evict_score_kernel<<<grid, 256, 0, st>>>(a, bp);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Bank commit: evict-if-full, then append (Section 3.3).  One block per listed stream.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) commit_kernel(CommitArgs a, BatchParams bp) {
+  const int b = blockIdx.x;
+  const int sid = bp.stream_id[b];
+  StreamMeta* meta = a.meta + sid;
+  if (a.M == 0) {
+    if (threadIdx.x == 0) { meta->frames_seen += 1; meta->last_victim_frame = -1; }
+    return;
+  }
+  int32_t* order = a.order + (size_t)sid * a.slots;
+  int32_t* slot_frame = a.slot_frame + (size_t)sid * a.slots;
+  int64_t* slot_pos = a.slot_pos + (size_t)sid * a.slots;
+  const int count = meta->count;
+  const int incoming = meta->free_slot;
+  const int64_t carrier_pos = bp.pos_base[b] + bp.rows_per_stream - 1;
+  if (count == a.M) {
+    const int v = meta->victim_logical;
+    const int victim_slot = order[v];
+    const int victim_frame = slot_frame[victim_slot];
+    __syncthreads();
+    // close the gap in the temporal order, one block-wide chunk at a time in ascending
+    // order: a chunk reads [base+1, base+256] before anything at or above base is written
+    for (int base = v; base < count - 1; base += blockDim.x) {
+      const int j = base + threadIdx.x;
+      const int32_t next = (j < count - 1) ? order[j + 1] : 0;
+      __syncthreads();
+      if (j < count - 1) order[j] = next;
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+      order[count - 1] = incoming;
+      slot_frame[victim_slot] = -1;
+      slot_frame[incoming] = (int32_t)bp.frame_id[b];
+      slot_pos[incoming] = carrier_pos;
+      if (a.log_cap > 0) {
+        int32_t* e = a.evict_log + ((size_t)sid * a.log_cap + (meta->log_count % a.log_cap)) * 2;
+        e[0] = (int32_t)bp.frame_id[b];
+        e[1] = victim_frame;
+      }
+      meta->log_count += 1;
+      meta->evictions += 1;
+      meta->last_victim_frame = victim_frame;
+      meta->free_slot = victim_slot;
+      meta->victim_logical = -1;
+      meta->frames_seen += 1;
+    }
+  } else if (threadIdx.x == 0) {
+    order[count] = incoming;
+    slot_frame[incoming] = (int32_t)bp.frame_id[b];
+    slot_pos[incoming] = carrier_pos;
+    meta->count = count + 1;
+    meta->free_slot = count + 1;            // slots fill in order until the bank is full
+    meta->last_victim_frame = -1;
+    meta->frames_seen += 1;
+  }
+}
+
+cudaError_t launch_commit(const CommitArgs& a, const BatchParams& bp, cudaStream_t st) {
+  commit_kernel<<<bp.n_active, 256, 0, st>>>(a, bp);
+  return cudaGetLastError();
+}
+
+__global__ void poison_kernel(uint32_t* p, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    p[i] = 0xFFFFFFFFu;
+}
+
+cudaError_t launch_poison(void* p, size_t bytes, cudaStream_t st) {
+  poison_kernel<<<592, 256, 0, st>>>(reinterpret_cast<uint32_t*>(p), bytes / 4);
+  return cudaGetLastError();
+}
+
+}  // namespace vs
