@@ -43,7 +43,8 @@ struct BatchParams {
 // ---- shapes ----------------------------------------------------------------------------
 struct Dims {
   int L, d, Hq, Hkv, D, G, E_out;
-  int maxN, maxP, maxT, maxStepT, M, slots, S;
+  int maxN, maxP, maxT, maxStepT, M, slots, S;   // maxP / maxT: allocated rows (>= 1)
+  int capP, capT;                                // caller's prefix / tail capacities
   int rows_per_stream_max, R_max;
   int log_cap;
   int agg_mode, evict_policy, use_rmsnorm, residual;

@@ -1,0 +1,584 @@
+// Host layer of the C ABI: argument checks, workspace carve-up, launch sequencing.
+// Per frame (Section 3.3, prefilling): pool -> per layer [norm] -> QKV GEMM -> finalize
+// (RoPE, carrier K/V into the bank's free slot) -> attention [-> residual] -> eviction
+// scoring (only when the bank is full) -> bank commit.  Per text step (Section 3.3,
+// decoding): RoPE table -> per layer [norm] -> GEMM -> finalize (K/V appended to prefix or
+// tail) -> attention.  Nothing here allocates device memory or synchronises, except
+// create / bank_state / last_step_kv.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "vs_common.cuh"
+
+using namespace vs;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct HostStream {
+  int64_t frames_seen = 0, next_pos = 0, prefix_len = 0, text_len = 0;
+};
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int fill_dims(const vs_config* c, Dims& D) {
+  if (c == nullptr) return VS_ERR_INVALID_ARG;
+  if (c->n_layers < 1 || c->d_model < 64 || c->n_q_heads < 1 || c->n_kv_heads < 1) return VS_ERR_INVALID_ARG;
+  if (c->n_streams < 1 || c->n_streams > VS_MAX_BATCH) return VS_ERR_INVALID_ARG;
+  if (c->max_tokens_per_frame < 1 || c->max_prefix < 0 || c->max_text < 0 || c->bank_capacity < 0) return VS_ERR_INVALID_ARG;
+  if (c->max_step_tokens < 1 || c->evict_log_capacity < 0) return VS_ERR_INVALID_ARG;
+  if (c->agg_mode < 0 || c->agg_mode > 1 || c->evict_policy < 0 || c->evict_policy > 2) return VS_ERR_INVALID_ARG;
+  if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f)) return VS_ERR_INVALID_ARG;
+  if (c->d_model % 64 != 0) return VS_ERR_UNSUPPORTED;
+  if (c->head_dim != 64 && c->head_dim != 128) return VS_ERR_UNSUPPORTED;
+  if (c->n_q_heads % c->n_kv_heads != 0 || c->n_q_heads / c->n_kv_heads > 8) return VS_ERR_UNSUPPORTED;
+  if (c->max_tokens_per_frame + 1 > 256) return VS_ERR_UNSUPPORTED;
+  if (c->n_layers > 1 && !c->residual) return VS_ERR_INVALID_ARG;
+  if (c->residual && c->n_q_heads * c->head_dim != c->d_model) return VS_ERR_INVALID_ARG;
+  D.L = c->n_layers; D.d = c->d_model; D.Hq = c->n_q_heads; D.Hkv = c->n_kv_heads; D.D = c->head_dim;
+  D.G = D.Hq / D.Hkv; D.E_out = (D.Hq + 2 * D.Hkv) * D.D;
+  D.maxN = c->max_tokens_per_frame; D.maxP = c->max_prefix > 0 ? c->max_prefix : 1;
+  D.maxT = c->max_text > 0 ? c->max_text : 1; D.maxStepT = c->max_step_tokens;
+  D.capP = c->max_prefix; D.capT = c->max_text;
+  D.M = c->bank_capacity; D.slots = D.M + 1; D.S = c->n_streams;
+  D.rows_per_stream_max = (D.maxN + 1 > D.maxStepT) ? D.maxN + 1 : D.maxStepT;
+  D.R_max = D.rows_per_stream_max * D.S;
+  D.log_cap = c->evict_log_capacity;
+  D.agg_mode = c->agg_mode; D.evict_policy = c->evict_policy; D.use_rmsnorm = c->use_rmsnorm ? 1 : 0;
+  D.residual = c->residual ? 1 : 0; D.rope_theta = c->rope_theta; D.rms_eps = c->rms_eps;
+  return VS_OK;
+}
+
+void fill_layout(const Dims& D, Layout& Lo) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t kv_bank = (size_t)D.L * D.S * D.Hkv * D.slots * D.D * 2;
+  const size_t kv_pre = (size_t)D.L * D.S * D.Hkv * D.maxP * D.D * 2;
+  const size_t kv_tail = (size_t)D.L * D.S * D.Hkv * D.maxT * D.D * 2;
+  Lo.bank_k = take(kv_bank); Lo.bank_v = take(kv_bank);
+  Lo.prefix_k = take(kv_pre); Lo.prefix_v = take(kv_pre);
+  Lo.tail_k = take(kv_tail); Lo.tail_v = take(kv_tail);
+  Lo.emb = take((size_t)D.S * D.slots * D.d * 2);
+  Lo.meta = take((size_t)D.S * sizeof(StreamMeta));
+  Lo.order = take((size_t)D.S * D.slots * 4);
+  Lo.slot_frame = take((size_t)D.S * D.slots * 4);
+  Lo.slot_pos = take((size_t)D.S * D.slots * 8);
+  Lo.evict_log = take((size_t)D.S * (D.log_cap > 0 ? D.log_cap : 1) * 8);
+  Lo.scores = take((size_t)D.S * D.slots * 8);
+  Lo.inv_freq = take((size_t)(D.D / 2) * 8);
+  Lo.status = take(8 * 4);
+  Lo.tickets = take((size_t)D.S * D.Hkv * 4);
+  Lo.persistent_end = off;
+  Lo.scratch_begin = off;
+  Lo.hbuf[0] = take((size_t)D.R_max * D.d * 2);
+  Lo.hbuf[1] = take((size_t)D.R_max * D.d * 2);
+  Lo.xn = take((size_t)D.R_max * D.d * 2);
+  Lo.partials = take((size_t)KSPLIT_MAX * D.R_max * D.E_out * 4);
+  Lo.q = take((size_t)D.R_max * D.Hq * D.D * 2);
+  Lo.kf = take((size_t)D.R_max * D.Hkv * D.D * 2);
+  Lo.vf = take((size_t)D.R_max * D.Hkv * D.D * 2);
+  Lo.rope = take((size_t)D.R_max * (D.D / 2) * 8);
+  Lo.obuf = take((size_t)D.R_max * D.Hq * D.D * 2);
+  Lo.dec_part = take((size_t)DEC_SPLIT_MAX * D.S * D.Hq * (D.D + 2) * 4);
+  Lo.scratch_end = off;
+  Lo.total = off;
+}
+
+}  // namespace
+
+struct vs_stream {
+  Dims dm;
+  Layout lo;
+  uint8_t* ws = nullptr;
+  size_t ws_bytes = 0;
+  int device = 0;
+  std::vector<const bf16*> w, bias, gain;
+  std::vector<CUtensorMap> tm_w;
+  std::vector<HostStream> hs;
+  EncodeTiledFn encode = nullptr;
+  cudaStream_t last_stream = nullptr;
+  int last_rows = 0;
+
+  template <typename T>
+  T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+};
+
+namespace {
+
+int encode_2d(vs_stream* h, CUtensorMap* tm, const void* base, uint64_t inner, uint64_t rows, uint32_t box_rows) {
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {inner * 2};
+  cuuint32_t box[2] = {(cuuint32_t)GEMM_BLOCK_K, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = h->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? VS_OK : VS_ERR_CUDA;
+}
+
+void choose_tiles(const Dims& D, int rows, int& tile_n, int& n_tiles, int& ksplit) {
+  n_tiles = (rows + 255) / 256;
+  const int per = (rows + n_tiles - 1) / n_tiles;
+  tile_n = (per + 15) / 16 * 16;
+  const int m_tiles = (D.E_out + GEMM_BLOCK_M - 1) / GEMM_BLOCK_M;
+  const int total_kb = D.d / GEMM_BLOCK_K;
+  ksplit = 1;
+  for (int ks = 1; ks <= KSPLIT_MAX; ++ks) {
+    if (total_kb % ks != 0) continue;
+    if (m_tiles * n_tiles * ks <= 148) ksplit = ks;
+  }
+}
+
+int check_ids(vs_stream* h, const int32_t* ids, int32_t n) {
+  if (h == nullptr || ids == nullptr || n < 1 || n > h->dm.S) return VS_ERR_INVALID_ARG;
+  bool seen[VS_MAX_BATCH] = {false};
+  for (int i = 0; i < n; ++i) {
+    if (ids[i] < 0 || ids[i] >= h->dm.S || seen[ids[i]]) return VS_ERR_INVALID_ARG;
+    seen[ids[i]] = true;
+  }
+  return VS_OK;
+}
+
+#define VS_CK(expr) do { if ((expr) != cudaSuccess) return VS_ERR_CUDA; } while (0)
+
+// QKV projection of `rows` token rows read from `src` ([rows][d] bf16) for layer l.
+int run_projection(vs_stream* h, int l, const bf16* src, int rows, int& ksplit_out, cudaStream_t st) {
+  const Dims& D = h->dm;
+  GemmArgs g;
+  choose_tiles(D, rows, g.tile_n, g.n_tiles, g.ksplit);
+  g.tm_w = h->tm_w[l];
+  if (encode_2d(h, &g.tm_x, src, (uint64_t)D.d, (uint64_t)rows, (uint32_t)g.tile_n) != VS_OK) return VS_ERR_CUDA;
+  g.partials = h->at<float>(h->lo.partials);
+  g.rows = rows; g.E_out = D.E_out; g.d = D.d;
+  g.status = h->at<int>(h->lo.status);
+  ksplit_out = g.ksplit;
+  VS_CK(launch_qkv_gemm(g, st));
+  return VS_OK;
+}
+
+size_t layer_stride_bank(const Dims& D) { return (size_t)D.S * D.Hkv * D.slots * D.D; }
+size_t layer_stride_prefix(const Dims& D) { return (size_t)D.S * D.Hkv * D.maxP * D.D; }
+size_t layer_stride_tail(const Dims& D) { return (size_t)D.S * D.Hkv * D.maxT * D.D; }
+
+}  // namespace
+
+extern "C" {
+
+const char* vs_status_string(int status) {
+  switch (status) {
+    case VS_OK: return "ok";
+    case VS_ERR_INVALID_ARG: return "invalid argument";
+    case VS_ERR_STATE: return "call not legal in the stream's current phase";
+    case VS_ERR_CAPACITY: return "capacity exceeded";
+    case VS_ERR_CUDA: return "CUDA call failed";
+    case VS_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case VS_ERR_UNSUPPORTED: return "unsupported shape";
+    default: return "unknown status";
+  }
+}
+
+int vs_workspace_bytes(const vs_config* cfg, size_t* out_bytes) {
+  if (out_bytes == nullptr) return VS_ERR_INVALID_ARG;
+  Dims D;
+  const int rc = fill_dims(cfg, D);
+  if (rc != VS_OK) return rc;
+  Layout lo;
+  fill_layout(D, lo);
+  *out_bytes = lo.total;
+  return VS_OK;
+}
+
+int vs_create_stream(const vs_config* cfg, const vs_weights* weights, void* workspace, size_t workspace_bytes,
+                     vs_stream** out) {
+  if (out == nullptr) return VS_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (weights == nullptr || weights->w_qkv == nullptr || workspace == nullptr) return VS_ERR_INVALID_ARG;
+  Dims D;
+  const int rc = fill_dims(cfg, D);
+  if (rc != VS_OK) return rc;
+  Layout lo;
+  fill_layout(D, lo);
+  if (workspace_bytes < lo.total) return VS_ERR_CAPACITY;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return VS_ERR_INVALID_ARG;
+  for (int l = 0; l < D.L; ++l) {
+    if (weights->w_qkv[l] == nullptr) return VS_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(weights->w_qkv[l]) & 15u) != 0) return VS_ERR_INVALID_ARG;
+  }
+  VS_CK(cudaSetDevice(cfg->device));
+  vs_stream* h = new (std::nothrow) vs_stream();
+  if (h == nullptr) return VS_ERR_INVALID_ARG;
+  h->dm = D; h->lo = lo; h->ws = static_cast<uint8_t*>(workspace); h->ws_bytes = workspace_bytes;
+  h->device = cfg->device;
+  h->hs.assign(D.S, HostStream());
+  for (int l = 0; l < D.L; ++l) {
+    h->w.push_back(static_cast<const bf16*>(weights->w_qkv[l]));
+    h->bias.push_back(weights->b_qkv ? static_cast<const bf16*>(weights->b_qkv[l]) : nullptr);
+    h->gain.push_back(weights->norm_w ? static_cast<const bf16*>(weights->norm_w[l]) : nullptr);
+  }
+  auto fail = [&](int code) { delete h; return code; };
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr ||
+      qres != cudaDriverEntryPointSuccess)
+    return fail(VS_ERR_CUDA);
+  h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  h->tm_w.resize(D.L);
+  for (int l = 0; l < D.L; ++l)
+    if (encode_2d(h, &h->tm_w[l], h->w[l], (uint64_t)D.d, (uint64_t)D.E_out, GEMM_BLOCK_M) != VS_OK) return fail(VS_ERR_CUDA);
+  if (qkv_gemm_init() != cudaSuccess || prefill_attention_init() != cudaSuccess) return fail(VS_ERR_CUDA);
+  // clear the whole workspace, then write the non-zero initial metadata
+  if (cudaMemset(h->ws, 0, lo.total) != cudaSuccess) return fail(VS_ERR_CUDA);
+  if (cudaMemset(h->ws + lo.slot_frame, 0xFF, (size_t)D.S * D.slots * 4) != cudaSuccess) return fail(VS_ERR_CUDA);
+  std::vector<StreamMeta> metas(D.S);
+  for (auto& m : metas) { std::memset(&m, 0, sizeof(m)); m.victim_logical = -1; m.last_victim_frame = -1; }
+  if (cudaMemcpy(h->ws + lo.meta, metas.data(), metas.size() * sizeof(StreamMeta), cudaMemcpyHostToDevice) != cudaSuccess)
+    return fail(VS_ERR_CUDA);
+  std::vector<double> inv(D.D / 2);
+  for (int k = 0; k < D.D / 2; ++k) inv[k] = std::pow((double)D.rope_theta, -2.0 * (double)k / (double)D.D);
+  if (cudaMemcpy(h->ws + lo.inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice) != cudaSuccess)
+    return fail(VS_ERR_CUDA);
+  if (cudaDeviceSynchronize() != cudaSuccess) return fail(VS_ERR_CUDA);
+  *out = h;
+  return VS_OK;
+}
+
+int vs_destroy_stream(vs_stream* h) {
+  if (h == nullptr) return VS_ERR_INVALID_ARG;
+  delete h;
+  return VS_OK;
+}
+
+int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, const void* hidden, int32_t N,
+                     const void* carrier_override, void* out, void* cuda_stream) {
+  int rc = check_ids(h, stream_ids, n_active);
+  if (rc != VS_OK) return rc;
+  if (hidden == nullptr || N < 1) return VS_ERR_INVALID_ARG;
+  const Dims& D = h->dm;
+  const Layout& lo = h->lo;
+  if (N > D.maxN) return VS_ERR_CAPACITY;
+  for (int i = 0; i < n_active; ++i)
+    if (h->hs[stream_ids[i]].text_len != 0) return VS_ERR_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  VS_CK(cudaSetDevice(h->device));
+
+  BatchParams bp;
+  std::memset(&bp, 0, sizeof(bp));
+  bp.n_active = n_active;
+  bp.rows_per_stream = N + 1;
+  bool any_full = false;
+  for (int i = 0; i < n_active; ++i) {
+    const HostStream& s = h->hs[stream_ids[i]];
+    bp.stream_id[i] = stream_ids[i];
+    bp.count[i] = (int32_t)(s.frames_seen < D.M ? s.frames_seen : D.M);
+    bp.prefix_len[i] = (int32_t)s.prefix_len;
+    bp.text_len[i] = 0;
+    bp.pos_base[i] = s.next_pos;
+    bp.frame_id[i] = s.frames_seen;
+    if (D.M > 0 && bp.count[i] == D.M) any_full = true;
+  }
+  const int rows = n_active * (N + 1);
+  StreamMeta* meta = h->at<StreamMeta>(lo.meta);
+
+  PoolArgs pa;
+  pa.hidden = static_cast<const bf16*>(hidden);
+  pa.carrier_override = static_cast<const bf16*>(carrier_override);
+  pa.x = h->at<bf16>(lo.hbuf[0]);
+  pa.emb = h->at<bf16>(lo.emb);
+  pa.meta = meta;
+  pa.inv_freq = h->at<double>(lo.inv_freq);
+  pa.rope = h->at<float2>(lo.rope);
+  pa.N = N; pa.d = D.d; pa.D = D.D; pa.slots = D.slots; pa.M = D.M; pa.agg_mode = D.agg_mode;
+  VS_CK(launch_pool(pa, bp, st));
+
+  bf16* out_final = out ? static_cast<bf16*>(out) : h->at<bf16>(lo.obuf);
+  int cur = 0;
+  for (int l = 0; l < D.L; ++l) {
+    const bf16* h_in = h->at<bf16>(lo.hbuf[cur]);
+    const bf16* src = h_in;
+    if (D.use_rmsnorm) {
+      VS_CK(launch_rmsnorm(h_in, h->gain[l], h->at<bf16>(lo.xn), rows, D.d, D.rms_eps, st));
+      src = h->at<bf16>(lo.xn);
+    }
+    int ksplit = 1;
+    rc = run_projection(h, l, src, rows, ksplit, st);
+    if (rc != VS_OK) return rc;
+
+    FinalizeArgs fa;
+    fa.partials = h->at<float>(lo.partials);
+    fa.bias = h->bias[l];
+    fa.rope = h->at<float2>(lo.rope);
+    fa.q = h->at<bf16>(lo.q); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
+    fa.bank_k = h->at<bf16>(lo.bank_k) + (size_t)l * layer_stride_bank(D);
+    fa.bank_v = h->at<bf16>(lo.bank_v) + (size_t)l * layer_stride_bank(D);
+    fa.text_k = nullptr; fa.text_v = nullptr;
+    fa.meta = meta;
+    fa.rows = rows; fa.ksplit = ksplit; fa.E_out = D.E_out; fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D;
+    fa.slots = D.slots; fa.text_cap = 0; fa.mode = 0; fa.M = D.M;
+    VS_CK(launch_finalize(fa, bp, st));
+
+    AttnArgs aa;
+    std::memset(&aa, 0, sizeof(aa));
+    aa.q = fa.q;
+    aa.seg[0] = {h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D),
+                 h->at<bf16>(lo.prefix_v) + (size_t)l * layer_stride_prefix(D),
+                 (long long)D.Hkv * D.maxP * D.D, (long long)D.maxP * D.D, (long long)D.D, 0, 0};
+    aa.seg[1] = {fa.bank_k, fa.bank_v, (long long)D.Hkv * D.slots * D.D, (long long)D.slots * D.D, (long long)D.D, 1, 0};
+    aa.seg[2] = {fa.kf, fa.vf, (long long)(N + 1) * D.Hkv * D.D, (long long)D.D, (long long)D.Hkv * D.D, 3, 1};
+    aa.n_seg = 3;
+    const bool last = (l == D.L - 1);
+    aa.out = last ? out_final : h->at<bf16>(lo.obuf);
+    aa.h_in = D.residual ? h_in : nullptr;
+    aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
+    aa.meta = meta;
+    aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
+    aa.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
+    VS_CK(launch_prefill_attention(aa, bp, st));
+    if (D.residual) cur ^= 1;
+  }
+
+  if (any_full) {
+    EvictArgs ea;
+    ea.emb = h->at<bf16>(lo.emb); ea.meta = meta;
+    ea.order = h->at<int32_t>(lo.order); ea.scores = h->at<double>(lo.scores);
+    ea.d = D.d; ea.slots = D.slots; ea.M = D.M; ea.policy = D.evict_policy;
+    VS_CK(launch_evict_score(ea, bp, st));
+  }
+  CommitArgs ca;
+  ca.meta = meta; ca.order = h->at<int32_t>(lo.order); ca.slot_frame = h->at<int32_t>(lo.slot_frame);
+  ca.slot_pos = h->at<int64_t>(lo.slot_pos); ca.evict_log = h->at<int32_t>(lo.evict_log);
+  ca.slots = D.slots; ca.M = D.M; ca.log_cap = D.log_cap;
+  VS_CK(launch_commit(ca, bp, st));
+
+  for (int i = 0; i < n_active; ++i) {
+    HostStream& s = h->hs[stream_ids[i]];
+    s.next_pos += N + 1;
+    s.frames_seen += 1;
+  }
+  h->last_stream = st;
+  h->last_rows = rows;
+  return VS_OK;
+}
+
+int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, const void* hidden, int32_t T,
+                   void* out, void* cuda_stream) {
+  int rc = check_ids(h, stream_ids, n_active);
+  if (rc != VS_OK) return rc;
+  if (hidden == nullptr || out == nullptr || T < 1) return VS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(hidden) & 15u) != 0) return VS_ERR_INVALID_ARG;
+  const Dims& D = h->dm;
+  const Layout& lo = h->lo;
+  if (T > D.maxStepT) return VS_ERR_CAPACITY;
+  const bool to_prefix = h->hs[stream_ids[0]].frames_seen == 0;
+  for (int i = 0; i < n_active; ++i) {
+    const HostStream& s = h->hs[stream_ids[i]];
+    if ((s.frames_seen == 0) != to_prefix) return VS_ERR_STATE;
+    if (to_prefix ? (s.prefix_len + T > D.capP) : (s.text_len + T > D.capT)) return VS_ERR_CAPACITY;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  VS_CK(cudaSetDevice(h->device));
+
+  BatchParams bp;
+  std::memset(&bp, 0, sizeof(bp));
+  bp.n_active = n_active;
+  bp.rows_per_stream = T;
+  int max_keys = 0;
+  for (int i = 0; i < n_active; ++i) {
+    const HostStream& s = h->hs[stream_ids[i]];
+    bp.stream_id[i] = stream_ids[i];
+    bp.count[i] = (int32_t)(s.frames_seen < D.M ? s.frames_seen : D.M);
+    bp.prefix_len[i] = (int32_t)s.prefix_len;
+    bp.text_len[i] = (int32_t)s.text_len;
+    bp.pos_base[i] = to_prefix ? s.next_pos : s.next_pos + s.text_len;
+    bp.frame_id[i] = s.frames_seen;
+    const int keys = (int)s.prefix_len + bp.count[i] + 1 + (int)s.text_len + T;
+    if (keys > max_keys) max_keys = keys;
+  }
+  const int rows = n_active * T;
+  StreamMeta* meta = h->at<StreamMeta>(lo.meta);
+
+  RopeArgs ra;
+  ra.inv_freq = h->at<double>(lo.inv_freq); ra.rope = h->at<float2>(lo.rope); ra.D = D.D;
+  VS_CK(launch_rope_table(ra, bp, st));
+
+  const bf16* h_in = static_cast<const bf16*>(hidden);
+  int next_buf = 0;
+  for (int l = 0; l < D.L; ++l) {
+    const bf16* src = h_in;
+    if (D.use_rmsnorm) {
+      VS_CK(launch_rmsnorm(h_in, h->gain[l], h->at<bf16>(lo.xn), rows, D.d, D.rms_eps, st));
+      src = h->at<bf16>(lo.xn);
+    }
+    int ksplit = 1;
+    rc = run_projection(h, l, src, rows, ksplit, st);
+    if (rc != VS_OK) return rc;
+
+    bf16* pk = h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D);
+    bf16* pv = h->at<bf16>(lo.prefix_v) + (size_t)l * layer_stride_prefix(D);
+    bf16* tk = h->at<bf16>(lo.tail_k) + (size_t)l * layer_stride_tail(D);
+    bf16* tv = h->at<bf16>(lo.tail_v) + (size_t)l * layer_stride_tail(D);
+    bf16* bk = h->at<bf16>(lo.bank_k) + (size_t)l * layer_stride_bank(D);
+    bf16* bv = h->at<bf16>(lo.bank_v) + (size_t)l * layer_stride_bank(D);
+
+    FinalizeArgs fa;
+    fa.partials = h->at<float>(lo.partials);
+    fa.bias = h->bias[l];
+    fa.rope = h->at<float2>(lo.rope);
+    fa.q = h->at<bf16>(lo.q); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
+    fa.bank_k = bk; fa.bank_v = bv;
+    fa.text_k = to_prefix ? pk : tk; fa.text_v = to_prefix ? pv : tv;
+    fa.meta = meta;
+    fa.rows = rows; fa.ksplit = ksplit; fa.E_out = D.E_out; fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D;
+    fa.slots = D.slots; fa.text_cap = to_prefix ? D.maxP : D.maxT; fa.mode = to_prefix ? 1 : 2; fa.M = D.M;
+    VS_CK(launch_finalize(fa, bp, st));
+
+    bf16* h_out = D.residual ? h->at<bf16>(lo.hbuf[next_buf]) : nullptr;
+    const float scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
+    if (T == 1) {
+      DecodeArgs da;
+      da.q = fa.q;
+      da.prefix_k = pk; da.prefix_v = pv; da.bank_k = bk; da.bank_v = bv; da.tail_k = tk; da.tail_v = tv;
+      da.partials = h->at<float>(lo.dec_part);
+      da.tickets = h->at<int>(lo.tickets);
+      da.out = static_cast<bf16*>(out);
+      da.h_in = D.residual ? h_in : nullptr; da.h_out = h_out;
+      da.meta = meta;
+      da.Hq = D.Hq; da.Hkv = D.Hkv; da.D = D.D; da.slots = D.slots; da.M = D.M; da.maxP = D.maxP; da.maxT = D.maxT;
+      int ns = (max_keys + 63) / 64;
+      if (ns < 1) ns = 1;
+      if (ns > DEC_SPLIT_MAX) ns = DEC_SPLIT_MAX;
+      da.nsplit = ns;
+      da.to_prefix = to_prefix ? 1 : 0;
+      da.scale_log2e = scale_log2e;
+      VS_CK(launch_decode_attention(da, bp, st));
+    } else {
+      AttnArgs aa;
+      std::memset(&aa, 0, sizeof(aa));
+      aa.q = fa.q;
+      int ns = 0;
+      aa.seg[ns++] = {pk, pv, (long long)D.Hkv * D.maxP * D.D, (long long)D.maxP * D.D, (long long)D.D, 0, 0};
+      if (!to_prefix) {
+        aa.seg[ns++] = {bk, bv, (long long)D.Hkv * D.slots * D.D, (long long)D.slots * D.D, (long long)D.D, 1, 0};
+        aa.seg[ns++] = {tk, tv, (long long)D.Hkv * D.maxT * D.D, (long long)D.maxT * D.D, (long long)D.D, 2, 0};
+      }
+      aa.seg[ns++] = {fa.kf, fa.vf, (long long)T * D.Hkv * D.D, (long long)D.D, (long long)D.Hkv * D.D, 3, 1};
+      aa.n_seg = ns;
+      aa.out = static_cast<bf16*>(out);
+      aa.h_in = D.residual ? h_in : nullptr;
+      aa.h_out = h_out;
+      aa.meta = meta;
+      aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
+      aa.scale_log2e = scale_log2e;
+      VS_CK(launch_prefill_attention(aa, bp, st));
+    }
+    if (D.residual) { h_in = h_out; next_buf ^= 1; }
+  }
+
+  for (int i = 0; i < n_active; ++i) {
+    HostStream& s = h->hs[stream_ids[i]];
+    if (to_prefix) { s.prefix_len += T; s.next_pos += T; }
+    else s.text_len += T;
+  }
+  h->last_stream = st;
+  h->last_rows = rows;
+  return VS_OK;
+}
+
+int vs_end_turn(vs_stream* h, const int32_t* stream_ids, int32_t n_active) {
+  const int rc = check_ids(h, stream_ids, n_active);
+  if (rc != VS_OK) return rc;
+  for (int i = 0; i < n_active; ++i) h->hs[stream_ids[i]].text_len = 0;
+  return VS_OK;
+}
+
+int vs_bank_state(vs_stream* h, int32_t stream_id, vs_bank_info* info, int32_t* frame_ids, int64_t* positions,
+                  int32_t* slots, int32_t* evict_log, int32_t evict_log_cap, int32_t* evict_log_n, void* emb_out,
+                  int32_t layer, void* k_out, void* v_out) {
+  if (h == nullptr || stream_id < 0 || stream_id >= h->dm.S) return VS_ERR_INVALID_ARG;
+  const Dims& D = h->dm;
+  const Layout& lo = h->lo;
+  if ((k_out != nullptr || v_out != nullptr) && (layer < 0 || layer >= D.L)) return VS_ERR_INVALID_ARG;
+  VS_CK(cudaSetDevice(h->device));
+  VS_CK(cudaStreamSynchronize(h->last_stream));
+  StreamMeta m;
+  VS_CK(cudaMemcpy(&m, h->ws + lo.meta + (size_t)stream_id * sizeof(StreamMeta), sizeof(m), cudaMemcpyDeviceToHost));
+  int status[8];
+  VS_CK(cudaMemcpy(status, h->ws + lo.status, sizeof(status), cudaMemcpyDeviceToHost));
+  std::vector<int32_t> order(D.slots), sframe(D.slots);
+  std::vector<int64_t> spos(D.slots);
+  VS_CK(cudaMemcpy(order.data(), h->ws + lo.order + (size_t)stream_id * D.slots * 4, (size_t)D.slots * 4, cudaMemcpyDeviceToHost));
+  VS_CK(cudaMemcpy(sframe.data(), h->ws + lo.slot_frame + (size_t)stream_id * D.slots * 4, (size_t)D.slots * 4, cudaMemcpyDeviceToHost));
+  VS_CK(cudaMemcpy(spos.data(), h->ws + lo.slot_pos + (size_t)stream_id * D.slots * 8, (size_t)D.slots * 8, cudaMemcpyDeviceToHost));
+  const HostStream& s = h->hs[stream_id];
+  if (info != nullptr) {
+    info->count = m.count; info->capacity = D.M;
+    info->frames_seen = m.frames_seen; info->evictions = m.evictions;
+    info->next_pos = s.next_pos; info->prefix_len = s.prefix_len; info->text_len = s.text_len;
+    info->last_victim_frame = m.last_victim_frame;
+    info->device_status = status[0];
+    info->persistent_bytes = lo.persistent_end;
+    info->workspace_bytes = lo.total;
+  }
+  for (int j = 0; j < m.count; ++j) {
+    const int sl = order[j];
+    if (frame_ids) frame_ids[j] = sframe[sl];
+    if (positions) positions[j] = spos[sl];
+    if (slots) slots[j] = sl;
+  }
+  if (evict_log != nullptr && evict_log_cap > 0 && D.log_cap > 0) {
+    std::vector<int32_t> ring((size_t)D.log_cap * 2);
+    VS_CK(cudaMemcpy(ring.data(), h->ws + lo.evict_log + (size_t)stream_id * D.log_cap * 8, ring.size() * 4, cudaMemcpyDeviceToHost));
+    int kept = m.log_count < D.log_cap ? m.log_count : D.log_cap;
+    if (kept > evict_log_cap) kept = evict_log_cap;
+    for (int i = 0; i < kept; ++i) {
+      const int src = (m.log_count - kept + i) % D.log_cap;
+      evict_log[2 * i] = ring[2 * src]; evict_log[2 * i + 1] = ring[2 * src + 1];
+    }
+    if (evict_log_n) *evict_log_n = kept;
+  } else if (evict_log_n) {
+    *evict_log_n = 0;
+  }
+  if (emb_out != nullptr) {
+    for (int j = 0; j < m.count; ++j)
+      VS_CK(cudaMemcpy(static_cast<uint8_t*>(emb_out) + (size_t)j * D.d * 2,
+                       h->ws + lo.emb + ((size_t)stream_id * D.slots + order[j]) * D.d * 2, (size_t)D.d * 2, cudaMemcpyDeviceToHost));
+  }
+  for (int which = 0; which < 2; ++which) {
+    uint8_t* dst = static_cast<uint8_t*>(which == 0 ? k_out : v_out);
+    if (dst == nullptr) continue;
+    const size_t base = (which == 0 ? lo.bank_k : lo.bank_v) + (size_t)layer * layer_stride_bank(D) * 2;
+    for (int j = 0; j < m.count; ++j)
+      for (int hk = 0; hk < D.Hkv; ++hk)
+        VS_CK(cudaMemcpy(dst + ((size_t)j * D.Hkv + hk) * D.D * 2,
+                         h->ws + base + ((((size_t)stream_id * D.Hkv + hk) * D.slots) + order[j]) * D.D * 2,
+                         (size_t)D.D * 2, cudaMemcpyDeviceToHost));
+  }
+  return status[0] == 0 ? VS_OK : status[0];
+}
+
+int vs_last_step_kv(vs_stream* h, void* k_out, void* v_out, int32_t rows) {
+  if (h == nullptr || rows < 1 || rows > h->last_rows) return VS_ERR_INVALID_ARG;
+  VS_CK(cudaSetDevice(h->device));
+  VS_CK(cudaStreamSynchronize(h->last_stream));
+  const size_t bytes = (size_t)rows * h->dm.Hkv * h->dm.D * 2;
+  if (k_out) VS_CK(cudaMemcpy(k_out, h->ws + h->lo.kf, bytes, cudaMemcpyDeviceToHost));
+  if (v_out) VS_CK(cudaMemcpy(v_out, h->ws + h->lo.vf, bytes, cudaMemcpyDeviceToHost));
+  return VS_OK;
+}
+
+int vs_poison_scratch(vs_stream* h, void* cuda_stream) {
+  if (h == nullptr) return VS_ERR_INVALID_ARG;
+  VS_CK(cudaSetDevice(h->device));
+  VS_CK(launch_poison(h->ws + h->lo.scratch_begin, h->lo.scratch_end - h->lo.scratch_begin,
+                      static_cast<cudaStream_t>(cuda_stream)));
+  h->last_stream = static_cast<cudaStream_t>(cuda_stream);
+  return VS_OK;
+}
+
+}  // extern "C"
