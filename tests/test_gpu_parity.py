@@ -19,7 +19,7 @@ def run_stream(p: Pair, w: synth.Workload, n_frames=None, check_every=1, questio
     for t in range(F):
         p.frame([0], [w.frame_hidden(t, shared=shared)], f"frame {t}")
         if t % check_every == 0 or t == F - 1:
-            st = p.check_bank(0)
+            st = p.check_bank(0, layer=w.n_layers - 1)
             k, v = p.gpu.last_step_kv(w.tokens_per_frame + 1)
             if st["count"]:      # the append is a pure copy of the carrier row of this step
                 assert np.array_equal(k[-1].reshape(w.n_kv_heads, w.head_dim), st["k"][-1])
