@@ -8,7 +8,7 @@
  *    throws, aborts or sets errno.  vs_status_string() names a code.
  *  - Pointers marked DEVICE are CUDA device pointers on `vs_config.device`; pointers
  *    marked HOST are ordinary host memory.  All tensors are bf16 (2 bytes, upper half of
- *    an IEEE fp32), row-major, densely packed.
+ *    an IEEE fp32) unless stated otherwise, row-major, densely packed.
  *  - The library borrows memory, it owns none on the device: weights, the workspace,
  *    inputs and outputs are allocated and freed by the caller, and weights and workspace
  *    must outlive the handle.  No call allocates device memory.
@@ -69,6 +69,9 @@ typedef struct {
   float   rms_eps;               /* RMSNorm epsilon                                                  */
   int32_t device;                /* CUDA device ordinal                                              */
   int32_t evict_log_capacity;    /* eviction-log entries kept per stream (most recent); may be 0     */
+  int32_t out_dtype;             /* element type of `out`: 0 = bf16, 1 = fp32.  Attention outputs reach
+                                    |y| > 4 on LLaVA-Video-shaped inputs, where bf16 storage alone
+                                    rounds by up to 1.6e-2; fp32 keeps the fp32-accumulated value    */
 } vs_config;
 
 /* DEVICE pointers to bf16 weights, one entry per layer.  The arrays of pointers themselves
@@ -117,8 +120,8 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights,
  * hidden:     DEVICE bf16 [n_active][N][d_model].
  * carrier_override: DEVICE bf16 [n_active][d_model] used as the carrier token instead of
  *             the mean (e.g. projector(mean) computed by the caller), or NULL.
- * out:        DEVICE bf16 [n_active][N+1][Hq*D], last layer's attention output, row N being
- *             the carrier's; may be NULL.
+ * out:        DEVICE [n_active][N+1][Hq*D] of `out_dtype`, last layer's attention output, row N
+ *             being the carrier's; may be NULL.
  * Errors: VS_ERR_STATE if a listed stream has an open text turn (call vs_end_turn first);
  *         VS_ERR_CAPACITY if N > max_tokens_per_frame. */
 int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
@@ -130,7 +133,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
  * itself]; no visual-token K/V exists any more.  Before a stream's first frame the tokens
  * extend the prompt prefix instead (the system instruction comes first, Section 3.3) and
  * stay for the life of the stream.
- * hidden: DEVICE bf16 [n_active][T][d_model];  out: DEVICE bf16 [n_active][T][Hq*D].
+ * hidden: DEVICE bf16 [n_active][T][d_model];  out: DEVICE [n_active][T][Hq*D] of `out_dtype`.
  * All listed streams must be in the same phase (all before or all after their first frame).
  * Errors: VS_ERR_CAPACITY on prefix / tail overflow or T > max_step_tokens. */
 int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active,

@@ -37,7 +37,7 @@ class VsConfig(C.Structure):
         "max_prefix", "max_text", "max_step_tokens", "bank_capacity", "n_streams", "agg_mode",
         "evict_policy", "use_rmsnorm", "residual")] + [
         ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("device", C.c_int32),
-        ("evict_log_capacity", C.c_int32)]
+        ("evict_log_capacity", C.c_int32), ("out_dtype", C.c_int32)]
 
 
 class VsWeights(C.Structure):
@@ -231,6 +231,7 @@ class StreamBatch:
             [g.data_ptr() if g is not None else None for g in norm_weights] if norm_weights is not None else None,
             self._ws_ptr, nbytes)
         self.out_width = cfg.n_q_heads * cfg.head_dim
+        self.out_torch_dtype = torch.float32 if cfg.out_dtype == 1 else torch.bfloat16
 
     def _stream(self) -> int:
         return self.torch.cuda.current_stream(self.device).cuda_stream
@@ -240,7 +241,7 @@ class StreamBatch:
         N = hidden.shape[-2]
         assert hidden.is_contiguous() and hidden.numel() == n * N * self.cfg.d_model
         if out is None and want_out:
-            out = self.torch.empty((n, N + 1, self.out_width), dtype=self.torch.bfloat16, device=self.device)
+            out = self.torch.empty((n, N + 1, self.out_width), dtype=self.out_torch_dtype, device=self.device)
         vs_frame_prefill(self.handle, stream_ids, hidden.data_ptr(), N,
                          carrier_override.data_ptr() if carrier_override is not None else None,
                          out.data_ptr() if out is not None else None, self._stream())
@@ -251,7 +252,7 @@ class StreamBatch:
         T = hidden.shape[-2]
         assert hidden.is_contiguous() and hidden.numel() == n * T * self.cfg.d_model
         if out is None:
-            out = self.torch.empty((n, T, self.out_width), dtype=self.torch.bfloat16, device=self.device)
+            out = self.torch.empty((n, T, self.out_width), dtype=self.out_torch_dtype, device=self.device)
         vs_decode_step(self.handle, stream_ids, hidden.data_ptr(), T, out.data_ptr(), self._stream())
         return out
 
@@ -282,7 +283,7 @@ class StreamBatch:
 def make_config(n_layers, d_model, n_q_heads, n_kv_heads, head_dim, max_tokens_per_frame, max_prefix,
                 max_text, bank_capacity, n_streams=1, max_step_tokens=64, agg_mode=0, evict_policy=0,
                 use_rmsnorm=0, residual=0, rope_theta=1.0e6, rms_eps=1.0e-6, device=0,
-                evict_log_capacity=4096) -> VsConfig:
+                evict_log_capacity=4096, out_dtype=1) -> VsConfig:
     return VsConfig(n_layers, d_model, n_q_heads, n_kv_heads, head_dim, max_tokens_per_frame, max_prefix,
                     max_text, max_step_tokens, bank_capacity, n_streams, agg_mode, evict_policy, use_rmsnorm,
-                    residual, rope_theta, rms_eps, device, evict_log_capacity)
+                    residual, rope_theta, rms_eps, device, evict_log_capacity, out_dtype)

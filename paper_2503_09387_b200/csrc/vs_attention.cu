@@ -255,11 +255,12 @@ __global__ void __launch_bounds__(256) prefill_attn_kernel(AttnArgs a, BatchPara
     if (row >= rps) continue;
     const float inv = (l_run[h] > 0.f) ? 1.f / l_run[h] : 0.f;
     const size_t grow = (size_t)b * rps + row;
-    bf16* dst = a.out + grow * a.Hq * D + (size_t)qhead * D + 2 * (lane & 3);
+    const size_t obase = grow * a.Hq * D + (size_t)qhead * D + 2 * (lane & 3);
 #pragma unroll
     for (int i = 0; i < D / 8; ++i) {
       const float v0 = o[i][2 * h] * inv, v1 = o[i][2 * h + 1] * inv;
-      *reinterpret_cast<__nv_bfloat162*>(dst + i * 8) = __floats2bfloat162_rn(v0, v1);
+      if (a.out_fp32) *reinterpret_cast<float2*>(static_cast<float*>(a.out) + obase + i * 8) = make_float2(v0, v1);
+      else *reinterpret_cast<__nv_bfloat162*>(static_cast<bf16*>(a.out) + obase + i * 8) = __floats2bfloat162_rn(v0, v1);
       if (a.h_out != nullptr) {
         const size_t hoff = grow * a.Hq * D + (size_t)qhead * D + 2 * (lane & 3) + i * 8;
         const float2 hv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(a.h_in + hoff));
@@ -434,7 +435,8 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(DecodeArgs a, BatchPar
     }
     const float val = (L > 0.f) ? O / L : 0.f;
     const size_t off = (size_t)b * a.Hq * D + (size_t)qh * D + c;
-    a.out[off] = __float2bfloat16_rn(val);
+    if (a.out_fp32) static_cast<float*>(a.out)[off] = val;
+    else static_cast<bf16*>(a.out)[off] = __float2bfloat16_rn(val);
     if (a.h_out != nullptr) a.h_out[off] = __float2bfloat16_rn(__bfloat162float(a.h_in[off]) + val);
   }
   if (threadIdx.x == 0) a.tickets[sid * a.Hkv + hkv] = 0;

@@ -47,7 +47,7 @@ struct Dims {
   int capP, capT;                                // caller's prefix / tail capacities
   int rows_per_stream_max, R_max;
   int log_cap;
-  int agg_mode, evict_policy, use_rmsnorm, residual;
+  int agg_mode, evict_policy, use_rmsnorm, residual, out_fp32;
   float rope_theta, rms_eps;
 };
 
@@ -80,7 +80,7 @@ struct Layout {
   size_t q;                     // bf16 [R_max][Hq*D]
   size_t kf, vf;                // bf16 [R_max][Hkv*D]
   size_t rope;                  // float2 [R_max][D/2]
-  size_t obuf;                  // bf16 [R_max][Hq*D]
+  size_t obuf;                  // f32  [R_max][Hq*D] (holds bf16 or fp32 rows)
   size_t dec_part;              // f32  [DEC_SPLIT_MAX][S][Hq][D+2]
   size_t scratch_begin, scratch_end;
   size_t total;
@@ -148,7 +148,8 @@ struct AttnArgs {
   const bf16* q;                 // [rows][Hq*D]
   AttnSegment seg[4];
   int n_seg;
-  bf16* out;                     // [rows][Hq*D]
+  void* out;                     // [rows][Hq*D], bf16 or fp32
+  int out_fp32;
   const bf16* h_in;              // residual input [rows][d] or null
   bf16* h_out;                   // residual output or null
   const StreamMeta* meta;
@@ -165,7 +166,8 @@ struct DecodeArgs {
   const bf16* tail_k;   const bf16* tail_v;    // [S][Hkv][maxT][D]
   float* partials;               // [nsplit][n_active][Hq][D+2]
   int* tickets;                  // [S*Hkv]
-  bf16* out;                     // [n_active][Hq*D]
+  void* out;                     // [n_active][Hq*D], bf16 or fp32
+  int out_fp32;
   const bf16* h_in; bf16* h_out;
   const StreamMeta* meta;
   int Hq, Hkv, D, slots, M, maxP, maxT, nsplit;

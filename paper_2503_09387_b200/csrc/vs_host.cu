@@ -34,6 +34,7 @@ int fill_dims(const vs_config* c, Dims& D) {
   if (c->n_streams < 1 || c->n_streams > VS_MAX_BATCH) return VS_ERR_INVALID_ARG;
   if (c->max_tokens_per_frame < 1 || c->max_prefix < 0 || c->max_text < 0 || c->bank_capacity < 0) return VS_ERR_INVALID_ARG;
   if (c->max_step_tokens < 1 || c->evict_log_capacity < 0) return VS_ERR_INVALID_ARG;
+  if (c->out_dtype < 0 || c->out_dtype > 1) return VS_ERR_INVALID_ARG;
   if (c->agg_mode < 0 || c->agg_mode > 1 || c->evict_policy < 0 || c->evict_policy > 2) return VS_ERR_INVALID_ARG;
   if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f)) return VS_ERR_INVALID_ARG;
   if (c->d_model % 64 != 0) return VS_ERR_UNSUPPORTED;
@@ -52,7 +53,7 @@ int fill_dims(const vs_config* c, Dims& D) {
   D.R_max = D.rows_per_stream_max * D.S;
   D.log_cap = c->evict_log_capacity;
   D.agg_mode = c->agg_mode; D.evict_policy = c->evict_policy; D.use_rmsnorm = c->use_rmsnorm ? 1 : 0;
-  D.residual = c->residual ? 1 : 0; D.rope_theta = c->rope_theta; D.rms_eps = c->rms_eps;
+  D.residual = c->residual ? 1 : 0; D.out_fp32 = c->out_dtype == 1 ? 1 : 0; D.rope_theta = c->rope_theta; D.rms_eps = c->rms_eps;
   return VS_OK;
 }
 
@@ -85,7 +86,7 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.kf = take((size_t)D.R_max * D.Hkv * D.D * 2);
   Lo.vf = take((size_t)D.R_max * D.Hkv * D.D * 2);
   Lo.rope = take((size_t)D.R_max * (D.D / 2) * 8);
-  Lo.obuf = take((size_t)D.R_max * D.Hq * D.D * 2);
+  Lo.obuf = take((size_t)D.R_max * D.Hq * D.D * 4);
   Lo.dec_part = take((size_t)DEC_SPLIT_MAX * D.S * D.Hq * (D.D + 2) * 4);
   Lo.scratch_end = off;
   Lo.total = off;
@@ -297,7 +298,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
   pa.N = N; pa.d = D.d; pa.D = D.D; pa.slots = D.slots; pa.M = D.M; pa.agg_mode = D.agg_mode;
   VS_CK(launch_pool(pa, bp, st));
 
-  bf16* out_final = out ? static_cast<bf16*>(out) : h->at<bf16>(lo.obuf);
+  void* out_final = out ? out : h->at<void>(lo.obuf);
   int cur = 0;
   for (int l = 0; l < D.L; ++l) {
     const bf16* h_in = h->at<bf16>(lo.hbuf[cur]);
@@ -333,7 +334,8 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     aa.seg[2] = {fa.kf, fa.vf, (long long)(N + 1) * D.Hkv * D.D, (long long)D.D, (long long)D.Hkv * D.D, 3, 1};
     aa.n_seg = 3;
     const bool last = (l == D.L - 1);
-    aa.out = last ? out_final : h->at<bf16>(lo.obuf);
+    aa.out = last ? out_final : h->at<void>(lo.obuf);
+    aa.out_fp32 = D.out_fp32;
     aa.h_in = D.residual ? h_in : nullptr;
     aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
     aa.meta = meta;
@@ -446,7 +448,8 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       da.prefix_k = pk; da.prefix_v = pv; da.bank_k = bk; da.bank_v = bv; da.tail_k = tk; da.tail_v = tv;
       da.partials = h->at<float>(lo.dec_part);
       da.tickets = h->at<int>(lo.tickets);
-      da.out = static_cast<bf16*>(out);
+      da.out = (l == D.L - 1) ? out : h->at<void>(lo.obuf);
+      da.out_fp32 = D.out_fp32;
       da.h_in = D.residual ? h_in : nullptr; da.h_out = h_out;
       da.meta = meta;
       da.Hq = D.Hq; da.Hkv = D.Hkv; da.D = D.D; da.slots = D.slots; da.M = D.M; da.maxP = D.maxP; da.maxT = D.maxT;
@@ -469,7 +472,8 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       }
       aa.seg[ns++] = {fa.kf, fa.vf, (long long)T * D.Hkv * D.D, (long long)D.D, (long long)D.Hkv * D.D, 3, 1};
       aa.n_seg = ns;
-      aa.out = static_cast<bf16*>(out);
+      aa.out = (l == D.L - 1) ? out : h->at<void>(lo.obuf);
+      aa.out_fp32 = D.out_fp32;
       aa.h_in = D.residual ? h_in : nullptr;
       aa.h_out = h_out;
       aa.meta = meta;

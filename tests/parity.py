@@ -65,7 +65,7 @@ class Pair:
     def __init__(self, w: synth.Workload, n_streams: Optional[int] = None, max_step_tokens: int = 64,
                  evict_policy: int = 0, agg_mode: int = 0, with_bias: bool = False, with_gain: bool = False,
                  max_tokens_per_frame: Optional[int] = None, max_prefix: Optional[int] = None,
-                 max_text: Optional[int] = None):
+                 max_text: Optional[int] = None, out_dtype: int = 1):
         self.w = w
         S = n_streams or w.n_streams
         self.S = S
@@ -82,7 +82,7 @@ class Pair:
             max_text if max_text is not None else max(w.question_len + w.decode_tokens, 1),
             w.bank_capacity, n_streams=S, max_step_tokens=max_step_tokens, agg_mode=agg_mode,
             evict_policy=evict_policy, use_rmsnorm=w.use_rmsnorm, residual=w.residual,
-            rope_theta=w.rope_theta, rms_eps=w.rms_eps)
+            rope_theta=w.rope_theta, rms_eps=w.rms_eps, out_dtype=out_dtype)
         self.gpu = binding.StreamBatch(self.cfg, [to_dev(b) for b in wbits],
                                        [to_dev(b) for b in bbits] if bbits else None,
                                        [to_dev(b) for b in gbits] if gbits else None)
@@ -146,10 +146,11 @@ class Pair:
         if kv and st["count"] and ora.bank[0].K is not None:
             wk = np.stack([e.K[layer] for e in ora.bank])
             wv = np.stack([e.V[layer] for e in ora.bank])
-            if layer == 0:
+            if layer == 0 and not self.w.use_rmsnorm:
                 assert_within_one_ulp(st["k"], wk, "bank K")
                 assert_within_one_ulp(st["v"], wv, "bank V")
-            else:   # deeper layers inherit bf16 rounding differences of the residual stream
+            else:   # the bf16 normalised input and, deeper down, the bf16 residual stream are
+                    # GPU-internal roundings the oracle does not mirror
                 assert_close(synth.bf16_bits_to_f64(st["k"]), wk, f"bank K layer {layer}")
                 assert_close(synth.bf16_bits_to_f64(st["v"]), wv, f"bank V layer {layer}")
         return st

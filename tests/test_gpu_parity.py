@@ -62,6 +62,25 @@ def test_bias_last_token_aggregation_and_carrier_override():
     p.close()
 
 
+def test_bf16_output_mode_adds_only_storage_rounding():
+    w = synth.workload("tiny", seed=3)
+    a, b = Pair(w, out_dtype=1), Pair(w, out_dtype=0)
+    xs = [w.prefix_hidden()] + [w.frame_hidden(t) for t in range(4)] + [w.decode_hidden(0)]
+    for i, x in enumerate(xs):
+        fn = (lambda p: p.frame([0], [x])) if 1 <= i <= 4 else (lambda p: p.text([0], [x], compare=False))
+        if not (1 <= i <= 4):
+            full = a.text([0], [x])
+            half = to_f64(b.gpu.decode_step([0], to_dev(x[None])))
+            b.ora[0].text_step(synth.bf16_bits_to_f64(x))
+        else:
+            full = a.frame([0], [x])
+            half = to_f64(b.gpu.frame_prefill([0], to_dev(x[None])))
+            b.ora[0].frame_step(synth.bf16_bits_to_f64(x))
+        want = torch.from_numpy(full).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+        assert np.array_equal(half, want)          # bf16 mode == fp32 mode rounded once
+    a.close(); b.close()
+
+
 def test_multi_layer_residual_rmsnorm_small():
     w = synth.workload("deep", n_layers=4, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64,
                        tokens_per_frame=21, n_frames=9, bank_capacity=4, prefix_len=6, question_len=7,
