@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the streaming attention path on B200.
+
+A step = one whole stream of the one-layer Qwen2-7B-shaped workload through the C ABI:
+reset, 64-token prompt prefix, 64 frames x 169 visual tokens (one vs_frame_prefill call per
+frame, bank capacity 64), 32 single-token decode steps.  Inputs are seeded synthetic tensors
+(paper_2503_09387_b200.synth) already resident in HBM; L2 is flushed between steps.  Device
+time is taken with CUDA events around the three phases; `value` = frames / frame-phase time.
+
+Extra legs (same process, same workload):
+  e2e          -- the same step with HOST (pinned) inputs: per-call H2D copy of the hidden
+                  states and D2H copy of the output inside the timed region.
+  roofline     -- the dominant kernel's average launch duration from CUDA events recorded
+                  around every launch (vs_profile_enable) in one extra pass of the step.
+  cpu_baseline -- the CPU oracle, as it stands, on a bounded sample of the same workload.
+`--impl reference` times the oracle alone (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2503_09387_b200 import synth  # noqa: E402
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------ algorithmic work
+def frame_flops(w, n_bank):
+    rows = w.tokens_per_frame + 1
+    proj = 2.0 * rows * w.d_model * w.e_out
+    keys_ctx = w.prefix_len + n_bank
+    attn = 4.0 * w.n_q_heads * w.head_dim * (rows * keys_ctx + rows * (rows + 1) / 2.0)
+    return proj, attn
+
+
+def frame_bytes(w, n_bank, out_bytes_per_el, weights_from_hbm):
+    rows = w.tokens_per_frame + 1
+    b = w.tokens_per_frame * w.d_model * 2                       # hidden in
+    b += rows * w.n_q_heads * w.head_dim * out_bytes_per_el      # attention out
+    b += (w.prefix_len + n_bank) * 2 * w.n_kv_heads * w.head_dim * 2   # prefix + bank K/V
+    b += 2 * w.n_kv_heads * w.head_dim * 2 + w.d_model * 2       # carrier K/V + embedding append
+    if weights_from_hbm:
+        b += w.e_out * w.d_model * 2
+    return float(b)
+
+
+def decode_bytes(w, n_keys, out_bytes_per_el):
+    b = w.e_out * w.d_model * 2                                  # weights
+    b += n_keys * 2 * w.n_kv_heads * w.head_dim * 2              # K/V read
+    b += 2 * w.n_kv_heads * w.head_dim * 2                       # tail append
+    b += w.d_model * 2 + w.n_q_heads * w.head_dim * out_bytes_per_el
+    return float(b)
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+# ------------------------------------------------------------------ the oracle legs
+def oracle_stream(w):
+    from oracle import videoscan_oracle as vo
+    cfg = vo.OracleConfig(w.n_layers, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, w.bank_capacity,
+                          use_rmsnorm=w.use_rmsnorm, residual=w.residual, rope_theta=w.rope_theta, rms_eps=w.rms_eps)
+    return vo.OracleStream(cfg, [synth.bf16_bits_to_f64(w.weight(l)) for l in range(w.n_layers)])
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle_sample(w, n_frames, n_decode):
+    """Times the oracle on prefix + n_frames frames + n_decode tokens; returns (frames/s, tok/s, seconds)."""
+    f64 = synth.bf16_bits_to_f64
+    st = oracle_stream(w)
+    shared = w.frame_shared(0, n_frames) if w.frame_model != "iid" else None
+    frames = [f64(w.frame_hidden(t, shared=shared)) for t in range(n_frames)]
+    prefix = f64(w.prefix_hidden())
+    dec = [f64(w.decode_hidden(i)) for i in range(n_decode)]
+    t0 = time.perf_counter()
+    st.text_step(prefix)
+    t1 = time.perf_counter()
+    for E in frames:
+        st.frame_step(E)
+    t2 = time.perf_counter()
+    for x in dec:
+        st.text_step(x)
+    t3 = time.perf_counter()
+    return n_frames / (t2 - t1), (n_decode / (t3 - t2) if n_decode else 0.0), t3 - t0
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_frames, n_decode = 4, 4
+    for _ in range(args.warmup):
+        time_oracle_sample(w, 1, 1)
+    t_frames = t_total = 0.0
+    fps_list, tps_list = [], []
+    for _ in range(args.steps):
+        fps, tps, secs = time_oracle_sample(w, n_frames, n_decode)
+        fps_list.append(fps); tps_list.append(tps); t_total += secs
+    fps = len(fps_list) / sum(1.0 / f for f in fps_list)
+    tps = len(tps_list) / sum(1.0 / f for f in tps_list)
+    cores = blas_threads()
+    sample = f"per step: {w.prefix_len}-token prefix, first {n_frames} frames, {n_decode} decode tokens of the workload"
+    print(json.dumps({
+        "impl": "reference", "metric": "streamed_frames_per_s", "value": fps, "unit": "frames/s",
+        "decode_tokens_per_s": tps, "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * t_total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w),
+        "cpu_baseline": {"value": fps, "unit": "frames/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": fps, "unit": "frames/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def workload_config(w):
+    return {"workload": f"{w.name}: {w.n_layers} Qwen2-7B-shaped attention layer(s), d={w.d_model}, "
+                        f"{w.n_q_heads}/{w.n_kv_heads} heads x {w.head_dim}, {w.prefix_len}-token prefix, "
+                        f"{w.n_frames} frames x {w.tokens_per_frame} tokens, bank {w.bank_capacity}, "
+                        f"{w.decode_tokens} decode tokens; one vs_frame_prefill call per frame",
+            "l2": "flushed between steps (256 MiB write); inside a step the 33 MB weight matrix stays L2-resident",
+            "out_dtype": "fp32"}
+
+
+# ------------------------------------------------------------------ our arm
+def run_ours(args, w):
+    import ctypes as C
+    import torch
+    import torch.distributed as dist
+    from paper_2503_09387_b200 import binding, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if rank == 0:
+        build.build_library()
+    if world > 1:
+        dist.barrier()
+    lib = binding.load_library()
+
+    def to_dev(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).to(dev)
+
+    # ---- inputs (replicas only: every rank streams its own copy of the workload) ----------
+    weights = [to_dev(w.weight(l)) for l in range(w.n_layers)]
+    shared = w.frame_shared() if w.frame_model != "iid" else None
+    frames_host = np.stack([w.frame_hidden(t, shared=shared) for t in range(w.n_frames)])
+    frames = to_dev(frames_host)                                   # [F, N, d]
+    prefix = to_dev(w.prefix_hidden())
+    dec = to_dev(np.concatenate([w.decode_hidden(i) for i in range(w.decode_tokens)]))   # [n_dec, d]
+    cfg = binding.make_config(w.n_layers, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens_per_frame,
+                              max(w.prefix_len, 1), max(w.question_len + w.decode_tokens, 1), w.bank_capacity,
+                              n_streams=1, max_step_tokens=max(64, w.prefix_len), use_rmsnorm=w.use_rmsnorm,
+                              residual=w.residual, rope_theta=w.rope_theta, rms_eps=w.rms_eps, device=local)
+    sb = binding.StreamBatch(cfg, weights)
+    N, d, HD = w.tokens_per_frame, w.d_model, w.n_q_heads * w.head_dim
+    out_frame = torch.empty((N + 1, HD), dtype=torch.float32, device=dev)
+    out_prefix = torch.empty((max(w.prefix_len, 1), HD), dtype=torch.float32, device=dev)
+    out_dec = torch.empty((1, HD), dtype=torch.float32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    sptr = C.c_void_p(stream.cuda_stream)
+    ids = (C.c_int32 * 1)(0)
+    h = C.c_void_p(sb.handle)
+    frame_ptrs = [C.c_void_p(frames[t].data_ptr()) for t in range(w.n_frames)]
+    dec_ptrs = [C.c_void_p(dec[i:i + 1].data_ptr()) for i in range(w.decode_tokens)]
+    p_prefix, p_out_prefix = C.c_void_p(prefix.data_ptr()), C.c_void_p(out_prefix.data_ptr())
+    p_out_frame, p_out_dec = C.c_void_p(out_frame.data_ptr()), C.c_void_p(out_dec.data_ptr())
+
+    def ck(code):
+        if code != 0:
+            raise RuntimeError("library call failed: %s" % binding.status_string(code))
+
+    def one_step(events=None, on_phase=None):
+        ck(lib.vs_reset_stream(h, ids, 1, sptr))
+        if events: events[0].record(stream)
+        if w.prefix_len:
+            ck(lib.vs_decode_step(h, ids, 1, p_prefix, w.prefix_len, p_out_prefix, sptr))
+        if events: events[1].record(stream)
+        if on_phase: on_phase("prefix")
+        for t in range(w.n_frames):
+            ck(lib.vs_frame_prefill(h, ids, 1, frame_ptrs[t], N, None, p_out_frame, sptr))
+        if events: events[2].record(stream)
+        if on_phase: on_phase("frames")
+        for i in range(w.decode_tokens):
+            ck(lib.vs_decode_step(h, ids, 1, dec_ptrs[i], 1, p_out_dec, sptr))
+        if events: events[3].record(stream)
+        if on_phase: on_phase("decode")
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize(dev)
+
+    for _ in range(max(args.warmup, 3)):
+        flush.zero_()
+        one_step()
+    sb.profile_read()                                   # clear launch counters
+    sampler = ClockSampler(local)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    barrier()
+    sampler.start()
+    wall0 = time.perf_counter()
+    for k in range(args.steps):
+        flush.zero_()
+        one_step(ev[k])
+    barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.stop()
+    counts = sb.profile_read()
+    gpu_launches = sum(v[2] for v in counts.values())
+    ms_prefix = sum(e[0].elapsed_time(e[1]) for e in ev)
+    ms_frames = sum(e[1].elapsed_time(e[2]) for e in ev)
+    ms_decode = sum(e[2].elapsed_time(e[3]) for e in ev)
+    times = torch.tensor([ms_prefix, ms_frames, ms_decode], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_prefix, ms_frames, ms_decode = times.tolist()
+    fps = world * args.steps * w.n_frames / (ms_frames * 1e-3)
+    tps = world * args.steps * w.decode_tokens / (ms_decode * 1e-3) if w.decode_tokens else 0.0
+
+    # ---- per-kernel pass: events around every launch, one extra step ------------------------
+    per_phase = {}
+    launches_per_step = gpu_launches // max(args.steps, 1) + 16
+    sb.profile_enable(True, launches_per_step)
+    flush.zero_()
+    one_step(on_phase=lambda name: per_phase.__setitem__(name, sb.profile_read()))
+    sb.profile_enable(False)
+
+    result = None
+    if rank == 0:
+        peaks = load_peaks()
+        fr = per_phase["frames"]
+        kernels = {k: {"launches": v[1], "total_ms": round(v[0], 4), "avg_us": round(1e3 * v[0] / v[1], 3)}
+                   for k, v in fr.items() if v[1]}
+        tot = sum(v["total_ms"] for v in kernels.values())
+        for v in kernels.values():
+            v["share"] = round(v["total_ms"] / tot, 4)
+        dom = max(kernels, key=lambda k: kernels[k]["total_ms"])
+        proj_flops, _ = frame_flops(w, 0)
+        avg_bank = (min(w.n_frames, w.bank_capacity) - 1) / 2.0 if w.bank_capacity else 0.0
+        _, attn_flops = frame_flops(w, avg_bank)
+        if dom == "qkv_gemm":
+            ach = proj_flops / (kernels[dom]["avg_us"] * 1e-6) / 1e12
+            roof = {"kernel": dom, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
+                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None,
+                    "peak_source": peaks["source"] + " (sustained bf16; kernel timed inside the step)",
+                    "avg_launch_us": kernels[dom]["avg_us"]}
+        else:
+            # every other kernel of the frame step moves bytes: report against HBM
+            rows = N + 1
+            alg = {"prefill_attention": rows * (HD * 2 * 2 + 2 * w.n_kv_heads * w.head_dim * 2) + rows * HD * 4
+                   + (w.prefix_len + avg_bank) * 2 * w.n_kv_heads * w.head_dim * 2,
+                   "finalize": 4 * rows * w.e_out * 4 + rows * w.e_out * 2 + rows * HD * 2,
+                   "pool": 2 * N * d * 2 + d * 4}.get(dom, 0.0)
+            ach = alg / (kernels[dom]["avg_us"] * 1e-6) / 1e9
+            roof = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                    "avg_launch_us": kernels[dom]["avg_us"]}
+        us_frame = 1e3 * ms_frames / (args.steps * w.n_frames)
+        ideal_c = (proj_flops + attn_flops) * w.n_layers / (peaks["bf16_tflops_sustained"] * 1e12) * 1e6
+        ideal_h = frame_bytes(w, avg_bank, 4, weights_from_hbm=w.n_layers > 1) / (peaks["hbm_gbs"] * 1e9) * 1e6
+        ideal = max(ideal_c, ideal_h)
+        n_keys = w.prefix_len + min(w.n_frames, w.bank_capacity) + w.decode_tokens / 2.0
+        us_tok = 1e3 * ms_decode / (args.steps * max(w.decode_tokens, 1))
+        dec_ideal = decode_bytes(w, n_keys, 4) * w.n_layers / (peaks["hbm_gbs"] * 1e9) * 1e6
+        result = {
+            "metric": "streamed_frames_per_s", "value": fps, "unit": "frames/s",
+            "decode_tokens_per_s": tps, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": (ms_prefix + ms_frames + ms_decode) / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_config(w),
+            "phase_ms_per_step": {"prefix": ms_prefix / args.steps, "frames": ms_frames / args.steps,
+                                  "decode": ms_decode / args.steps},
+            "wall_s": wall, "clocks": clocks, "gpu_launches": gpu_launches,
+            "roofline": roof, "kernels_frame_phase": kernels,
+            "step_roofline": {
+                "frame": {"us_per_frame": us_frame, "ideal_us": ideal, "frac": ideal / us_frame,
+                          "ideal_compute_us": ideal_c, "ideal_hbm_us": ideal_h,
+                          "note": "ideal = max(flops / sustained bf16 peak, bytes / HBM peak); single-layer "
+                                  "weights are L2-resident so they are not counted as HBM bytes"},
+                "decode": {"us_per_token": us_tok, "ideal_hbm_us": dec_ideal, "frac": dec_ideal / us_tok,
+                           "note": "bytes = weights + K/V + append; the weights are L2-resident in the "
+                                   "one-layer workload, so this fraction is not a DRAM fraction"}},
+        }
+
+    # ---- end to end: host inputs, H2D + D2H inside the timed region ---------------------------
+    pin_frames = torch.from_numpy(frames_host.view(np.int16)).pin_memory()
+    pin_out = torch.empty((N + 1, HD), dtype=torch.float32).pin_memory()
+    dev_in = torch.empty((N, d), dtype=torch.int16, device=dev)
+    p_dev_in = C.c_void_p(dev_in.data_ptr())
+
+    def e2e_step():
+        ck(lib.vs_reset_stream(h, ids, 1, sptr))
+        if w.prefix_len:
+            ck(lib.vs_decode_step(h, ids, 1, p_prefix, w.prefix_len, p_out_prefix, sptr))
+        for t in range(w.n_frames):
+            dev_in.copy_(pin_frames[t], non_blocking=True)
+            ck(lib.vs_frame_prefill(h, ids, 1, p_dev_in, N, None, p_out_frame, sptr))
+            pin_out.copy_(out_frame, non_blocking=True)
+        stream.synchronize()
+
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    e_steps = max(1, min(args.steps, 3))
+    for _ in range(e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = torch.tensor([time.perf_counter() - t0], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
+    if rank == 0:
+        result["e2e"] = {"value": world * e_steps * w.n_frames / e2e_s.item(), "unit": "frames/s",
+                         "h2d_bytes_per_step": int(w.n_frames * N * d * 2),
+                         "d2h_bytes_per_step": int(w.n_frames * (N + 1) * HD * 4),
+                         "note": "frames phase only; per frame: pinned H2D of the hidden states, "
+                                 "vs_frame_prefill, D2H of the fp32 output; wall clock incl. launch cost"}
+        if not args.no_cpu_baseline and world == 1:
+            n_frames, n_decode = 16, 8
+            fps_cpu, tps_cpu, secs = time_oracle_sample(w, n_frames, n_decode)
+            result["cpu_baseline"] = {"value": fps_cpu, "unit": "frames/s", "decode_tokens_per_s": tps_cpu,
+                                      "cores": blas_threads(), "kind": "oracle", "seconds": secs,
+                                      "sample": f"{w.prefix_len}-token prefix, first {n_frames} frames and "
+                                                f"{n_decode} decode tokens of the same workload"}
+        print(json.dumps(result))
+    sb.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="layer")
+    ap.add_argument("--frames", type=int, default=None, help="override the number of frames (exploration only)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    kw = {}
+    if args.frames:
+        kw["n_frames"] = args.frames
+    w = synth.workload(args.workload, **kw)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

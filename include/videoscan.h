@@ -39,6 +39,7 @@ extern "C" {
 #define VS_ERR_UNSUPPORTED     -6   /* shape outside what the kernels are built for         */
 
 #define VS_MAX_BATCH           64   /* most streams one call may list                       */
+#define VS_N_KERNEL_CLASSES    10   /* kernel classes reported by vs_profile_read           */
 
 typedef struct vs_stream vs_stream;   /* opaque handle: a batch of n_streams independent video streams */
 
@@ -143,6 +144,10 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
  * positions do not move.  Host-only bookkeeping. */
 int vs_end_turn(vs_stream* h, const int32_t* stream_ids, int32_t n_active);
 
+/* Starts the listed streams over (a new video): empty bank, no prefix, positions from 0.
+ * Asynchronous on cuda_stream; the memory mechanism of Section 3.3 simply begins again. */
+int vs_reset_stream(vs_stream* h, const int32_t* stream_ids, int32_t n_active, void* cuda_stream);
+
 /* Synchronises the handle's CUDA stream and reports one stream's bank (Section 3.3,
  * memory mechanism) in temporal order (oldest carrier first).  All outputs are HOST and
  * optional (NULL skips them):
@@ -165,6 +170,17 @@ int vs_bank_state(vs_stream* h, int32_t stream_id, vs_bank_info* info,
  * must not change, which shows that no visual-token state survives a step. */
 int vs_last_step_kv(vs_stream* h, void* k_out, void* v_out, int32_t rows);
 int vs_poison_scratch(vs_stream* h, void* cuda_stream);
+
+/* Launch accounting (no counterpart in the paper; measurement aid).  Every kernel launch is
+ * counted per class.  With profiling enabled each launch is also bracketed by a pair of CUDA
+ * events on the launching stream, at most `max_launches` pairs between two reads (host-side
+ * event objects are created on enable; no device memory).  vs_profile_read synchronises and
+ * returns, per class and since the previous read: summed device milliseconds of the timed
+ * launches (HOST double[VS_N_KERNEL_CLASSES]), how many were timed, and how many were
+ * launched (HOST int64[VS_N_KERNEL_CLASSES] each); any pointer may be NULL. */
+int vs_profile_enable(vs_stream* h, int32_t on, int32_t max_launches);
+int vs_profile_read(vs_stream* h, double* ms, int64_t* timed, int64_t* launches);
+const char* vs_kernel_class_name(int32_t k);
 
 int vs_destroy_stream(vs_stream* h);
 

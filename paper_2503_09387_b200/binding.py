@@ -28,7 +28,9 @@ VS_MAX_BATCH = 64
 
 EXPORTS = ["vs_workspace_bytes", "vs_create_stream", "vs_frame_prefill", "vs_decode_step",
            "vs_end_turn", "vs_bank_state", "vs_last_step_kv", "vs_poison_scratch",
-           "vs_destroy_stream", "vs_status_string"]
+           "vs_destroy_stream", "vs_status_string", "vs_reset_stream", "vs_profile_enable",
+           "vs_profile_read", "vs_kernel_class_name"]
+VS_N_KERNEL_CLASSES = 10
 
 
 class VsConfig(C.Structure):
@@ -86,8 +88,13 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.vs_destroy_stream.argtypes = [vp]
     lib.vs_status_string.argtypes = [C.c_int]
     lib.vs_status_string.restype = C.c_char_p
+    lib.vs_reset_stream.argtypes = [vp, i32p, i32, vp]
+    lib.vs_profile_enable.argtypes = [vp, i32, i32]
+    lib.vs_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+    lib.vs_kernel_class_name.argtypes = [i32]
+    lib.vs_kernel_class_name.restype = C.c_char_p
     for name in EXPORTS:
-        if name != "vs_status_string":
+        if name not in ("vs_status_string", "vs_kernel_class_name"):
             getattr(lib, name).restype = C.c_int
     if path is None:
         _lib = lib
@@ -147,6 +154,26 @@ def vs_decode_step(handle: int, stream_ids: Sequence[int], hidden_ptr: int, T: i
 def vs_end_turn(handle: int, stream_ids: Sequence[int]) -> None:
     ids, n = _ids(stream_ids)
     _check(load_library().vs_end_turn(handle, ids, n), "vs_end_turn")
+
+
+def vs_reset_stream(handle: int, stream_ids: Sequence[int], cuda_stream: int = 0) -> None:
+    ids, n = _ids(stream_ids)
+    _check(load_library().vs_reset_stream(handle, ids, n, cuda_stream or None), "vs_reset_stream")
+
+
+def vs_profile_enable(handle: int, on: bool, max_launches: int = 0) -> None:
+    _check(load_library().vs_profile_enable(handle, 1 if on else 0, max_launches), "vs_profile_enable")
+
+
+def vs_profile_read(handle: int) -> dict:
+    """{class name: (summed ms of timed launches, timed launches, all launches)} since the last read."""
+    lib = load_library()
+    ms = (C.c_double * VS_N_KERNEL_CLASSES)()
+    timed = (C.c_int64 * VS_N_KERNEL_CLASSES)()
+    launches = (C.c_int64 * VS_N_KERNEL_CLASSES)()
+    _check(lib.vs_profile_read(handle, ms, timed, launches), "vs_profile_read")
+    return {lib.vs_kernel_class_name(k).decode(): (ms[k], int(timed[k]), int(launches[k]))
+            for k in range(VS_N_KERNEL_CLASSES)}
 
 
 def vs_destroy_stream(handle: int) -> None:
@@ -264,6 +291,15 @@ class StreamBatch:
 
     def last_step_kv(self, rows):
         return vs_last_step_kv(self.handle, rows, self.cfg.n_kv_heads, self.cfg.head_dim)
+
+    def reset(self, stream_ids):
+        vs_reset_stream(self.handle, stream_ids, self._stream())
+
+    def profile_enable(self, on, max_launches=0):
+        vs_profile_enable(self.handle, on, max_launches)
+
+    def profile_read(self):
+        return vs_profile_read(self.handle)
 
     def poison_scratch(self):
         vs_poison_scratch(self.handle, self._stream())

@@ -126,17 +126,22 @@ __global__ void __launch_bounds__(256) prefill_attn_kernel(AttnArgs a, BatchPara
   };
 
   // Q fragments (A operand): rows r0 + lane/4 and + 8, all D/16 k-steps
-  uint32_t qf[D / 16][4];
+  // (hi and lo halves: Q = qf + ql carries 16 mantissa bits into the scores)
+  uint32_t qf[D / 16][4], ql[D / 16][4];
   {
     const int ra = r0 + (lane >> 2), rb = ra + 8;
-    const bf16* qa = a.q + ((size_t)b * rps + ra) * a.Hq * D + (size_t)qhead * D + 2 * (lane & 3);
-    const bf16* qb = a.q + ((size_t)b * rps + rb) * a.Hq * D + (size_t)qhead * D + 2 * (lane & 3);
+    const size_t oa = ((size_t)b * rps + ra) * a.Hq * D + (size_t)qhead * D + 2 * (lane & 3);
+    const size_t ob = ((size_t)b * rps + rb) * a.Hq * D + (size_t)qhead * D + 2 * (lane & 3);
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
-      qf[ks][0] = (ra < rps) ? *reinterpret_cast<const uint32_t*>(qa + ks * 16) : 0u;
-      qf[ks][1] = (rb < rps) ? *reinterpret_cast<const uint32_t*>(qb + ks * 16) : 0u;
-      qf[ks][2] = (ra < rps) ? *reinterpret_cast<const uint32_t*>(qa + ks * 16 + 8) : 0u;
-      qf[ks][3] = (rb < rps) ? *reinterpret_cast<const uint32_t*>(qb + ks * 16 + 8) : 0u;
+      qf[ks][0] = (ra < rps) ? *reinterpret_cast<const uint32_t*>(a.q + oa + ks * 16) : 0u;
+      qf[ks][1] = (rb < rps) ? *reinterpret_cast<const uint32_t*>(a.q + ob + ks * 16) : 0u;
+      qf[ks][2] = (ra < rps) ? *reinterpret_cast<const uint32_t*>(a.q + oa + ks * 16 + 8) : 0u;
+      qf[ks][3] = (rb < rps) ? *reinterpret_cast<const uint32_t*>(a.q + ob + ks * 16 + 8) : 0u;
+      ql[ks][0] = (ra < rps) ? *reinterpret_cast<const uint32_t*>(a.q_lo + oa + ks * 16) : 0u;
+      ql[ks][1] = (rb < rps) ? *reinterpret_cast<const uint32_t*>(a.q_lo + ob + ks * 16) : 0u;
+      ql[ks][2] = (ra < rps) ? *reinterpret_cast<const uint32_t*>(a.q_lo + oa + ks * 16 + 8) : 0u;
+      ql[ks][3] = (rb < rps) ? *reinterpret_cast<const uint32_t*>(a.q_lo + ob + ks * 16 + 8) : 0u;
     }
   }
 
@@ -178,6 +183,8 @@ __global__ void __launch_bounds__(256) prefill_attn_kernel(AttnArgs a, BatchPara
         ldmatrix_x4(kbase + tile_off<D>(key, chunk), b0, b1, b2, b3);
         mma_bf16(sc[2 * jp], qf[ks], b0, b1);
         mma_bf16(sc[2 * jp + 1], qf[ks], b2, b3);
+        mma_bf16(sc[2 * jp], ql[ks], b0, b1);
+        mma_bf16(sc[2 * jp + 1], ql[ks], b2, b3);
       }
     }
     // mask, scale (log2 domain), running max
@@ -311,12 +318,16 @@ __global__ void __launch_bounds__(128) decode_attn_kernel(DecodeArgs a, BatchPar
 #pragma unroll
   for (int g = 0; g < GMAX; ++g) {
     if (g < G) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(a.q + (size_t)b * a.Hq * D + (size_t)(hkv * G + g) * D + li * 8);
+      const size_t qo = (size_t)b * a.Hq * D + (size_t)(hkv * G + g) * D + li * 8;
+      const uint4 raw = *reinterpret_cast<const uint4*>(a.q + qo);
+      const uint4 raw_lo = *reinterpret_cast<const uint4*>(a.q_lo + qo);
       const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+      const __nv_bfloat162* l2 = reinterpret_cast<const __nv_bfloat162*>(&raw_lo);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const float2 f = __bfloat1622float2(h2[i]);
-        q[g][2 * i] = f.x * a.scale_log2e; q[g][2 * i + 1] = f.y * a.scale_log2e;
+        const float2 fl = __bfloat1622float2(l2[i]);
+        q[g][2 * i] = (f.x + fl.x) * a.scale_log2e; q[g][2 * i + 1] = (f.y + fl.y) * a.scale_log2e;
       }
     } else {
 #pragma unroll

@@ -78,6 +78,7 @@ struct Layout {
   size_t xn;                    // bf16 [R_max][d]  normalised layer input
   size_t partials;              // f32  [KSPLIT_MAX][R_max][E_out]
   size_t q;                     // bf16 [R_max][Hq*D]
+  size_t q_lo;                  // bf16 [R_max][Hq*D]  low-order half of the rotated query
   size_t kf, vf;                // bf16 [R_max][Hkv*D]
   size_t rope;                  // float2 [R_max][D/2]
   size_t obuf;                  // f32  [R_max][Hq*D] (holds bf16 or fp32 rows)
@@ -124,7 +125,8 @@ struct FinalizeArgs {
   const float* partials;         // [ksplit][rows][E_out]
   const bf16* bias;              // [E_out] or null
   const float2* rope;            // [rows][D/2]
-  bf16* q;                       // [rows][Hq*D]
+  bf16* q;                       // [rows][Hq*D]  rotated query, leading bf16 part
+  bf16* q_lo;                    // [rows][Hq*D]  bf16(query - q): the pair carries 16 mantissa bits
   bf16* kf;                      // [rows][Hkv*D]
   bf16* vf;
   bf16* bank_k; bf16* bank_v;    // layer base [S][Hkv][slots][D]
@@ -146,6 +148,7 @@ struct AttnSegment {
 };
 struct AttnArgs {
   const bf16* q;                 // [rows][Hq*D]
+  const bf16* q_lo;
   AttnSegment seg[4];
   int n_seg;
   void* out;                     // [rows][Hq*D], bf16 or fp32
@@ -161,6 +164,7 @@ cudaError_t prefill_attention_init();
 
 struct DecodeArgs {
   const bf16* q;                 // [n_active][Hq*D]
+  const bf16* q_lo;
   const bf16* prefix_k; const bf16* prefix_v;  // layer base [S][Hkv][maxP][D]
   const bf16* bank_k;   const bf16* bank_v;    // [S][Hkv][slots][D]
   const bf16* tail_k;   const bf16* tail_v;    // [S][Hkv][maxT][D]
@@ -192,5 +196,6 @@ struct CommitArgs {
 cudaError_t launch_commit(const CommitArgs& a, const BatchParams& bp, cudaStream_t st);
 
 cudaError_t launch_poison(void* p, size_t bytes, cudaStream_t st);
+cudaError_t launch_reset(StreamMeta* meta, int32_t* slot_frame, int slots, const BatchParams& bp, cudaStream_t st);
 
 }  // namespace vs

@@ -83,6 +83,7 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.xn = take((size_t)D.R_max * D.d * 2);
   Lo.partials = take((size_t)KSPLIT_MAX * D.R_max * D.E_out * 4);
   Lo.q = take((size_t)D.R_max * D.Hq * D.D * 2);
+  Lo.q_lo = take((size_t)D.R_max * D.Hq * D.D * 2);
   Lo.kf = take((size_t)D.R_max * D.Hkv * D.D * 2);
   Lo.vf = take((size_t)D.R_max * D.Hkv * D.D * 2);
   Lo.rope = take((size_t)D.R_max * (D.D / 2) * 8);
@@ -106,6 +107,12 @@ struct vs_stream {
   EncodeTiledFn encode = nullptr;
   cudaStream_t last_stream = nullptr;
   int last_rows = 0;
+  // launch accounting: counts always, CUDA-event timing of every launch when enabled
+  int64_t launches[VS_N_KERNEL_CLASSES] = {0};
+  bool prof_on = false;
+  std::vector<cudaEvent_t> prof_ev;          // pairs (start, stop)
+  std::vector<int> prof_class;               // class of pair i
+  size_t prof_used = 0;                      // pairs in use
 
   template <typename T>
   T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
@@ -149,6 +156,23 @@ int check_ids(vs_stream* h, const int32_t* ids, int32_t n) {
 
 #define VS_CK(expr) do { if ((expr) != cudaSuccess) return VS_ERR_CUDA; } while (0)
 
+enum KernelClass { KC_POOL = 0, KC_ROPE, KC_RMSNORM, KC_GEMM, KC_FINALIZE, KC_PREFILL_ATTN, KC_DECODE_ATTN,
+                   KC_EVICT, KC_COMMIT, KC_OTHER };
+static_assert(KC_OTHER + 1 == VS_N_KERNEL_CLASSES, "kernel class table");
+
+// One launch: counted, and bracketed by CUDA events on the launching stream when profiling is on.
+#define VS_LAUNCH(h, st, kc, expr)                                                          \
+  do {                                                                                      \
+    const bool vs_t_ = (h)->prof_on && (h)->prof_used * 2 + 1 < (h)->prof_ev.size();        \
+    if (vs_t_) VS_CK(cudaEventRecord((h)->prof_ev[(h)->prof_used * 2], (st)));              \
+    VS_CK(expr);                                                                            \
+    if (vs_t_) {                                                                            \
+      VS_CK(cudaEventRecord((h)->prof_ev[(h)->prof_used * 2 + 1], (st)));                   \
+      (h)->prof_class[(h)->prof_used++] = (kc);                                             \
+    }                                                                                       \
+    (h)->launches[(kc)] += 1;                                                               \
+  } while (0)
+
 // QKV projection of `rows` token rows read from `src` ([rows][d] bf16) for layer l.
 int run_projection(vs_stream* h, int l, const bf16* src, int rows, int& ksplit_out, cudaStream_t st) {
   const Dims& D = h->dm;
@@ -160,7 +184,7 @@ int run_projection(vs_stream* h, int l, const bf16* src, int rows, int& ksplit_o
   g.rows = rows; g.E_out = D.E_out; g.d = D.d;
   g.status = h->at<int>(h->lo.status);
   ksplit_out = g.ksplit;
-  VS_CK(launch_qkv_gemm(g, st));
+  VS_LAUNCH(h, st, KC_GEMM, launch_qkv_gemm(g, st));
   return VS_OK;
 }
 
@@ -252,6 +276,7 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights, void* work
 
 int vs_destroy_stream(vs_stream* h) {
   if (h == nullptr) return VS_ERR_INVALID_ARG;
+  for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);
   delete h;
   return VS_OK;
 }
@@ -296,7 +321,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
   pa.inv_freq = h->at<double>(lo.inv_freq);
   pa.rope = h->at<float2>(lo.rope);
   pa.N = N; pa.d = D.d; pa.D = D.D; pa.slots = D.slots; pa.M = D.M; pa.agg_mode = D.agg_mode;
-  VS_CK(launch_pool(pa, bp, st));
+  VS_LAUNCH(h, st, KC_POOL, launch_pool(pa, bp, st));
 
   void* out_final = out ? out : h->at<void>(lo.obuf);
   int cur = 0;
@@ -304,7 +329,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     const bf16* h_in = h->at<bf16>(lo.hbuf[cur]);
     const bf16* src = h_in;
     if (D.use_rmsnorm) {
-      VS_CK(launch_rmsnorm(h_in, h->gain[l], h->at<bf16>(lo.xn), rows, D.d, D.rms_eps, st));
+      VS_LAUNCH(h, st, KC_RMSNORM, launch_rmsnorm(h_in, h->gain[l], h->at<bf16>(lo.xn), rows, D.d, D.rms_eps, st));
       src = h->at<bf16>(lo.xn);
     }
     int ksplit = 1;
@@ -315,18 +340,18 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     fa.partials = h->at<float>(lo.partials);
     fa.bias = h->bias[l];
     fa.rope = h->at<float2>(lo.rope);
-    fa.q = h->at<bf16>(lo.q); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
+    fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
     fa.bank_k = h->at<bf16>(lo.bank_k) + (size_t)l * layer_stride_bank(D);
     fa.bank_v = h->at<bf16>(lo.bank_v) + (size_t)l * layer_stride_bank(D);
     fa.text_k = nullptr; fa.text_v = nullptr;
     fa.meta = meta;
     fa.rows = rows; fa.ksplit = ksplit; fa.E_out = D.E_out; fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D;
     fa.slots = D.slots; fa.text_cap = 0; fa.mode = 0; fa.M = D.M;
-    VS_CK(launch_finalize(fa, bp, st));
+    VS_LAUNCH(h, st, KC_FINALIZE, launch_finalize(fa, bp, st));
 
     AttnArgs aa;
     std::memset(&aa, 0, sizeof(aa));
-    aa.q = fa.q;
+    aa.q = fa.q; aa.q_lo = fa.q_lo;
     aa.seg[0] = {h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D),
                  h->at<bf16>(lo.prefix_v) + (size_t)l * layer_stride_prefix(D),
                  (long long)D.Hkv * D.maxP * D.D, (long long)D.maxP * D.D, (long long)D.D, 0, 0};
@@ -341,7 +366,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     aa.meta = meta;
     aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
     aa.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
-    VS_CK(launch_prefill_attention(aa, bp, st));
+    VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention(aa, bp, st));
     if (D.residual) cur ^= 1;
   }
 
@@ -350,13 +375,13 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     ea.emb = h->at<bf16>(lo.emb); ea.meta = meta;
     ea.order = h->at<int32_t>(lo.order); ea.scores = h->at<double>(lo.scores);
     ea.d = D.d; ea.slots = D.slots; ea.M = D.M; ea.policy = D.evict_policy;
-    VS_CK(launch_evict_score(ea, bp, st));
+    VS_LAUNCH(h, st, KC_EVICT, launch_evict_score(ea, bp, st));
   }
   CommitArgs ca;
   ca.meta = meta; ca.order = h->at<int32_t>(lo.order); ca.slot_frame = h->at<int32_t>(lo.slot_frame);
   ca.slot_pos = h->at<int64_t>(lo.slot_pos); ca.evict_log = h->at<int32_t>(lo.evict_log);
   ca.slots = D.slots; ca.M = D.M; ca.log_cap = D.log_cap;
-  VS_CK(launch_commit(ca, bp, st));
+  VS_LAUNCH(h, st, KC_COMMIT, launch_commit(ca, bp, st));
 
   for (int i = 0; i < n_active; ++i) {
     HostStream& s = h->hs[stream_ids[i]];
@@ -407,14 +432,14 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
 
   RopeArgs ra;
   ra.inv_freq = h->at<double>(lo.inv_freq); ra.rope = h->at<float2>(lo.rope); ra.D = D.D;
-  VS_CK(launch_rope_table(ra, bp, st));
+  VS_LAUNCH(h, st, KC_ROPE, launch_rope_table(ra, bp, st));
 
   const bf16* h_in = static_cast<const bf16*>(hidden);
   int next_buf = 0;
   for (int l = 0; l < D.L; ++l) {
     const bf16* src = h_in;
     if (D.use_rmsnorm) {
-      VS_CK(launch_rmsnorm(h_in, h->gain[l], h->at<bf16>(lo.xn), rows, D.d, D.rms_eps, st));
+      VS_LAUNCH(h, st, KC_RMSNORM, launch_rmsnorm(h_in, h->gain[l], h->at<bf16>(lo.xn), rows, D.d, D.rms_eps, st));
       src = h->at<bf16>(lo.xn);
     }
     int ksplit = 1;
@@ -432,19 +457,19 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
     fa.partials = h->at<float>(lo.partials);
     fa.bias = h->bias[l];
     fa.rope = h->at<float2>(lo.rope);
-    fa.q = h->at<bf16>(lo.q); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
+    fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
     fa.bank_k = bk; fa.bank_v = bv;
     fa.text_k = to_prefix ? pk : tk; fa.text_v = to_prefix ? pv : tv;
     fa.meta = meta;
     fa.rows = rows; fa.ksplit = ksplit; fa.E_out = D.E_out; fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D;
     fa.slots = D.slots; fa.text_cap = to_prefix ? D.maxP : D.maxT; fa.mode = to_prefix ? 1 : 2; fa.M = D.M;
-    VS_CK(launch_finalize(fa, bp, st));
+    VS_LAUNCH(h, st, KC_FINALIZE, launch_finalize(fa, bp, st));
 
     bf16* h_out = D.residual ? h->at<bf16>(lo.hbuf[next_buf]) : nullptr;
     const float scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
     if (T == 1) {
       DecodeArgs da;
-      da.q = fa.q;
+      da.q = fa.q; da.q_lo = fa.q_lo;
       da.prefix_k = pk; da.prefix_v = pv; da.bank_k = bk; da.bank_v = bv; da.tail_k = tk; da.tail_v = tv;
       da.partials = h->at<float>(lo.dec_part);
       da.tickets = h->at<int>(lo.tickets);
@@ -459,11 +484,11 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       da.nsplit = ns;
       da.to_prefix = to_prefix ? 1 : 0;
       da.scale_log2e = scale_log2e;
-      VS_CK(launch_decode_attention(da, bp, st));
+      VS_LAUNCH(h, st, KC_DECODE_ATTN, launch_decode_attention(da, bp, st));
     } else {
       AttnArgs aa;
       std::memset(&aa, 0, sizeof(aa));
-      aa.q = fa.q;
+      aa.q = fa.q; aa.q_lo = fa.q_lo;
       int ns = 0;
       aa.seg[ns++] = {pk, pv, (long long)D.Hkv * D.maxP * D.D, (long long)D.maxP * D.D, (long long)D.D, 0, 0};
       if (!to_prefix) {
@@ -479,7 +504,7 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       aa.meta = meta;
       aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
       aa.scale_log2e = scale_log2e;
-      VS_CK(launch_prefill_attention(aa, bp, st));
+      VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention(aa, bp, st));
     }
     if (D.residual) { h_in = h_out; next_buf ^= 1; }
   }
@@ -492,6 +517,65 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
   h->last_stream = st;
   h->last_rows = rows;
   return VS_OK;
+}
+
+int vs_reset_stream(vs_stream* h, const int32_t* stream_ids, int32_t n_active, void* cuda_stream) {
+  const int rc = check_ids(h, stream_ids, n_active);
+  if (rc != VS_OK) return rc;
+  const Dims& D = h->dm;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  VS_CK(cudaSetDevice(h->device));
+  BatchParams bp;
+  std::memset(&bp, 0, sizeof(bp));
+  bp.n_active = n_active;
+  for (int i = 0; i < n_active; ++i) bp.stream_id[i] = stream_ids[i];
+  VS_LAUNCH(h, st, KC_OTHER, launch_reset(h->at<StreamMeta>(h->lo.meta), h->at<int32_t>(h->lo.slot_frame), D.slots, bp, st));
+  for (int i = 0; i < n_active; ++i) h->hs[stream_ids[i]] = HostStream();
+  h->last_stream = st;
+  return VS_OK;
+}
+
+int vs_profile_enable(vs_stream* h, int32_t on, int32_t max_launches) {
+  if (h == nullptr || max_launches < 0) return VS_ERR_INVALID_ARG;
+  VS_CK(cudaSetDevice(h->device));
+  if (on) {
+    while (h->prof_ev.size() < (size_t)max_launches * 2) {
+      cudaEvent_t e;
+      VS_CK(cudaEventCreate(&e));
+      h->prof_ev.push_back(e);
+    }
+    h->prof_class.resize(h->prof_ev.size() / 2);
+  }
+  h->prof_on = on != 0;
+  h->prof_used = 0;
+  return VS_OK;
+}
+
+int vs_profile_read(vs_stream* h, double* ms, int64_t* timed, int64_t* launches) {
+  if (h == nullptr) return VS_ERR_INVALID_ARG;
+  VS_CK(cudaSetDevice(h->device));
+  VS_CK(cudaStreamSynchronize(h->last_stream));
+  for (int k = 0; k < VS_N_KERNEL_CLASSES; ++k) {
+    if (ms) ms[k] = 0.0;
+    if (timed) timed[k] = 0;
+    if (launches) { launches[k] = h->launches[k]; }
+    h->launches[k] = 0;
+  }
+  for (size_t i = 0; i < h->prof_used; ++i) {
+    float t = 0.f;
+    VS_CK(cudaEventElapsedTime(&t, h->prof_ev[2 * i], h->prof_ev[2 * i + 1]));
+    if (ms) ms[h->prof_class[i]] += (double)t;
+    if (timed) timed[h->prof_class[i]] += 1;
+  }
+  h->prof_used = 0;
+  return VS_OK;
+}
+
+const char* vs_kernel_class_name(int32_t k) {
+  static const char* names[VS_N_KERNEL_CLASSES] = {"pool", "rope_table", "rmsnorm", "qkv_gemm", "finalize",
+                                                   "prefill_attention", "decode_attention", "evict_score",
+                                                   "bank_commit", "other"};
+  return (k >= 0 && k < VS_N_KERNEL_CLASSES) ? names[k] : "?";
 }
 
 int vs_end_turn(vs_stream* h, const int32_t* stream_ids, int32_t n_active) {
@@ -579,8 +663,9 @@ int vs_last_step_kv(vs_stream* h, void* k_out, void* v_out, int32_t rows) {
 int vs_poison_scratch(vs_stream* h, void* cuda_stream) {
   if (h == nullptr) return VS_ERR_INVALID_ARG;
   VS_CK(cudaSetDevice(h->device));
-  VS_CK(launch_poison(h->ws + h->lo.scratch_begin, h->lo.scratch_end - h->lo.scratch_begin,
-                      static_cast<cudaStream_t>(cuda_stream)));
+  VS_LAUNCH(h, static_cast<cudaStream_t>(cuda_stream), KC_OTHER,
+            launch_poison(h->ws + h->lo.scratch_begin, h->lo.scratch_end - h->lo.scratch_begin,
+                          static_cast<cudaStream_t>(cuda_stream)));
   h->last_stream = static_cast<cudaStream_t>(cuda_stream);
   return VS_OK;
 }

@@ -173,8 +173,12 @@ __global__ void __launch_bounds__(256) finalize_kernel(FinalizeArgs a, BatchPara
   }
   const bf16 o1 = __float2bfloat16_rn(x1), o2 = __float2bfloat16_rn(x2);
   if (hs < a.Hq) {
-    bf16* q = a.q + (size_t)row * a.Hq * a.D + hs * a.D;
-    q[k] = o1; q[k + half] = o2;
+    // the query never leaves the step, so it is kept as a bf16 pair (hi + lo): the score
+    // Q K^T then sees a 16-bit mantissa instead of 8 at the cost of a second MMA
+    const size_t qo = (size_t)row * a.Hq * a.D + hs * a.D;
+    a.q[qo + k] = o1; a.q[qo + k + half] = o2;
+    a.q_lo[qo + k] = __float2bfloat16_rn(x1 - __bfloat162float(o1));
+    a.q_lo[qo + k + half] = __float2bfloat16_rn(x2 - __bfloat162float(o2));
     return;
   }
   const bool is_k = hs < a.Hq + a.Hkv;
@@ -361,6 +365,25 @@ __global__ void poison_kernel(uint32_t* p, size_t n) {
 
 cudaError_t launch_poison(void* p, size_t bytes, cudaStream_t st) {
   poison_kernel<<<592, 256, 0, st>>>(reinterpret_cast<uint32_t*>(p), bytes / 4);
+  return cudaGetLastError();
+}
+
+// a stream starts over (new video): empty bank, no history; K/V payloads need no clearing
+// because nothing reads a slot that the metadata does not list
+__global__ void reset_kernel(StreamMeta* meta, int32_t* slot_frame, int slots, BatchParams bp) {
+  const int sid = bp.stream_id[blockIdx.x];
+  for (int i = threadIdx.x; i < slots; i += blockDim.x) slot_frame[(size_t)sid * slots + i] = -1;
+  if (threadIdx.x == 0) {
+    StreamMeta m;
+    m.count = 0; m.free_slot = 0; m.victim_logical = -1; m.last_victim_frame = -1;
+    m.frames_seen = 0; m.evictions = 0; m.log_count = 0; m.score_ticket = 0;
+    m.pad[0] = m.pad[1] = m.pad[2] = m.pad[3] = 0;
+    meta[sid] = m;
+  }
+}
+
+cudaError_t launch_reset(StreamMeta* meta, int32_t* slot_frame, int slots, const BatchParams& bp, cudaStream_t st) {
+  reset_kernel<<<bp.n_active, 256, 0, st>>>(meta, slot_frame, slots, bp);
   return cudaGetLastError();
 }
 
