@@ -40,6 +40,7 @@ extern "C" {
 
 #define VS_MAX_BATCH           64   /* most streams one call may list                       */
 #define VS_N_KERNEL_CLASSES    10   /* kernel classes reported by vs_profile_read           */
+#define VS_STATIC_MAX_BANK   4096   /* most carriers vs_evict_choose_static can score       */
 
 typedef struct vs_stream vs_stream;   /* opaque handle: a batch of n_streams independent video streams */
 
@@ -181,6 +182,29 @@ int vs_poison_scratch(vs_stream* h, void* cuda_stream);
 int vs_profile_enable(vs_stream* h, int32_t on, int32_t max_launches);
 int vs_profile_read(vs_stream* h, double* ms, int64_t* timed, int64_t* launches);
 const char* vs_kernel_class_name(int32_t k);
+
+/* Eviction decision without any allocation (the paper has no counterpart; it is the rule of
+ * Section 3.3's memory mechanism offered as a stand-alone call).  It is meant for callers
+ * that hold no workspace and may not call cudaMalloc: a real-time frame loop, where an
+ * allocation would stall the device; a component that was handed a fixed memory budget up
+ * front; a plug-in that must not go around its host framework's allocator.  Such a caller
+ * can still ask which stored carrier the bank would discard for an incoming one.
+ *   bank_emb  : DEVICE bf16 [count][d_model], carriers in temporal order (oldest first);
+ *   incoming  : DEVICE bf16 [d_model];
+ *   policy    : as vs_config.evict_policy (0 similarity to the incoming carrier, 1 most
+ *               similar adjacent pair, 2 FIFO);
+ *   victim_out: DEVICE int32[1], receives the temporal index to discard (ties: oldest).
+ * The call only enqueues work on cuda_stream.  Its scratch (count fp64 scores and one block
+ * counter) lives in a static device array of the library, VS_STATIC_MAX_BANK * 8 + 256
+ * bytes, which every GPU that loads the library holds until the process exits; count above
+ * VS_STATIC_MAX_BANK returns VS_ERR_CAPACITY.  The first call on a device looks the array's
+ * device address up (cudaGetSymbolAddress, with that device current) and should therefore
+ * come before any stream capture.  All calls on a device share the array: it keeps the last
+ * call's scores, the counter is cleared at the start of every call, and two calls that
+ * overlap on the GPU (different streams) race -- order them.  Calls no cudaMalloc, cudaFree
+ * or other allocating routine. */
+int vs_evict_choose_static(const void* bank_emb, const void* incoming, int32_t count, int32_t d_model,
+                           int32_t policy, int32_t* victim_out, void* cuda_stream);
 
 int vs_destroy_stream(vs_stream* h);
 

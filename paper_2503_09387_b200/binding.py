@@ -29,7 +29,8 @@ VS_MAX_BATCH = 64
 EXPORTS = ["vs_workspace_bytes", "vs_create_stream", "vs_frame_prefill", "vs_decode_step",
            "vs_end_turn", "vs_bank_state", "vs_last_step_kv", "vs_poison_scratch",
            "vs_destroy_stream", "vs_status_string", "vs_reset_stream", "vs_profile_enable",
-           "vs_profile_read", "vs_kernel_class_name"]
+           "vs_profile_read", "vs_kernel_class_name", "vs_evict_choose_static"]
+VS_STATIC_MAX_BANK = 4096
 VS_N_KERNEL_CLASSES = 10
 
 
@@ -91,6 +92,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.vs_reset_stream.argtypes = [vp, i32p, i32, vp]
     lib.vs_profile_enable.argtypes = [vp, i32, i32]
     lib.vs_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+    lib.vs_evict_choose_static.argtypes = [vp, vp, i32, i32, i32, vp, vp]
     lib.vs_kernel_class_name.argtypes = [i32]
     lib.vs_kernel_class_name.restype = C.c_char_p
     for name in EXPORTS:
@@ -174,6 +176,13 @@ def vs_profile_read(handle: int) -> dict:
     _check(lib.vs_profile_read(handle, ms, timed, launches), "vs_profile_read")
     return {lib.vs_kernel_class_name(k).decode(): (ms[k], int(timed[k]), int(launches[k]))
             for k in range(VS_N_KERNEL_CLASSES)}
+
+
+def vs_evict_choose_static(bank_emb_ptr: int, incoming_ptr: int, count: int, d_model: int, policy: int,
+                           victim_out_ptr: int, cuda_stream: int = 0) -> None:
+    """Enqueues the allocation-free eviction decision; the result lands in the int32 at victim_out_ptr."""
+    _check(load_library().vs_evict_choose_static(bank_emb_ptr, incoming_ptr, count, d_model, policy,
+                                                 victim_out_ptr, cuda_stream or None), "vs_evict_choose_static")
 
 
 def vs_destroy_stream(handle: int) -> None:
