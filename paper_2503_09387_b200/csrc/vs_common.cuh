@@ -180,20 +180,13 @@ struct DecodeArgs {
 };
 cudaError_t launch_decode_attention(const DecodeArgs& a, const BatchParams& bp, cudaStream_t st);
 
-struct EvictArgs {
+struct BankUpdateArgs {
   const bf16* emb;               // [S][slots][d]
   StreamMeta* meta;
-  const int32_t* order; double* scores;  // per-stream arrays, stride `slots`
-  int d, slots, M, policy;
+  int32_t* order; int32_t* slot_frame; int64_t* slot_pos; int32_t* evict_log; double* scores;
+  int d, slots, M, policy, log_cap;
 };
-cudaError_t launch_evict_score(const EvictArgs& a, const BatchParams& bp, cudaStream_t st);
-
-struct CommitArgs {
-  StreamMeta* meta;
-  int32_t* order; int32_t* slot_frame; int64_t* slot_pos; int32_t* evict_log;
-  int slots, M, log_cap;
-};
-cudaError_t launch_commit(const CommitArgs& a, const BatchParams& bp, cudaStream_t st);
+cudaError_t launch_bank_update(const BankUpdateArgs& a, const BatchParams& bp, bool any_full, cudaStream_t st);
 
 cudaError_t launch_poison(void* p, size_t bytes, cudaStream_t st);
 cudaError_t launch_reset(StreamMeta* meta, int32_t* slot_frame, int slots, const BatchParams& bp, cudaStream_t st);

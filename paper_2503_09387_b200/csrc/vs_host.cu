@@ -370,18 +370,13 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     if (D.residual) cur ^= 1;
   }
 
-  if (any_full) {
-    EvictArgs ea;
-    ea.emb = h->at<bf16>(lo.emb); ea.meta = meta;
-    ea.order = h->at<int32_t>(lo.order); ea.scores = h->at<double>(lo.scores);
-    ea.d = D.d; ea.slots = D.slots; ea.M = D.M; ea.policy = D.evict_policy;
-    VS_LAUNCH(h, st, KC_EVICT, launch_evict_score(ea, bp, st));
-  }
-  CommitArgs ca;
-  ca.meta = meta; ca.order = h->at<int32_t>(lo.order); ca.slot_frame = h->at<int32_t>(lo.slot_frame);
-  ca.slot_pos = h->at<int64_t>(lo.slot_pos); ca.evict_log = h->at<int32_t>(lo.evict_log);
-  ca.slots = D.slots; ca.M = D.M; ca.log_cap = D.log_cap;
-  VS_LAUNCH(h, st, KC_COMMIT, launch_commit(ca, bp, st));
+  BankUpdateArgs ba;
+  ba.emb = h->at<bf16>(lo.emb); ba.meta = meta;
+  ba.order = h->at<int32_t>(lo.order); ba.slot_frame = h->at<int32_t>(lo.slot_frame);
+  ba.slot_pos = h->at<int64_t>(lo.slot_pos); ba.evict_log = h->at<int32_t>(lo.evict_log);
+  ba.scores = h->at<double>(lo.scores);
+  ba.d = D.d; ba.slots = D.slots; ba.M = D.M; ba.policy = D.evict_policy; ba.log_cap = D.log_cap;
+  VS_LAUNCH(h, st, KC_COMMIT, launch_bank_update(ba, bp, any_full, st));
 
   for (int i = 0; i < n_active; ++i) {
     HostStream& s = h->hs[stream_ids[i]];
@@ -573,8 +568,8 @@ int vs_profile_read(vs_stream* h, double* ms, int64_t* timed, int64_t* launches)
 
 const char* vs_kernel_class_name(int32_t k) {
   static const char* names[VS_N_KERNEL_CLASSES] = {"pool", "rope_table", "rmsnorm", "qkv_gemm", "finalize",
-                                                   "prefill_attention", "decode_attention", "evict_score",
-                                                   "bank_commit", "other"};
+                                                   "prefill_attention", "decode_attention", "unused",
+                                                   "bank_update", "other"};
   return (k >= 0 && k < VS_N_KERNEL_CLASSES) ? names[k] : "?";
 }
 

@@ -17,9 +17,10 @@ __device__ __forceinline__ bf16 f64_to_bf16_rne(double x) {
 
 // ------------------------------------------------------------------------------------------
 // Carrier aggregation + layer-0 input assembly + RoPE table.
-// grid = (pool_blocks + rope_blocks, n_active); block = 256 = 8 row groups x 32 lanes, each
-// lane owns 2 adjacent channels, so one block covers 64 channels of every row.  The sum of
-// <= 256 bf16 values in fp64 is exact, hence independent of the order used here.
+// grid = (pool_blocks + rope_blocks, n_active).  A pool block owns 64 channels of every row:
+// 256 threads = 32 row groups x 8 lanes of 16 bytes (8 channels).  Every thread issues all of
+// its <= 8 row loads before using any of them, so the whole frame (1.2 MB) is in flight at
+// once.  The sum of <= 256 bf16 values in fp64 is exact, hence independent of the order.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, int pool_blocks) {
   const int b = blockIdx.y;
@@ -38,46 +39,61 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, i
     }
     return;
   }
-  __shared__ double red[8][64];
-  const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
-  const int ch = blockIdx.x * 64 + lane * 2;
-  const bf16* src = a.hidden + (size_t)b * N * d;
-  bf16* dst = a.x + (size_t)b * (N + 1) * d;
-  double s0 = 0.0, s1 = 0.0;
-  if (ch < d) {
-    for (int r = grp; r < N; r += 8) {
-      const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(src + (size_t)r * d + ch);
-      *reinterpret_cast<__nv_bfloat162*>(dst + (size_t)r * d + ch) = v;
-      s0 += (double)__bfloat162float(v.x);
-      s1 += (double)__bfloat162float(v.y);
+  constexpr int RG = 32;                    // row groups
+  constexpr int MAXR = 8;                   // rows per thread (N <= 255)
+  __shared__ double red[RG][64];
+  const int cl = threadIdx.x & 7, grp = threadIdx.x >> 3;
+  const int ch = blockIdx.x * 64 + cl * 8;  // d is a multiple of 64
+  const bf16* src = a.hidden + (size_t)b * N * d + ch;
+  bf16* dst = a.x + (size_t)b * (N + 1) * d + ch;
+  uint4 v[MAXR];
+#pragma unroll
+  for (int i = 0; i < MAXR; ++i) {
+    const int r = grp + i * RG;
+    v[i] = (r < N) ? *reinterpret_cast<const uint4*>(src + (size_t)r * d) : make_uint4(0, 0, 0, 0);
+  }
+  double acc[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc[j] = 0.0;
+#pragma unroll
+  for (int i = 0; i < MAXR; ++i) {
+    const int r = grp + i * RG;
+    if (r < N) {
+      *reinterpret_cast<uint4*>(dst + (size_t)r * d) = v[i];
+      const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&v[i]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        acc[2 * j] += (double)__bfloat162float(h2[j].x);
+        acc[2 * j + 1] += (double)__bfloat162float(h2[j].y);
+      }
     }
   }
-  red[grp][lane * 2] = s0;
-  red[grp][lane * 2 + 1] = s1;
-  __syncthreads();
-  if (grp == 0 && ch < d) {
-    __nv_bfloat162 c;
-    if (a.carrier_override != nullptr) {
-      c = *reinterpret_cast<const __nv_bfloat162*>(a.carrier_override + (size_t)b * d + ch);
-    } else if (a.agg_mode == 1) {
-      c = *reinterpret_cast<const __nv_bfloat162*>(src + (size_t)(N - 1) * d + ch);
-    } else {
-      double t0 = 0.0, t1 = 0.0;
 #pragma unroll
-      for (int g = 0; g < 8; ++g) { t0 += red[g][lane * 2]; t1 += red[g][lane * 2 + 1]; }
-      c.x = f64_to_bf16_rne(t0 / (double)N);
-      c.y = f64_to_bf16_rne(t1 / (double)N);
+  for (int j = 0; j < 8; ++j) red[grp][cl * 8 + j] = acc[j];
+  __syncthreads();
+  if (threadIdx.x < 64) {
+    const int c = blockIdx.x * 64 + threadIdx.x;
+    bf16 cv;
+    if (a.carrier_override != nullptr) {
+      cv = a.carrier_override[(size_t)b * d + c];
+    } else if (a.agg_mode == 1) {
+      cv = a.hidden[(size_t)b * N * d + (size_t)(N - 1) * d + c];
+    } else {
+      double t = 0.0;
+#pragma unroll
+      for (int g = 0; g < RG; ++g) t += red[g][threadIdx.x];
+      cv = f64_to_bf16_rne(t / (double)N);
     }
-    *reinterpret_cast<__nv_bfloat162*>(dst + (size_t)N * d + ch) = c;   // carrier = last token of the frame
+    a.x[(size_t)b * (N + 1) * d + (size_t)N * d + c] = cv;   // carrier = last token of the frame
     if (a.M > 0) {
       const int slot = a.meta[sid].free_slot;
-      *reinterpret_cast<__nv_bfloat162*>(a.emb + ((size_t)sid * a.slots + slot) * d + ch) = c;
+      a.emb[((size_t)sid * a.slots + slot) * d + c] = cv;
     }
   }
 }
 
 cudaError_t launch_pool(const PoolArgs& a, const BatchParams& bp, cudaStream_t st) {
-  const int pool_blocks = (a.d + 63) / 64;
+  const int pool_blocks = a.d / 64;
   const int rope_blocks = ((a.N + 1) * (a.D / 2) + 255) / 256;
   dim3 grid(pool_blocks + rope_blocks, bp.n_active);
   pool_kernel<<<grid, 256, 0, st>>>(a, bp, pool_blocks);
@@ -209,12 +225,16 @@ cudaError_t launch_finalize(const FinalizeArgs& a, const BatchParams& bp, cudaSt
 }
 
 // ------------------------------------------------------------------------------------------
-// Eviction scoring (Section 3.3: discard the older carrier with the largest cosine
-// similarity).  One warp per temporal index j.  Dot products are accumulated in fp64 in a
-// fixed order -- lane p sums elements k = p (mod 32) in ascending k, then a butterfly
-// 16, 8, 4, 2, 1 -- so that the score, and with it the argmax, is reproducible bit for bit.
-// Products of two bf16 values are exact in fp64, so fused and unfused accumulation agree.
-// The last block to finish picks the victim: largest score, oldest on ties.
+// Bank update (Section 3.3, memory mechanism): evict-if-full, then append.  One launch per
+// frame step, grid = (blocks, n_active).
+// Bank not full: block 0 appends; the other blocks exit.
+// Bank full: one warp per temporal index j scores cos(e_j, e_other) -- e_other is the incoming
+// carrier (policy 0) or the next carrier in temporal order (policy 1).  Dot products are
+// accumulated in fp64 in a fixed order -- lane p sums elements k = p (mod 32) in ascending k,
+// then a butterfly 16, 8, 4, 2, 1 -- so that the score, and with it the argmax, is
+// reproducible bit for bit; products of two bf16 values are exact in fp64, so fused and
+// unfused accumulation agree.  The last block of a stream to finish picks the victim (largest
+// score, oldest on ties), closes the gap in the temporal order and appends.
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ double warp_tree_sum(double v) {
 #pragma unroll
@@ -222,18 +242,39 @@ __device__ __forceinline__ double warp_tree_sum(double v) {
   return v;
 }
 
-__global__ void __launch_bounds__(256) evict_score_kernel(EvictArgs a, BatchParams bp) {
+__global__ void __launch_bounds__(256) bank_update_kernel(BankUpdateArgs a, BatchParams bp) {
   const int b = blockIdx.y;
   const int sid = bp.stream_id[b];
-  const int count = bp.count[b];
-  if (count < a.M || a.M == 0) return;             // bank not full: nothing to score
   StreamMeta* meta = a.meta + sid;
-  const int32_t* order = a.order + (size_t)sid * a.slots;
+  if (a.M == 0) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) { meta->frames_seen += 1; meta->last_victim_frame = -1; }
+    return;
+  }
+  int32_t* order = a.order + (size_t)sid * a.slots;
+  int32_t* slot_frame = a.slot_frame + (size_t)sid * a.slots;
+  int64_t* slot_pos = a.slot_pos + (size_t)sid * a.slots;
+  const int count = bp.count[b];
+  const int incoming = meta->free_slot;
+  const int64_t carrier_pos = bp.pos_base[b] + bp.rows_per_stream - 1;
+  if (count < a.M) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      order[count] = incoming;
+      slot_frame[incoming] = (int32_t)bp.frame_id[b];
+      slot_pos[incoming] = carrier_pos;
+      meta->count = count + 1;
+      meta->free_slot = count + 1;          // slots fill in order until the bank is full
+      meta->last_victim_frame = -1;
+      meta->frames_seen += 1;
+    }
+    return;
+  }
+  // ---- bank full: score, then the last block commits --------------------------------------
   double* scores = a.scores + (size_t)sid * a.slots;
   const int lane = threadIdx.x & 31;
+  const int n_score_blocks = (a.M + 7) / 8;
+  if ((int)blockIdx.x >= n_score_blocks) return;
   const int j = blockIdx.x * 8 + (threadIdx.x >> 5);
-  const int incoming = meta->free_slot;
-  if (j < count) {
+  if (j < count && a.policy != 2) {
     const int sa = order[j];
     const int sb = (a.policy == 1 && j + 1 < count) ? order[j + 1] : incoming;
     const bf16* va = a.emb + ((size_t)sid * a.slots + sa) * a.d;
@@ -253,23 +294,21 @@ __global__ void __launch_bounds__(256) evict_score_kernel(EvictArgs a, BatchPara
       scores[j] = s;
     }
   }
-  // the last block of this stream to finish does the argmax
   __shared__ int is_last;
   __threadfence();
   __syncthreads();
-  if (threadIdx.x == 0) {
-    const int done = atomicAdd(&meta->score_ticket, 1);
-    is_last = (done == (int)gridDim.x - 1);
-  }
+  if (threadIdx.x == 0) is_last = (atomicAdd(&meta->score_ticket, 1) == n_score_blocks - 1);
   __syncthreads();
   if (!is_last) return;
   __threadfence();
   __shared__ double best_s[256];
   __shared__ int best_j[256];
   double bs = -2.0; int bj = 0x7fffffff;
-  for (int i = threadIdx.x; i < count; i += blockDim.x) {
-    const double s = __ldcg(scores + i);
-    if (s > bs) { bs = s; bj = i; }                 // ascending i: first maximum kept
+  if (a.policy != 2) {
+    for (int i = threadIdx.x; i < count; i += blockDim.x) {
+      const double s = __ldcg(scores + i);
+      if (s > bs) { bs = s; bj = i; }                 // ascending i: first maximum kept
+    }
   }
   best_s[threadIdx.x] = bs; best_j[threadIdx.x] = bj;
   __syncthreads();
@@ -282,79 +321,42 @@ __global__ void __launch_bounds__(256) evict_score_kernel(EvictArgs a, BatchPara
     }
     __syncthreads();
   }
+  const int v = (a.policy == 2) ? 0 : best_j[0];
+  const int victim_slot = order[v];
+  const int victim_frame = slot_frame[victim_slot];
+  __syncthreads();
+  // close the gap in the temporal order, one block-wide chunk at a time in ascending
+  // order: a chunk reads [base+1, base+256] before anything at or above base is written
+  for (int base = v; base < count - 1; base += blockDim.x) {
+    const int jj = base + threadIdx.x;
+    const int32_t next = (jj < count - 1) ? order[jj + 1] : 0;
+    __syncthreads();
+    if (jj < count - 1) order[jj] = next;
+    __syncthreads();
+  }
   if (threadIdx.x == 0) {
-    meta->victim_logical = (a.policy == 2) ? 0 : best_j[0];
+    order[count - 1] = incoming;
+    slot_frame[victim_slot] = -1;
+    slot_frame[incoming] = (int32_t)bp.frame_id[b];
+    slot_pos[incoming] = carrier_pos;
+    if (a.log_cap > 0) {
+      int32_t* e = a.evict_log + ((size_t)sid * a.log_cap + (meta->log_count % a.log_cap)) * 2;
+      e[0] = (int32_t)bp.frame_id[b];
+      e[1] = victim_frame;
+    }
+    meta->log_count += 1;
+    meta->evictions += 1;
+    meta->last_victim_frame = victim_frame;
+    meta->free_slot = victim_slot;
+    meta->victim_logical = -1;
+    meta->frames_seen += 1;
     meta->score_ticket = 0;
   }
 }
 
-cudaError_t launch_evict_score(const EvictArgs& a, const BatchParams& bp, cudaStream_t st) {
-  dim3 grid((a.M + 7) / 8, bp.n_active);
-  evict_score_kernel<<<grid, 256, 0, st>>>(a, bp);
-  return cudaGetLastError();
-}
-
-// ------------------------------------------------------------------------------------------
-// Bank commit: evict-if-full, then append (Section 3.3).  One block per listed stream.
-// ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) commit_kernel(CommitArgs a, BatchParams bp) {
-  const int b = blockIdx.x;
-  const int sid = bp.stream_id[b];
-  StreamMeta* meta = a.meta + sid;
-  if (a.M == 0) {
-    if (threadIdx.x == 0) { meta->frames_seen += 1; meta->last_victim_frame = -1; }
-    return;
-  }
-  int32_t* order = a.order + (size_t)sid * a.slots;
-  int32_t* slot_frame = a.slot_frame + (size_t)sid * a.slots;
-  int64_t* slot_pos = a.slot_pos + (size_t)sid * a.slots;
-  const int count = meta->count;
-  const int incoming = meta->free_slot;
-  const int64_t carrier_pos = bp.pos_base[b] + bp.rows_per_stream - 1;
-  if (count == a.M) {
-    const int v = meta->victim_logical;
-    const int victim_slot = order[v];
-    const int victim_frame = slot_frame[victim_slot];
-    __syncthreads();
-    // close the gap in the temporal order, one block-wide chunk at a time in ascending
-    // order: a chunk reads [base+1, base+256] before anything at or above base is written
-    for (int base = v; base < count - 1; base += blockDim.x) {
-      const int j = base + threadIdx.x;
-      const int32_t next = (j < count - 1) ? order[j + 1] : 0;
-      __syncthreads();
-      if (j < count - 1) order[j] = next;
-      __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-      order[count - 1] = incoming;
-      slot_frame[victim_slot] = -1;
-      slot_frame[incoming] = (int32_t)bp.frame_id[b];
-      slot_pos[incoming] = carrier_pos;
-      if (a.log_cap > 0) {
-        int32_t* e = a.evict_log + ((size_t)sid * a.log_cap + (meta->log_count % a.log_cap)) * 2;
-        e[0] = (int32_t)bp.frame_id[b];
-        e[1] = victim_frame;
-      }
-      meta->log_count += 1;
-      meta->evictions += 1;
-      meta->last_victim_frame = victim_frame;
-      meta->free_slot = victim_slot;
-      meta->victim_logical = -1;
-      meta->frames_seen += 1;
-    }
-  } else if (threadIdx.x == 0) {
-    order[count] = incoming;
-    slot_frame[incoming] = (int32_t)bp.frame_id[b];
-    slot_pos[incoming] = carrier_pos;
-    meta->count = count + 1;
-    meta->free_slot = count + 1;            // slots fill in order until the bank is full
-    meta->last_victim_frame = -1;
-    meta->frames_seen += 1;
-  }
-}
-
-cudaError_t launch_commit(const CommitArgs& a, const BatchParams& bp, cudaStream_t st) {
-  commit_kernel<<<bp.n_active, 256, 0, st>>>(a, bp);
+cudaError_t launch_bank_update(const BankUpdateArgs& a, const BatchParams& bp, bool any_full, cudaStream_t st) {
+  dim3 grid(any_full ? (a.M + 7) / 8 : 1, bp.n_active);
+  bank_update_kernel<<<grid, 256, 0, st>>>(a, bp);
   return cudaGetLastError();
 }
 
