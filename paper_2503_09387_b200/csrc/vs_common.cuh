@@ -161,6 +161,8 @@ struct AttnArgs {
 };
 cudaError_t launch_prefill_attention(const AttnArgs& a, const BatchParams& bp, cudaStream_t st);
 cudaError_t prefill_attention_init();
+cudaError_t launch_prefill_attention_tc(const AttnArgs& a, const BatchParams& bp, int* status, cudaStream_t st);
+cudaError_t prefill_attention_tc_init();
 
 struct DecodeArgs {
   const bf16* q;                 // [n_active][Hq*D]

@@ -257,7 +257,7 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights, void* work
   h->tm_w.resize(D.L);
   for (int l = 0; l < D.L; ++l)
     if (encode_2d(h, &h->tm_w[l], h->w[l], (uint64_t)D.d, (uint64_t)D.E_out, GEMM_BLOCK_M) != VS_OK) return fail(VS_ERR_CUDA);
-  if (qkv_gemm_init() != cudaSuccess || prefill_attention_init() != cudaSuccess) return fail(VS_ERR_CUDA);
+  if (qkv_gemm_init() != cudaSuccess || prefill_attention_init() != cudaSuccess || prefill_attention_tc_init() != cudaSuccess) return fail(VS_ERR_CUDA);
   // clear the whole workspace, then write the non-zero initial metadata
   if (cudaMemset(h->ws, 0, lo.total) != cudaSuccess) return fail(VS_ERR_CUDA);
   if (cudaMemset(h->ws + lo.slot_frame, 0xFF, (size_t)D.S * D.slots * 4) != cudaSuccess) return fail(VS_ERR_CUDA);
@@ -366,7 +366,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     aa.meta = meta;
     aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
     aa.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
-    VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention(aa, bp, st));
+    VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, bp, h->at<int>(lo.status), st));
     if (D.residual) cur ^= 1;
   }
 
@@ -499,7 +499,7 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       aa.meta = meta;
       aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
       aa.scale_log2e = scale_log2e;
-      VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention(aa, bp, st));
+      VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, bp, h->at<int>(lo.status), st));
     }
     if (D.residual) { h_in = h_out; next_buf ^= 1; }
   }
