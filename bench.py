@@ -322,7 +322,6 @@ def run_ours(args, w):
             rows = N + 1
             alg = {"prefill_attention": rows * (HD * 2 * 2 + 2 * w.n_kv_heads * w.head_dim * 2) + rows * HD * 4
                    + (w.prefix_len + avg_bank) * 2 * w.n_kv_heads * w.head_dim * 2,
-                   "finalize": 4 * rows * w.e_out * 4 + rows * w.e_out * 2 + rows * HD * 2,
                    "pool": 2 * N * d * 2 + d * 4}.get(dom, 0.0)
             ach = alg / (kernels[dom]["avg_us"] * 1e-6) / 1e9
             roof = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -76,7 +76,6 @@ struct Layout {
   // per-step scratch
   size_t hbuf[2];               // bf16 [R_max][d]  residual ping-pong; hbuf[0] holds [E; carrier]
   size_t xn;                    // bf16 [R_max][d]  normalised layer input
-  size_t partials;              // f32  [KSPLIT_MAX][R_max][E_out]
   size_t q;                     // bf16 [R_max][Hq*D]
   size_t q_lo;                  // bf16 [R_max][Hq*D]  low-order half of the rotated query
   size_t kf, vf;                // bf16 [R_max][Hkv*D]
@@ -110,33 +109,31 @@ cudaError_t launch_rope_table(const RopeArgs& a, const BatchParams& bp, cudaStre
 cudaError_t launch_rmsnorm(const bf16* h, const bf16* gain, bf16* xn, int rows, int d, float eps,
                            cudaStream_t st);
 
-struct GemmArgs {
-  CUtensorMap tm_w;              // [E_out, d] bf16, box 64 x 128, 128-byte swizzle
-  CUtensorMap tm_x;              // [rows, d] bf16, box 64 x tile_n, 128-byte swizzle
-  float* partials;               // [ksplit][rows][E_out]
-  int rows, E_out, d;
-  int tile_n, n_tiles, ksplit;
-  int* status;
-};
-cudaError_t launch_qkv_gemm(const GemmArgs& a, cudaStream_t st);
-cudaError_t qkv_gemm_init();     // opt-in shared memory attribute, once per process/device
-
-struct FinalizeArgs {
-  const float* partials;         // [ksplit][rows][E_out]
+// What the projection epilogue writes (finished rows: bias, RoPE, bf16) and where rows persist.
+struct ProjectionOut {
   const bf16* bias;              // [E_out] or null
-  const float2* rope;            // [rows][D/2]
+  const float2* rope;            // [rows][D/2] (cos, sin)
   bf16* q;                       // [rows][Hq*D]  rotated query, leading bf16 part
   bf16* q_lo;                    // [rows][Hq*D]  bf16(query - q): the pair carries 16 mantissa bits
-  bf16* kf;                      // [rows][Hkv*D]
-  bf16* vf;
+  bf16* kf;                      // [rows][Hkv*D] rotated keys of this step
+  bf16* vf;                      // [rows][Hkv*D]
   bf16* bank_k; bf16* bank_v;    // layer base [S][Hkv][slots][D]
   bf16* text_k; bf16* text_v;    // layer base [S][Hkv][text_cap][D]: prefix or tail
   const StreamMeta* meta;
-  int rows, ksplit, E_out, Hq, Hkv, D, slots, text_cap;
+  int Hq, Hkv, D, slots, text_cap, M;
   int mode;                      // 0 frame step (carrier row -> bank), 1 text -> prefix, 2 text -> tail
-  int M;
 };
-cudaError_t launch_finalize(const FinalizeArgs& a, const BatchParams& bp, cudaStream_t st);
+
+struct GemmArgs {
+  CUtensorMap tm_w;              // [E_out, d] bf16, box 64 x 128, 128-byte swizzle
+  CUtensorMap tm_x;              // [rows, d] bf16, box 64 x tile_n, 128-byte swizzle
+  ProjectionOut out;
+  int rows, E_out, d;
+  int tile_n, n_tiles, ksplit;   // ksplit = cluster size: 1, 2, 4 or 8
+  int* status;
+};
+cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream_t st);
+cudaError_t qkv_gemm_init();     // opt-in shared memory attribute, once per process/device
 
 struct AttnSegment {
   const bf16* k; const bf16* v;

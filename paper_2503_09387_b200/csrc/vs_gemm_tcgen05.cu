@@ -7,14 +7,24 @@
 // (128 weight rows per CTA, read K-major straight from the caller's [E_out, d] matrix) and
 // the *tokens* take the MMA's N axis (any multiple of 16 up to 256: 170 tokens cost 176
 // columns, 3.5 % padding instead of 33 % with 128-row token tiles).  The reduction dimension
-// d is split over `ksplit` CTAs so that m_tiles * n_tiles * ksplit fills the 148 SMs; each
-// CTA writes an fp32 partial tile which the finalize kernel sums.
+// d is split over `ksplit` CTAs so that m_tiles * n_tiles * ksplit fills the 148 SMs.  The
+// ksplit CTAs of one output tile form a thread-block cluster: each dumps its fp32 partial
+// accumulator to its own shared memory, and after a cluster barrier CTA r sums token slice r
+// of all partials through distributed shared memory.  The same epilogue adds the bias,
+// applies RoPE (a 128-row tile holds whole heads, so both elements of a rotation pair are at
+// hand), writes Q as a bf16 hi + lo pair and K, V as bf16, and persists what the method keeps:
+// the carrier row's K/V goes straight into the bank's free slot (Section 3.2: only the
+// carrier keeps its K/V), text rows are appended to the prefix or to the turn's tail.
 //
 // Per CTA: 6 warps.  Warp 0 lane 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer
-// (lane 0), warps 2..5 = epilogue (tcgen05.ld of their 32-lane quarter -> global).
+// (lane 0), warps 2..5 = epilogue (tcgen05.ld of their 32-lane quarter).
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, records
 // VS_ERR_DEVICE_TIMEOUT, lets in-flight copies land, frees its tensor memory and exits.
+#include <cooperative_groups.h>
+
 #include "vs_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace vs {
 
@@ -105,21 +115,28 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 
 struct KernelParams {
-  float* partials;
+  ProjectionOut o;
   int* status;
-  int rows, E_out, tile_n, kblocks, stages, tmem_cols;
+  int rows, E_out, tile_n, kblocks, stages, tmem_cols, ksplit;
+  uint32_t data_bytes;          // shared memory ahead of the barriers: max(pipeline stages, fp32 partial tile)
 };
 
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __global__ void __launch_bounds__(kThreads, 1)
-qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, KernelParams p) {
+qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, KernelParams p,
+                BatchParams bp) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  // carve: [stages][A 16 KiB | B tile_n*128] | full[stages] | empty[stages] | tmem_full | tmem slot | abort
+  // carve: [stages][A 16 KiB | B tile_n*128] (later reused as the fp32 partial tile
+  // [token][128 features]) | full[stages] | empty[stages] | tmem_full | tmem slot | abort
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t stage_b_bytes = (uint32_t)p.tile_n * 128u;
   const uint32_t stage_bytes = kStageABytes + stage_b_bytes;
-  const uint32_t bar_base = base + (uint32_t)p.stages * stage_bytes;
+  const uint32_t bar_base = base + p.data_bytes;
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
-  uint8_t* ctl = gen_base + (size_t)p.stages * stage_bytes + 16 * p.stages;
+  uint8_t* ctl = gen_base + p.data_bytes + 16 * p.stages;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctl + 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + 12);
   auto full_bar = [&](int s) { return bar_base + 8u * (uint32_t)s; };
@@ -129,7 +146,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * GEMM_BLOCK_M;
   const int n0 = blockIdx.y * p.tile_n;
-  const int kb0 = blockIdx.z * p.kblocks;
+  const int kb0 = blockIdx.z * p.kblocks;      // blockIdx.z = rank in the cluster (cluster dims 1 x 1 x ksplit)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -197,30 +214,136 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
       if (ok) umma_commit(tmem_full_bar);   // accumulator complete
     }
   } else {
-    // epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31 (one lane = one output feature)
+    // epilogue, phase A: accumulator -> this CTA's fp32 partial tile in shared memory,
+    // [token][128 features]; warp w may touch TMEM lanes 32*(w%4) .. +31 (lane = feature).
+    // Every MMA has completed, hence every TMA write has landed and the stages are free.
     const int quarter = warp & 3;
     const bool ok = __all_sync(0xffffffffu, mbar_wait(tmem_full_bar, 0, abort_flag));   // warp-uniform
     tcgen05_fence_after();
     if (ok) {
-      const int feat = m0 + quarter * 32 + lane;
-      float* dst = p.partials + ((size_t)blockIdx.z * p.rows) * p.E_out + feat;
+      float* part = reinterpret_cast<float*>(gen_base) + quarter * 32 + lane;
       for (int c = 0; c < p.tile_n; c += 16) {
         if (n0 + c >= p.rows) break;               // uniform across the warp
         uint32_t r[16];
         tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, r);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (feat < p.E_out) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int tok = n0 + c + j;
-            if (tok < p.rows) dst[(size_t)tok * p.E_out] = __uint_as_float(r[j]);
+        for (int j = 0; j < 16; ++j) part[(c + j) * GEMM_BLOCK_M] = __uint_as_float(r[j]);
+      }
+    }
+  }
+
+  // phase B: every CTA of the cluster has its partial tile in place
+  tcgen05_fence_before();
+  __syncthreads();
+  if (p.ksplit > 1) cluster_sync_all();
+
+  // phase C: CTA r reduces token slice r, finishes the rows and stores them.  Thread =
+  // (group of 4 rotation pairs, token lane): float4 reads of every CTA's partial tile through
+  // distributed shared memory, all issued before they are summed.
+  if (warp >= 2 && !*abort_flag) {
+    const int te = threadIdx.x - 64;               // 0..127
+    const int D = p.o.D, half = D >> 1;
+    const int p0 = (te & 15) * 4;                  // first of 4 rotation pairs inside the 128-feature tile
+    const int hl = p0 / half, k0 = p0 - hl * half; // local head, index inside the half head
+    const int f1 = hl * D + k0, f2 = f1 + half;
+    const int hs = (m0 + f1) / D;                  // head slot: Q heads, then K heads, then V heads
+    const int slice = (p.tile_n + p.ksplit - 1) / p.ksplit;
+    const int t_begin = (int)blockIdx.z * slice;
+    const int t_end = min(t_begin + slice, p.tile_n);
+    const float* part_local = reinterpret_cast<const float*>(gen_base);
+    const float* part[8];
+    cg::cluster_group cluster = cg::this_cluster();
+#pragma unroll
+    for (int r = 0; r < 8; ++r)
+      part[r] = (p.ksplit > 1 && r < p.ksplit) ? cluster.map_shared_rank(part_local, r) : part_local;
+    if (m0 + f2 + 3 < p.E_out) {
+      float bb1[4] = {0.f, 0.f, 0.f, 0.f}, bb2[4] = {0.f, 0.f, 0.f, 0.f};
+      if (p.o.bias != nullptr) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          bb1[i] = __bfloat162float(p.o.bias[m0 + f1 + i]);
+          bb2[i] = __bfloat162float(p.o.bias[m0 + f2 + i]);
+        }
+      }
+      const int rps = bp.rows_per_stream;
+      for (int t = t_begin + (te >> 4); t < t_end; t += 8) {
+        const int row = n0 + t;
+        if (row >= p.rows) break;
+        float4 v1[8], v2[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+          if (r < p.ksplit) {
+            v1[r] = *reinterpret_cast<const float4*>(part[r] + t * GEMM_BLOCK_M + f1);
+            v2[r] = *reinterpret_cast<const float4*>(part[r] + t * GEMM_BLOCK_M + f2);
+          }
+        }
+        float x1[4] = {bb1[0], bb1[1], bb1[2], bb1[3]}, x2[4] = {bb2[0], bb2[1], bb2[2], bb2[3]};
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+          if (r < p.ksplit) {
+            x1[0] += v1[r].x; x1[1] += v1[r].y; x1[2] += v1[r].z; x1[3] += v1[r].w;
+            x2[0] += v2[r].x; x2[1] += v2[r].y; x2[2] += v2[r].z; x2[3] += v2[r].w;
+          }
+        }
+        if (hs < p.o.Hq + p.o.Hkv) {
+          const float4 ra = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0);
+          const float4 rb = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0 + 2);
+          const float cs[4] = {ra.x, ra.z, rb.x, rb.z}, sn[4] = {ra.y, ra.w, rb.y, rb.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float y1 = x1[i] * cs[i] - x2[i] * sn[i];
+            const float y2 = x2[i] * cs[i] + x1[i] * sn[i];
+            x1[i] = y1; x2[i] = y2;
+          }
+        }
+        __align__(8) bf16 o1[4], o2[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { o1[i] = __float2bfloat16_rn(x1[i]); o2[i] = __float2bfloat16_rn(x2[i]); }
+        const uint2 w1 = *reinterpret_cast<const uint2*>(o1), w2 = *reinterpret_cast<const uint2*>(o2);
+        if (hs < p.o.Hq) {
+          // the query never leaves the step, so it is kept as a bf16 pair (hi + lo): the score
+          // Q K^T then sees a 16-bit mantissa instead of 8 at the cost of a second MMA
+          const size_t qo = (size_t)row * p.o.Hq * D + (size_t)hs * D + k0;
+          *reinterpret_cast<uint2*>(p.o.q + qo) = w1;
+          *reinterpret_cast<uint2*>(p.o.q + qo + half) = w2;
+          __align__(8) bf16 l1[4], l2[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            l1[i] = __float2bfloat16_rn(x1[i] - __bfloat162float(o1[i]));
+            l2[i] = __float2bfloat16_rn(x2[i] - __bfloat162float(o2[i]));
+          }
+          *reinterpret_cast<uint2*>(p.o.q_lo + qo) = *reinterpret_cast<const uint2*>(l1);
+          *reinterpret_cast<uint2*>(p.o.q_lo + qo + half) = *reinterpret_cast<const uint2*>(l2);
+        } else {
+          const bool is_k = hs < p.o.Hq + p.o.Hkv;
+          const int hkv = is_k ? hs - p.o.Hq : hs - p.o.Hq - p.o.Hkv;
+          bf16* f = (is_k ? p.o.kf : p.o.vf) + (size_t)row * p.o.Hkv * D + (size_t)hkv * D + k0;
+          *reinterpret_cast<uint2*>(f) = w1;
+          *reinterpret_cast<uint2*>(f + half) = w2;
+          const int b = row / rps, tt = row - b * rps;
+          const int sid = bp.stream_id[b];
+          bf16* dst = nullptr;
+          if (p.o.mode == 0) {
+            if (tt == rps - 1 && p.o.M > 0) {
+              const int slot = p.o.meta[sid].free_slot;
+              dst = (is_k ? p.o.bank_k : p.o.bank_v) + (((size_t)sid * p.o.Hkv + hkv) * p.o.slots + slot) * D + k0;
+            }
+          } else {
+            const int tb = (p.o.mode == 1) ? bp.prefix_len[b] : bp.text_len[b];
+            dst = (is_k ? p.o.text_k : p.o.text_v) + (((size_t)sid * p.o.Hkv + hkv) * p.o.text_cap + tb + tt) * D + k0;
+          }
+          if (dst != nullptr) {
+            *reinterpret_cast<uint2*>(dst) = w1;
+            *reinterpret_cast<uint2*>(dst + half) = w2;
           }
         }
       }
     }
   }
 
-  tcgen05_fence_before();
+  // no CTA may leave while a peer still reads its partial tile
+  if (p.ksplit > 1) cluster_sync_all();
   __syncthreads();
   if (warp == 1) {
     tcgen05_fence_after();
@@ -234,22 +357,30 @@ constexpr int kMaxDynSmem = 227 * 1024;
 }  // namespace
 
 cudaError_t qkv_gemm_init() {
-  return cudaFuncSetAttribute(qkv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+  cudaError_t e = cudaFuncSetAttribute(qkv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(qkv_gemm_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 0);
 }
 
-cudaError_t launch_qkv_gemm(const GemmArgs& a, cudaStream_t st) {
+cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream_t st) {
   KernelParams p;
-  p.partials = a.partials;
+  p.o = a.out;
   p.status = a.status;
   p.rows = a.rows;
   p.E_out = a.E_out;
   p.tile_n = a.tile_n;
+  p.ksplit = a.ksplit;
   const int total_kb = a.d / GEMM_BLOCK_K;
-  if (a.ksplit < 1 || total_kb % a.ksplit != 0) return cudaErrorInvalidValue;
+  if (a.ksplit < 1 || a.ksplit > 8 || (a.ksplit & (a.ksplit - 1)) || total_kb % a.ksplit != 0) return cudaErrorInvalidValue;
   if (a.tile_n < 16 || a.tile_n > 256 || (a.tile_n & 15)) return cudaErrorInvalidValue;
+  if (128 % a.out.D != 0) return cudaErrorInvalidValue;
   p.kblocks = total_kb / a.ksplit;
   const int stage_bytes = kStageABytes + a.tile_n * 128;
-  int stages = (kMaxDynSmem - 2048) / stage_bytes;
+  // With one CTA per SM only 33 clusters of 4 can be resident on the 148 SMs (clusters do not
+  // straddle GPCs), fewer than the 36 weight tiles of the Qwen2-7B shape.  Keeping a CTA under
+  // half an SM's shared memory lets every cluster be resident in one wave.
+  const int smem_cap = (a.ksplit >= 4) ? 112 * 1024 : kMaxDynSmem;
+  int stages = (smem_cap - 2048) / stage_bytes;
   if (stages > 8) stages = 8;
   if (stages > p.kblocks) stages = p.kblocks;
   if (stages < 1) return cudaErrorInvalidValue;
@@ -257,10 +388,23 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, cudaStream_t st) {
   int cols = 32;
   while (cols < a.tile_n) cols <<= 1;
   p.tmem_cols = cols;
-  const size_t smem = 1024 + (size_t)stages * stage_bytes + 16 * stages + 64;
-  dim3 grid((a.E_out + GEMM_BLOCK_M - 1) / GEMM_BLOCK_M, a.n_tiles, a.ksplit);
-  qkv_gemm_kernel<<<grid, kThreads, smem, st>>>(a.tm_w, a.tm_x, p);
-  return cudaGetLastError();
+  size_t data = (size_t)stages * stage_bytes;
+  const size_t tile = (size_t)a.tile_n * GEMM_BLOCK_M * 4;
+  if (tile > data) data = (tile + 1023) / 1024 * 1024;
+  p.data_bytes = (uint32_t)data;
+  const size_t smem = 1024 + data + 16 * stages + 64;
+  if (smem > (size_t)kMaxDynSmem) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((a.E_out + GEMM_BLOCK_M - 1) / GEMM_BLOCK_M, a.n_tiles, a.ksplit);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = a.ksplit;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel, a.tm_w, a.tm_x, p, bp);
 }
 
 }  // namespace vs

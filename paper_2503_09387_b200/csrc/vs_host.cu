@@ -1,9 +1,8 @@
 // Host layer of the C ABI: argument checks, workspace carve-up, launch sequencing.
-// Per frame (Section 3.3, prefilling): pool -> per layer [norm] -> QKV GEMM -> finalize
-// (RoPE, carrier K/V into the bank's free slot) -> attention [-> residual] -> eviction
-// scoring (only when the bank is full) -> bank commit.  Per text step (Section 3.3,
-// decoding): RoPE table -> per layer [norm] -> GEMM -> finalize (K/V appended to prefix or
-// tail) -> attention.  Nothing here allocates device memory or synchronises, except
+// Per frame (Section 3.3, prefilling): pool -> per layer [norm] -> QKV GEMM (epilogue: RoPE,
+// carrier K/V into the bank's free slot) -> attention [-> residual] -> bank update (eviction
+// scoring when the bank is full, then append).  Per text step (Section 3.3, decoding): RoPE
+// table -> per layer [norm] -> GEMM (epilogue: K/V appended to prefix or tail) -> attention.  Nothing here allocates device memory or synchronises, except
 // create / bank_state / last_step_kv.
 #include <cmath>
 #include <cstdio>
@@ -81,7 +80,6 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.hbuf[0] = take((size_t)D.R_max * D.d * 2);
   Lo.hbuf[1] = take((size_t)D.R_max * D.d * 2);
   Lo.xn = take((size_t)D.R_max * D.d * 2);
-  Lo.partials = take((size_t)KSPLIT_MAX * D.R_max * D.E_out * 4);
   Lo.q = take((size_t)D.R_max * D.Hq * D.D * 2);
   Lo.q_lo = take((size_t)D.R_max * D.Hq * D.D * 2);
   Lo.kf = take((size_t)D.R_max * D.Hkv * D.D * 2);
@@ -137,8 +135,8 @@ void choose_tiles(const Dims& D, int rows, int& tile_n, int& n_tiles, int& kspli
   tile_n = (per + 15) / 16 * 16;
   const int m_tiles = (D.E_out + GEMM_BLOCK_M - 1) / GEMM_BLOCK_M;
   const int total_kb = D.d / GEMM_BLOCK_K;
-  ksplit = 1;
-  for (int ks = 1; ks <= KSPLIT_MAX; ++ks) {
+  ksplit = 1;                                  // cluster size along K: 1, 2, 4 or 8
+  for (int ks = 1; ks <= KSPLIT_MAX; ks *= 2) {
     if (total_kb % ks != 0) continue;
     if (m_tiles * n_tiles * ks <= 148) ksplit = ks;
   }
@@ -173,18 +171,19 @@ static_assert(KC_OTHER + 1 == VS_N_KERNEL_CLASSES, "kernel class table");
     (h)->launches[(kc)] += 1;                                                               \
   } while (0)
 
-// QKV projection of `rows` token rows read from `src` ([rows][d] bf16) for layer l.
-int run_projection(vs_stream* h, int l, const bf16* src, int rows, int& ksplit_out, cudaStream_t st) {
+// QKV projection of `rows` token rows read from `src` ([rows][d] bf16) for layer l, finished
+// rows written as `po` says.
+int run_projection(vs_stream* h, int l, const bf16* src, int rows, const ProjectionOut& po, const BatchParams& bp,
+                   cudaStream_t st) {
   const Dims& D = h->dm;
   GemmArgs g;
   choose_tiles(D, rows, g.tile_n, g.n_tiles, g.ksplit);
   g.tm_w = h->tm_w[l];
   if (encode_2d(h, &g.tm_x, src, (uint64_t)D.d, (uint64_t)rows, (uint32_t)g.tile_n) != VS_OK) return VS_ERR_CUDA;
-  g.partials = h->at<float>(h->lo.partials);
+  g.out = po;
   g.rows = rows; g.E_out = D.E_out; g.d = D.d;
   g.status = h->at<int>(h->lo.status);
-  ksplit_out = g.ksplit;
-  VS_LAUNCH(h, st, KC_GEMM, launch_qkv_gemm(g, st));
+  VS_LAUNCH(h, st, KC_GEMM, launch_qkv_gemm(g, bp, st));
   return VS_OK;
 }
 
@@ -332,12 +331,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
       VS_LAUNCH(h, st, KC_RMSNORM, launch_rmsnorm(h_in, h->gain[l], h->at<bf16>(lo.xn), rows, D.d, D.rms_eps, st));
       src = h->at<bf16>(lo.xn);
     }
-    int ksplit = 1;
-    rc = run_projection(h, l, src, rows, ksplit, st);
-    if (rc != VS_OK) return rc;
-
-    FinalizeArgs fa;
-    fa.partials = h->at<float>(lo.partials);
+    ProjectionOut fa;
     fa.bias = h->bias[l];
     fa.rope = h->at<float2>(lo.rope);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
@@ -345,9 +339,9 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     fa.bank_v = h->at<bf16>(lo.bank_v) + (size_t)l * layer_stride_bank(D);
     fa.text_k = nullptr; fa.text_v = nullptr;
     fa.meta = meta;
-    fa.rows = rows; fa.ksplit = ksplit; fa.E_out = D.E_out; fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D;
-    fa.slots = D.slots; fa.text_cap = 0; fa.mode = 0; fa.M = D.M;
-    VS_LAUNCH(h, st, KC_FINALIZE, launch_finalize(fa, bp, st));
+    fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D; fa.slots = D.slots; fa.text_cap = 0; fa.mode = 0; fa.M = D.M;
+    rc = run_projection(h, l, src, rows, fa, bp, st);
+    if (rc != VS_OK) return rc;
 
     AttnArgs aa;
     std::memset(&aa, 0, sizeof(aa));
@@ -437,10 +431,6 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       VS_LAUNCH(h, st, KC_RMSNORM, launch_rmsnorm(h_in, h->gain[l], h->at<bf16>(lo.xn), rows, D.d, D.rms_eps, st));
       src = h->at<bf16>(lo.xn);
     }
-    int ksplit = 1;
-    rc = run_projection(h, l, src, rows, ksplit, st);
-    if (rc != VS_OK) return rc;
-
     bf16* pk = h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D);
     bf16* pv = h->at<bf16>(lo.prefix_v) + (size_t)l * layer_stride_prefix(D);
     bf16* tk = h->at<bf16>(lo.tail_k) + (size_t)l * layer_stride_tail(D);
@@ -448,17 +438,17 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
     bf16* bk = h->at<bf16>(lo.bank_k) + (size_t)l * layer_stride_bank(D);
     bf16* bv = h->at<bf16>(lo.bank_v) + (size_t)l * layer_stride_bank(D);
 
-    FinalizeArgs fa;
-    fa.partials = h->at<float>(lo.partials);
+    ProjectionOut fa;
     fa.bias = h->bias[l];
     fa.rope = h->at<float2>(lo.rope);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
     fa.bank_k = bk; fa.bank_v = bv;
     fa.text_k = to_prefix ? pk : tk; fa.text_v = to_prefix ? pv : tv;
     fa.meta = meta;
-    fa.rows = rows; fa.ksplit = ksplit; fa.E_out = D.E_out; fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D;
-    fa.slots = D.slots; fa.text_cap = to_prefix ? D.maxP : D.maxT; fa.mode = to_prefix ? 1 : 2; fa.M = D.M;
-    VS_LAUNCH(h, st, KC_FINALIZE, launch_finalize(fa, bp, st));
+    fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D; fa.slots = D.slots;
+    fa.text_cap = to_prefix ? D.maxP : D.maxT; fa.mode = to_prefix ? 1 : 2; fa.M = D.M;
+    rc = run_projection(h, l, src, rows, fa, bp, st);
+    if (rc != VS_OK) return rc;
 
     bf16* h_out = D.residual ? h->at<bf16>(lo.hbuf[next_buf]) : nullptr;
     const float scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
@@ -567,7 +557,7 @@ int vs_profile_read(vs_stream* h, double* ms, int64_t* timed, int64_t* launches)
 }
 
 const char* vs_kernel_class_name(int32_t k) {
-  static const char* names[VS_N_KERNEL_CLASSES] = {"pool", "rope_table", "rmsnorm", "qkv_gemm", "finalize",
+  static const char* names[VS_N_KERNEL_CLASSES] = {"pool", "rope_table", "rmsnorm", "qkv_gemm", "unused_a",
                                                    "prefill_attention", "decode_attention", "unused",
                                                    "bank_update", "other"};
   return (k >= 0 && k < VS_N_KERNEL_CLASSES) ? names[k] : "?";

@@ -1,7 +1,6 @@
 // Memory-bound and bookkeeping kernels of the frame / text step:
-//   carrier aggregation (Section 3.3: C = (1/N) sum_i E_i), RoPE table, RMSNorm,
-//   split-K reduction + RoPE + K/V persistence, eviction scoring and bank commit
-//   (Section 3.3, memory mechanism).
+//   carrier aggregation (Section 3.3: C = (1/N) sum_i E_i), RoPE table, RMSNorm, eviction
+//   scoring and bank commit (Section 3.3, memory mechanism).
 #include "vs_common.cuh"
 
 namespace vs {
@@ -153,74 +152,6 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const bf16* __restrict__ h
 cudaError_t launch_rmsnorm(const bf16* h, const bf16* gain, bf16* xn, int rows, int d, float eps,
                            cudaStream_t st) {
   rmsnorm_kernel<<<rows, 256, 0, st>>>(h, gain, xn, d, eps);
-  return cudaGetLastError();
-}
-
-// ------------------------------------------------------------------------------------------
-// Split-K reduction + bias + RoPE + bf16 + persistence of K/V rows.
-// One thread per (row, head slot, rotation pair k): elements k and k + D/2 of one head.
-// Frame step: the carrier row's K/V (last token of each stream's N+1 rows) goes straight
-// into the bank's free slot (Section 3.2: only the carrier keeps its K/V in the cache).
-// Text step: every row's K/V is appended to the prefix or to the turn's tail.
-// ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) finalize_kernel(FinalizeArgs a, BatchParams bp) {
-  const int row = blockIdx.y;
-  const int half = a.D / 2;
-  const int pair = blockIdx.x * blockDim.x + threadIdx.x;
-  const int n_pairs = (a.Hq + 2 * a.Hkv) * half;
-  if (pair >= n_pairs) return;
-  const int hs = pair / half, k = pair - hs * half;
-  const int e1 = hs * a.D + k, e2 = e1 + half;
-  float x1 = 0.f, x2 = 0.f;
-  for (int s = 0; s < a.ksplit; ++s) {
-    const float* p = a.partials + ((size_t)s * a.rows + row) * a.E_out;
-    x1 += p[e1];
-    x2 += p[e2];
-  }
-  if (a.bias != nullptr) {
-    x1 += __bfloat162float(a.bias[e1]);
-    x2 += __bfloat162float(a.bias[e2]);
-  }
-  if (hs < a.Hq + a.Hkv) {
-    const float2 cs = a.rope[(size_t)row * half + k];
-    const float y1 = x1 * cs.x - x2 * cs.y;
-    const float y2 = x2 * cs.x + x1 * cs.y;
-    x1 = y1; x2 = y2;
-  }
-  const bf16 o1 = __float2bfloat16_rn(x1), o2 = __float2bfloat16_rn(x2);
-  if (hs < a.Hq) {
-    // the query never leaves the step, so it is kept as a bf16 pair (hi + lo): the score
-    // Q K^T then sees a 16-bit mantissa instead of 8 at the cost of a second MMA
-    const size_t qo = (size_t)row * a.Hq * a.D + hs * a.D;
-    a.q[qo + k] = o1; a.q[qo + k + half] = o2;
-    a.q_lo[qo + k] = __float2bfloat16_rn(x1 - __bfloat162float(o1));
-    a.q_lo[qo + k + half] = __float2bfloat16_rn(x2 - __bfloat162float(o2));
-    return;
-  }
-  const bool is_k = hs < a.Hq + a.Hkv;
-  const int hkv = is_k ? hs - a.Hq : hs - a.Hq - a.Hkv;
-  bf16* f = (is_k ? a.kf : a.vf) + (size_t)row * a.Hkv * a.D + hkv * a.D;
-  f[k] = o1; f[k + half] = o2;
-  const int rps = bp.rows_per_stream;
-  const int b = row / rps, t = row - b * rps;
-  const int sid = bp.stream_id[b];
-  if (a.mode == 0) {
-    if (t == rps - 1 && a.M > 0) {
-      const int slot = a.meta[sid].free_slot;
-      bf16* dst = (is_k ? a.bank_k : a.bank_v) + (((size_t)sid * a.Hkv + hkv) * a.slots + slot) * a.D;
-      dst[k] = o1; dst[k + half] = o2;
-    }
-  } else {
-    const int base = (a.mode == 1) ? bp.prefix_len[b] : bp.text_len[b];
-    bf16* dst = (is_k ? a.text_k : a.text_v) + (((size_t)sid * a.Hkv + hkv) * a.text_cap + base + t) * a.D;
-    dst[k] = o1; dst[k + half] = o2;
-  }
-}
-
-cudaError_t launch_finalize(const FinalizeArgs& a, const BatchParams& bp, cudaStream_t st) {
-  const int n_pairs = (a.Hq + 2 * a.Hkv) * (a.D / 2);
-  dim3 grid((n_pairs + 255) / 256, a.rows);
-  finalize_kernel<<<grid, 256, 0, st>>>(a, bp);
   return cudaGetLastError();
 }
 
