@@ -125,7 +125,8 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__global__ void __launch_bounds__(kThreads, 1)
+// (two CTAs per SM must fit: see the shared-memory cap at the launch site)
+__global__ void __launch_bounds__(kThreads, 2)
 qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, KernelParams p,
                 BatchParams bp) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -213,34 +214,60 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
       }
       if (ok) umma_commit(tmem_full_bar);   // accumulator complete
     }
-  } else {
-    // epilogue, phase A: accumulator -> this CTA's fp32 partial tile in shared memory,
-    // [token][128 features]; warp w may touch TMEM lanes 32*(w%4) .. +31 (lane = feature).
-    // Every MMA has completed, hence every TMA write has landed and the stages are free.
-    const int quarter = warp & 3;
-    const bool ok = __all_sync(0xffffffffu, mbar_wait(tmem_full_bar, 0, abort_flag));   // warp-uniform
-    tcgen05_fence_after();
-    if (ok) {
-      float* part = reinterpret_cast<float*>(gen_base) + quarter * 32 + lane;
-      for (int c = 0; c < p.tile_n; c += 16) {
-        if (n0 + c >= p.rows) break;               // uniform across the warp
-        uint32_t r[16];
-        tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, r);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-        for (int j = 0; j < 16; ++j) part[(c + j) * GEMM_BLOCK_M] = __uint_as_float(r[j]);
-      }
-    }
   }
 
-  // phase B: every CTA of the cluster has its partial tile in place
+  // ---- epilogue ---------------------------------------------------------------------------
+  // The tile's tokens are cut into ksplit slices; CTA r of the cluster owns slice r.
+  // A  every CTA waits for its own accumulator (all its MMAs done, so all its TMA writes have
+  //    landed and its stages are dead) and copies it, fp32, into its own shared memory as
+  //    [token][128 features]; a cluster barrier publishes the partial tiles.
+  // C  the owner of a slice sums the ksplit partials of its tokens (float4 reads of the peers'
+  //    shared memory), adds the bias, rotates, rounds and stores; a last cluster barrier keeps
+  //    every CTA's shared memory alive until its peers have read it.
+  const int slice = p.tile_n / p.ksplit;          // tile_n is a multiple of 16, ksplit of 1, 2, 4, 8
+  constexpr int kPre = 6;                          // rows whose RoPE entries a thread fetches ahead
+  float4 rope_a[kPre], rope_b[kPre];
+  bool acc_ok = true;
+  if (warp >= 2) {
+    // while the main loop runs: fetch the (cos, sin) entries this thread will need in phase C
+    const int te = threadIdx.x - 64;
+    const int half = p.o.D >> 1;
+    const int p0 = (te & 15) * 4;
+    const int k0 = p0 - (p0 / half) * half;
+#pragma unroll
+    for (int i = 0; i < kPre; ++i) {
+      const int t = (int)blockIdx.z * slice + (te >> 4) + 8 * i;
+      const int row = n0 + t;
+      if (8 * i + (te >> 4) < slice && row < p.rows) {
+        rope_a[i] = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0);
+        rope_b[i] = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0 + 2);
+      } else {
+        rope_a[i] = make_float4(1.f, 0.f, 1.f, 0.f); rope_b[i] = rope_a[i];
+      }
+    }
+    acc_ok = __all_sync(0xffffffffu, mbar_wait(tmem_full_bar, 0, abort_flag));   // warp-uniform
+  }
+  tcgen05_fence_after();
+
+  float* part_local = reinterpret_cast<float*>(gen_base);      // [token][128 features]
+  if (warp >= 2 && acc_ok) {
+    // warp w may touch TMEM lanes 32*(w%4) .. +31 (lane = feature)
+    const int quarter = warp & 3;
+    float* dst = part_local + quarter * 32 + lane;
+    for (int c = 0; c < p.tile_n; c += 16) {
+      if (n0 + c >= p.rows) break;                             // uniform across the warp
+      uint32_t r[16];
+      tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, r);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+      for (int j = 0; j < 16; ++j) dst[(c + j) * GEMM_BLOCK_M] = __uint_as_float(r[j]);
+    }
+  }
   tcgen05_fence_before();
   __syncthreads();
   if (p.ksplit > 1) cluster_sync_all();
 
-  // phase C: CTA r reduces token slice r, finishes the rows and stores them.  Thread =
-  // (group of 4 rotation pairs, token lane): float4 reads of every CTA's partial tile through
-  // distributed shared memory, all issued before they are summed.
+  // phase C.  Thread = (group of 4 rotation pairs, token lane); float4 reads.
   if (warp >= 2 && !*abort_flag) {
     const int te = threadIdx.x - 64;               // 0..127
     const int D = p.o.D, half = D >> 1;
@@ -248,10 +275,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
     const int hl = p0 / half, k0 = p0 - hl * half; // local head, index inside the half head
     const int f1 = hl * D + k0, f2 = f1 + half;
     const int hs = (m0 + f1) / D;                  // head slot: Q heads, then K heads, then V heads
-    const int slice = (p.tile_n + p.ksplit - 1) / p.ksplit;
     const int t_begin = (int)blockIdx.z * slice;
-    const int t_end = min(t_begin + slice, p.tile_n);
-    const float* part_local = reinterpret_cast<const float*>(gen_base);
     const float* part[8];
     cg::cluster_group cluster = cg::this_cluster();
 #pragma unroll
@@ -267,7 +291,9 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
         }
       }
       const int rps = bp.rows_per_stream;
-      for (int t = t_begin + (te >> 4); t < t_end; t += 8) {
+#pragma unroll 1
+      for (int it = 0; it * 8 + (te >> 4) < slice; ++it) {
+        const int t = t_begin + (te >> 4) + 8 * it;
         const int row = n0 + t;
         if (row >= p.rows) break;
         float4 v1[8], v2[8];
@@ -287,8 +313,15 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
           }
         }
         if (hs < p.o.Hq + p.o.Hkv) {
-          const float4 ra = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0);
-          const float4 rb = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0 + 2);
+          float4 ra, rb;
+          if (it < kPre) {
+            ra = rope_a[0]; rb = rope_b[0];
+#pragma unroll
+            for (int i = 1; i < kPre; ++i) if (i == it) { ra = rope_a[i]; rb = rope_b[i]; }
+          } else {
+            ra = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0);
+            rb = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0 + 2);
+          }
           const float cs[4] = {ra.x, ra.z, rb.x, rb.z}, sn[4] = {ra.y, ra.w, rb.y, rb.w};
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
