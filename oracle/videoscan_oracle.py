@@ -245,6 +245,8 @@ class OracleStream:
         self.evictions = 0
         self.evict_log: List[tuple] = []        # (frame step, victim frame id)
         self.last_victim_frame = -1
+        # test aid: when set to a list, every step appends {"kind", "h": [layer inputs], "O": [layer outputs]}
+        self.record: Optional[list] = None
 
     # -- pieces -------------------------------------------------------------------------
     def _layer_input(self, h: np.ndarray, layer: int) -> np.ndarray:
@@ -303,7 +305,9 @@ class OracleStream:
             cK = np.zeros((L, Hkv, D))
             cV = np.zeros((L, Hkv, D))
             h = X
+            rec = {"kind": "frame", "h": [], "O": []}
             for l in range(L):
+                rec["h"].append(h)
                 Q, K, V = self._project(self._layer_input(h, l), l)
                 Q = apply_rope(Q, ang)
                 K = apply_rope(K, ang)
@@ -317,8 +321,11 @@ class OracleStream:
                 cK[l] = round_to_bf16(K[N])
                 cV[l] = round_to_bf16(V[N])
                 out = O
+                rec["O"].append(O)
                 if cfg.residual:
                     h = round_to_bf16(h + O)
+            if self.record is not None:
+                self.record.append(rec)
         elif mode == "carrier":
             if L != 1 or cfg.use_rmsnorm:
                 raise ValueError("carrier-only mode needs a single layer without norm")
@@ -359,7 +366,9 @@ class OracleStream:
         ang = rope_angles([base + i for i in range(T)], D, cfg.rope_theta)
         h = X
         out = None
+        rec = {"kind": "text", "h": [], "O": []}
         for l in range(L):
+            rec["h"].append(h)
             Q, K, V = self._project(self._layer_input(h, l), l)
             Q = apply_rope(Q, ang)
             K = round_to_bf16(apply_rope(K, ang))
@@ -381,8 +390,11 @@ class OracleStream:
                 self.tail_K[l] = np.concatenate([self.tail_K[l], K], axis=0)
                 self.tail_V[l] = np.concatenate([self.tail_V[l], V], axis=0)
             out = O
+            rec["O"].append(O)
             if cfg.residual:
                 h = round_to_bf16(h + O)
+        if self.record is not None:
+            self.record.append(rec)
         if to_prefix:
             self.next_pos += T
         else:

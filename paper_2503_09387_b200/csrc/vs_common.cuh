@@ -75,7 +75,8 @@ struct Layout {
   size_t persistent_end;
   // per-step scratch
   size_t hbuf[2];               // bf16 [R_max][d]  residual ping-pong; hbuf[0] holds [E; carrier]
-  size_t xn;                    // bf16 [R_max][d]  normalised layer input
+  size_t xn;                    // bf16 [R_max][d]  layer input times the RMSNorm gain (only with a gain vector)
+  size_t row_scale;             // f32  [R_max]     RMSNorm row scales
   size_t q;                     // bf16 [R_max][Hq*D]
   size_t q_lo;                  // bf16 [R_max][Hq*D]  low-order half of the rotated query
   size_t kf, vf;                // bf16 [R_max][Hkv*D]
@@ -106,12 +107,13 @@ struct RopeArgs {
 };
 cudaError_t launch_rope_table(const RopeArgs& a, const BatchParams& bp, cudaStream_t st);
 
-cudaError_t launch_rmsnorm(const bf16* h, const bf16* gain, bf16* xn, int rows, int d, float eps,
-                           cudaStream_t st);
+cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* row_scale, int rows, int d,
+                             float eps, cudaStream_t st);
 
 // What the projection epilogue writes (finished rows: bias, RoPE, bf16) and where rows persist.
 struct ProjectionOut {
   const bf16* bias;              // [E_out] or null
+  const float* row_scale;        // [rows] RMSNorm scale applied to the accumulated row, or null
   const float2* rope;            // [rows][D/2] (cos, sin)
   bf16* q;                       // [rows][Hq*D]  rotated query, leading bf16 part
   bf16* q_lo;                    // [rows][Hq*D]  bf16(query - q): the pair carries 16 mantissa bits

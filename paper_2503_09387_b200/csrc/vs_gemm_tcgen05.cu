@@ -304,7 +304,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
             v2[r] = *reinterpret_cast<const float4*>(part[r] + t * GEMM_BLOCK_M + f2);
           }
         }
-        float x1[4] = {bb1[0], bb1[1], bb1[2], bb1[3]}, x2[4] = {bb2[0], bb2[1], bb2[2], bb2[3]};
+        float x1[4] = {0.f, 0.f, 0.f, 0.f}, x2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int r = 0; r < 8; ++r) {
           if (r < p.ksplit) {
@@ -312,6 +312,10 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
             x2[0] += v2[r].x; x2[1] += v2[r].y; x2[2] += v2[r].z; x2[3] += v2[r].w;
           }
         }
+        // RMSNorm's row scale commutes with the projection: applied here, in fp32
+        const float rsc = (p.o.row_scale != nullptr) ? p.o.row_scale[row] : 1.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { x1[i] = fmaf(x1[i], rsc, bb1[i]); x2[i] = fmaf(x2[i], rsc, bb2[i]); }
         if (hs < p.o.Hq + p.o.Hkv) {
           float4 ra, rb;
           if (it < kPre) {

@@ -80,6 +80,7 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.hbuf[0] = take((size_t)D.R_max * D.d * 2);
   Lo.hbuf[1] = take((size_t)D.R_max * D.d * 2);
   Lo.xn = take((size_t)D.R_max * D.d * 2);
+  Lo.row_scale = take((size_t)D.R_max * 4);
   Lo.q = take((size_t)D.R_max * D.Hq * D.D * 2);
   Lo.q_lo = take((size_t)D.R_max * D.Hq * D.D * 2);
   Lo.kf = take((size_t)D.R_max * D.Hkv * D.D * 2);
@@ -328,11 +329,13 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     const bf16* h_in = h->at<bf16>(lo.hbuf[cur]);
     const bf16* src = h_in;
     if (D.use_rmsnorm) {
-      VS_LAUNCH(h, st, KC_RMSNORM, launch_rmsnorm(h_in, h->gain[l], h->at<bf16>(lo.xn), rows, D.d, D.rms_eps, st));
-      src = h->at<bf16>(lo.xn);
+      VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_scale),
+                                                    rows, D.d, D.rms_eps, st));
+      if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
     }
     ProjectionOut fa;
     fa.bias = h->bias[l];
+    fa.row_scale = D.use_rmsnorm ? h->at<float>(lo.row_scale) : nullptr;
     fa.rope = h->at<float2>(lo.rope);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
     fa.bank_k = h->at<bf16>(lo.bank_k) + (size_t)l * layer_stride_bank(D);
@@ -428,8 +431,9 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
   for (int l = 0; l < D.L; ++l) {
     const bf16* src = h_in;
     if (D.use_rmsnorm) {
-      VS_LAUNCH(h, st, KC_RMSNORM, launch_rmsnorm(h_in, h->gain[l], h->at<bf16>(lo.xn), rows, D.d, D.rms_eps, st));
-      src = h->at<bf16>(lo.xn);
+      VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_scale),
+                                                    rows, D.d, D.rms_eps, st));
+      if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
     }
     bf16* pk = h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D);
     bf16* pv = h->at<bf16>(lo.prefix_v) + (size_t)l * layer_stride_prefix(D);
@@ -440,6 +444,7 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
 
     ProjectionOut fa;
     fa.bias = h->bias[l];
+    fa.row_scale = D.use_rmsnorm ? h->at<float>(lo.row_scale) : nullptr;
     fa.rope = h->at<float2>(lo.rope);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
     fa.bank_k = bk; fa.bank_v = bv;

@@ -118,40 +118,42 @@ cudaError_t launch_rope_table(const RopeArgs& a, const BatchParams& bp, cudaStre
 }
 
 // ------------------------------------------------------------------------------------------
-// RMSNorm of the layer input: xn = h / sqrt(mean(h^2) + eps) * gain.  One block per row.
+// RMSNorm statistics of the layer input.  xn = h * r * gain with r = 1 / sqrt(mean(h^2) + eps).
+// The row scale r commutes with the projection, so it is applied in fp32 in the GEMM epilogue
+// and the GEMM reads the bf16 residual stream itself: no rounded copy of the normalised
+// activations exists (with a gain vector, bf16(h * gain) is written and read instead).
+// One block per row.
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) rmsnorm_kernel(const bf16* __restrict__ h, const bf16* __restrict__ gain,
-                                                      bf16* __restrict__ xn, int d, float eps) {
+__global__ void __launch_bounds__(256) rms_stats_kernel(const bf16* __restrict__ h, const bf16* __restrict__ gain,
+                                                        bf16* __restrict__ hg, float* __restrict__ row_scale,
+                                                        int d, float eps) {
   const size_t row = blockIdx.x;
   const bf16* src = h + row * d;
   float ss = 0.f;
   for (int c = threadIdx.x * 2; c < d; c += 512) {
     const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(src + c));
     ss += v.x * v.x + v.y * v.y;
+    if (gain != nullptr) {
+      const float2 g = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(gain + c));
+      *reinterpret_cast<__nv_bfloat162*>(hg + row * d + c) = __floats2bfloat162_rn(v.x * g.x, v.y * g.y);
+    }
   }
   __shared__ float red[8];
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
-  float tot = 0.f;
+  if (threadIdx.x == 0) {
+    float tot = 0.f;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) tot += red[i];
-  const float r = rsqrtf(tot / (float)d + eps);
-  for (int c = threadIdx.x * 2; c < d; c += 512) {
-    float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(src + c));
-    v.x *= r; v.y *= r;
-    if (gain != nullptr) {
-      const float2 g = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(gain + c));
-      v.x *= g.x; v.y *= g.y;
-    }
-    *reinterpret_cast<__nv_bfloat162*>(xn + row * d + c) = __floats2bfloat162_rn(v.x, v.y);
+    for (int i = 0; i < 8; ++i) tot += red[i];
+    row_scale[row] = rsqrtf(tot / (float)d + eps);
   }
 }
 
-cudaError_t launch_rmsnorm(const bf16* h, const bf16* gain, bf16* xn, int rows, int d, float eps,
-                           cudaStream_t st) {
-  rmsnorm_kernel<<<rows, 256, 0, st>>>(h, gain, xn, d, eps);
+cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* row_scale, int rows, int d, float eps,
+                             cudaStream_t st) {
+  rms_stats_kernel<<<rows, 256, 0, st>>>(h, gain, hg, row_scale, d, eps);
   return cudaGetLastError();
 }
 

@@ -172,3 +172,129 @@ def test_one_layer_qwen_shape_full_stream():
     assert st["count"] == 64 and st["persistent_bytes"] < st["workspace_bytes"]
     print("worst errors (max_abs, rel_rms):", p.worst)
     p.close()
+
+
+# ------------------------------------------------------------------ full-size workloads
+def test_long_stream_full_size_sampled():
+    """1024 frames x 169 tokens, bank 256 (768 evictions), 64-token question, 64 decode tokens.
+    Bank bookkeeping, eviction trace, embeddings and K/V are checked over the WHOLE stream (the
+    oracle projects only the carrier row on frames that are not sampled); full attention parity
+    on a seeded sample: first and last frames, both sides of the first eviction, random rest."""
+    w = synth.workload("long")
+    p = Pair(w, max_text=w.question_len + w.decode_tokens)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    shared = w.frame_shared()
+    rng = np.random.default_rng(3)
+    sample = {0, 1, 2, 254, 255, 256, 257, 258, 511, 1021, 1022, 1023} | set(rng.integers(3, 1021, 22).tolist())
+    for t in range(w.n_frames):
+        full = t in sample
+        p.frame([0], [w.frame_hidden(t, shared=shared)], f"frame {t}", mode="full" if full else "carrier")
+        if full or t % 128 == 0:
+            p.check_bank(0)
+    st = p.check_bank(0)
+    assert st["count"] == 256 and st["evictions"] == 768 and st["frames_seen"] == 1024
+    assert len(set(p.ora[0].bank_frame_ids()) - set(range(768, 1024))) > 0       # not plain FIFO
+    p.text([0], [w.question_hidden()], "question")
+    for i in range(w.decode_tokens):
+        p.text([0], [w.decode_hidden(i)], f"decode {i}")
+    p.check_bank(0)
+    print("long: sampled frames", sorted(sample), "worst", p.worst)
+    p.close()
+
+
+# Chained layers.  Both sides store the residual stream in bf16.  A difference of ~2e-3 in one
+# layer's attention output flips the bf16 rounding of h + O for roughly one element in eight
+# (spacing 1.6e-2 at |h| ~ 3), i.e. it injects noise of the size of one more bf16 rounding per
+# layer, which the next layer's logits (std ~ 19 with N(0, 0.02) weights) amplify.  The
+# per-operation tolerance therefore cannot hold for the 28th layer of a free-running chain; it is
+# checked layer by layer with the oracle's own layer inputs fed to a one-layer handle (below), and
+# the free-running chain gets the depth-scaled bound max |err| <= 2e-2 * sqrt(L), rel RMS <= 2e-2.
+def chain_bounds(n_layers):
+    return 2e-2 * np.sqrt(n_layers), 2e-2
+
+
+def run_chain(w, max_text):
+    """Free-running multi-layer stream on both sides; returns the oracle's per-layer record."""
+    from tests import parity
+    p = Pair(w, max_text=max_text)
+    p.ora[0].record = []
+    saved = (parity.MAX_ABS, parity.REL_RMS)
+    parity.MAX_ABS, parity.REL_RMS = chain_bounds(w.n_layers)
+    try:
+        steps = [("text", w.prefix_hidden(), None)]
+        p.text([0], [w.prefix_hidden()], "prefix")
+        shared = w.frame_shared()
+        for t in range(w.n_frames):
+            x = w.frame_hidden(t, shared=shared)
+            p.frame([0], [x], f"frame {t}")
+        if w.question_len:
+            p.text([0], [w.question_hidden()], "question")
+        for i in range(w.decode_tokens):
+            p.text([0], [w.decode_hidden(i)], f"decode {i}")
+        for layer in sorted({0, w.n_layers // 2, w.n_layers - 1}):
+            p.check_bank(0, layer=layer)
+    finally:
+        parity.MAX_ABS, parity.REL_RMS = saved
+    rec = p.ora[0].record
+    worst = list(p.worst)
+    p.close()
+    return rec, worst
+
+
+def teacher_forced_layer(w, layer, rec):
+    """One-layer handle holding layer `layer`'s weights, fed the oracle's inputs of that layer
+    (bf16 values: the residual stream is a storage point); outputs must meet the strict tolerance."""
+    from oracle import videoscan_oracle as vo
+    w1 = synth.workload(w.name, n_layers=1, n_frames=w.n_frames, decode_tokens=w.decode_tokens,
+                        question_len=w.question_len, tokens_per_frame=w.tokens_per_frame, d_model=w.d_model,
+                        n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
+                        bank_capacity=w.bank_capacity, prefix_len=w.prefix_len, seed=w.seed)
+    cfg = binding.make_config(1, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens_per_frame,
+                              max(w.prefix_len, 1), max(w.question_len + w.decode_tokens, 1), w.bank_capacity,
+                              use_rmsnorm=w.use_rmsnorm, residual=w.residual, rope_theta=w.rope_theta,
+                              rms_eps=w.rms_eps)
+    sb = binding.StreamBatch(cfg, [to_dev(w.weight(layer))])
+    worst = [0.0, 0.0]
+    for i, r in enumerate(rec):
+        h = vo.bf16_bits_of(r["h"][layer])
+        if r["kind"] == "text":
+            got = to_f64(sb.decode_step([0], to_dev(h[None])))[0]
+        else:
+            got = to_f64(sb.frame_prefill([0], to_dev(h[None, :-1]), carrier_override=to_dev(h[None, -1])))[0]
+        e = assert_close(got, r["O"][layer], f"layer {layer} step {i} ({r['kind']})")
+        worst = [max(worst[0], e[0]), max(worst[1], e[1])]
+    sb.close()
+    return worst
+
+
+def test_deep_stack_full_shape_first_frames():
+    """28 layers at the Qwen2-7B shape (RMSNorm, residual, no MLP), bank 512: the first 6 frames,
+    the 32-token question and 4 decode tokens, free-running and teacher-forced per layer."""
+    w = synth.workload("deep", n_frames=6, decode_tokens=4)
+    rec, worst = run_chain(w, w.question_len + w.decode_tokens)
+    print("deep chain: worst", worst)
+    for layer in (0, 1, 13, 27):
+        print("deep layer", layer, "teacher-forced worst", teacher_forced_layer(w, layer, rec))
+
+
+def test_batched_streams_full_shape():
+    """16 streams x 196 tokens at the Qwen2-7B shape, bank capacity 1024, ragged lengths (scaled to
+    [6, 24] frames so the oracle finishes in seconds), then batched single-token decode."""
+    w = synth.workload("batched", n_frames=24, min_frames=6, decode_tokens=4)
+    lengths = w.stream_lengths()
+    p = Pair(w)
+    ids = list(range(w.n_streams))
+    p.text(ids, [w.prefix_hidden(s) for s in ids], "prefix")
+    shared = [w.frame_shared(s) for s in ids]
+    for t in range(max(lengths)):
+        act = [s for s in ids if lengths[s] > t]
+        full = t in (0, 5, max(lengths) - 1) or len(act) < 4
+        p.frame(act, [w.frame_hidden(t, s, shared=shared[s]) for s in act], f"frame {t}",
+                mode="full" if full else "carrier")
+    for i in range(w.decode_tokens):
+        p.text(ids, [w.decode_hidden(i, s) for s in ids], f"decode {i}")
+    for s in ids:
+        st = p.check_bank(s)
+        assert st["frames_seen"] == lengths[s] and st["count"] == lengths[s]
+    print("batched: lengths", lengths, "worst", p.worst)
+    p.close()
