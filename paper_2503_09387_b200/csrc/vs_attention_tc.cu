@@ -3,24 +3,25 @@
 //
 // One CTA = 16 query tokens x one KV head x one stream.  The G query heads of the group are
 // stacked on the MMA's M axis (row = g * 16 + token, G * 16 <= 128), so K and V are staged
-// once for the whole group and one thread owns one row: its maximum, its sum and its 128
-// output values live in that thread's registers and need no shuffles.
-// Per 64-key tile:  S = Q K^T  (tcgen05.mma, M 128 x N 64, Q as a bf16 hi + lo pair)  -> TMEM
-//                   softmax of the row in registers, P (bf16) -> shared memory
-//                   O_tile = P V (tcgen05.mma, M 128 x N D, V read MN-major)          -> TMEM
-//                   o_row = o_row * alpha + O_tile                                       (registers)
-// Key tiles come from up to four segments: prompt prefix, carrier bank (the free slot is
-// masked), earlier text of the turn, and the step's own rows (causal).  The carrier is the
-// last row of its frame (Section 3.2), so the causal rule alone gives it the whole frame.
-// K/V tiles are fetched with cp.async into the 128-byte-swizzled layout the MMA descriptors
-// expect and are double buffered.  All mbarrier waits are bounded.
+// once for the whole group.  Keys come from up to four segments -- prompt prefix, carrier bank
+// (the free slot is masked), earlier text of the turn, the step's own rows (causal) -- laid end
+// to end and cut into dense tiles of 128 keys.  The carrier is the last row of its frame
+// (Section 3.2), so the causal rule alone gives it the whole frame.
+// Per tile:  S = Q K^T  (tcgen05.mma, M 128 x N 128, Q as a bf16 hi + lo pair)     -> TMEM
+//            softmax of the row in registers, P (bf16) -> shared memory (over the dead K tile)
+//            O_tile = P V  (tcgen05.mma, M 128 x N D, V read MN-major)             -> TMEM
+//            o_row = o_row * alpha + O_tile                                          (registers)
+// Warps 0..7: two threads per row (each owns 64 keys of a tile and D/2 output dims), they also
+// fetch K/V with cp.async into the 128-byte-swizzled layout the MMA descriptors expect.
+// Warp 8: one thread issues every MMA, one tile of Q K^T ahead of the softmax (S is double
+// buffered in TMEM).  All mbarrier waits are bounded.
 #include "vs_common.cuh"
 
 namespace vs {
 
 namespace {
 
-constexpr int kKeys = 64;        // keys per tile
+constexpr int kKeys = 128;       // keys per tile
 constexpr int kRows = 128;       // MMA M
 constexpr int kTok = 16;         // query tokens per CTA
 constexpr unsigned long long kWaitLimitNs = 400ull * 1000ull * 1000ull;
@@ -127,14 +128,14 @@ template <int D>
 struct Smem {
   static constexpr int kQBytes = kRows * D * 2;           // one of hi / lo
   static constexpr int kKVBytes = kKeys * D * 2;          // one of K / V, one stage
-  static constexpr int kPBytes = kRows * kKeys * 2;
   static constexpr int kQhi = 0;
   static constexpr int kQlo = kQBytes;
-  static constexpr int kKV = 2 * kQBytes;                 // [stage][K | V]
-  static constexpr int kStages = 3;
-  static constexpr int kP = kKV + 2 * kStages * kKVBytes;
-  static constexpr int kMax = kP + kPBytes;               // float [2][128]: row maxima of the two key halves
-  static constexpr int kCtl = kMax + 2048;                // (two parities of the maxima)                // barriers, tmem slot, abort flag
+  static constexpr int kPBytes = kRows * kKeys * 2;
+  static constexpr int kKStage = kKVBytes > kPBytes ? kKVBytes : kPBytes;   // K tile; P is written over it once S is done
+  static constexpr int kK = 2 * kQBytes;                  // [stage] K tile / P
+  static constexpr int kV = kK + 2 * kKStage;             // [stage] V tile
+  static constexpr int kMax = kV + 2 * kKVBytes;          // float [2][2][128]: row maxima exchange
+  static constexpr int kCtl = kMax + 2048;                // barriers, tmem slot, abort flag
   static constexpr int kTotal = kCtl + 64 + 1024;         // + alignment slack
 };
 
@@ -143,20 +144,38 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// barrier 1 over the 256 softmax threads, AND-reducing a predicate (keeps their exits uniform)
+__device__ __forceinline__ bool softmax_barrier_and(bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, 256, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"((uint32_t)pred) : "memory");
+  return r != 0;
+}
 
-// 256 threads: two threads per row of the stacked query block.  Thread (row, half) owns keys
-// [32*half, 32*half + 32) of every S tile and output dims [D/2*half, D/2*half + D/2).
+constexpr int kSoftmaxThreads = 256;
+constexpr int kAttnThreads = kSoftmaxThreads + 32;
+
 template <int D>
-__global__ void __launch_bounds__(256, 1) prefill_attn_tc_kernel(AttnArgs a, BatchParams bp, int* status) {
+__global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnArgs a, BatchParams bp, int* status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   using L = Smem<D>;
   constexpr int CPR = D / 8;
   constexpr int DH = D / 2;
+  constexpr int KH = kKeys / 2;                 // keys of a tile owned by one thread of a row pair
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t bar_s0 = base + L::kCtl, bar_o = base + L::kCtl + 16;   // bar_s0, bar_s0 + 8: the two S buffers
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + L::kCtl + 24);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kCtl + 28);
+  const uint32_t bar_s0 = base + L::kCtl;       // +0, +8: S buffer ready (tcgen05.commit)
+  const uint32_t bar_o = base + L::kCtl + 16;   // O tile ready (tcgen05.commit)
+  const uint32_t bar_p = base + L::kCtl + 24;   // P written and next K/V tile landed (256 arrivals)
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + L::kCtl + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kCtl + 36);
   float* max_x = reinterpret_cast<float*>(gbase + L::kMax);
 
   const int b = blockIdx.z, hkv = blockIdx.y;
@@ -165,58 +184,58 @@ __global__ void __launch_bounds__(256, 1) prefill_attn_tc_kernel(AttnArgs a, Bat
   const int sid = bp.stream_id[b];
   const int G = a.Hq / a.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5;
-  const int row = tid & 127, half = tid >> 7;
+  const bool is_softmax = tid < kSoftmaxThreads;
+  const int row = tid & 127, half = (tid >> 7) & 1;
   const int count = bp.count[b];
   const bool bank_full = (a.M > 0 && count == a.M);
-  const int free_slot = bank_full ? a.meta[sid].free_slot : -1;
 
   const int g = row >> 4;
   const int tok = r0 + (row & 15);
-  const bool row_valid = (g < G) && (tok < rps);
+  const bool row_valid = is_softmax && (g < G) && (tok < rps);
 
-  int seg_len[4], seg_kind[4], seg_chunk0[5];
+  // ---- the virtual key axis: segments end to end ----------------------------------------------
+  int seg_end[4];                                // exclusive prefix sums of the segment lengths
   const bf16* seg_k[4];
   const bf16* seg_v[4];
   long long seg_stride[4];
-  int n_chunks = 0;
+  int total = 0, causal_start = 0x3fffffff, hole = -1;
 #pragma unroll
   for (int s = 0; s < 4; ++s) {
-    seg_len[s] = 0; seg_kind[s] = 0; seg_k[s] = nullptr; seg_v[s] = nullptr; seg_stride[s] = 0;
-    seg_chunk0[s] = n_chunks;
+    seg_k[s] = nullptr; seg_v[s] = nullptr; seg_stride[s] = 0;
     if (s < a.n_seg) {
       const AttnSegment sg = a.seg[s];
       int len;
       if (sg.kind == 0) len = bp.prefix_len[b];
-      else if (sg.kind == 1) len = (a.M == 0) ? 0 : (bank_full ? a.M + 1 : count);
+      else if (sg.kind == 1) {
+        len = (a.M == 0) ? 0 : (bank_full ? a.M + 1 : count);
+        if (bank_full) hole = total + a.meta[sid].free_slot;     // the slot being refilled holds no carrier
+      }
       else if (sg.kind == 2) len = bp.text_len[b];
-      else len = min(rps, r0 + kTok);            // causal: later keys are visible to no row of this tile
+      else { len = min(rps, r0 + kTok); causal_start = total; }  // later keys are visible to no row of this tile
       const long long off = (long long)(sg.by_batch ? b : sid) * sg.stream_stride + (long long)hkv * sg.head_stride;
-      seg_len[s] = len; seg_kind[s] = sg.kind; seg_k[s] = sg.k + off; seg_v[s] = sg.v + off;
-      seg_stride[s] = sg.row_stride;
-      n_chunks += (len + kKeys - 1) / kKeys;
+      seg_k[s] = sg.k + off; seg_v[s] = sg.v + off; seg_stride[s] = sg.row_stride;
+      total += len;
     }
+    seg_end[s] = total;
   }
-  seg_chunk0[4] = n_chunks;
-  auto locate = [&](int ci, int& s, int& start) {
-    s = 0;
-#pragma unroll
-    for (int t = 1; t < 4; ++t) if (ci >= seg_chunk0[t]) s = t;
-    start = (ci - seg_chunk0[s]) * kKeys;
-  };
-  auto load_chunk = [&](int ci, int stage) {
-    int s, start;
-    locate(ci, s, start);
-    const bf16* kp = seg_k[s]; const bf16* vp = seg_v[s];
-    const long long stride = seg_stride[s];
-    const int len = seg_len[s];
-    const uint32_t kdst = base + L::kKV + (uint32_t)stage * 2u * L::kKVBytes;
-    const uint32_t vdst = kdst + L::kKVBytes;
-    for (int idx = tid; idx < kKeys * CPR; idx += 256) {
+  const int n_tiles = (total + kKeys - 1) / kKeys;
+
+  auto load_tile = [&](int ti, int stage) {
+    const uint32_t kdst = base + L::kK + (uint32_t)stage * L::kKStage;
+    const uint32_t vdst = base + L::kV + (uint32_t)stage * L::kKVBytes;
+    for (int idx = tid; idx < kKeys * CPR; idx += kSoftmaxThreads) {
       const int r = idx / CPR, c = idx - r * CPR;
-      const bool valid = (start + r) < len;
-      const long long goff = valid ? ((long long)(start + r) * stride + c * 8) : 0;
-      cp_async16(kdst + sw_off<kKeys>(r, c), kp + goff, valid);
-      cp_async16(vdst + sw_off<kKeys>(r, c), vp + goff, valid);
+      const int v = ti * kKeys + r;
+      int s = 0;
+#pragma unroll
+      for (int t = 0; t < 3; ++t) if (v >= seg_end[t]) s = t + 1;
+      const bool valid = v < total;
+      const bf16* kp = seg_k[0]; const bf16* vp = seg_v[0]; long long stride = seg_stride[0]; int first = 0;
+#pragma unroll
+      for (int t = 1; t < 4; ++t) if (s == t) { kp = seg_k[t]; vp = seg_v[t]; stride = seg_stride[t]; first = seg_end[t - 1]; }
+      const long long goff = valid ? ((long long)(v - first) * stride + c * 8) : 0;
+      cp_async16(kdst + sw_off<kKeys>(r, c), (valid ? kp : a.q) + goff, valid);
+      cp_async16(vdst + sw_off<kKeys>(r, c), (valid ? vp : a.q) + goff, valid);
     }
   };
 
@@ -225,188 +244,201 @@ __global__ void __launch_bounds__(256, 1) prefill_attn_tc_kernel(AttnArgs a, Bat
     mbar_init(bar_s0, 1);
     mbar_init(bar_s0 + 8, 1);
     mbar_init(bar_o, 1);
+    mbar_init(bar_p, kSoftmaxThreads);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 0) {
+  if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32((const void*)tmem_slot)), "r"(256u) : "memory");
+                 ::"r"(smem_u32((const void*)tmem_slot)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  for (int idx = tid; idx < kRows * CPR; idx += 256) {
-    const int r = idx / CPR, c = idx - r * CPR;
-    const int gg = r >> 4, tt = r0 + (r & 15);
-    const bool valid = (gg < G) && (tt < rps);
-    const size_t off = valid ? (((size_t)b * rps + tt) * a.Hq + (size_t)hkv * G + gg) * D + c * 8 : 0;
-    cp_async16(base + L::kQhi + sw_off<kRows>(r, c), a.q + off, valid);
-    cp_async16(base + L::kQlo + sw_off<kRows>(r, c), a.q_lo + off, valid);
+  if (is_softmax) {
+    for (int idx = tid; idx < kRows * CPR; idx += kSoftmaxThreads) {
+      const int r = idx / CPR, c = idx - r * CPR;
+      const int gg = r >> 4, tt = r0 + (r & 15);
+      const bool valid = (gg < G) && (tt < rps);
+      const size_t off = valid ? (((size_t)b * rps + tt) * a.Hq + (size_t)hkv * G + gg) * D + c * 8 : 0;
+      cp_async16(base + L::kQhi + sw_off<kRows>(r, c), a.q + off, valid);
+      cp_async16(base + L::kQlo + sw_off<kRows>(r, c), a.q_lo + off, valid);
+    }
+    load_tile(0, 0);
+    cp_async_commit();                                   // group: Q + tile 0
+    if (n_tiles > 1) load_tile(1, 1);
+    cp_async_commit();                                   // group: tile 1
+    cp_async_wait<1>();
+    fence_async_proxy();                                 // cp.async writes -> visible to the tensor-core proxy
   }
-  if (n_chunks > 0) load_chunk(0, 0);
-  cp_async_commit();                                   // group 0: Q + tile 0
-  if (n_chunks > 1) load_chunk(1, 1);
-  cp_async_commit();                                   // group 1: tile 1
-  cp_async_wait<1>();
-  fence_async_proxy();                                 // cp.async writes -> visible to the tensor-core proxy
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_o = tmem + 128;                  // S buffers at columns 0 and 64
-  const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;   // warp w may touch TMEM lanes 32*(w%4)..+31
+  const uint32_t tmem_o = tmem + 256;                    // S buffers at columns 0 and 128
 
-  float o_acc[DH];
+  if (warp == 8) {
+    // ---- MMA issuer -----------------------------------------------------------------------------
+    if ((tid & 31) == 0) {
+      const uint32_t idesc_qk = make_idesc(kKeys, 0);
+      const uint32_t idesc_pv = make_idesc(D, 1);
+      auto issue_qk = [&](int t) {
+        const uint32_t k_addr = base + L::kK + (uint32_t)(t & 1) * L::kKStage;
+        const uint32_t tmem_s = tmem + 128u * (uint32_t)(t & 1);
 #pragma unroll
-  for (int i = 0; i < DH; ++i) o_acc[i] = 0.f;
-  float m_run = -INFINITY, l_run = 0.f;      // m_run in the log2 domain (score * scale_log2e)
-  const uint32_t idesc_qk = make_idesc(kKeys, 0);
-  const uint32_t idesc_pv = make_idesc(D, 1);
-  const float scale = a.scale_log2e;
-  bool ok = true;
-
-  // S(c) = Q K(c)^T into S buffer c&1; issued one tile ahead of its softmax
-  auto issue_qk = [&](int c) {
-    const uint32_t k_addr = base + L::kKV + (uint32_t)(c % L::kStages) * 2u * L::kKVBytes;
-    const uint32_t tmem_s = tmem + 64u * (uint32_t)(c & 1);
+        for (int ks = 0; ks < D / 16; ++ks) {
+          // k-step ks: block ks/4 of 64 elements, 32 bytes per step inside the 128-byte row
+          const uint32_t qo = (uint32_t)(ks >> 2) * (kRows * 128) + (uint32_t)(ks & 3) * 32u;
+          const uint32_t ko = (uint32_t)(ks >> 2) * (kKeys * 128) + (uint32_t)(ks & 3) * 32u;
+          const uint64_t dk = make_desc(k_addr + ko, 16, 1024);
+          umma(tmem_s, make_desc(base + L::kQhi + qo, 16, 1024), dk, idesc_qk, ks != 0);
+          umma(tmem_s, make_desc(base + L::kQlo + qo, 16, 1024), dk, idesc_qk, 1);
+        }
+        umma_commit(bar_s0 + 8u * (uint32_t)(t & 1));
+      };
+      issue_qk(0);
+      for (int ti = 0; ti < n_tiles; ++ti) {
+        if (!mbar_wait(bar_p, (uint32_t)(ti & 1), abort_flag)) break;   // P(ti) in place, tile ti+1 landed
+        tc_fence_after();
+        const uint32_t p_addr = base + L::kK + (uint32_t)(ti & 1) * L::kKStage;
+        const uint32_t v_addr = base + L::kV + (uint32_t)(ti & 1) * L::kKVBytes;
 #pragma unroll
-    for (int ks = 0; ks < D / 16; ++ks) {
-      // k-step ks: block ks/4 of 64 elements, 32 bytes per step inside the 128-byte row
-      const uint32_t qo = (uint32_t)(ks >> 2) * (kRows * 128) + (uint32_t)(ks & 3) * 32u;
-      const uint32_t ko = (uint32_t)(ks >> 2) * (kKeys * 128) + (uint32_t)(ks & 3) * 32u;
-      const uint64_t dk = make_desc(k_addr + ko, 16, 1024);
-      umma(tmem_s, make_desc(base + L::kQhi + qo, 16, 1024), dk, idesc_qk, ks != 0);
-      umma(tmem_s, make_desc(base + L::kQlo + qo, 16, 1024), dk, idesc_qk, 1);
-    }
-    umma_commit(bar_s0 + 8u * (uint32_t)(c & 1));
-  };
-  if (tid == 0 && n_chunks > 0) issue_qk(0);
-
-  for (int ci = 0; ci < n_chunks; ++ci) {
-    // tile ci+2 goes into the stage tile ci-1 used; its P V finished before the last wait on bar_o
-    if (ci + 2 < n_chunks) load_chunk(ci + 2, (ci + 2) % L::kStages);
-    cp_async_commit();
-
-    int s_idx, start;
-    locate(ci, s_idx, start);
-    const int len = seg_len[s_idx], kind = seg_kind[s_idx];
-    const uint32_t v_addr = base + L::kKV + (uint32_t)(ci % L::kStages) * 2u * L::kKVBytes + L::kKVBytes;
-    const uint32_t tmem_s = tmem + 64u * (uint32_t)(ci & 1);
-
-    ok = __syncthreads_and(mbar_wait(bar_s0 + 8u * (uint32_t)(ci & 1), (uint32_t)((ci >> 1) & 1), abort_flag));
-    if (!ok) break;
-    tc_fence_after();
-
-    // ---- softmax: this thread's 32 keys of its row ---------------------------------------------
-    float sc[32];
-    tmem_ld32(tmem_s + lane_base + 32 * half, sc);
-    tmem_ld_wait();
-    // a tile needs masking only at a segment's ragged end, around the bank's free slot, or on
-    // the causal diagonal (uniform over the CTA)
-    const bool need_mask = (start + kKeys > len) || (kind == 1 && free_slot >= start && free_slot < start + kKeys) ||
-                           (kind == 3 && start + kKeys - 1 > r0);
-    float mx = -INFINITY;
-    if (need_mask) {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const int key = start + 32 * half + j;
-        bool vis = key < len;
-        if (kind == 1) vis = vis && (key != free_slot);
-        if (kind == 3) vis = vis && (key <= tok);
-        sc[j] = vis ? sc[j] : -INFINITY;
-        mx = fmaxf(mx, sc[j]);
+        for (int kk = 0; kk < kKeys / 16; ++kk) {
+          // A = P, K-major: 64-key blocks of kRows*128 bytes, 32 bytes per 16 keys inside a block.
+          // B = V, MN-major: 16 key rows = 2048 bytes, 64-wide d blocks kKeys*128 bytes apart,
+          // 8-key groups 1024 bytes apart.
+          umma(tmem_o, make_desc(p_addr + (uint32_t)(kk >> 2) * (kRows * 128) + (uint32_t)(kk & 3) * 32u, 16, 1024),
+               make_desc(v_addr + (uint32_t)kk * 2048u, kKeys * 128, 1024), idesc_pv, kk != 0);
+        }
+        umma_commit(bar_o);
+        if (ti + 1 < n_tiles) issue_qk(ti + 1);
       }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) mx = fmaxf(mx, sc[j]);
     }
-    max_x[(ci & 1) * 256 + half * 128 + row] = mx;
-    __syncthreads();
-    mx = fmaxf(mx, max_x[(ci & 1) * 256 + (half ^ 1) * 128 + row]) * scale;     // scale > 0: max commutes with it
-    const float m_new = fmaxf(m_run, mx);
-    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-    const float alpha = ex2_approx(m_run - m_use);               // ex2(-inf) = 0 on the first tile
-    m_run = m_new;
-    float rs = 0.f;
-    uint8_t* ptile = gbase + L::kP;
+  } else {
+    // ---- softmax / accumulation / loader threads ----------------------------------------------------
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;   // warp w may touch TMEM lanes 32*(w%4)..+31
+    float o_acc[DH];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      float p[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) { p[j] = ex2_approx(fmaf(sc[c * 8 + j], scale, -m_use)); rs += p[j]; }
-      uint4 pk;
-      __nv_bfloat162 t0 = __floats2bfloat162_rn(p[0], p[1]), t1 = __floats2bfloat162_rn(p[2], p[3]);
-      __nv_bfloat162 t2 = __floats2bfloat162_rn(p[4], p[5]), t3 = __floats2bfloat162_rn(p[6], p[7]);
-      pk.x = *reinterpret_cast<uint32_t*>(&t0); pk.y = *reinterpret_cast<uint32_t*>(&t1);
-      pk.z = *reinterpret_cast<uint32_t*>(&t2); pk.w = *reinterpret_cast<uint32_t*>(&t3);
-      *reinterpret_cast<uint4*>(ptile + sw_off<kRows>(row, 4 * half + c)) = pk;
-    }
-    l_run = l_run * alpha + rs;
-    cp_async_wait<1>();            // tile ci+1 has landed (needed by the Q K^T issued below)
-    fence_async_proxy();           // P stores and cp.async writes -> visible to the tensor-core proxy
-    tc_fence_before();
-    __syncthreads();
+    for (int i = 0; i < DH; ++i) o_acc[i] = 0.f;
+    float m_run = -INFINITY, l_run = 0.f;      // m_run in the log2 domain (score * scale_log2e)
+    const float scale = a.scale_log2e;
+    const int lim = min(total, (causal_start == 0x3fffffff) ? total : causal_start + tok + 1);  // first invisible key
+    bool ok = true;
 
-    if (tid == 0) {
+    for (int ti = 0; ti < n_tiles; ++ti) {
+      const uint32_t tmem_s = tmem + 128u * (uint32_t)(ti & 1);
+      ok = ok && mbar_wait(bar_s0 + 8u * (uint32_t)(ti & 1), (uint32_t)((ti >> 1) & 1), abort_flag);
       tc_fence_after();
+      const int v0 = ti * kKeys + KH * half;       // first key of this thread's half tile
+      // a tile needs masking at the ragged end of the key axis, around the bank's free slot and
+      // on the causal diagonal (uniform over the CTA)
+      const bool need_mask = ((ti + 1) * kKeys > min(total, causal_start + r0 + 1)) ||
+                             (hole >= ti * kKeys && hole < (ti + 1) * kKeys);
+      float mx = -INFINITY;
+      float sc[KH];
+      if (ok) {
+        tmem_ld32(tmem_s + lane_base + KH * half, sc);
+        tmem_ld32(tmem_s + lane_base + KH * half + 32, sc + 32);
+        tmem_ld_wait();
+        if (need_mask) {
+          const int nvis = lim - v0, hj = hole - v0;
 #pragma unroll
-      for (int kk = 0; kk < kKeys / 16; ++kk) {
-        // A = P, K-major: 32 bytes per 16 keys.  B = V, MN-major: 16 key rows = 2048 bytes,
-        // 64-wide d blocks kKeys*128 bytes apart, 8-key groups 1024 bytes apart.
-        umma(tmem_o, make_desc(base + L::kP + (uint32_t)kk * 32u, 16, 1024),
-             make_desc(v_addr + (uint32_t)kk * 2048u, kKeys * 128, 1024), idesc_pv, kk != 0);
+          for (int j = 0; j < KH; ++j) {
+            sc[j] = (j < nvis && j != hj) ? sc[j] : -INFINITY;
+            mx = fmaxf(mx, sc[j]);
+          }
+        } else {
+          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < KH; j += 4) {
+            m0 = fmaxf(m0, sc[j]); m1 = fmaxf(m1, sc[j + 1]); m2 = fmaxf(m2, sc[j + 2]); m3 = fmaxf(m3, sc[j + 3]);
+          }
+          mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+        }
       }
-      umma_commit(bar_o);
-      if (ci + 1 < n_chunks) issue_qk(ci + 1);     // overlaps with the accumulation below
-    }
-    ok = __syncthreads_and(mbar_wait(bar_o, (uint32_t)(ci & 1), abort_flag));
-    if (!ok) break;
-    tc_fence_after();
+      max_x[(ti & 1) * 256 + half * 128 + row] = mx;
+      if (!softmax_barrier_and(ok)) { ok = false; break; }      // uniform over the 256 threads
+      mx = fmaxf(mx, max_x[(ti & 1) * 256 + (half ^ 1) * 128 + row]) * scale;   // scale > 0: max commutes with it
+      const float m_new = fmaxf(m_run, mx);
+      const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+      const float alpha = ex2_approx(m_run - m_use);               // ex2(-inf) = 0 on the first tile
+      m_run = m_new;
+      float rs0 = 0.f, rs1 = 0.f;
+      // S(ti) is complete, so the K tile is dead: P takes its place
+      uint8_t* ptile = gbase + L::kK + (size_t)(ti & 1) * L::kKStage;
 #pragma unroll
-    for (int c0 = 0; c0 < DH; c0 += 32) {
-      float t[32];
-      tmem_ld32(tmem_o + lane_base + DH * half + c0, t);
-      tmem_ld_wait();
+      for (int c = 0; c < KH / 8; ++c) {
+        float p[8];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) o_acc[c0 + j] = fmaf(o_acc[c0 + j], alpha, t[j]);
-    }
-    tc_fence_before();             // orders these TMEM reads before the next tile's MMAs (issued after a barrier)
-  }
-  cp_async_wait<0>();
+        for (int j = 0; j < 8; ++j) p[j] = ex2_approx(fmaf(sc[c * 8 + j], scale, -m_use));
+        rs0 += (p[0] + p[1]) + (p[2] + p[3]);
+        rs1 += (p[4] + p[5]) + (p[6] + p[7]);
+        uint4 pk;
+        __nv_bfloat162 t0 = __floats2bfloat162_rn(p[0], p[1]), t1 = __floats2bfloat162_rn(p[2], p[3]);
+        __nv_bfloat162 t2 = __floats2bfloat162_rn(p[4], p[5]), t3 = __floats2bfloat162_rn(p[6], p[7]);
+        pk.x = *reinterpret_cast<uint32_t*>(&t0); pk.y = *reinterpret_cast<uint32_t*>(&t1);
+        pk.z = *reinterpret_cast<uint32_t*>(&t2); pk.w = *reinterpret_cast<uint32_t*>(&t3);
+        *reinterpret_cast<uint4*>(ptile + sw_off<kRows>(row, (KH / 8) * half + c)) = pk;
+      }
+      l_run = l_run * alpha + (rs0 + rs1);
+      cp_async_wait<0>();            // tile ti+1 has landed (the next Q K^T reads it)
+      fence_async_proxy();           // P stores and cp.async writes -> visible to the tensor-core proxy
+      tc_fence_before();
+      mbar_arrive(bar_p);
 
-  // the two halves of a row hold partial sums of the softmax denominator
-  max_x[half * 128 + row] = l_run;
-  __syncthreads();
-  l_run += max_x[(half ^ 1) * 128 + row];
-
-  if (ok && row_valid) {
-    const float inv = (l_run > 0.f) ? 1.f / l_run : 0.f;
-    const size_t obase = (((size_t)b * rps + tok) * a.Hq + (size_t)hkv * G + g) * D + DH * half;
-    if (a.out_fp32) {
-      float* dst = static_cast<float*>(a.out) + obase;
+      ok = mbar_wait(bar_o, (uint32_t)(ti & 1), abort_flag);
+      tc_fence_after();
+      if (ok) {
 #pragma unroll
-      for (int c = 0; c < DH; c += 4)
-        *reinterpret_cast<float4*>(dst + c) =
-            make_float4(o_acc[c] * inv, o_acc[c + 1] * inv, o_acc[c + 2] * inv, o_acc[c + 3] * inv);
-    } else {
-      bf16* dst = static_cast<bf16*>(a.out) + obase;
+        for (int c0 = 0; c0 < DH; c0 += 32) {
+          float t[32];
+          tmem_ld32(tmem_o + lane_base + DH * half + c0, t);
+          tmem_ld_wait();
 #pragma unroll
-      for (int c = 0; c < DH; c += 2)
-        *reinterpret_cast<__nv_bfloat162*>(dst + c) = __floats2bfloat162_rn(o_acc[c] * inv, o_acc[c + 1] * inv);
+          for (int j = 0; j < 32; ++j) o_acc[c0 + j] = fmaf(o_acc[c0 + j], alpha, t[j]);
+        }
+        tc_fence_before();
+        // P V (ti) is done: its K/P and V stage may take tile ti+2
+        if (ti + 2 < n_tiles) load_tile(ti + 2, ti & 1);
+        cp_async_commit();
+      }
     }
-    if (a.h_out != nullptr) {
+    cp_async_wait<0>();
+
+    // the two halves of a row hold partial sums of the softmax denominator
+    max_x[half * 128 + row] = l_run;
+    const bool all_ok = softmax_barrier_and(ok);
+    l_run += max_x[(half ^ 1) * 128 + row];
+
+    if (all_ok && row_valid) {
+      const float inv = (l_run > 0.f) ? 1.f / l_run : 0.f;
+      const size_t obase = (((size_t)b * rps + tok) * a.Hq + (size_t)hkv * G + g) * D + DH * half;
+      if (a.out_fp32) {
+        float* dst = static_cast<float*>(a.out) + obase;
 #pragma unroll
-      for (int c = 0; c < DH; c += 2) {
-        const float2 hv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(a.h_in + obase + c));
-        *reinterpret_cast<__nv_bfloat162*>(a.h_out + obase + c) =
-            __floats2bfloat162_rn(hv.x + o_acc[c] * inv, hv.y + o_acc[c + 1] * inv);
+        for (int c = 0; c < DH; c += 4)
+          *reinterpret_cast<float4*>(dst + c) =
+              make_float4(o_acc[c] * inv, o_acc[c + 1] * inv, o_acc[c + 2] * inv, o_acc[c + 3] * inv);
+      } else {
+        bf16* dst = static_cast<bf16*>(a.out) + obase;
+#pragma unroll
+        for (int c = 0; c < DH; c += 2)
+          *reinterpret_cast<__nv_bfloat162*>(dst + c) = __floats2bfloat162_rn(o_acc[c] * inv, o_acc[c + 1] * inv);
+      }
+      if (a.h_out != nullptr) {
+#pragma unroll
+        for (int c = 0; c < DH; c += 2) {
+          const float2 hv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(a.h_in + obase + c));
+          *reinterpret_cast<__nv_bfloat162*>(a.h_out + obase + c) =
+              __floats2bfloat162_rn(hv.x + o_acc[c] * inv, hv.y + o_acc[c + 1] * inv);
+        }
       }
     }
   }
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == 8) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
   }
   if (tid == 0 && *abort_flag) atomicExch(status, VS_ERR_DEVICE_TIMEOUT);
 }
@@ -423,8 +455,8 @@ cudaError_t prefill_attention_tc_init() {
 
 cudaError_t launch_prefill_attention_tc(const AttnArgs& a, const BatchParams& bp, int* status, cudaStream_t st) {
   dim3 grid((bp.rows_per_stream + kTok - 1) / kTok, a.Hkv, bp.n_active);
-  if (a.D == 128) prefill_attn_tc_kernel<128><<<grid, 256, Smem<128>::kTotal, st>>>(a, bp, status);
-  else if (a.D == 64) prefill_attn_tc_kernel<64><<<grid, 256, Smem<64>::kTotal, st>>>(a, bp, status);
+  if (a.D == 128) prefill_attn_tc_kernel<128><<<grid, kAttnThreads, Smem<128>::kTotal, st>>>(a, bp, status);
+  else if (a.D == 64) prefill_attn_tc_kernel<64><<<grid, kAttnThreads, Smem<64>::kTotal, st>>>(a, bp, status);
   else return cudaErrorInvalidValue;
   return cudaGetLastError();
 }
