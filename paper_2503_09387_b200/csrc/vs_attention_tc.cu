@@ -11,10 +11,11 @@
 //            softmax of the row in registers, P (bf16) -> shared memory (over the dead K tile)
 //            O_tile = P V  (tcgen05.mma, M 128 x N D, V read MN-major)             -> TMEM
 //            o_row = o_row * alpha + O_tile                                          (registers)
-// Warps 0..7: two threads per row (each owns 64 keys of a tile and D/2 output dims), they also
-// fetch K/V with cp.async into the 128-byte-swizzled layout the MMA descriptors expect.
+// Warps 0..7: two threads per row (each owns 64 keys of a tile and D/2 output dims).
 // Warp 8: one thread issues every MMA, one tile of Q K^T ahead of the softmax (S is double
-// buffered in TMEM).  All mbarrier waits are bounded.
+// buffered in TMEM); descriptors are built once.  Warps 9..11 fetch K/V with cp.async into the
+// 128-byte-swizzled layout the MMA descriptors expect, one tile ahead.  Finished rows leave
+// through shared memory as whole contiguous rows.  All mbarrier waits are bounded.
 #include "vs_common.cuh"
 
 namespace vs {
@@ -159,8 +160,22 @@ __device__ __forceinline__ bool softmax_barrier_and(bool pred) {
   return r != 0;
 }
 
-constexpr int kSoftmaxThreads = 256;
-constexpr int kAttnThreads = kSoftmaxThreads + 32;
+constexpr int kSoftmaxThreads = 256;                     // warps 0..7
+constexpr int kLoaderThreads = 96;                       // warps 9, 10, 11
+constexpr int kAttnThreads = kSoftmaxThreads + 32 + kLoaderThreads;
+
+__device__ __forceinline__ void umma_acc(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.eq.u32 p, 1, 1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc) : "memory");
+}
+__device__ __forceinline__ void umma_new(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, 1, 1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc) : "memory");
+}
 
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnArgs a, BatchParams bp, int* status) {
@@ -173,9 +188,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bar_s0 = base + L::kCtl;       // +0, +8: S buffer ready (tcgen05.commit)
   const uint32_t bar_o = base + L::kCtl + 16;   // O tile ready (tcgen05.commit)
-  const uint32_t bar_p = base + L::kCtl + 24;   // P written and next K/V tile landed (256 arrivals)
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + L::kCtl + 32);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kCtl + 36);
+  const uint32_t bar_p = base + L::kCtl + 24;   // P written (256 arrivals)
+  const uint32_t bar_kv0 = base + L::kCtl + 32; // +0, +8: K/V tile landed in a stage (one arrival per loader thread)
+  const uint32_t bar_free0 = base + L::kCtl + 48;  // +0, +8: stage free again (tcgen05.commit after P V)
+  const uint32_t bar_q = base + L::kCtl + 64;   // Q tile landed (256 arrivals)
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + L::kCtl + 72);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kCtl + 76);
   float* max_x = reinterpret_cast<float*>(gbase + L::kMax);
 
   const int b = blockIdx.z, hkv = blockIdx.y;
@@ -184,24 +202,20 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   const int sid = bp.stream_id[b];
   const int G = a.Hq / a.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5;
-  const bool is_softmax = tid < kSoftmaxThreads;
-  const int row = tid & 127, half = (tid >> 7) & 1;
   const int count = bp.count[b];
   const bool bank_full = (a.M > 0 && count == a.M);
 
-  const int g = row >> 4;
-  const int tok = r0 + (row & 15);
-  const bool row_valid = is_softmax && (g < G) && (tok < rps);
-
   // ---- the virtual key axis: segments end to end ----------------------------------------------
-  int seg_end[4];                                // exclusive prefix sums of the segment lengths
+  // key v of segment s lives at seg_k[s] + v * seg_stride[s] (the segment's first key index is
+  // folded into the pointer)
+  int seg_end[4];
   const bf16* seg_k[4];
   const bf16* seg_v[4];
-  long long seg_stride[4];
+  int seg_stride[4];
   int total = 0, causal_start = 0x3fffffff, hole = -1;
 #pragma unroll
   for (int s = 0; s < 4; ++s) {
-    seg_k[s] = nullptr; seg_v[s] = nullptr; seg_stride[s] = 0;
+    seg_k[s] = a.q; seg_v[s] = a.q; seg_stride[s] = 0;
     if (s < a.n_seg) {
       const AttnSegment sg = a.seg[s];
       int len;
@@ -212,39 +226,23 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
       }
       else if (sg.kind == 2) len = bp.text_len[b];
       else { len = min(rps, r0 + kTok); causal_start = total; }  // later keys are visible to no row of this tile
-      const long long off = (long long)(sg.by_batch ? b : sid) * sg.stream_stride + (long long)hkv * sg.head_stride;
-      seg_k[s] = sg.k + off; seg_v[s] = sg.v + off; seg_stride[s] = sg.row_stride;
+      const long long off = (long long)(sg.by_batch ? b : sid) * sg.stream_stride + (long long)hkv * sg.head_stride -
+                            (long long)total * sg.row_stride;
+      seg_k[s] = sg.k + off; seg_v[s] = sg.v + off; seg_stride[s] = (int)sg.row_stride;
       total += len;
     }
     seg_end[s] = total;
   }
   const int n_tiles = (total + kKeys - 1) / kKeys;
 
-  auto load_tile = [&](int ti, int stage) {
-    const uint32_t kdst = base + L::kK + (uint32_t)stage * L::kKStage;
-    const uint32_t vdst = base + L::kV + (uint32_t)stage * L::kKVBytes;
-    for (int idx = tid; idx < kKeys * CPR; idx += kSoftmaxThreads) {
-      const int r = idx / CPR, c = idx - r * CPR;
-      const int v = ti * kKeys + r;
-      int s = 0;
-#pragma unroll
-      for (int t = 0; t < 3; ++t) if (v >= seg_end[t]) s = t + 1;
-      const bool valid = v < total;
-      const bf16* kp = seg_k[0]; const bf16* vp = seg_v[0]; long long stride = seg_stride[0]; int first = 0;
-#pragma unroll
-      for (int t = 1; t < 4; ++t) if (s == t) { kp = seg_k[t]; vp = seg_v[t]; stride = seg_stride[t]; first = seg_end[t - 1]; }
-      const long long goff = valid ? ((long long)(v - first) * stride + c * 8) : 0;
-      cp_async16(kdst + sw_off<kKeys>(r, c), (valid ? kp : a.q) + goff, valid);
-      cp_async16(vdst + sw_off<kKeys>(r, c), (valid ? vp : a.q) + goff, valid);
-    }
-  };
-
-  // ---- set-up: barriers, TMEM, Q tile ------------------------------------------------------
+  // ---- set-up ---------------------------------------------------------------------------------
   if (tid == 0) {
-    mbar_init(bar_s0, 1);
-    mbar_init(bar_s0 + 8, 1);
+    mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1);
     mbar_init(bar_o, 1);
     mbar_init(bar_p, kSoftmaxThreads);
+    mbar_init(bar_kv0, kLoaderThreads); mbar_init(bar_kv0 + 8, kLoaderThreads);
+    mbar_init(bar_free0, 1); mbar_init(bar_free0 + 8, 1);
+    mbar_init(bar_q, kSoftmaxThreads);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -253,7 +251,112 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
                  ::"r"(smem_u32((const void*)tmem_slot)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (is_softmax) {
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem_o = tmem + 256;                    // S buffers at columns 0 and 128
+
+  if (warp >= 9) {
+    // ---- K/V loaders: cp.async into the swizzled tiles, one tile ahead ---------------------------
+    const int lt = tid - (kSoftmaxThreads + 32);         // 0..95
+    auto issue_tile = [&](int ti) {
+      const int stage = ti & 1;
+      const uint32_t kdst = base + L::kK + (uint32_t)stage * L::kKStage;
+      const uint32_t vdst = base + L::kV + (uint32_t)stage * L::kKVBytes;
+      constexpr int kRowStep = kLoaderThreads / CPR;     // key rows covered per pass
+      const int c = lt % CPR;
+      for (int r = lt / CPR; r < kKeys; r += kRowStep) {
+        const int v = ti * kKeys + r;
+        const bool valid = v < total;
+        const bf16* kp = seg_k[0]; const bf16* vp = seg_v[0]; int stride = seg_stride[0];
+#pragma unroll
+        for (int t = 1; t < 4; ++t)
+          if (v >= seg_end[t - 1]) { kp = seg_k[t]; vp = seg_v[t]; stride = seg_stride[t]; }
+        const long long goff = valid ? ((long long)v * stride + c * 8) : 0;
+        cp_async16(kdst + sw_off<kKeys>(r, c), (valid ? kp : a.q) + goff, valid);
+        cp_async16(vdst + sw_off<kKeys>(r, c), (valid ? vp : a.q) + goff, valid);
+      }
+      cp_async_commit();
+    };
+    // Two tiles are put in flight at once; afterwards tile ti+2 can only be fetched once P V of
+    // tile ti has released its stage.  A tile is always published BEFORE the loader waits for a
+    // stage to be released: the issuer runs Q K^T of tile ti+1 ahead of P V of tile ti, so the
+    // release of tile ti's stage depends on tile ti+1 having been published.
+    issue_tile(0);
+    if (n_tiles > 1) { issue_tile(1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
+    fence_async_proxy();             // cp.async writes -> visible to the tensor-core proxy
+    mbar_arrive(bar_kv0);            // tile 0
+    for (int ti = 0; ti + 1 < n_tiles; ++ti) {
+      cp_async_wait<0>();            // tile ti+1 has landed
+      fence_async_proxy();
+      mbar_arrive(bar_kv0 + 8u * (uint32_t)((ti + 1) & 1));
+      if (ti + 2 < n_tiles) {
+        if (!mbar_wait(bar_free0 + 8u * (uint32_t)(ti & 1), (uint32_t)((ti >> 1) & 1), abort_flag)) break;
+        issue_tile(ti + 2);
+      }
+    }
+    cp_async_wait<0>();
+  } else if (warp == 8) {
+    // ---- MMA issuer: descriptors are built once, each MMA costs one add ----------------------------
+    if ((tid & 31) == 0) {
+      const uint32_t idesc_qk = make_idesc(kKeys, 0);
+      const uint32_t idesc_pv = make_idesc(D, 1);
+      uint64_t dq_hi[D / 16], dq_lo[D / 16];
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks) {
+        // k-step ks: block ks/4 of 64 elements, 32 bytes per step inside the 128-byte row
+        const uint32_t qo = (uint32_t)(ks >> 2) * (kRows * 128) + (uint32_t)(ks & 3) * 32u;
+        dq_hi[ks] = make_desc(base + L::kQhi + qo, 16, 1024);
+        dq_lo[ks] = make_desc(base + L::kQlo + qo, 16, 1024);
+      }
+      uint64_t dk0[2], dv0[2];
+#pragma unroll
+      for (int st = 0; st < 2; ++st) {
+        dk0[st] = make_desc(base + L::kK + (uint32_t)st * L::kKStage, 16, 1024);            // K tile (later P), K-major
+        dv0[st] = make_desc(base + L::kV + (uint32_t)st * L::kKVBytes, kKeys * 128, 1024);  // V tile, MN-major
+      }
+      auto issue_qk = [&](int t) {
+        const uint32_t tmem_s = tmem + 128u * (uint32_t)(t & 1);
+        const uint64_t dk = dk0[t & 1];
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint64_t dkk = dk + (uint64_t)(((ks >> 2) * (kKeys * 128) + (ks & 3) * 32) >> 4);
+          if (ks == 0) umma_new(tmem_s, dq_hi[ks], dkk, idesc_qk); else umma_acc(tmem_s, dq_hi[ks], dkk, idesc_qk);
+          umma_acc(tmem_s, dq_lo[ks], dkk, idesc_qk);
+        }
+        umma_commit(bar_s0 + 8u * (uint32_t)(t & 1));
+      };
+      bool ok = mbar_wait(bar_q, 0, abort_flag) && mbar_wait(bar_kv0, 0, abort_flag);
+      if (ok) { tc_fence_after(); issue_qk(0); }
+      for (int ti = 0; ti < n_tiles && ok; ++ti) {
+        if (ti + 1 < n_tiles) {      // next S tile first: it has a whole softmax of lead time
+          ok = mbar_wait(bar_kv0 + 8u * (uint32_t)((ti + 1) & 1), (uint32_t)(((ti + 1) >> 1) & 1), abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          issue_qk(ti + 1);
+        }
+        ok = mbar_wait(bar_p, (uint32_t)(ti & 1), abort_flag);   // P(ti) in place
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t dp = dk0[ti & 1], dv = dv0[ti & 1];
+#pragma unroll
+        for (int kk = 0; kk < kKeys / 16; ++kk) {
+          // A = P, K-major: 64-key blocks of kRows*128 bytes, 32 bytes per 16 keys inside a block.
+          // B = V, MN-major: 16 key rows = 2048 bytes further per step.
+          const uint64_t dpk = dp + (uint64_t)(((kk >> 2) * (kRows * 128) + (kk & 3) * 32) >> 4);
+          const uint64_t dvk = dv + (uint64_t)((kk * 2048) >> 4);
+          if (kk == 0) umma_new(tmem_o, dpk, dvk, idesc_pv); else umma_acc(tmem_o, dpk, dvk, idesc_pv);
+        }
+        umma_commit(bar_o);
+        umma_commit(bar_free0 + 8u * (uint32_t)(ti & 1));
+      }
+    }
+  } else {
+    // ---- softmax / accumulation threads: two per row --------------------------------------------------
+    const int row = tid & 127, half = tid >> 7;
+    const int tok = r0 + (row & 15);
+    // Q tile (hi and lo) -> shared memory
     for (int idx = tid; idx < kRows * CPR; idx += kSoftmaxThreads) {
       const int r = idx / CPR, c = idx - r * CPR;
       const int gg = r >> 4, tt = r0 + (r & 15);
@@ -262,58 +365,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
       cp_async16(base + L::kQhi + sw_off<kRows>(r, c), a.q + off, valid);
       cp_async16(base + L::kQlo + sw_off<kRows>(r, c), a.q_lo + off, valid);
     }
-    load_tile(0, 0);
-    cp_async_commit();                                   // group: Q + tile 0
-    if (n_tiles > 1) load_tile(1, 1);
-    cp_async_commit();                                   // group: tile 1
-    cp_async_wait<1>();
-    fence_async_proxy();                                 // cp.async writes -> visible to the tensor-core proxy
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_o = tmem + 256;                    // S buffers at columns 0 and 128
+    cp_async_commit();
+    cp_async_wait<0>();
+    fence_async_proxy();
+    mbar_arrive(bar_q);
 
-  if (warp == 8) {
-    // ---- MMA issuer -----------------------------------------------------------------------------
-    if ((tid & 31) == 0) {
-      const uint32_t idesc_qk = make_idesc(kKeys, 0);
-      const uint32_t idesc_pv = make_idesc(D, 1);
-      auto issue_qk = [&](int t) {
-        const uint32_t k_addr = base + L::kK + (uint32_t)(t & 1) * L::kKStage;
-        const uint32_t tmem_s = tmem + 128u * (uint32_t)(t & 1);
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          // k-step ks: block ks/4 of 64 elements, 32 bytes per step inside the 128-byte row
-          const uint32_t qo = (uint32_t)(ks >> 2) * (kRows * 128) + (uint32_t)(ks & 3) * 32u;
-          const uint32_t ko = (uint32_t)(ks >> 2) * (kKeys * 128) + (uint32_t)(ks & 3) * 32u;
-          const uint64_t dk = make_desc(k_addr + ko, 16, 1024);
-          umma(tmem_s, make_desc(base + L::kQhi + qo, 16, 1024), dk, idesc_qk, ks != 0);
-          umma(tmem_s, make_desc(base + L::kQlo + qo, 16, 1024), dk, idesc_qk, 1);
-        }
-        umma_commit(bar_s0 + 8u * (uint32_t)(t & 1));
-      };
-      issue_qk(0);
-      for (int ti = 0; ti < n_tiles; ++ti) {
-        if (!mbar_wait(bar_p, (uint32_t)(ti & 1), abort_flag)) break;   // P(ti) in place, tile ti+1 landed
-        tc_fence_after();
-        const uint32_t p_addr = base + L::kK + (uint32_t)(ti & 1) * L::kKStage;
-        const uint32_t v_addr = base + L::kV + (uint32_t)(ti & 1) * L::kKVBytes;
-#pragma unroll
-        for (int kk = 0; kk < kKeys / 16; ++kk) {
-          // A = P, K-major: 64-key blocks of kRows*128 bytes, 32 bytes per 16 keys inside a block.
-          // B = V, MN-major: 16 key rows = 2048 bytes, 64-wide d blocks kKeys*128 bytes apart,
-          // 8-key groups 1024 bytes apart.
-          umma(tmem_o, make_desc(p_addr + (uint32_t)(kk >> 2) * (kRows * 128) + (uint32_t)(kk & 3) * 32u, 16, 1024),
-               make_desc(v_addr + (uint32_t)kk * 2048u, kKeys * 128, 1024), idesc_pv, kk != 0);
-        }
-        umma_commit(bar_o);
-        if (ti + 1 < n_tiles) issue_qk(ti + 1);
-      }
-    }
-  } else {
-    // ---- softmax / accumulation / loader threads ----------------------------------------------------
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;   // warp w may touch TMEM lanes 32*(w%4)..+31
     float o_acc[DH];
 #pragma unroll
@@ -379,8 +435,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
         *reinterpret_cast<uint4*>(ptile + sw_off<kRows>(row, (KH / 8) * half + c)) = pk;
       }
       l_run = l_run * alpha + (rs0 + rs1);
-      cp_async_wait<0>();            // tile ti+1 has landed (the next Q K^T reads it)
-      fence_async_proxy();           // P stores and cp.async writes -> visible to the tensor-core proxy
+      fence_async_proxy();           // P stores -> visible to the tensor-core proxy
       tc_fence_before();
       mbar_arrive(bar_p);
 
@@ -396,39 +451,50 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
           for (int j = 0; j < 32; ++j) o_acc[c0 + j] = fmaf(o_acc[c0 + j], alpha, t[j]);
         }
         tc_fence_before();
-        // P V (ti) is done: its K/P and V stage may take tile ti+2
-        if (ti + 2 < n_tiles) load_tile(ti + 2, ti & 1);
-        cp_async_commit();
       }
     }
-    cp_async_wait<0>();
 
     // the two halves of a row hold partial sums of the softmax denominator
     max_x[half * 128 + row] = l_run;
     const bool all_ok = softmax_barrier_and(ok);
     l_run += max_x[(half ^ 1) * 128 + row];
 
-    if (all_ok && row_valid) {
+    // Every MMA has completed, so the Q tiles are dead: the normalised rows go through them
+    // (fp32, 16-byte units XOR-swizzled by the row) and leave as whole contiguous rows.
+    constexpr int F4 = D / 4;                                      // float4 units per row
+    if (all_ok) {
+      float4* stage_o = reinterpret_cast<float4*>(gbase + L::kQhi);
       const float inv = (l_run > 0.f) ? 1.f / l_run : 0.f;
-      const size_t obase = (((size_t)b * rps + tok) * a.Hq + (size_t)hkv * G + g) * D + DH * half;
-      if (a.out_fp32) {
-        float* dst = static_cast<float*>(a.out) + obase;
 #pragma unroll
-        for (int c = 0; c < DH; c += 4)
-          *reinterpret_cast<float4*>(dst + c) =
-              make_float4(o_acc[c] * inv, o_acc[c + 1] * inv, o_acc[c + 2] * inv, o_acc[c + 3] * inv);
-      } else {
-        bf16* dst = static_cast<bf16*>(a.out) + obase;
-#pragma unroll
-        for (int c = 0; c < DH; c += 2)
-          *reinterpret_cast<__nv_bfloat162*>(dst + c) = __floats2bfloat162_rn(o_acc[c] * inv, o_acc[c + 1] * inv);
-      }
-      if (a.h_out != nullptr) {
-#pragma unroll
-        for (int c = 0; c < DH; c += 2) {
-          const float2 hv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(a.h_in + obase + c));
-          *reinterpret_cast<__nv_bfloat162*>(a.h_out + obase + c) =
-              __floats2bfloat162_rn(hv.x + o_acc[c] * inv, hv.y + o_acc[c + 1] * inv);
+      for (int c = 0; c < DH; c += 4)
+        stage_o[row * F4 + (((DH * half + c) >> 2) ^ (row & (F4 - 1)))] =
+            make_float4(o_acc[c] * inv, o_acc[c + 1] * inv, o_acc[c + 2] * inv, o_acc[c + 3] * inv);
+    }
+    softmax_barrier_and(true);
+    if (all_ok) {
+      const float4* stage_o = reinterpret_cast<const float4*>(gbase + L::kQhi);
+      const int lane = tid & 31;
+      for (int r = warp * 16; r < warp * 16 + 16; ++r) {           // 8 warps x 16 rows
+        const int gg = r >> 4, tt = r0 + (r & 15);
+        if (gg >= G || tt >= rps) continue;                        // uniform over the warp
+        const size_t obase = (((size_t)b * rps + tt) * a.Hq + (size_t)hkv * G + gg) * D;
+        for (int u = lane; u < F4; u += 32) {
+          const float4 v = stage_o[r * F4 + (u ^ (r & (F4 - 1)))];
+          if (a.out_fp32) {
+            *reinterpret_cast<float4*>(static_cast<float*>(a.out) + obase + 4 * u) = v;
+          } else {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+            uint2 w; w.x = *reinterpret_cast<uint32_t*>(&lo); w.y = *reinterpret_cast<uint32_t*>(&hi);
+            *reinterpret_cast<uint2*>(static_cast<bf16*>(a.out) + obase + 4 * u) = w;
+          }
+          if (a.h_out != nullptr) {
+            const uint2 hraw = *reinterpret_cast<const uint2*>(a.h_in + obase + 4 * u);
+            const float2 h0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hraw.x));
+            const float2 h1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hraw.y));
+            __nv_bfloat162 lo = __floats2bfloat162_rn(h0.x + v.x, h0.y + v.y), hi = __floats2bfloat162_rn(h1.x + v.z, h1.y + v.w);
+            uint2 w; w.x = *reinterpret_cast<uint32_t*>(&lo); w.y = *reinterpret_cast<uint32_t*>(&hi);
+            *reinterpret_cast<uint2*>(a.h_out + obase + 4 * u) = w;
+          }
         }
       }
     }
