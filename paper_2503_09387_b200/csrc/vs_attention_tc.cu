@@ -260,22 +260,38 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   if (warp >= 9) {
     // ---- K/V loaders: cp.async into the swizzled tiles, one tile ahead ---------------------------
     const int lt = tid - (kSoftmaxThreads + 32);         // 0..95
+    // A thread owns one 16-byte column c of the key rows r = rsub, rsub + kRowStep, ...; it walks
+    // the tile segment by segment so that inside a segment a row costs one pointer step.
+    constexpr int kRowStep = kLoaderThreads / CPR;       // key rows covered per pass
+    const int c = lt % CPR, rsub = lt / CPR;
     auto issue_tile = [&](int ti) {
       const int stage = ti & 1;
-      const uint32_t kdst = base + L::kK + (uint32_t)stage * L::kKStage;
-      const uint32_t vdst = base + L::kV + (uint32_t)stage * L::kKVBytes;
-      constexpr int kRowStep = kLoaderThreads / CPR;     // key rows covered per pass
-      const int c = lt % CPR;
-      for (int r = lt / CPR; r < kKeys; r += kRowStep) {
-        const int v = ti * kKeys + r;
-        const bool valid = v < total;
-        const bf16* kp = seg_k[0]; const bf16* vp = seg_v[0]; int stride = seg_stride[0];
+      const uint32_t kdst = base + L::kK + (uint32_t)stage * L::kKStage + (uint32_t)((c >> 3) * (kKeys * 128));
+      const uint32_t vdst = base + L::kV + (uint32_t)stage * L::kKVBytes + (uint32_t)((c >> 3) * (kKeys * 128));
+      const int t_begin = ti * kKeys;
+      int seg_begin = 0;
 #pragma unroll
-        for (int t = 1; t < 4; ++t)
-          if (v >= seg_end[t - 1]) { kp = seg_k[t]; vp = seg_v[t]; stride = seg_stride[t]; }
-        const long long goff = valid ? ((long long)v * stride + c * 8) : 0;
-        cp_async16(kdst + sw_off<kKeys>(r, c), (valid ? kp : a.q) + goff, valid);
-        cp_async16(vdst + sw_off<kKeys>(r, c), (valid ? vp : a.q) + goff, valid);
+      for (int sgi = 0; sgi < 4; ++sgi) {
+        const int lo = max(seg_begin, t_begin) - t_begin;            // rows of this segment inside the tile
+        const int hi = min(seg_end[sgi], t_begin + kKeys) - t_begin;
+        seg_begin = seg_end[sgi];
+        if (lo >= hi) continue;
+        int r = lo + ((rsub - lo) % kRowStep + kRowStep) % kRowStep;  // first row >= lo owned by this thread
+        const long long step = (long long)kRowStep * seg_stride[sgi];
+        const bf16* kp = seg_k[sgi] + (long long)(t_begin + r) * seg_stride[sgi] + c * 8;
+        const bf16* vp = seg_v[sgi] + (long long)(t_begin + r) * seg_stride[sgi] + c * 8;
+        for (; r < hi; r += kRowStep, kp += step, vp += step) {
+          const uint32_t so = (uint32_t)(r * 128 + (((c & 7) ^ (r & 7)) << 4));
+          cp_async16(kdst + so, kp, true);
+          cp_async16(vdst + so, vp, true);
+        }
+      }
+      // rows past the end of the key axis (last tile only): zero-filled
+      for (int r = max(total - t_begin, 0) + ((rsub - max(total - t_begin, 0)) % kRowStep + kRowStep) % kRowStep; r < kKeys;
+           r += kRowStep) {
+        const uint32_t so = (uint32_t)(r * 128 + (((c & 7) ^ (r & 7)) << 4));
+        cp_async16(kdst + so, a.q, false);
+        cp_async16(vdst + so, a.q, false);
       }
       cp_async_commit();
     };
