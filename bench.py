@@ -307,6 +307,8 @@ def run_ours(args, w):
         tot = sum(v["total_ms"] for v in kernels.values())
         for v in kernels.values():
             v["share"] = round(v["total_ms"] / tot, 4)
+        kernels_dec = {k: {"launches": v[1], "total_ms": round(v[0], 4), "avg_us": round(1e3 * v[0] / v[1], 3)}
+                       for k, v in per_phase["decode"].items() if v[1]}
         dom = max(kernels, key=lambda k: kernels[k]["total_ms"])
         proj_flops, _ = frame_flops(w, 0)
         avg_bank = (min(w.n_frames, w.bank_capacity) - 1) / 2.0 if w.bank_capacity else 0.0
@@ -343,7 +345,7 @@ def run_ours(args, w):
             "phase_ms_per_step": {"prefix": ms_prefix / args.steps, "frames": ms_frames / args.steps,
                                   "decode": ms_decode / args.steps},
             "wall_s": wall, "clocks": clocks, "gpu_launches": gpu_launches,
-            "roofline": roof, "kernels_frame_phase": kernels,
+            "roofline": roof, "kernels_frame_phase": kernels, "kernels_decode_phase": kernels_dec,
             "step_roofline": {
                 "frame": {"us_per_frame": us_frame, "ideal_us": ideal, "frac": ideal / us_frame,
                           "ideal_compute_us": ideal_c, "ideal_hbm_us": ideal_h,

@@ -158,8 +158,6 @@ struct AttnArgs {
   int Hq, Hkv, D, slots, M;
   float scale_log2e;
 };
-cudaError_t launch_prefill_attention(const AttnArgs& a, const BatchParams& bp, cudaStream_t st);
-cudaError_t prefill_attention_init();
 cudaError_t launch_prefill_attention_tc(const AttnArgs& a, const BatchParams& bp, int* status, cudaStream_t st);
 cudaError_t prefill_attention_tc_init();
 

@@ -257,7 +257,7 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights, void* work
   h->tm_w.resize(D.L);
   for (int l = 0; l < D.L; ++l)
     if (encode_2d(h, &h->tm_w[l], h->w[l], (uint64_t)D.d, (uint64_t)D.E_out, GEMM_BLOCK_M) != VS_OK) return fail(VS_ERR_CUDA);
-  if (qkv_gemm_init() != cudaSuccess || prefill_attention_init() != cudaSuccess || prefill_attention_tc_init() != cudaSuccess) return fail(VS_ERR_CUDA);
+  if (qkv_gemm_init() != cudaSuccess || prefill_attention_tc_init() != cudaSuccess) return fail(VS_ERR_CUDA);
   // clear the whole workspace, then write the non-zero initial metadata
   if (cudaMemset(h->ws, 0, lo.total) != cudaSuccess) return fail(VS_ERR_CUDA);
   if (cudaMemset(h->ws + lo.slot_frame, 0xFF, (size_t)D.S * D.slots * 4) != cudaSuccess) return fail(VS_ERR_CUDA);
@@ -468,8 +468,9 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       da.h_in = D.residual ? h_in : nullptr; da.h_out = h_out;
       da.meta = meta;
       da.Hq = D.Hq; da.Hkv = D.Hkv; da.D = D.D; da.slots = D.slots; da.M = D.M; da.maxP = D.maxP; da.maxT = D.maxT;
-      int ns = (max_keys + 63) / 64;
-      if (ns < 1) ns = 1;
+      // short contexts: one CTA per (stream, KV head) writes the result directly; longer ones are
+      // split so that a CTA walks about 128 keys
+      int ns = (max_keys <= 256) ? 1 : (max_keys + 127) / 128;
       if (ns > DEC_SPLIT_MAX) ns = DEC_SPLIT_MAX;
       da.nsplit = ns;
       da.to_prefix = to_prefix ? 1 : 0;
