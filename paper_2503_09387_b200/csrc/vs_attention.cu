@@ -29,6 +29,8 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
   __shared__ float sp_w[DEC_SPLIT_MAX][GMAX];
   __shared__ int is_last;
 
+  pdl_wait();
+  pdl_launch_dependents();
   const int split = blockIdx.x, hkv = blockIdx.y, b = blockIdx.z;
   const int sid = bp.stream_id[b];
   const int G = a.Hq / a.Hkv;
@@ -270,10 +272,9 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
 cudaError_t launch_decode_attention(const DecodeArgs& a, const BatchParams& bp, cudaStream_t st) {
   if (a.nsplit < 1 || a.nsplit > DEC_SPLIT_MAX || a.Hq / a.Hkv > GMAX) return cudaErrorInvalidValue;
   dim3 grid(a.nsplit, a.Hkv, bp.n_active);
-  if (a.D == 128) decode_attn_kernel<128><<<grid, kDecThreads, 0, st>>>(a, bp);
-  else if (a.D == 64) decode_attn_kernel<64><<<grid, kDecThreads, 0, st>>>(a, bp);
-  else return cudaErrorInvalidValue;
-  return cudaGetLastError();
+  if (a.D == 128) return launch_pdl(decode_attn_kernel<128>, grid, dim3(kDecThreads), 0, st, a, bp);
+  if (a.D == 64) return launch_pdl(decode_attn_kernel<64>, grid, dim3(kDecThreads), 0, st, a, bp);
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace vs

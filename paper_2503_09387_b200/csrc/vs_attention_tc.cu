@@ -196,12 +196,31 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kCtl + 76);
   float* max_x = reinterpret_cast<float*>(gbase + L::kMax);
 
+  const int tid = threadIdx.x, warp = tid >> 5;
+  // ---- set-up that needs nothing from earlier kernels: barriers, tensor memory ------------------
+  if (tid == 0) {
+    mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1);
+    mbar_init(bar_o, 1);
+    mbar_init(bar_p, kSoftmaxThreads);
+    mbar_init(bar_kv0, kLoaderThreads); mbar_init(bar_kv0 + 8, kLoaderThreads);
+    mbar_init(bar_free0, 1); mbar_init(bar_free0 + 8, 1);
+    mbar_init(bar_q, kSoftmaxThreads);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32((const void*)tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  pdl_wait();                       // earlier kernels of the stream have completed
+  pdl_launch_dependents();
+
   const int b = blockIdx.z, hkv = blockIdx.y;
   const int r0 = blockIdx.x * kTok;
   const int rps = bp.rows_per_stream;
   const int sid = bp.stream_id[b];
   const int G = a.Hq / a.Hkv;
-  const int tid = threadIdx.x, warp = tid >> 5;
   const int count = bp.count[b];
   const bool bank_full = (a.M > 0 && count == a.M);
 
@@ -235,22 +254,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   }
   const int n_tiles = (total + kKeys - 1) / kKeys;
 
-  // ---- set-up ---------------------------------------------------------------------------------
-  if (tid == 0) {
-    mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1);
-    mbar_init(bar_o, 1);
-    mbar_init(bar_p, kSoftmaxThreads);
-    mbar_init(bar_kv0, kLoaderThreads); mbar_init(bar_kv0 + 8, kLoaderThreads);
-    mbar_init(bar_free0, 1); mbar_init(bar_free0 + 8, 1);
-    mbar_init(bar_q, kSoftmaxThreads);
-    *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 8) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32((const void*)tmem_slot)), "r"(512u) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -537,10 +540,9 @@ cudaError_t prefill_attention_tc_init() {
 
 cudaError_t launch_prefill_attention_tc(const AttnArgs& a, const BatchParams& bp, int* status, cudaStream_t st) {
   dim3 grid((bp.rows_per_stream + kTok - 1) / kTok, a.Hkv, bp.n_active);
-  if (a.D == 128) prefill_attn_tc_kernel<128><<<grid, kAttnThreads, Smem<128>::kTotal, st>>>(a, bp, status);
-  else if (a.D == 64) prefill_attn_tc_kernel<64><<<grid, kAttnThreads, Smem<64>::kTotal, st>>>(a, bp, status);
-  else return cudaErrorInvalidValue;
-  return cudaGetLastError();
+  if (a.D == 128) return launch_pdl(prefill_attn_tc_kernel<128>, grid, dim3(kAttnThreads), (size_t)Smem<128>::kTotal, st, a, bp, status);
+  if (a.D == 64) return launch_pdl(prefill_attn_tc_kernel<64>, grid, dim3(kAttnThreads), (size_t)Smem<64>::kTotal, st, a, bp, status);
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace vs

@@ -87,6 +87,28 @@ struct Layout {
   size_t total;
 };
 
+// ---- programmatic dependent launch ------------------------------------------------------
+// Every kernel of a step is launched with programmatic stream serialisation: it may be
+// scheduled while its predecessor in the stream is still running, does its set-up (barriers,
+// tensor memory, descriptor prefetch), and only then waits for the predecessor to have
+// completed and flushed.  No kernel touches global memory before pdl_wait(), and every kernel
+// calls it, so completion is transitive along the stream.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 // ---- launch wrappers (each returns the cudaError_t of the launch) -----------------------
 struct PoolArgs {
   const bf16* hidden;            // [n_active][N][d]

@@ -22,6 +22,8 @@ __device__ __forceinline__ bf16 f64_to_bf16_rne(double x) {
 // once.  The sum of <= 256 bf16 values in fp64 is exact, hence independent of the order.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, int pool_blocks) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int b = blockIdx.y;
   const int sid = bp.stream_id[b];
   const int N = a.N, d = a.d;
@@ -95,11 +97,12 @@ cudaError_t launch_pool(const PoolArgs& a, const BatchParams& bp, cudaStream_t s
   const int pool_blocks = a.d / 64;
   const int rope_blocks = ((a.N + 1) * (a.D / 2) + 255) / 256;
   dim3 grid(pool_blocks + rope_blocks, bp.n_active);
-  pool_kernel<<<grid, 256, 0, st>>>(a, bp, pool_blocks);
-  return cudaGetLastError();
+  return launch_pdl(pool_kernel, grid, dim3(256), 0, st, a, bp, pool_blocks);
 }
 
 __global__ void __launch_bounds__(256) rope_table_kernel(RopeArgs a, BatchParams bp) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int b = blockIdx.y;
   const int half = a.D / 2, T = bp.rows_per_stream;
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -113,8 +116,7 @@ __global__ void __launch_bounds__(256) rope_table_kernel(RopeArgs a, BatchParams
 
 cudaError_t launch_rope_table(const RopeArgs& a, const BatchParams& bp, cudaStream_t st) {
   dim3 grid((bp.rows_per_stream * (a.D / 2) + 255) / 256, bp.n_active);
-  rope_table_kernel<<<grid, 256, 0, st>>>(a, bp);
-  return cudaGetLastError();
+  return launch_pdl(rope_table_kernel, grid, dim3(256), 0, st, a, bp);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -127,6 +129,8 @@ cudaError_t launch_rope_table(const RopeArgs& a, const BatchParams& bp, cudaStre
 __global__ void __launch_bounds__(256) rms_stats_kernel(const bf16* __restrict__ h, const bf16* __restrict__ gain,
                                                         bf16* __restrict__ hg, float* __restrict__ row_scale,
                                                         int d, float eps) {
+  pdl_wait();
+  pdl_launch_dependents();
   const size_t row = blockIdx.x;
   const bf16* src = h + row * d;
   float ss = 0.f;
@@ -153,8 +157,7 @@ __global__ void __launch_bounds__(256) rms_stats_kernel(const bf16* __restrict__
 
 cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* row_scale, int rows, int d, float eps,
                              cudaStream_t st) {
-  rms_stats_kernel<<<rows, 256, 0, st>>>(h, gain, hg, row_scale, d, eps);
-  return cudaGetLastError();
+  return launch_pdl(rms_stats_kernel, dim3(rows), dim3(256), 0, st, h, gain, hg, row_scale, d, eps);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -176,6 +179,8 @@ __device__ __forceinline__ double warp_tree_sum(double v) {
 }
 
 __global__ void __launch_bounds__(256) bank_update_kernel(BankUpdateArgs a, BatchParams bp) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int b = blockIdx.y;
   const int sid = bp.stream_id[b];
   StreamMeta* meta = a.meta + sid;
@@ -289,11 +294,11 @@ __global__ void __launch_bounds__(256) bank_update_kernel(BankUpdateArgs a, Batc
 
 cudaError_t launch_bank_update(const BankUpdateArgs& a, const BatchParams& bp, bool any_full, cudaStream_t st) {
   dim3 grid(any_full ? (a.M + 7) / 8 : 1, bp.n_active);
-  bank_update_kernel<<<grid, 256, 0, st>>>(a, bp);
-  return cudaGetLastError();
+  return launch_pdl(bank_update_kernel, grid, dim3(256), 0, st, a, bp);
 }
 
 __global__ void poison_kernel(uint32_t* p, size_t n) {
+  pdl_wait();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
     p[i] = 0xFFFFFFFFu;
 }
@@ -306,6 +311,7 @@ cudaError_t launch_poison(void* p, size_t bytes, cudaStream_t st) {
 // a stream starts over (new video): empty bank, no history; K/V payloads need no clearing
 // because nothing reads a slot that the metadata does not list
 __global__ void reset_kernel(StreamMeta* meta, int32_t* slot_frame, int slots, BatchParams bp) {
+  pdl_wait();
   const int sid = bp.stream_id[blockIdx.x];
   for (int i = threadIdx.x; i < slots; i += blockDim.x) slot_frame[(size_t)sid * slots + i] = -1;
   if (threadIdx.x == 0) {
