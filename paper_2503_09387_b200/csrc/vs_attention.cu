@@ -2,12 +2,11 @@
 // query token per stream attends over [prompt prefix | carrier bank | text of the turn].  No
 // visual-token K/V exists at this point -- only carriers.
 //
-// grid = (key splits, KV heads, streams), 256 threads.  A group of D/8 lanes owns one key row
-// and reads it with 128-bit loads; every lane issues the K and V loads of four keys before it
-// uses any of them, so a warp has 8 key rows (4 KB) in flight.  The G query heads of the group
-// are kept in registers and share each key.  Warps merge their running (m, l, o) through
-// shared memory; with several key splits the last CTA of a (stream, KV head) to finish
-// combines the partial triples -- no CTA ever waits for another.
+// grid = (key splits, query heads, streams), 256 threads.  A group of D/8 lanes owns one key
+// row and reads it with 128-bit loads; every lane issues the K and V loads of four keys before
+// it uses any of them, so a warp has 8 key rows (4 KB) in flight.  Warps merge their running
+// (m, l, o) by shuffles and through shared memory; with several key splits the last CTA of a
+// (stream, query head) to finish combines the partial triples -- no CTA ever waits for another.
 #include "vs_common.cuh"
 
 namespace vs {
@@ -16,24 +15,26 @@ namespace {
 
 constexpr int kDecThreads = 256;
 constexpr int kDecWarps = kDecThreads / 32;
-constexpr int GMAX = 8;
 constexpr int kBatch = 4;     // keys a lane group loads before computing
 
+// One CTA = one query head x one key split x one stream.  The heads of a KV group read the
+// same K/V rows from L2; spreading them over CTAs keeps every SM's instruction stream short,
+// which is what bounds this kernel (a few hundred keys of 256 bytes each).
 template <int D>
 __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, BatchParams bp) {
   constexpr int LPK = D / 8;            // lanes that share one key row (16 bytes each)
   constexpr int KPW = 32 / LPK;         // lane groups (keys in parallel) per warp
-  __shared__ float st_m[kDecWarps][GMAX];
-  __shared__ float st_l[kDecWarps][GMAX];
-  __shared__ float st_o[kDecWarps][GMAX][D];
-  __shared__ float sp_w[DEC_SPLIT_MAX][GMAX];
+  __shared__ float st_m[kDecWarps];
+  __shared__ float st_l[kDecWarps];
+  __shared__ float st_o[kDecWarps][D];
+  __shared__ float sp_w[DEC_SPLIT_MAX];
   __shared__ int is_last;
 
   pdl_wait();
   pdl_launch_dependents();
-  const int split = blockIdx.x, hkv = blockIdx.y, b = blockIdx.z;
+  const int split = blockIdx.x, qh = blockIdx.y, b = blockIdx.z;
   const int sid = bp.stream_id[b];
-  const int G = a.Hq / a.Hkv;
+  const int hkv = qh / (a.Hq / a.Hkv);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sub = lane / LPK, li = lane % LPK;
   const int count = bp.count[b];
@@ -55,34 +56,24 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
   const bf16* tk = a.tail_k + hoff * a.maxT * D + li * 8;
   const bf16* tv = a.tail_v + hoff * a.maxT * D + li * 8;
 
-  // query (bf16 hi + lo pair) of the G heads, pre-scaled into the log2 domain
-  float q[GMAX][8];
+  // this lane's 8 dims of the query (bf16 hi + lo pair), pre-scaled into the log2 domain
+  float q[8];
+  {
+    const size_t qo = (size_t)b * a.Hq * D + (size_t)qh * D + li * 8;
+    const uint4 raw = *reinterpret_cast<const uint4*>(a.q + qo);
+    const uint4 raw_lo = *reinterpret_cast<const uint4*>(a.q_lo + qo);
+    const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+    const __nv_bfloat162* l2 = reinterpret_cast<const __nv_bfloat162*>(&raw_lo);
 #pragma unroll
-  for (int g = 0; g < GMAX; ++g) {
-    if (g < G) {
-      const size_t qo = (size_t)b * a.Hq * D + (size_t)(hkv * G + g) * D + li * 8;
-      const uint4 raw = *reinterpret_cast<const uint4*>(a.q + qo);
-      const uint4 raw_lo = *reinterpret_cast<const uint4*>(a.q_lo + qo);
-      const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
-      const __nv_bfloat162* l2 = reinterpret_cast<const __nv_bfloat162*>(&raw_lo);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float2 f = __bfloat1622float2(h2[i]);
-        const float2 fl = __bfloat1622float2(l2[i]);
-        q[g][2 * i] = (f.x + fl.x) * a.scale_log2e; q[g][2 * i + 1] = (f.y + fl.y) * a.scale_log2e;
-      }
-    } else {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) q[g][i] = 0.f;
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __bfloat1622float2(h2[i]);
+      const float2 fl = __bfloat1622float2(l2[i]);
+      q[2 * i] = (f.x + fl.x) * a.scale_log2e; q[2 * i + 1] = (f.y + fl.y) * a.scale_log2e;
     }
   }
-  float m[GMAX], l[GMAX], o[GMAX][8];
+  float m = -INFINITY, l = 0.f, o[8];
 #pragma unroll
-  for (int g = 0; g < GMAX; ++g) {
-    m[g] = -INFINITY; l[g] = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) o[g][i] = 0.f;
-  }
+  for (int i = 0; i < 8; ++i) o[i] = 0.f;
 
   // keys of this CTA are dealt to (warp, lane group) round-robin, kBatch at a time
   constexpr int kStride = kDecWarps * KPW;
@@ -106,49 +97,38 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
       kr[u] = act[u] ? *reinterpret_cast<const uint4*>(kp) : make_uint4(0, 0, 0, 0);
       vr[u] = act[u] ? *reinterpret_cast<const uint4*>(vp) : make_uint4(0, 0, 0, 0);
     }
-    float s[kBatch][GMAX];
+    float s[kBatch];
+    float mx = m;
 #pragma unroll
     for (int u = 0; u < kBatch; ++u) {
-      float kf[8];
       const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kr[u]);
+      float d = 0.f;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(k2[i]); kf[2 * i] = f.x; kf[2 * i + 1] = f.y; }
-#pragma unroll
-      for (int g = 0; g < GMAX; ++g) {
-        float d = 0.f;
-        if (g < G) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) d = fmaf(q[g][i], kf[i], d);
-#pragma unroll
-          for (int off = LPK / 2; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
-        }
-        s[u][g] = act[u] ? d : -INFINITY;
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __bfloat1622float2(k2[i]);
+        d = fmaf(q[2 * i], f.x, d); d = fmaf(q[2 * i + 1], f.y, d);
       }
+#pragma unroll
+      for (int off = LPK / 2; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+      s[u] = act[u] ? d : -INFINITY;
+      mx = fmaxf(mx, s[u]);
     }
+    if (mx > -INFINITY) {
+      const float sc = exp2f(m - mx);                    // exp2f(-inf) = 0 on the first keys
+      l *= sc;
 #pragma unroll
-    for (int g = 0; g < GMAX; ++g) {
-      if (g < G) {
-        float mx = m[g];
+      for (int i = 0; i < 8; ++i) o[i] *= sc;
+      m = mx;
 #pragma unroll
-        for (int u = 0; u < kBatch; ++u) mx = fmaxf(mx, s[u][g]);
-        if (mx > -INFINITY) {
-          const float sc = exp2f(m[g] - mx);             // exp2f(-inf) = 0 on the first keys
-          l[g] *= sc;
+      for (int u = 0; u < kBatch; ++u) {
+        const float p = exp2f(s[u] - mx);
+        l += p;
+        const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&vr[u]);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) o[g][i] *= sc;
-          m[g] = mx;
-#pragma unroll
-          for (int u = 0; u < kBatch; ++u) {
-            const float p = exp2f(s[u][g] - mx);
-            l[g] += p;
-            const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&vr[u]);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const float2 f = __bfloat1622float2(v2[i]);
-              o[g][2 * i] = fmaf(p, f.x, o[g][2 * i]);
-              o[g][2 * i + 1] = fmaf(p, f.y, o[g][2 * i + 1]);
-            }
-          }
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __bfloat1622float2(v2[i]);
+          o[2 * i] = fmaf(p, f.x, o[2 * i]);
+          o[2 * i + 1] = fmaf(p, f.y, o[2 * i + 1]);
         }
       }
     }
@@ -157,121 +137,107 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
   // lane groups of a warp merge by shuffles (they own the same dims of different keys)
 #pragma unroll
   for (int off = LPK; off < 32; off <<= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, off);
+    const float l2 = __shfl_xor_sync(0xffffffffu, l, off);
+    const float mn = fmaxf(m, m2);
+    const float w1 = (m == -INFINITY) ? 0.f : exp2f(m - mn);
+    const float w2 = (m2 == -INFINITY) ? 0.f : exp2f(m2 - mn);
+    l = l * w1 + l2 * w2;
 #pragma unroll
-    for (int g = 0; g < GMAX; ++g) {
-      if (g < G) {
-        const float m2 = __shfl_xor_sync(0xffffffffu, m[g], off);
-        const float l2 = __shfl_xor_sync(0xffffffffu, l[g], off);
-        const float mn = fmaxf(m[g], m2);
-        const float w1 = (m[g] == -INFINITY) ? 0.f : exp2f(m[g] - mn);
-        const float w2 = (m2 == -INFINITY) ? 0.f : exp2f(m2 - mn);
-        l[g] = l[g] * w1 + l2 * w2;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float o2 = __shfl_xor_sync(0xffffffffu, o[g][i], off);
-          o[g][i] = o[g][i] * w1 + o2 * w2;
-        }
-        m[g] = mn;
-      }
+    for (int i = 0; i < 8; ++i) {
+      const float o2 = __shfl_xor_sync(0xffffffffu, o[i], off);
+      o[i] = o[i] * w1 + o2 * w2;
     }
+    m = mn;
   }
   if (sub == 0) {
+    if (li == 0) { st_m[warp] = m; st_l[warp] = l; }
 #pragma unroll
-    for (int g = 0; g < GMAX; ++g) {
-      if (g < G) {
-        if (li == 0) { st_m[warp][g] = m[g]; st_l[warp][g] = l[g]; }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) st_o[warp][g][li * 8 + i] = o[g][i];
-      }
-    }
+    for (int i = 0; i < 8; ++i) st_o[warp][li * 8 + i] = o[i];
   }
   __syncthreads();
 
   // warps -> CTA
   const bool direct = a.nsplit == 1;
-  float* part = a.partials + (((size_t)split * bp.n_active + b) * a.Hq + (size_t)hkv * G) * (D + 2);
-  for (int idx = threadIdx.x; idx < G * D; idx += kDecThreads) {
-    const int g = idx / D, c = idx - g * D;
+  float* part = a.partials + (((size_t)split * bp.n_active + b) * a.Hq + qh) * (D + 2);
+  const size_t out_off = (size_t)b * a.Hq * D + (size_t)qh * D;
+  if (threadIdx.x < D) {
+    const int c = threadIdx.x;
     float M = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < kDecWarps; ++w) M = fmaxf(M, st_m[w][g]);
+    for (int w = 0; w < kDecWarps; ++w) M = fmaxf(M, st_m[w]);
     float L = 0.f, O = 0.f;
 #pragma unroll
     for (int w = 0; w < kDecWarps; ++w) {
-      const float wt = (st_m[w][g] == -INFINITY) ? 0.f : exp2f(st_m[w][g] - M);
-      L += st_l[w][g] * wt;
-      O += st_o[w][g][c] * wt;
+      const float wt = (st_m[w] == -INFINITY) ? 0.f : exp2f(st_m[w] - M);
+      L += st_l[w] * wt;
+      O += st_o[w][c] * wt;
     }
     if (direct) {
       const float val = (L > 0.f) ? O / L : 0.f;
-      const size_t off = (size_t)b * a.Hq * D + (size_t)(hkv * G + g) * D + c;
-      if (a.out_fp32) static_cast<float*>(a.out)[off] = val;
-      else static_cast<bf16*>(a.out)[off] = __float2bfloat16_rn(val);
-      if (a.h_out != nullptr) a.h_out[off] = __float2bfloat16_rn(__bfloat162float(a.h_in[off]) + val);
+      if (a.out_fp32) static_cast<float*>(a.out)[out_off + c] = val;
+      else static_cast<bf16*>(a.out)[out_off + c] = __float2bfloat16_rn(val);
+      if (a.h_out != nullptr) a.h_out[out_off + c] = __float2bfloat16_rn(__bfloat162float(a.h_in[out_off + c]) + val);
     } else {
-      part[(size_t)g * (D + 2) + c] = O;
-      if (c == 0) { part[(size_t)g * (D + 2) + D] = M; part[(size_t)g * (D + 2) + D + 1] = L; }
+      part[c] = O;
+      if (c == 0) { part[D] = M; part[D + 1] = L; }
     }
   }
   if (direct) return;
 
-  // last CTA of this (stream, KV head) combines the splits
+  // last CTA of this (stream, query head) combines the splits
   __threadfence();
   __syncthreads();
-  if (threadIdx.x == 0) is_last = (atomicAdd(a.tickets + sid * a.Hkv + hkv, 1) == a.nsplit - 1);
+  if (threadIdx.x == 0) is_last = (atomicAdd(a.tickets + sid * a.Hq + qh, 1) == a.nsplit - 1);
   __syncthreads();
   if (!is_last) return;
   __threadfence();
-  // weights of the splits per head, then every output element with all its loads in flight
-  if (threadIdx.x < G) {
-    const int g = threadIdx.x, qh = hkv * G + g;
+  if (threadIdx.x == 0) {
     float ms[DEC_SPLIT_MAX], ls[DEC_SPLIT_MAX];
     float M = -INFINITY;
 #pragma unroll
-    for (int s = 0; s < DEC_SPLIT_MAX; ++s) {
-      if (s < a.nsplit) {
-        const float* pp = a.partials + (((size_t)s * bp.n_active + b) * a.Hq + qh) * (D + 2);
-        ms[s] = __ldcg(pp + D); ls[s] = __ldcg(pp + D + 1);
-        M = fmaxf(M, ms[s]);
+    for (int s2 = 0; s2 < DEC_SPLIT_MAX; ++s2) {
+      if (s2 < a.nsplit) {
+        const float* pp = a.partials + (((size_t)s2 * bp.n_active + b) * a.Hq + qh) * (D + 2);
+        ms[s2] = __ldcg(pp + D); ls[s2] = __ldcg(pp + D + 1);
+        M = fmaxf(M, ms[s2]);
       }
     }
     float L = 0.f;
 #pragma unroll
-    for (int s = 0; s < DEC_SPLIT_MAX; ++s) {
-      if (s < a.nsplit) {
-        const float wt = (ms[s] == -INFINITY) ? 0.f : exp2f(ms[s] - M);
-        L += ls[s] * wt;
-        sp_w[s][g] = wt;
+    for (int s2 = 0; s2 < DEC_SPLIT_MAX; ++s2) {
+      if (s2 < a.nsplit) {
+        const float wt = (ms[s2] == -INFINITY) ? 0.f : exp2f(ms[s2] - M);
+        L += ls[s2] * wt;
+        sp_w[s2] = wt;
       }
     }
     const float inv = (L > 0.f) ? 1.f / L : 0.f;
 #pragma unroll
-    for (int s = 0; s < DEC_SPLIT_MAX; ++s) if (s < a.nsplit) sp_w[s][g] *= inv;
+    for (int s2 = 0; s2 < DEC_SPLIT_MAX; ++s2) if (s2 < a.nsplit) sp_w[s2] *= inv;
   }
   __syncthreads();
-  for (int idx = threadIdx.x; idx < G * D; idx += kDecThreads) {
-    const int g = idx / D, c = idx - g * D;
-    const int qh = hkv * G + g;
+  if (threadIdx.x < D) {
+    const int c = threadIdx.x;
     float v[DEC_SPLIT_MAX];
 #pragma unroll
-    for (int s = 0; s < DEC_SPLIT_MAX; ++s)
-      v[s] = (s < a.nsplit) ? __ldcg(a.partials + (((size_t)s * bp.n_active + b) * a.Hq + qh) * (D + 2) + c) : 0.f;
+    for (int s2 = 0; s2 < DEC_SPLIT_MAX; ++s2)
+      v[s2] = (s2 < a.nsplit) ? __ldcg(a.partials + (((size_t)s2 * bp.n_active + b) * a.Hq + qh) * (D + 2) + c) : 0.f;
     float val = 0.f;
 #pragma unroll
-    for (int s = 0; s < DEC_SPLIT_MAX; ++s) if (s < a.nsplit) val = fmaf(v[s], sp_w[s][g], val);
-    const size_t off = (size_t)b * a.Hq * D + (size_t)qh * D + c;
-    if (a.out_fp32) static_cast<float*>(a.out)[off] = val;
-    else static_cast<bf16*>(a.out)[off] = __float2bfloat16_rn(val);
-    if (a.h_out != nullptr) a.h_out[off] = __float2bfloat16_rn(__bfloat162float(a.h_in[off]) + val);
+    for (int s2 = 0; s2 < DEC_SPLIT_MAX; ++s2) if (s2 < a.nsplit) val = fmaf(v[s2], sp_w[s2], val);
+    if (a.out_fp32) static_cast<float*>(a.out)[out_off + c] = val;
+    else static_cast<bf16*>(a.out)[out_off + c] = __float2bfloat16_rn(val);
+    if (a.h_out != nullptr) a.h_out[out_off + c] = __float2bfloat16_rn(__bfloat162float(a.h_in[out_off + c]) + val);
   }
-  if (threadIdx.x == 0) a.tickets[sid * a.Hkv + hkv] = 0;
+  if (threadIdx.x == 0) a.tickets[sid * a.Hq + qh] = 0;
 }
 
 }  // namespace
 
 cudaError_t launch_decode_attention(const DecodeArgs& a, const BatchParams& bp, cudaStream_t st) {
-  if (a.nsplit < 1 || a.nsplit > DEC_SPLIT_MAX || a.Hq / a.Hkv > GMAX) return cudaErrorInvalidValue;
-  dim3 grid(a.nsplit, a.Hkv, bp.n_active);
+  if (a.nsplit < 1 || a.nsplit > DEC_SPLIT_MAX) return cudaErrorInvalidValue;
+  dim3 grid(a.nsplit, a.Hq, bp.n_active);
   if (a.D == 128) return launch_pdl(decode_attn_kernel<128>, grid, dim3(kDecThreads), 0, st, a, bp);
   if (a.D == 64) return launch_pdl(decode_attn_kernel<64>, grid, dim3(kDecThreads), 0, st, a, bp);
   return cudaErrorInvalidValue;

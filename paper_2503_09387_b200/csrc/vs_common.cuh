@@ -71,7 +71,7 @@ struct Layout {
   size_t scores;                // f64   [S][slots]
   size_t inv_freq;              // f64   [D/2]
   size_t status;                // int32 [8]
-  size_t tickets;               // int32 [S*Hkv]
+  size_t tickets;               // int32 [S*Hq]  split-KV decode: CTAs finished per (stream, query head)
   size_t persistent_end;
   // per-step scratch
   size_t hbuf[2];               // bf16 [R_max][d]  residual ping-pong; hbuf[0] holds [E; carrier]
@@ -190,7 +190,7 @@ struct DecodeArgs {
   const bf16* bank_k;   const bf16* bank_v;    // [S][Hkv][slots][D]
   const bf16* tail_k;   const bf16* tail_v;    // [S][Hkv][maxT][D]
   float* partials;               // [nsplit][n_active][Hq][D+2]
-  int* tickets;                  // [S*Hkv]
+  int* tickets;                  // [S*Hq]
   void* out;                     // [n_active][Hq*D], bf16 or fp32
   int out_fp32;
   const bf16* h_in; bf16* h_out;

@@ -74,7 +74,7 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.scores = take((size_t)D.S * D.slots * 8);
   Lo.inv_freq = take((size_t)(D.D / 2) * 8);
   Lo.status = take(8 * 4);
-  Lo.tickets = take((size_t)D.S * D.Hkv * 4);
+  Lo.tickets = take((size_t)D.S * D.Hq * 4);
   Lo.persistent_end = off;
   Lo.scratch_begin = off;
   Lo.hbuf[0] = take((size_t)D.R_max * D.d * 2);
