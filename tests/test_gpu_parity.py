@@ -298,3 +298,55 @@ def test_batched_streams_full_shape():
         assert st["frames_seen"] == lengths[s] and st["count"] == lengths[s]
     print("batched: lengths", lengths, "worst", p.worst)
     p.close()
+
+
+# ------------------------------------------------------------------ limits and degenerate shapes
+def test_largest_frame_and_widest_group():
+    """N = 255 (256-column token tile, the MMA's widest), 8 query heads per KV head (a full
+    128-row stacked query block), head_dim 64, three KV heads (feature tiles end mid-way)."""
+    w = synth.workload("tiny", d_model=512, n_q_heads=24, n_kv_heads=3, head_dim=64, tokens_per_frame=255,
+                       prefix_len=5, n_frames=3, bank_capacity=2, question_len=64, decode_tokens=2, seed=9)
+    p = Pair(w, max_text=66)
+    run_stream(p, w)
+    p.close()
+
+
+def test_large_bank_with_evictions_and_long_decode_context():
+    """Bank of 300 carriers, 340 one-token... short frames: 40 evictions, decode over > 256 keys
+    (split-KV path with the last-CTA combine), both eviction policies."""
+    for policy in (0, 1):
+        w = synth.workload("long", d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64, tokens_per_frame=3,
+                           prefix_len=16, n_frames=340, bank_capacity=300, question_len=9, decode_tokens=3,
+                           cut_period=50, seed=30 + policy)
+        p = Pair(w, evict_policy=policy, max_text=12)
+        p.text([0], [w.prefix_hidden()], "prefix")
+        shared = w.frame_shared()
+        for t in range(w.n_frames):
+            p.frame([0], [w.frame_hidden(t, shared=shared)], f"frame {t}", mode="full" if t % 37 == 0 or t > 335 else "carrier")
+        st = p.check_bank(0)
+        assert st["evictions"] == 40 and st["count"] == 300
+        p.text([0], [w.question_hidden()], "question")
+        for i in range(w.decode_tokens):
+            p.text([0], [w.decode_hidden(i)], f"decode {i}")
+        p.close()
+
+
+def test_argument_errors_leave_the_stream_untouched():
+    w = synth.workload("tiny")
+    p = Pair(w)
+    x = to_dev(w.frame_hidden(0)[None])
+    for bad_ids in ([1], [0, 0], [-1]):
+        with pytest.raises(binding.VsError) as e:
+            p.gpu.frame_prefill(bad_ids, x if len(bad_ids) == 1 else torch.cat([x, x]))
+        assert e.value.code == binding.VS_ERR_INVALID_ARG
+    big = to_dev(synth.normal_bf16(1, synth.TAG_PREFIX, (1, 17, w.d_model)))
+    with pytest.raises(binding.VsError) as e:
+        p.gpu.frame_prefill([0], big)
+    assert e.value.code == binding.VS_ERR_CAPACITY
+    with pytest.raises(binding.VsError) as e:       # prefix capacity is 8
+        p.gpu.decode_step([0], to_dev(synth.normal_bf16(1, synth.TAG_PREFIX, (1, 9, w.d_model))))
+    assert e.value.code == binding.VS_ERR_CAPACITY
+    st = p.gpu.bank_state(0)
+    assert st["frames_seen"] == 0 and st["prefix_len"] == 0 and st["device_status"] == 0
+    run_stream(p, w)                                   # and the stream still works from scratch
+    p.close()
