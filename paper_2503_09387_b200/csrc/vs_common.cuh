@@ -51,7 +51,7 @@ struct Dims {
   float rope_theta, rms_eps;
 };
 
-constexpr int KSPLIT_MAX = 8;
+constexpr int KSPLIT_MAX = 4;   // cluster size of the projection along K
 constexpr int DEC_SPLIT_MAX = 16;
 constexpr int GEMM_BLOCK_M = 128;
 constexpr int GEMM_BLOCK_K = 64;
@@ -153,7 +153,7 @@ struct GemmArgs {
   CUtensorMap tm_x;              // [rows, d] bf16, box 64 x tile_n, 128-byte swizzle
   ProjectionOut out;
   int rows, E_out, d;
-  int tile_n, n_tiles, ksplit;   // ksplit = cluster size: 1, 2, 4 or 8
+  int tile_n, n_tiles, ksplit;   // ksplit = cluster size: 1, 2 or 4
   int* status;
 };
 cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream_t st);

@@ -226,27 +226,9 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   // C  the owner of a slice sums the ksplit partials of its tokens (float4 reads of the peers'
   //    shared memory), adds the bias, rotates, rounds and stores; a last cluster barrier keeps
   //    every CTA's shared memory alive until its peers have read it.
-  const int slice = p.tile_n / p.ksplit;          // tile_n is a multiple of 16, ksplit of 1, 2, 4, 8
-  constexpr int kPre = 6;                          // rows whose RoPE entries a thread fetches ahead
-  float4 rope_a[kPre], rope_b[kPre];
+  const int slice = p.tile_n / p.ksplit;          // tile_n is a multiple of 16, ksplit is 1, 2 or 4
   bool acc_ok = true;
   if (warp >= 2) {
-    // while the main loop runs: fetch the (cos, sin) entries this thread will need in phase C
-    const int te = threadIdx.x - 64;
-    const int half = p.o.D >> 1;
-    const int p0 = (te & 15) * 4;
-    const int k0 = p0 - (p0 / half) * half;
-#pragma unroll
-    for (int i = 0; i < kPre; ++i) {
-      const int t = (int)blockIdx.z * slice + (te >> 4) + 8 * i;
-      const int row = n0 + t;
-      if (8 * i + (te >> 4) < slice && row < p.rows) {
-        rope_a[i] = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0);
-        rope_b[i] = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0 + 2);
-      } else {
-        rope_a[i] = make_float4(1.f, 0.f, 1.f, 0.f); rope_b[i] = rope_a[i];
-      }
-    }
     acc_ok = __all_sync(0xffffffffu, mbar_wait(tmem_full_bar, 0, abort_flag));   // warp-uniform
   }
   tcgen05_fence_after();
@@ -269,7 +251,9 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   __syncthreads();
   if (p.ksplit > 1) cluster_sync_all();
 
-  // phase C.  Thread = (group of 4 rotation pairs, token lane); float4 reads.
+  // phase C.  Thread = (group of 4 rotation pairs, token lane).  The reads of a row -- float4
+  // pieces of every CTA's partial tile through distributed shared memory, and the row's RoPE
+  // entries -- are issued one row ahead of the arithmetic (two register buffers).
   if (warp >= 2 && !*abort_flag) {
     const int te = threadIdx.x - 64;               // 0..127
     const int D = p.o.D, half = D >> 1;
@@ -277,11 +261,12 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
     const int hl = p0 / half, k0 = p0 - hl * half; // local head, index inside the half head
     const int f1 = hl * D + k0, f2 = f1 + half;
     const int hs = (m0 + f1) / D;                  // head slot: Q heads, then K heads, then V heads
+    const bool rotate = hs < p.o.Hq + p.o.Hkv;
     const int t_begin = (int)blockIdx.z * slice;
-    const float* part[8];
+    const float* part[KSPLIT_MAX];
     cg::cluster_group cluster = cg::this_cluster();
 #pragma unroll
-    for (int r = 0; r < 8; ++r)
+    for (int r = 0; r < KSPLIT_MAX; ++r)
       part[r] = (p.ksplit > 1 && r < p.ksplit) ? cluster.map_shared_rank(part_local, r) : part_local;
     if (m0 + f2 + 3 < p.E_out) {
       float bb1[4] = {0.f, 0.f, 0.f, 0.f}, bb2[4] = {0.f, 0.f, 0.f, 0.f};
@@ -293,42 +278,41 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
         }
       }
       const int rps = bp.rows_per_stream;
-#pragma unroll 1
-      for (int it = 0; it * 8 + (te >> 4) < slice; ++it) {
+      const int n_it = (slice - (te >> 4) + 7) / 8;          // rows this thread finishes
+      struct RowRegs { float4 v1[KSPLIT_MAX], v2[KSPLIT_MAX], ra, rb; float rsc; };
+      auto valid_it = [&](int it) { return it < n_it && n0 + t_begin + (te >> 4) + 8 * it < p.rows; };
+      auto load_row = [&](RowRegs& R, int it) {
         const int t = t_begin + (te >> 4) + 8 * it;
         const int row = n0 + t;
-        if (row >= p.rows) break;
-        float4 v1[8], v2[8];
 #pragma unroll
-        for (int r = 0; r < 8; ++r) {
+        for (int r = 0; r < KSPLIT_MAX; ++r) {
           if (r < p.ksplit) {
-            v1[r] = *reinterpret_cast<const float4*>(part[r] + t * GEMM_BLOCK_M + f1);
-            v2[r] = *reinterpret_cast<const float4*>(part[r] + t * GEMM_BLOCK_M + f2);
+            R.v1[r] = *reinterpret_cast<const float4*>(part[r] + t * GEMM_BLOCK_M + f1);
+            R.v2[r] = *reinterpret_cast<const float4*>(part[r] + t * GEMM_BLOCK_M + f2);
           }
         }
-        float x1[4] = {0.f, 0.f, 0.f, 0.f}, x2[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int r = 0; r < 8; ++r) {
-          if (r < p.ksplit) {
-            x1[0] += v1[r].x; x1[1] += v1[r].y; x1[2] += v1[r].z; x1[3] += v1[r].w;
-            x2[0] += v2[r].x; x2[1] += v2[r].y; x2[2] += v2[r].z; x2[3] += v2[r].w;
-          }
+        if (rotate) {
+          R.ra = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0);
+          R.rb = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0 + 2);
         }
         // RMSNorm's row scale commutes with the projection: applied here, in fp32
-        const float rsc = (p.o.row_scale != nullptr) ? p.o.row_scale[row] : 1.f;
+        R.rsc = (p.o.row_scale != nullptr) ? p.o.row_scale[row] : 1.f;
+      };
+      auto finish_row = [&](const RowRegs& R, int it) {
+        const int t = t_begin + (te >> 4) + 8 * it;
+        const int row = n0 + t;
+        float x1[4] = {0.f, 0.f, 0.f, 0.f}, x2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { x1[i] = fmaf(x1[i], rsc, bb1[i]); x2[i] = fmaf(x2[i], rsc, bb2[i]); }
-        if (hs < p.o.Hq + p.o.Hkv) {
-          float4 ra, rb;
-          if (it < kPre) {
-            ra = rope_a[0]; rb = rope_b[0];
-#pragma unroll
-            for (int i = 1; i < kPre; ++i) if (i == it) { ra = rope_a[i]; rb = rope_b[i]; }
-          } else {
-            ra = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0);
-            rb = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0 + 2);
+        for (int r = 0; r < KSPLIT_MAX; ++r) {
+          if (r < p.ksplit) {
+            x1[0] += R.v1[r].x; x1[1] += R.v1[r].y; x1[2] += R.v1[r].z; x1[3] += R.v1[r].w;
+            x2[0] += R.v2[r].x; x2[1] += R.v2[r].y; x2[2] += R.v2[r].z; x2[3] += R.v2[r].w;
           }
-          const float cs[4] = {ra.x, ra.z, rb.x, rb.z}, sn[4] = {ra.y, ra.w, rb.y, rb.w};
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { x1[i] = fmaf(x1[i], R.rsc, bb1[i]); x2[i] = fmaf(x2[i], R.rsc, bb2[i]); }
+        if (rotate) {
+          const float cs[4] = {R.ra.x, R.ra.z, R.rb.x, R.rb.z}, sn[4] = {R.ra.y, R.ra.w, R.rb.y, R.rb.w};
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const float y1 = x1[i] * cs[i] - x2[i] * sn[i];
@@ -377,6 +361,15 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
             *reinterpret_cast<uint2*>(dst + half) = w2;
           }
         }
+      };
+      RowRegs A, B;
+      if (valid_it(0)) load_row(A, 0);
+#pragma unroll 1
+      for (int it = 0; valid_it(it); it += 2) {
+        if (valid_it(it + 1)) load_row(B, it + 1);
+        finish_row(A, it);
+        if (valid_it(it + 2)) load_row(A, it + 2);
+        if (valid_it(it + 1)) finish_row(B, it + 1);
       }
     }
   }
@@ -410,7 +403,7 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   p.tile_n = a.tile_n;
   p.ksplit = a.ksplit;
   const int total_kb = a.d / GEMM_BLOCK_K;
-  if (a.ksplit < 1 || a.ksplit > 8 || (a.ksplit & (a.ksplit - 1)) || total_kb % a.ksplit != 0) return cudaErrorInvalidValue;
+  if (a.ksplit < 1 || a.ksplit > KSPLIT_MAX || (a.ksplit & (a.ksplit - 1)) || total_kb % a.ksplit != 0) return cudaErrorInvalidValue;
   if (a.tile_n < 16 || a.tile_n > 256 || (a.tile_n & 15)) return cudaErrorInvalidValue;
   if (128 % a.out.D != 0) return cudaErrorInvalidValue;
   p.kblocks = total_kb / a.ksplit;

@@ -136,7 +136,7 @@ void choose_tiles(const Dims& D, int rows, int& tile_n, int& n_tiles, int& kspli
   tile_n = (per + 15) / 16 * 16;
   const int m_tiles = (D.E_out + GEMM_BLOCK_M - 1) / GEMM_BLOCK_M;
   const int total_kb = D.d / GEMM_BLOCK_K;
-  ksplit = 1;                                  // cluster size along K: 1, 2, 4 or 8
+  ksplit = 1;                                  // cluster size along K: 1, 2 or 4
   for (int ks = 1; ks <= KSPLIT_MAX; ks *= 2) {
     if (total_kb % ks != 0) continue;
     if (m_tiles * n_tiles * ks <= 148) ksplit = ks;
