@@ -51,10 +51,11 @@ struct Dims {
   float rope_theta, rms_eps;
 };
 
-constexpr int KSPLIT_MAX = 4;   // cluster size of the projection along K
+constexpr int KSPLIT_MAX = 4;   // CTAs sharing one output tile of the projection along K
 constexpr int DEC_SPLIT_MAX = 16;
 constexpr int GEMM_BLOCK_M = 128;
 constexpr int GEMM_BLOCK_K = 64;
+constexpr int GEMM_XCHG_CTAS = 160;   // most CTAs a K-split projection launches (one per SM)
 
 // ---- workspace layout (byte offsets from the workspace base) ----------------------------
 struct Layout {
@@ -72,6 +73,7 @@ struct Layout {
   size_t inv_freq;              // f64   [D/2]
   size_t status;                // int32 [8]
   size_t tickets;               // int32 [S*Hq]  split-KV decode: CTAs finished per (stream, query head)
+  size_t gemm_flags;            // int32 [GEMM_XCHG_CTAS]  projection K split: partials delivered per slice owner
   size_t persistent_end;
   // per-step scratch
   size_t hbuf[2];               // bf16 [R_max][d]  residual ping-pong; hbuf[0] holds [E; carrier]
@@ -83,6 +85,7 @@ struct Layout {
   size_t rope;                  // float2 [R_max][D/2]
   size_t obuf;                  // f32  [R_max][Hq*D] (holds bf16 or fp32 rows)
   size_t dec_part;              // f32  [DEC_SPLIT_MAX][S][Hq][D+2]
+  size_t gemm_xchg;             // f32  [GEMM_XCHG_CTAS][256][128]  projection K split: partial tiles
   size_t scratch_begin, scratch_end;
   size_t total;
 };
@@ -153,7 +156,10 @@ struct GemmArgs {
   CUtensorMap tm_x;              // [rows, d] bf16, box 64 x tile_n, 128-byte swizzle
   ProjectionOut out;
   int rows, E_out, d;
-  int tile_n, n_tiles, ksplit;   // ksplit = cluster size: 1, 2 or 4
+  int tile_n, n_tiles, ksplit;   // ksplit = CTAs per output tile along K: 1, 2 or 4
+  float* xchg;                   // [m_tiles*n_tiles][ksplit][tile_n][128] fp32, needed when ksplit > 1
+  int* flags;                    // [m_tiles*n_tiles][ksplit], zero between launches
+  int n_sms;
   int* status;
 };
 cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream_t st);

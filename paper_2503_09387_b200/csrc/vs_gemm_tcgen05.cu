@@ -8,10 +8,12 @@
 // the *tokens* take the MMA's N axis (any multiple of 16 up to 256: 170 tokens cost 176
 // columns, 3.5 % padding instead of 33 % with 128-row token tiles).  The reduction dimension
 // d is split over `ksplit` CTAs so that m_tiles * n_tiles * ksplit fills the 148 SMs.  The
-// ksplit CTAs of one output tile form a thread-block cluster: each dumps its fp32 partial
-// accumulator to its own shared memory, and after a cluster barrier CTA r sums token slice r
-// of all partials through distributed shared memory.  The same epilogue adds the bias,
-// applies RoPE (a 128-row tile holds whole heads, so both elements of a rotation pair are at
+// tile's tokens are cut into ksplit slices and CTA r finishes slice r: every CTA stores the
+// other slices of its fp32 partial accumulator to an exchange buffer in global memory (it
+// stays in L2), counts itself in on the owners' flags, and the owner of a slice, once its
+// flag shows ksplit - 1 arrivals, adds the peers' partials to its own.  All CTAs of the grid
+// are resident at once (the launch checks it), so the wait on the flag ends; it is bounded
+// like every other wait.  The same epilogue adds the bias, applies RoPE (a 128-row tile holds whole heads, so both elements of a rotation pair are at
 // hand), writes Q as a bf16 hi + lo pair and K, V as bf16, and persists what the method keeps:
 // the carrier row's K/V goes straight into the bank's free slot (Section 3.2: only the
 // carrier keeps its K/V), text rows are appended to the prefix or to the turn's tail.
@@ -20,11 +22,7 @@
 // (lane 0), warps 2..5 = epilogue (tcgen05.ld of their 32-lane quarter).
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, records
 // VS_ERR_DEVICE_TIMEOUT, lets in-flight copies land, frees its tensor memory and exits.
-#include <cooperative_groups.h>
-
 #include "vs_common.cuh"
-
-namespace cg = cooperative_groups;
 
 namespace vs {
 
@@ -118,20 +116,24 @@ struct KernelParams {
   ProjectionOut o;
   int* status;
   int rows, E_out, tile_n, kblocks, stages, tmem_cols, ksplit;
-  uint32_t data_bytes;          // shared memory ahead of the barriers: max(pipeline stages, fp32 partial tile)
+  uint32_t data_bytes;          // shared memory ahead of the barriers: max(pipeline stages, own fp32 slice)
+  float* xchg;                  // [group][rank][tile_n][128] partial tiles of the K split
+  int* flags;                   // [group][rank] peers that have delivered their part of slice `rank`
 };
 
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
 }
-// (two CTAs per SM must fit: see the shared-memory cap at the launch site)
-__global__ void __launch_bounds__(kThreads, 2)
+
+__global__ void __launch_bounds__(kThreads, 1)
 qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, KernelParams p,
                 BatchParams bp) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  // carve: [stages][A 16 KiB | B tile_n*128] (later reused as the fp32 partial tile
-  // [token][128 features]) | full[stages] | empty[stages] | tmem_full | tmem slot | abort
+  // carve: [stages][A 16 KiB | B tile_n*128] (later reused for this CTA's own token slice of
+  // the fp32 partial tile, [token][128 features]) | full[stages] | empty[stages] | tmem_full |
+  // tmem slot | abort
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t stage_b_bytes = (uint32_t)p.tile_n * 128u;
   const uint32_t stage_bytes = kStageABytes + stage_b_bytes;
@@ -147,13 +149,13 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * GEMM_BLOCK_M;
   const int n0 = blockIdx.y * p.tile_n;
-  const int kb0 = blockIdx.z * p.kblocks;      // blockIdx.z = rank in the cluster (cluster dims 1 x 1 x ksplit)
+  const int kb0 = blockIdx.z * p.kblocks;      // blockIdx.z = rank in the K split
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(tmem_full_bar, 1);
     *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");   // (the only scope this fence has)
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_x) : "memory");
@@ -219,41 +221,68 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   }
 
   // ---- epilogue ---------------------------------------------------------------------------
-  // The tile's tokens are cut into ksplit slices; CTA r of the cluster owns slice r.
+  // The tile's tokens are cut into ksplit slices; CTA r of the split owns slice r.
   // A  every CTA waits for its own accumulator (all its MMAs done, so all its TMA writes have
-  //    landed and its stages are dead) and copies it, fp32, into its own shared memory as
-  //    [token][128 features]; a cluster barrier publishes the partial tiles.
-  // C  the owner of a slice sums the ksplit partials of its tokens (float4 reads of the peers'
-  //    shared memory), adds the bias, rotates, rounds and stores; a last cluster barrier keeps
-  //    every CTA's shared memory alive until its peers have read it.
+  //    landed and its stages are dead) and copies it out, fp32, as [token][128 features]: its own
+  //    slice into its shared memory, the other slices into its part of the exchange buffer.
+  // B  it then counts itself in on the flag of every other slice's owner, and waits until the
+  //    ksplit - 1 peers have done the same on its own flag.
+  // C  the owner of a slice sums the ksplit partials of its tokens, adds the bias, rotates,
+  //    rounds and stores.
   const int slice = p.tile_n / p.ksplit;          // tile_n is a multiple of 16, ksplit is 1, 2 or 4
+  const int rank = (int)blockIdx.z;
+  const int group = (int)(blockIdx.y * gridDim.x + blockIdx.x);
+  const int t_begin = rank * slice;
   bool acc_ok = true;
   if (warp >= 2) {
     acc_ok = __all_sync(0xffffffffu, mbar_wait(tmem_full_bar, 0, abort_flag));   // warp-uniform
   }
   tcgen05_fence_after();
 
-  float* part_local = reinterpret_cast<float*>(gen_base);      // [token][128 features]
+  float* part_local = reinterpret_cast<float*>(gen_base);      // [token - t_begin][128 features]
   if (warp >= 2 && acc_ok) {
     // warp w may touch TMEM lanes 32*(w%4) .. +31 (lane = feature)
     const int quarter = warp & 3;
-    float* dst = part_local + quarter * 32 + lane;
+    float* dst_own = part_local + quarter * 32 + lane;
+    float* dst_far = p.xchg + ((size_t)group * p.ksplit + rank) * p.tile_n * GEMM_BLOCK_M + quarter * 32 + lane;
     for (int c = 0; c < p.tile_n; c += 16) {
       if (n0 + c >= p.rows) break;                             // uniform across the warp
       uint32_t r[16];
       tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, r);
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-      for (int j = 0; j < 16; ++j) dst[(c + j) * GEMM_BLOCK_M] = __uint_as_float(r[j]);
+      for (int j = 0; j < 16; ++j) {
+        const int t = c + j;
+        if ((unsigned)(t - t_begin) < (unsigned)slice) dst_own[(t - t_begin) * GEMM_BLOCK_M] = __uint_as_float(r[j]);
+        else dst_far[(size_t)t * GEMM_BLOCK_M] = __uint_as_float(r[j]);
+      }
     }
+    if (p.ksplit > 1) __threadfence();                         // the stores above, before the flag below
   }
   tcgen05_fence_before();
   __syncthreads();
-  if (p.ksplit > 1) cluster_sync_all();
+  if (p.ksplit > 1 && threadIdx.x == 64) {
+    if (!*abort_flag) {
+      for (int s = 0; s < p.ksplit; ++s)
+        if (s != rank) atomicAdd(p.flags + group * p.ksplit + s, 1);
+    }
+    int* mine = p.flags + group * p.ksplit + rank;
+    uint32_t spins = 0;
+    unsigned long long t0 = 0;
+    while (!*abort_flag && ld_acquire_gpu(mine) < p.ksplit - 1) {
+      if ((++spins & 255u) == 0u) {
+        const unsigned long long now = global_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > kWaitLimitNs) *abort_flag = 1;
+      }
+    }
+    *mine = 0;                                                 // next launch starts from zero
+  }
+  if (p.ksplit > 1) __syncthreads();
 
   // phase C.  Thread = (group of 4 rotation pairs, token lane).  The reads of a row -- float4
-  // pieces of every CTA's partial tile through distributed shared memory, and the row's RoPE
-  // entries -- are issued one row ahead of the arithmetic (two register buffers).
+  // pieces of the own slice in shared memory and of the peers' partials in the exchange buffer,
+  // and the row's RoPE entries -- are issued one row ahead of the arithmetic (two register buffers).
   if (warp >= 2 && !*abort_flag) {
     const int te = threadIdx.x - 64;               // 0..127
     const int D = p.o.D, half = D >> 1;
@@ -262,12 +291,8 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
     const int f1 = hl * D + k0, f2 = f1 + half;
     const int hs = (m0 + f1) / D;                  // head slot: Q heads, then K heads, then V heads
     const bool rotate = hs < p.o.Hq + p.o.Hkv;
-    const int t_begin = (int)blockIdx.z * slice;
-    const float* part[KSPLIT_MAX];
-    cg::cluster_group cluster = cg::this_cluster();
-#pragma unroll
-    for (int r = 0; r < KSPLIT_MAX; ++r)
-      part[r] = (p.ksplit > 1 && r < p.ksplit) ? cluster.map_shared_rank(part_local, r) : part_local;
+    const float* far = p.xchg + (size_t)group * p.ksplit * p.tile_n * GEMM_BLOCK_M;
+    const size_t far_stride = (size_t)p.tile_n * GEMM_BLOCK_M;
     if (m0 + f2 + 3 < p.E_out) {
       float bb1[4] = {0.f, 0.f, 0.f, 0.f}, bb2[4] = {0.f, 0.f, 0.f, 0.f};
       if (p.o.bias != nullptr) {
@@ -286,9 +311,13 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
         const int row = n0 + t;
 #pragma unroll
         for (int r = 0; r < KSPLIT_MAX; ++r) {
-          if (r < p.ksplit) {
-            R.v1[r] = *reinterpret_cast<const float4*>(part[r] + t * GEMM_BLOCK_M + f1);
-            R.v2[r] = *reinterpret_cast<const float4*>(part[r] + t * GEMM_BLOCK_M + f2);
+          if (r == rank) {
+            R.v1[r] = *reinterpret_cast<const float4*>(part_local + (t - t_begin) * GEMM_BLOCK_M + f1);
+            R.v2[r] = *reinterpret_cast<const float4*>(part_local + (t - t_begin) * GEMM_BLOCK_M + f2);
+          } else if (r < p.ksplit) {
+            // written by another SM during this launch: read past L1
+            R.v1[r] = __ldcg(reinterpret_cast<const float4*>(far + r * far_stride + (size_t)t * GEMM_BLOCK_M + f1));
+            R.v2[r] = __ldcg(reinterpret_cast<const float4*>(far + r * far_stride + (size_t)t * GEMM_BLOCK_M + f2));
           }
         }
         if (rotate) {
@@ -374,8 +403,6 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
     }
   }
 
-  // no CTA may leave while a peer still reads its partial tile
-  if (p.ksplit > 1) cluster_sync_all();
   __syncthreads();
   if (warp == 1) {
     tcgen05_fence_after();
@@ -389,9 +416,7 @@ constexpr int kMaxDynSmem = 227 * 1024;
 }  // namespace
 
 cudaError_t qkv_gemm_init() {
-  cudaError_t e = cudaFuncSetAttribute(qkv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(qkv_gemm_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 0);
+  return cudaFuncSetAttribute(qkv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
 }
 
 cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream_t st) {
@@ -407,12 +432,10 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   if (a.tile_n < 16 || a.tile_n > 256 || (a.tile_n & 15)) return cudaErrorInvalidValue;
   if (128 % a.out.D != 0) return cudaErrorInvalidValue;
   p.kblocks = total_kb / a.ksplit;
+  p.xchg = a.xchg;
+  p.flags = a.flags;
   const int stage_bytes = kStageABytes + a.tile_n * 128;
-  // With one CTA per SM only 33 clusters of 4 can be resident on the 148 SMs (clusters do not
-  // straddle GPCs), fewer than the 36 weight tiles of the Qwen2-7B shape.  Keeping a CTA under
-  // half an SM's shared memory lets every cluster be resident in one wave.
-  const int smem_cap = (a.ksplit >= 4) ? 112 * 1024 : kMaxDynSmem;
-  int stages = (smem_cap - 2048) / stage_bytes;
+  int stages = (kMaxDynSmem - 2048) / stage_bytes;
   if (stages > 8) stages = 8;
   if (stages > p.kblocks) stages = p.kblocks;
   if (stages < 1) return cudaErrorInvalidValue;
@@ -421,23 +444,30 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   while (cols < a.tile_n) cols <<= 1;
   p.tmem_cols = cols;
   size_t data = (size_t)stages * stage_bytes;
-  const size_t tile = (size_t)a.tile_n * GEMM_BLOCK_M * 4;
-  if (tile > data) data = (tile + 1023) / 1024 * 1024;
+  const size_t own = (size_t)(a.tile_n / a.ksplit) * GEMM_BLOCK_M * 4;
+  if (own > data) data = (own + 1023) / 1024 * 1024;
   p.data_bytes = (uint32_t)data;
   const size_t smem = 1024 + data + 16 * stages + 64;
   if (smem > (size_t)kMaxDynSmem) return cudaErrorInvalidValue;
+  const dim3 grid((a.E_out + GEMM_BLOCK_M - 1) / GEMM_BLOCK_M, a.n_tiles, a.ksplit);
+  if (a.ksplit > 1) {
+    // the CTAs of a K split wait for one another: the whole grid has to be resident at once
+    if (a.xchg == nullptr || a.flags == nullptr) return cudaErrorInvalidValue;
+    int per_sm = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, qkv_gemm_kernel, kThreads, smem);
+    if (e != cudaSuccess) return e;
+    if ((long long)grid.x * grid.y * grid.z > (long long)per_sm * a.n_sms) return cudaErrorInvalidValue;
+  }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((a.E_out + GEMM_BLOCK_M - 1) / GEMM_BLOCK_M, a.n_tiles, a.ksplit);
+  cfg.gridDim = grid;
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = a.ksplit;
-  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 2;
+  cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel, a.tm_w, a.tm_x, p, bp);
 }
 

@@ -75,6 +75,7 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.inv_freq = take((size_t)(D.D / 2) * 8);
   Lo.status = take(8 * 4);
   Lo.tickets = take((size_t)D.S * D.Hq * 4);
+  Lo.gemm_flags = take((size_t)GEMM_XCHG_CTAS * 4);
   Lo.persistent_end = off;
   Lo.scratch_begin = off;
   Lo.hbuf[0] = take((size_t)D.R_max * D.d * 2);
@@ -88,6 +89,7 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.rope = take((size_t)D.R_max * (D.D / 2) * 8);
   Lo.obuf = take((size_t)D.R_max * D.Hq * D.D * 4);
   Lo.dec_part = take((size_t)DEC_SPLIT_MAX * D.S * D.Hq * (D.D + 2) * 4);
+  Lo.gemm_xchg = take((size_t)GEMM_XCHG_CTAS * 256 * GEMM_BLOCK_M * 4);
   Lo.scratch_end = off;
   Lo.total = off;
 }
@@ -100,6 +102,7 @@ struct vs_stream {
   uint8_t* ws = nullptr;
   size_t ws_bytes = 0;
   int device = 0;
+  int n_sms = 0;
   std::vector<const bf16*> w, bias, gain;
   std::vector<CUtensorMap> tm_w;
   std::vector<HostStream> hs;
@@ -130,16 +133,17 @@ int encode_2d(vs_stream* h, CUtensorMap* tm, const void* base, uint64_t inner, u
   return r == CUDA_SUCCESS ? VS_OK : VS_ERR_CUDA;
 }
 
-void choose_tiles(const Dims& D, int rows, int& tile_n, int& n_tiles, int& ksplit) {
+void choose_tiles(const Dims& D, int n_sms, int rows, int& tile_n, int& n_tiles, int& ksplit) {
   n_tiles = (rows + 255) / 256;
   const int per = (rows + n_tiles - 1) / n_tiles;
   tile_n = (per + 15) / 16 * 16;
   const int m_tiles = (D.E_out + GEMM_BLOCK_M - 1) / GEMM_BLOCK_M;
   const int total_kb = D.d / GEMM_BLOCK_K;
-  ksplit = 1;                                  // cluster size along K: 1, 2 or 4
+  const int resident = n_sms < GEMM_XCHG_CTAS ? n_sms : GEMM_XCHG_CTAS;   // one CTA per SM
+  ksplit = 1;                                  // CTAs per output tile along K: 1, 2 or 4
   for (int ks = 1; ks <= KSPLIT_MAX; ks *= 2) {
     if (total_kb % ks != 0) continue;
-    if (m_tiles * n_tiles * ks <= 148) ksplit = ks;
+    if (m_tiles * n_tiles * ks <= resident) ksplit = ks;
   }
 }
 
@@ -178,7 +182,10 @@ int run_projection(vs_stream* h, int l, const bf16* src, int rows, const Project
                    cudaStream_t st) {
   const Dims& D = h->dm;
   GemmArgs g;
-  choose_tiles(D, rows, g.tile_n, g.n_tiles, g.ksplit);
+  choose_tiles(D, h->n_sms, rows, g.tile_n, g.n_tiles, g.ksplit);
+  g.xchg = h->at<float>(h->lo.gemm_xchg);
+  g.flags = h->at<int>(h->lo.gemm_flags);
+  g.n_sms = h->n_sms;
   g.tm_w = h->tm_w[l];
   if (encode_2d(h, &g.tm_x, src, (uint64_t)D.d, (uint64_t)rows, (uint32_t)g.tile_n) != VS_OK) return VS_ERR_CUDA;
   g.out = po;
@@ -241,6 +248,7 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights, void* work
   if (h == nullptr) return VS_ERR_INVALID_ARG;
   h->dm = D; h->lo = lo; h->ws = static_cast<uint8_t*>(workspace); h->ws_bytes = workspace_bytes;
   h->device = cfg->device;
+  if (cudaDeviceGetAttribute(&h->n_sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess) { delete h; return VS_ERR_CUDA; }
   h->hs.assign(D.S, HostStream());
   for (int l = 0; l < D.L; ++l) {
     h->w.push_back(static_cast<const bf16*>(weights->w_qkv[l]));
