@@ -18,8 +18,9 @@
 // the carrier row's K/V goes straight into the bank's free slot (Section 3.2: only the
 // carrier keeps its K/V), text rows are appended to the prefix or to the turn's tail.
 //
-// Per CTA: 6 warps.  Warp 0 lane 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer
-// (lane 0), warps 2..5 = epilogue (tcgen05.ld of their 32-lane quarter).
+// Per CTA: 6 or 18 warps.  Warp 0 lane 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer
+// (lane 0), warps 2.. = epilogue, 4 or 16 of them (tcgen05.ld of the 32-lane quarter that
+// warp % 4 allows; with 16, four warps per quarter take every fourth block of 16 columns).
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, records
 // VS_ERR_DEVICE_TIMEOUT, lets in-flight copies land, frees its tensor memory and exits.
 #include "vs_common.cuh"
@@ -28,7 +29,8 @@ namespace vs {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kMaxEpiWarps = 16;                 // 4 per scheduler: the epilogue is bound by instruction latency
+constexpr int kMaxThreads = 64 + 32 * kMaxEpiWarps;
 constexpr int kStageABytes = GEMM_BLOCK_M * GEMM_BLOCK_K * 2;   // 16 KiB
 constexpr unsigned long long kWaitLimitNs = 400ull * 1000ull * 1000ull;
 
@@ -127,7 +129,7 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
   return v;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kMaxThreads, 1)
 qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, KernelParams p,
                 BatchParams bp) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -147,6 +149,8 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   const uint32_t tmem_full_bar = bar_base + 16u * (uint32_t)p.stages;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int epi_warps = ((int)blockDim.x >> 5) - 2;   // 4, 8 or 16
+  const int tok_lanes = 2 * epi_warps;                // token rows finished side by side
   const int m0 = blockIdx.x * GEMM_BLOCK_M;
   const int n0 = blockIdx.y * p.tile_n;
   const int kb0 = blockIdx.z * p.kblocks;      // blockIdx.z = rank in the K split
@@ -245,7 +249,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
     const int quarter = warp & 3;
     float* dst_own = part_local + quarter * 32 + lane;
     float* dst_far = p.xchg + ((size_t)group * p.ksplit + rank) * p.tile_n * GEMM_BLOCK_M + quarter * 32 + lane;
-    for (int c = 0; c < p.tile_n; c += 16) {
+    for (int c = 16 * ((warp - 2) >> 2); c < p.tile_n; c += 16 * (epi_warps >> 2)) {
       if (n0 + c >= p.rows) break;                             // uniform across the warp
       uint32_t r[16];
       tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, r);
@@ -282,9 +286,9 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
 
   // phase C.  Thread = (group of 4 rotation pairs, token lane).  The reads of a row -- float4
   // pieces of the own slice in shared memory and of the peers' partials in the exchange buffer,
-  // and the row's RoPE entries -- are issued one row ahead of the arithmetic (two register buffers).
+  // and the row's RoPE entries -- are all issued before the arithmetic.
   if (warp >= 2 && !*abort_flag) {
-    const int te = threadIdx.x - 64;               // 0..127
+    const int te = threadIdx.x - 64;               // 0 .. 32 * epi_warps - 1
     const int D = p.o.D, half = D >> 1;
     const int p0 = (te & 15) * 4;                  // first of 4 rotation pairs inside the 128-feature tile
     const int hl = p0 / half, k0 = p0 - hl * half; // local head, index inside the half head
@@ -303,11 +307,11 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
         }
       }
       const int rps = bp.rows_per_stream;
-      const int n_it = (slice - (te >> 4) + 7) / 8;          // rows this thread finishes
+      const int n_it = (slice - (te >> 4) + tok_lanes - 1) / tok_lanes;   // rows this thread finishes
       struct RowRegs { float4 v1[KSPLIT_MAX], v2[KSPLIT_MAX], ra, rb; float rsc; };
-      auto valid_it = [&](int it) { return it < n_it && n0 + t_begin + (te >> 4) + 8 * it < p.rows; };
+      auto valid_it = [&](int it) { return it < n_it && n0 + t_begin + (te >> 4) + tok_lanes * it < p.rows; };
       auto load_row = [&](RowRegs& R, int it) {
-        const int t = t_begin + (te >> 4) + 8 * it;
+        const int t = t_begin + (te >> 4) + tok_lanes * it;
         const int row = n0 + t;
 #pragma unroll
         for (int r = 0; r < KSPLIT_MAX; ++r) {
@@ -328,7 +332,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
         R.rsc = (p.o.row_scale != nullptr) ? p.o.row_scale[row] : 1.f;
       };
       auto finish_row = [&](const RowRegs& R, int it) {
-        const int t = t_begin + (te >> 4) + 8 * it;
+        const int t = t_begin + (te >> 4) + tok_lanes * it;
         const int row = n0 + t;
         float x1[4] = {0.f, 0.f, 0.f, 0.f}, x2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -391,14 +395,12 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
           }
         }
       };
-      RowRegs A, B;
-      if (valid_it(0)) load_row(A, 0);
+      // four warps per scheduler overlap one another's load latency; a thread holds one row at a time
 #pragma unroll 1
-      for (int it = 0; valid_it(it); it += 2) {
-        if (valid_it(it + 1)) load_row(B, it + 1);
+      for (int it = 0; valid_it(it); ++it) {
+        RowRegs A;
+        load_row(A, it);
         finish_row(A, it);
-        if (valid_it(it + 2)) load_row(A, it + 2);
-        if (valid_it(it + 1)) finish_row(B, it + 1);
       }
     }
   }
@@ -449,18 +451,21 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   p.data_bytes = (uint32_t)data;
   const size_t smem = 1024 + data + 16 * stages + 64;
   if (smem > (size_t)kMaxDynSmem) return cudaErrorInvalidValue;
+  // a token slice of a few rows is finished by 4 warps; wider ones by 16, which overlap one another's latency
+  const int slice_rows = a.tile_n / a.ksplit;
+  const int threads = 64 + 32 * (slice_rows <= 8 ? 4 : kMaxEpiWarps);
   const dim3 grid((a.E_out + GEMM_BLOCK_M - 1) / GEMM_BLOCK_M, a.n_tiles, a.ksplit);
   if (a.ksplit > 1) {
     // the CTAs of a K split wait for one another: the whole grid has to be resident at once
     if (a.xchg == nullptr || a.flags == nullptr) return cudaErrorInvalidValue;
     int per_sm = 0;
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, qkv_gemm_kernel, kThreads, smem);
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, qkv_gemm_kernel, threads, smem);
     if (e != cudaSuccess) return e;
     if ((long long)grid.x * grid.y * grid.z > (long long)per_sm * a.n_sms) return cudaErrorInvalidValue;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(threads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
