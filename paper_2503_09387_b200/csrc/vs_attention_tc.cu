@@ -10,12 +10,14 @@
 // Per tile:  S = Q K^T  (tcgen05.mma, M 128 x N 128, Q as a bf16 hi + lo pair)     -> TMEM
 //            softmax of the row in registers, P (bf16) -> shared memory (over the dead K tile)
 //            O_tile = P V  (tcgen05.mma, M 128 x N D, V read MN-major)             -> TMEM
-//            o_row = o_row * alpha + O_tile                                          (registers)
+//            o_row = o_row * alpha + O_tile, one tile late (two O buffers)         (registers)
 // Warps 0..7: two threads per row (each owns 64 keys of a tile and D/2 output dims).
 // Warp 8: one thread issues every MMA, one tile of Q K^T ahead of the softmax (S is double
 // buffered in TMEM); descriptors are built once.  Warps 9..11 fetch K/V with cp.async into the
 // 128-byte-swizzled layout the MMA descriptors expect, one tile ahead.  Finished rows leave
 // through shared memory as whole contiguous rows.  All mbarrier waits are bounded.
+#include <type_traits>
+
 #include "vs_common.cuh"
 
 namespace vs {
@@ -137,7 +139,7 @@ struct Smem {
   static constexpr int kV = kK + 2 * kKStage;             // [stage] V tile
   static constexpr int kMax = kV + 2 * kKVBytes;          // float [2][2][128]: row maxima exchange
   static constexpr int kCtl = kMax + 2048;                // barriers, tmem slot, abort flag
-  static constexpr int kTotal = kCtl + 64 + 1024;         // + alignment slack
+  static constexpr int kTotal = kCtl + 128 + 1024;        // + alignment slack
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -187,11 +189,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bar_s0 = base + L::kCtl;       // +0, +8: S buffer ready (tcgen05.commit)
-  const uint32_t bar_o = base + L::kCtl + 16;   // O tile ready (tcgen05.commit)
+  const uint32_t bar_o0 = base + L::kCtl + 16;  // +0, +64: O buffer ready (tcgen05.commit)
   const uint32_t bar_p = base + L::kCtl + 24;   // P written (256 arrivals)
   const uint32_t bar_kv0 = base + L::kCtl + 32; // +0, +8: K/V tile landed in a stage (one arrival per loader thread)
   const uint32_t bar_free0 = base + L::kCtl + 48;  // +0, +8: stage free again (tcgen05.commit after P V)
-  const uint32_t bar_q = base + L::kCtl + 64;   // Q tile landed (256 arrivals)
+  const uint32_t bar_q = base + L::kCtl + 64;   // Q tile and the K tile of key tile 0 landed (256 arrivals)
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + L::kCtl + 72);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kCtl + 76);
   float* max_x = reinterpret_cast<float*>(gbase + L::kMax);
@@ -200,7 +202,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   // ---- set-up that needs nothing from earlier kernels: barriers, tensor memory ------------------
   if (tid == 0) {
     mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1);
-    mbar_init(bar_o, 1);
+    mbar_init(bar_o0, 1); mbar_init(bar_o0 + 64, 1);
     mbar_init(bar_p, kSoftmaxThreads);
     mbar_init(bar_kv0, kLoaderThreads); mbar_init(bar_kv0 + 8, kLoaderThreads);
     mbar_init(bar_free0, 1); mbar_init(bar_free0 + 8, 1);
@@ -213,9 +215,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
                  ::"r"(smem_u32((const void*)tmem_slot)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  pdl_wait();                       // earlier kernels of the stream have completed
-  pdl_launch_dependents();
-
+  // (the key axis below is laid out from the kernel's parameters alone, so it too comes before the wait)
   const int b = blockIdx.z, hkv = blockIdx.y;
   const int r0 = blockIdx.x * kTok;
   const int rps = bp.rows_per_stream;
@@ -231,7 +231,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   const bf16* seg_k[4];
   const bf16* seg_v[4];
   int seg_stride[4];
-  int total = 0, causal_start = 0x3fffffff, hole = -1;
+  int total = 0, causal_start = 0x3fffffff, hole = -1, bank_begin = 0;
 #pragma unroll
   for (int s = 0; s < 4; ++s) {
     seg_k[s] = a.q; seg_v[s] = a.q; seg_stride[s] = 0;
@@ -241,7 +241,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
       if (sg.kind == 0) len = bp.prefix_len[b];
       else if (sg.kind == 1) {
         len = (a.M == 0) ? 0 : (bank_full ? a.M + 1 : count);
-        if (bank_full) hole = total + a.meta[sid].free_slot;     // the slot being refilled holds no carrier
+        bank_begin = total;
       }
       else if (sg.kind == 2) len = bp.text_len[b];
       else { len = min(rps, r0 + kTok); causal_start = total; }  // later keys are visible to no row of this tile
@@ -254,50 +254,59 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   }
   const int n_tiles = (total + kKeys - 1) / kKeys;
 
+  pdl_wait();                       // earlier kernels of the stream have completed
+  pdl_launch_dependents();
+  if (bank_full) hole = bank_begin + a.meta[sid].free_slot;      // the slot being refilled holds no carrier
+
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_o = tmem + 256;                    // S buffers at columns 0 and 128
+  const uint32_t tmem_o = tmem + 256;                    // S buffers at columns 0 and 128, O buffers at 256 and 384
+
+  // ---- K/V tile fetch: cp.async into the swizzled tiles ------------------------------------------
+  // Thread `lt` of `NT` cooperating threads owns one 16-byte column c of the key rows r = rsub,
+  // rsub + NT / CPR, ...; it walks the tile segment by segment so that inside a segment a row
+  // costs one pointer step.
+  auto fetch_tile = [&](int ti, int lt, auto nt_c, bool do_k, bool do_v) {
+    constexpr int kRowStep = decltype(nt_c)::value / CPR;     // key rows covered per pass
+    const int c = lt % CPR, rsub = lt / CPR;
+    const int stage = ti & 1;
+    const uint32_t kdst = base + L::kK + (uint32_t)stage * L::kKStage + (uint32_t)((c >> 3) * (kKeys * 128));
+    const uint32_t vdst = base + L::kV + (uint32_t)stage * L::kKVBytes + (uint32_t)((c >> 3) * (kKeys * 128));
+    const int t_begin = ti * kKeys;
+    int seg_begin = 0;
+#pragma unroll
+    for (int sgi = 0; sgi < 4; ++sgi) {
+      const int lo = max(seg_begin, t_begin) - t_begin;            // rows of this segment inside the tile
+      const int hi = min(seg_end[sgi], t_begin + kKeys) - t_begin;
+      seg_begin = seg_end[sgi];
+      if (lo >= hi) continue;
+      int r = lo + ((rsub - lo) % kRowStep + kRowStep) % kRowStep;  // first row >= lo owned by this thread
+      const long long step = (long long)kRowStep * seg_stride[sgi];
+      const bf16* kp = seg_k[sgi] + (long long)(t_begin + r) * seg_stride[sgi] + c * 8;
+      const bf16* vp = seg_v[sgi] + (long long)(t_begin + r) * seg_stride[sgi] + c * 8;
+      for (; r < hi; r += kRowStep, kp += step, vp += step) {
+        const uint32_t so = (uint32_t)(r * 128 + (((c & 7) ^ (r & 7)) << 4));
+        if (do_k) cp_async16(kdst + so, kp, true);
+        if (do_v) cp_async16(vdst + so, vp, true);
+      }
+    }
+    // rows past the end of the key axis (last tile only): zero-filled
+    for (int r = max(total - t_begin, 0) + ((rsub - max(total - t_begin, 0)) % kRowStep + kRowStep) % kRowStep; r < kKeys;
+         r += kRowStep) {
+      const uint32_t so = (uint32_t)(r * 128 + (((c & 7) ^ (r & 7)) << 4));
+      if (do_k) cp_async16(kdst + so, a.q, false);
+      if (do_v) cp_async16(vdst + so, a.q, false);
+    }
+  };
 
   if (warp >= 9) {
-    // ---- K/V loaders: cp.async into the swizzled tiles, one tile ahead ---------------------------
+    // ---- K/V loaders, one tile ahead.  The K tile of key tile 0 is fetched by the softmax threads
+    // together with Q (they are idle until the first scores exist); the loaders bring its V tile.
     const int lt = tid - (kSoftmaxThreads + 32);         // 0..95
-    // A thread owns one 16-byte column c of the key rows r = rsub, rsub + kRowStep, ...; it walks
-    // the tile segment by segment so that inside a segment a row costs one pointer step.
-    constexpr int kRowStep = kLoaderThreads / CPR;       // key rows covered per pass
-    const int c = lt % CPR, rsub = lt / CPR;
-    auto issue_tile = [&](int ti) {
-      const int stage = ti & 1;
-      const uint32_t kdst = base + L::kK + (uint32_t)stage * L::kKStage + (uint32_t)((c >> 3) * (kKeys * 128));
-      const uint32_t vdst = base + L::kV + (uint32_t)stage * L::kKVBytes + (uint32_t)((c >> 3) * (kKeys * 128));
-      const int t_begin = ti * kKeys;
-      int seg_begin = 0;
-#pragma unroll
-      for (int sgi = 0; sgi < 4; ++sgi) {
-        const int lo = max(seg_begin, t_begin) - t_begin;            // rows of this segment inside the tile
-        const int hi = min(seg_end[sgi], t_begin + kKeys) - t_begin;
-        seg_begin = seg_end[sgi];
-        if (lo >= hi) continue;
-        int r = lo + ((rsub - lo) % kRowStep + kRowStep) % kRowStep;  // first row >= lo owned by this thread
-        const long long step = (long long)kRowStep * seg_stride[sgi];
-        const bf16* kp = seg_k[sgi] + (long long)(t_begin + r) * seg_stride[sgi] + c * 8;
-        const bf16* vp = seg_v[sgi] + (long long)(t_begin + r) * seg_stride[sgi] + c * 8;
-        for (; r < hi; r += kRowStep, kp += step, vp += step) {
-          const uint32_t so = (uint32_t)(r * 128 + (((c & 7) ^ (r & 7)) << 4));
-          cp_async16(kdst + so, kp, true);
-          cp_async16(vdst + so, vp, true);
-        }
-      }
-      // rows past the end of the key axis (last tile only): zero-filled
-      for (int r = max(total - t_begin, 0) + ((rsub - max(total - t_begin, 0)) % kRowStep + kRowStep) % kRowStep; r < kKeys;
-           r += kRowStep) {
-        const uint32_t so = (uint32_t)(r * 128 + (((c & 7) ^ (r & 7)) << 4));
-        cp_async16(kdst + so, a.q, false);
-        cp_async16(vdst + so, a.q, false);
-      }
-      cp_async_commit();
-    };
+    using NT = std::integral_constant<int, kLoaderThreads>;
+    auto issue_tile = [&](int ti) { fetch_tile(ti, lt, NT(), ti != 0, true); cp_async_commit(); };
     // Two tiles are put in flight at once; afterwards tile ti+2 can only be fetched once P V of
     // tile ti has released its stage.  A tile is always published BEFORE the loader waits for a
     // stage to be released: the issuer runs Q K^T of tile ti+1 ahead of P V of tile ti, so the
@@ -346,8 +355,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
         }
         umma_commit(bar_s0 + 8u * (uint32_t)(t & 1));
       };
-      bool ok = mbar_wait(bar_q, 0, abort_flag) && mbar_wait(bar_kv0, 0, abort_flag);
+      bool ok = mbar_wait(bar_q, 0, abort_flag);                 // Q and K(0)
       if (ok) { tc_fence_after(); issue_qk(0); }
+      ok = ok && mbar_wait(bar_kv0, 0, abort_flag);              // V(0)
       for (int ti = 0; ti < n_tiles && ok; ++ti) {
         if (ti + 1 < n_tiles) {      // next S tile first: it has a whole softmax of lead time
           ok = mbar_wait(bar_kv0 + 8u * (uint32_t)((ti + 1) & 1), (uint32_t)(((ti + 1) >> 1) & 1), abort_flag);
@@ -365,9 +375,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
           // B = V, MN-major: 16 key rows = 2048 bytes further per step.
           const uint64_t dpk = dp + (uint64_t)(((kk >> 2) * (kRows * 128) + (kk & 3) * 32) >> 4);
           const uint64_t dvk = dv + (uint64_t)((kk * 2048) >> 4);
-          if (kk == 0) umma_new(tmem_o, dpk, dvk, idesc_pv); else umma_acc(tmem_o, dpk, dvk, idesc_pv);
+          const uint32_t tmem_ob = tmem_o + 128u * (uint32_t)(ti & 1);
+          if (kk == 0) umma_new(tmem_ob, dpk, dvk, idesc_pv); else umma_acc(tmem_ob, dpk, dvk, idesc_pv);
         }
-        umma_commit(bar_o);
+        umma_commit(bar_o0 + 64u * (uint32_t)(ti & 1));
         umma_commit(bar_free0 + 8u * (uint32_t)(ti & 1));
       }
     }
@@ -384,6 +395,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
       cp_async16(base + L::kQhi + sw_off<kRows>(r, c), a.q + off, valid);
       cp_async16(base + L::kQlo + sw_off<kRows>(r, c), a.q_lo + off, valid);
     }
+    fetch_tile(0, tid, std::integral_constant<int, kSoftmaxThreads>(), true, false);
     cp_async_commit();
     cp_async_wait<0>();
     fence_async_proxy();
@@ -397,6 +409,24 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
     const float scale = a.scale_log2e;
     const int lim = min(total, (causal_start == 0x3fffffff) ? total : causal_start + tok + 1);  // first invisible key
     bool ok = true;
+    // O(ti) = P(ti) V(ti) is folded into the row one tile late, after P(ti+1) has been handed to
+    // the tensor core, so the softmax of a tile overlaps the P V product of the tile before it
+    // (two O buffers in TMEM): o = o * alpha(ti) + O(ti) with alpha(ti) = 2^(m(ti-1) - m(ti)).
+    float alpha_prev = 0.f;
+    auto fold_o = [&](int t, float al) {
+      if (!mbar_wait(bar_o0 + 64u * (uint32_t)(t & 1), (uint32_t)((t >> 1) & 1), abort_flag)) return false;
+      tc_fence_after();
+#pragma unroll
+      for (int c0 = 0; c0 < DH; c0 += 32) {
+        float tv[32];
+        tmem_ld32(tmem_o + 128u * (uint32_t)(t & 1) + lane_base + DH * half + c0, tv);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) o_acc[c0 + j] = fmaf(o_acc[c0 + j], al, tv[j]);
+      }
+      tc_fence_before();
+      return true;
+    };
 
     for (int ti = 0; ti < n_tiles; ++ti) {
       const uint32_t tmem_s = tmem + 128u * (uint32_t)(ti & 1);
@@ -458,20 +488,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
       tc_fence_before();
       mbar_arrive(bar_p);
 
-      ok = mbar_wait(bar_o, (uint32_t)(ti & 1), abort_flag);
-      tc_fence_after();
-      if (ok) {
-#pragma unroll
-        for (int c0 = 0; c0 < DH; c0 += 32) {
-          float t[32];
-          tmem_ld32(tmem_o + lane_base + DH * half + c0, t);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) o_acc[c0 + j] = fmaf(o_acc[c0 + j], alpha, t[j]);
-        }
-        tc_fence_before();
-      }
+      if (ti >= 1) ok = fold_o(ti - 1, alpha_prev);
+      alpha_prev = alpha;
     }
+    if (ok && n_tiles >= 1) ok = fold_o(n_tiles - 1, alpha_prev);
 
     // the two halves of a row hold partial sums of the softmax denominator
     max_x[half * 128 + row] = l_run;

@@ -22,18 +22,20 @@ __device__ __forceinline__ bf16 f64_to_bf16_rne(double x) {
 // once.  The sum of <= 256 bf16 values in fp64 is exact, hence independent of the order.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, int pool_blocks) {
-  pdl_wait();
-  pdl_launch_dependents();
+  // what depends on the parameters alone comes before the wait on the stream's earlier kernels
   const int b = blockIdx.y;
   const int sid = bp.stream_id[b];
   const int N = a.N, d = a.d;
+  const long long pos0 = bp.pos_base[b];
   if ((int)blockIdx.x >= pool_blocks) {
+    pdl_wait();
+    pdl_launch_dependents();
     // RoPE table of this step's N + 1 positions: angle = pos * theta^(-2k/D), in fp64
     const int half = a.D / 2;
     const int idx = (blockIdx.x - pool_blocks) * blockDim.x + threadIdx.x;
     if (idx < (N + 1) * half) {
       const int r = idx / half, k = idx - r * half;
-      const double ang = (double)(bp.pos_base[b] + r) * a.inv_freq[k];
+      const double ang = (double)(pos0 + r) * a.inv_freq[k];
       double s, c;
       sincos(ang, &s, &c);
       a.rope[((size_t)b * (N + 1) + r) * half + k] = make_float2((float)c, (float)s);
@@ -47,6 +49,8 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, i
   const int ch = blockIdx.x * 64 + cl * 8;  // d is a multiple of 64
   const bf16* src = a.hidden + (size_t)b * N * d + ch;
   bf16* dst = a.x + (size_t)b * (N + 1) * d + ch;
+  pdl_wait();
+  pdl_launch_dependents();
   uint4 v[MAXR];
 #pragma unroll
   for (int i = 0; i < MAXR; ++i) {
