@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_DIR = os.path.join(HERE, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "libvideoscan.so")
-SOURCES = ["vs_host.cu", "vs_kernels_misc.cu", "vs_gemm_tcgen05.cu", "vs_attention.cu", "vs_attention_tc.cu", "vs_noalloc.cu"]
+SOURCES = ["vs_host.cu", "vs_kernels_misc.cu", "vs_gemm_tcgen05.cu", "vs_gemv.cu", "vs_attention.cu", "vs_attention_tc.cu", "vs_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 

@@ -139,7 +139,8 @@ cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* r
 struct ProjectionOut {
   const bf16* bias;              // [E_out] or null
   const float* row_scale;        // [rows] RMSNorm scale applied to the accumulated row, or null
-  const float2* rope;            // [rows][D/2] (cos, sin)
+  const float2* rope;            // [rows][D/2] (cos, sin); null: the kernel derives them from inv_freq (few rows only)
+  const double* inv_freq;        // [D/2]
   bf16* q;                       // [rows][Hq*D]  rotated query, leading bf16 part
   bf16* q_lo;                    // [rows][Hq*D]  bf16(query - q): the pair carries 16 mantissa bits
   bf16* kf;                      // [rows][Hkv*D] rotated keys of this step
@@ -164,6 +165,10 @@ struct GemmArgs {
 };
 cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream_t st);
 cudaError_t qkv_gemm_init();     // opt-in shared memory attribute, once per process/device
+// Projection of one to four rows of a text step as a matrix-vector product (no RoPE table needed).
+bool qkv_gemv_supported(const ProjectionOut& o, int rows, int d);
+cudaError_t launch_qkv_gemv(const bf16* W, const bf16* x, const ProjectionOut& o, const BatchParams& bp, int rows, int E_out,
+                            int d, cudaStream_t st);
 
 struct AttnSegment {
   const bf16* k; const bf16* v;

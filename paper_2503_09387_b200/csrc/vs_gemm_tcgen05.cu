@@ -129,6 +129,7 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
   return v;
 }
 
+template <bool kOwnRope>   // true: no RoPE table, every finishing thread derives the rotation of its one row
 __global__ void __launch_bounds__(kMaxThreads, 1)
 qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, KernelParams p,
                 BatchParams bp) {
@@ -237,6 +238,28 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   const int rank = (int)blockIdx.z;
   const int group = (int)(blockIdx.y * gridDim.x + blockIdx.x);
   const int t_begin = rank * slice;
+  // A step of a few rows brings no RoPE table: each finishing thread works out the (cos, sin) of
+  // the four rotation pairs of its one row, in fp64 like the table kernel, while the main loop runs.
+  float4 own_ra = make_float4(1.f, 0.f, 1.f, 0.f), own_rb = own_ra;
+  if (kOwnRope && warp >= 2) {
+    const int te = threadIdx.x - 64;
+    const int half = p.o.D >> 1;
+    const int p0 = (te & 15) * 4, hl = p0 / half, k0 = p0 - hl * half;
+    const int row = n0 + t_begin + (te >> 4);
+    if ((m0 + hl * p.o.D + k0) / p.o.D < p.o.Hq + p.o.Hkv && (te >> 4) < slice && row < p.rows) {
+      const int b = row / bp.rows_per_stream;
+      const double pos = (double)(bp.pos_base[b] + (row - b * bp.rows_per_stream));
+      double sn, cs;
+      float r[8];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        sincos(pos * p.o.inv_freq[k0 + i], &sn, &cs);
+        r[2 * i] = (float)cs; r[2 * i + 1] = (float)sn;
+      }
+      own_ra = make_float4(r[0], r[1], r[2], r[3]);
+      own_rb = make_float4(r[4], r[5], r[6], r[7]);
+    }
+  }
   bool acc_ok = true;
   if (warp >= 2) {
     acc_ok = __all_sync(0xffffffffu, mbar_wait(tmem_full_bar, 0, abort_flag));   // warp-uniform
@@ -325,8 +348,12 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
           }
         }
         if (rotate) {
-          R.ra = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0);
-          R.rb = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0 + 2);
+          if (!kOwnRope) {
+            R.ra = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0);
+            R.rb = *reinterpret_cast<const float4*>(p.o.rope + (size_t)row * half + k0 + 2);
+          } else {                       // the thread's only row (the launch checks it)
+            R.ra = own_ra; R.rb = own_rb;
+          }
         }
         // RMSNorm's row scale commutes with the projection: applied here, in fp32
         R.rsc = (p.o.row_scale != nullptr) ? p.o.row_scale[row] : 1.f;
@@ -418,7 +445,9 @@ constexpr int kMaxDynSmem = 227 * 1024;
 }  // namespace
 
 cudaError_t qkv_gemm_init() {
-  return cudaFuncSetAttribute(qkv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+  cudaError_t e = cudaFuncSetAttribute(qkv_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(qkv_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
 }
 
 cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream_t st) {
@@ -454,12 +483,16 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   // a token slice of a few rows is finished by 4 warps; wider ones by 16, which overlap one another's latency
   const int slice_rows = a.tile_n / a.ksplit;
   const int threads = 64 + 32 * (slice_rows <= 8 ? 4 : kMaxEpiWarps);
+  // without a RoPE table every finishing thread must have at most one row
+  if (a.out.rope == nullptr && (a.out.inv_freq == nullptr || slice_rows > 2 * (threads / 32 - 2))) return cudaErrorInvalidValue;
   const dim3 grid((a.E_out + GEMM_BLOCK_M - 1) / GEMM_BLOCK_M, a.n_tiles, a.ksplit);
   if (a.ksplit > 1) {
     // the CTAs of a K split wait for one another: the whole grid has to be resident at once
     if (a.xchg == nullptr || a.flags == nullptr) return cudaErrorInvalidValue;
     int per_sm = 0;
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, qkv_gemm_kernel, threads, smem);
+    cudaError_t e = (a.out.rope == nullptr)
+        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, qkv_gemm_kernel<true>, threads, smem)
+        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, qkv_gemm_kernel<false>, threads, smem);
     if (e != cudaSuccess) return e;
     if ((long long)grid.x * grid.y * grid.z > (long long)per_sm * a.n_sms) return cudaErrorInvalidValue;
   }
@@ -473,7 +506,8 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel, a.tm_w, a.tm_x, p, bp);
+  if (a.out.rope == nullptr) return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<true>, a.tm_w, a.tm_x, p, bp);
+  return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<false>, a.tm_w, a.tm_x, p, bp);
 }
 
 }  // namespace vs

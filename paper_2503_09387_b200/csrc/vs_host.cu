@@ -159,7 +159,7 @@ int check_ids(vs_stream* h, const int32_t* ids, int32_t n) {
 
 #define VS_CK(expr) do { if ((expr) != cudaSuccess) return VS_ERR_CUDA; } while (0)
 
-enum KernelClass { KC_POOL = 0, KC_ROPE, KC_RMSNORM, KC_GEMM, KC_FINALIZE, KC_PREFILL_ATTN, KC_DECODE_ATTN,
+enum KernelClass { KC_POOL = 0, KC_ROPE, KC_RMSNORM, KC_GEMM, KC_GEMV, KC_PREFILL_ATTN, KC_DECODE_ATTN,
                    KC_EVICT, KC_COMMIT, KC_OTHER };
 static_assert(KC_OTHER + 1 == VS_N_KERNEL_CLASSES, "kernel class table");
 
@@ -181,6 +181,11 @@ static_assert(KC_OTHER + 1 == VS_N_KERNEL_CLASSES, "kernel class table");
 int run_projection(vs_stream* h, int l, const bf16* src, int rows, const ProjectionOut& po, const BatchParams& bp,
                    cudaStream_t st) {
   const Dims& D = h->dm;
+  if (po.rope == nullptr && qkv_gemv_supported(po, rows, D.d) && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+    // a text step of a few rows: bound by reading W once, done on the CUDA cores
+    VS_LAUNCH(h, st, KC_GEMV, launch_qkv_gemv(h->w[l], src, po, bp, rows, D.E_out, D.d, st));
+    return VS_OK;
+  }
   GemmArgs g;
   choose_tiles(D, h->n_sms, rows, g.tile_n, g.n_tiles, g.ksplit);
   g.xchg = h->at<float>(h->lo.gemm_xchg);
@@ -345,6 +350,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     fa.bias = h->bias[l];
     fa.row_scale = D.use_rmsnorm ? h->at<float>(lo.row_scale) : nullptr;
     fa.rope = h->at<float2>(lo.rope);
+    fa.inv_freq = h->at<double>(lo.inv_freq);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
     fa.bank_k = h->at<bf16>(lo.bank_k) + (size_t)l * layer_stride_bank(D);
     fa.bank_v = h->at<bf16>(lo.bank_v) + (size_t)l * layer_stride_bank(D);
@@ -430,9 +436,13 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
   const int rows = n_active * T;
   StreamMeta* meta = h->at<StreamMeta>(lo.meta);
 
-  RopeArgs ra;
-  ra.inv_freq = h->at<double>(lo.inv_freq); ra.rope = h->at<float2>(lo.rope); ra.D = D.D;
-  VS_LAUNCH(h, st, KC_ROPE, launch_rope_table(ra, bp, st));
+  // a step of up to 16 rows needs no table: the projection works the rotation out itself
+  const bool rope_inline = rows <= 16;
+  if (!rope_inline) {
+    RopeArgs ra;
+    ra.inv_freq = h->at<double>(lo.inv_freq); ra.rope = h->at<float2>(lo.rope); ra.D = D.D;
+    VS_LAUNCH(h, st, KC_ROPE, launch_rope_table(ra, bp, st));
+  }
 
   const bf16* h_in = static_cast<const bf16*>(hidden);
   int next_buf = 0;
@@ -453,7 +463,8 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
     ProjectionOut fa;
     fa.bias = h->bias[l];
     fa.row_scale = D.use_rmsnorm ? h->at<float>(lo.row_scale) : nullptr;
-    fa.rope = h->at<float2>(lo.rope);
+    fa.rope = rope_inline ? nullptr : h->at<float2>(lo.rope);
+    fa.inv_freq = h->at<double>(lo.inv_freq);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
     fa.bank_k = bk; fa.bank_v = bv;
     fa.text_k = to_prefix ? pk : tk; fa.text_v = to_prefix ? pv : tv;
@@ -571,7 +582,7 @@ int vs_profile_read(vs_stream* h, double* ms, int64_t* timed, int64_t* launches)
 }
 
 const char* vs_kernel_class_name(int32_t k) {
-  static const char* names[VS_N_KERNEL_CLASSES] = {"pool", "rope_table", "rmsnorm", "qkv_gemm", "unused_a",
+  static const char* names[VS_N_KERNEL_CLASSES] = {"pool", "rope_table", "rmsnorm", "qkv_gemm", "qkv_gemv",
                                                    "prefill_attention", "decode_attention", "unused",
                                                    "bank_update", "other"};
   return (k >= 0 && k < VS_N_KERNEL_CLASSES) ? names[k] : "?";
