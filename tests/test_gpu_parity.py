@@ -92,6 +92,41 @@ def test_multi_layer_residual_rmsnorm_small():
     p.close()
 
 
+def test_text_steps_of_one_to_four_rows():
+    """Steps of 1..4 rows take the matrix-vector projection (no RoPE table); 5..16 rows the
+    tensor-core one with the rotation derived in the kernel.  Two layers with RMSNorm gain,
+    bias and residual, single streams and small batches."""
+    w = synth.workload("deep", n_layers=2, d_model=512, n_q_heads=4, n_kv_heads=2, head_dim=128,
+                       tokens_per_frame=23, n_frames=5, bank_capacity=3, prefix_len=3, question_len=0,
+                       decode_tokens=0, n_streams=3, frame_model="iid", seed=23)
+    p = Pair(w, with_gain=True, with_bias=True, max_prefix=8, max_text=40, max_step_tokens=16)
+    ids = [0, 1, 2]
+    p.gpu.profile_read()
+    draw = lambda tag, T, s: synth.normal_bf16(w.seed, synth.TAG_QUESTION, (T, w.d_model), 1.0, offset=(tag * 8 + s) * 16 * w.d_model)
+    p.text([0], [w.prefix_hidden(0)], "prefix of 3 rows")                                  # 3 rows -> prefix
+    p.text([1, 2], [w.prefix_hidden(1)[:1], w.prefix_hidden(2)[:1]], "two one-row prefixes")  # 2 rows
+    p.text([1], [draw(0, 4, 1)], "prefix extended by 4 rows")                              # 4 rows
+    for t in range(5):
+        p.frame(ids, [w.frame_hidden(t, s) for s in ids], f"frame {t}")
+    launches = p.gpu.profile_read()
+    assert launches["qkv_gemv"][2] == 3 * w.n_layers and launches["rope_table"][2] == 0
+    p.text([0], [draw(1, 2, 0)], "2-row question")
+    p.text(ids, [draw(2, 1, s) for s in ids], "3 streams x 1 token")
+    p.text([2], [draw(3, 4, 2)], "4-row step")
+    p.text([0, 1], [draw(4, 1, s) for s in (0, 1)], "2 streams x 1 token")
+    p.text([1], [draw(5, 1, 1)], "single token")
+    launches = p.gpu.profile_read()
+    assert launches["qkv_gemv"][2] == 5 * w.n_layers and launches["qkv_gemm"][2] == 0
+    p.text([0], [draw(6, 7, 0)], "7-row step")                                             # tensor cores, no table
+    p.text([1, 2], [draw(7, 8, s) for s in (1, 2)], "2 streams x 8 rows")                  # 16 rows, no table
+    launches = p.gpu.profile_read()
+    assert launches["qkv_gemm"][2] == 2 * w.n_layers and launches["rope_table"][2] == 0
+    for s in ids:
+        for layer in range(2):
+            p.check_bank(s, layer=layer)
+    p.close()
+
+
 def test_scratch_holds_no_state_between_steps():
     """Section 3.3: visual tokens are discarded after prefill.  Overwriting every per-step
     scratch region with NaN between steps must not change any later output."""
