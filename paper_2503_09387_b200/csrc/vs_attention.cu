@@ -3,8 +3,8 @@
 // visual-token K/V exists at this point -- only carriers.
 //
 // grid = (key splits, query heads, streams), 256 threads.  A group of D/8 lanes owns one key
-// row and reads it with 128-bit loads; every lane issues the K and V loads of four keys before
-// it uses any of them, so a warp has 8 key rows (4 KB) in flight.  Warps merge their running
+// row and reads it with 128-bit loads; every lane issues the K and V loads of eight keys before
+// it uses any of them, so a warp has 16 key rows (8 KB) in flight.  Warps merge their running
 // (m, l, o) by shuffles and through shared memory; with several key splits the last CTA of a
 // (stream, query head) to finish combines the partial triples -- no CTA ever waits for another.
 #include "vs_common.cuh"
@@ -15,7 +15,7 @@ namespace {
 
 constexpr int kDecThreads = 256;
 constexpr int kDecWarps = kDecThreads / 32;
-constexpr int kBatch = 4;     // keys a lane group loads before computing
+constexpr int kBatch = 8;     // keys a lane group loads before computing
 
 // One CTA = one query head x one key split x one stream.  The heads of a KV group read the
 // same K/V rows from L2; spreading them over CTAs keeps every SM's instruction stream short,
@@ -30,8 +30,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
   __shared__ float sp_w[DEC_SPLIT_MAX];
   __shared__ int is_last;
 
-  pdl_wait();
-  pdl_launch_dependents();
+  // what follows from the parameters alone comes before the wait on the stream's earlier kernels
   const int split = blockIdx.x, qh = blockIdx.y, b = blockIdx.z;
   const int sid = bp.stream_id[b];
   const int hkv = qh / (a.Hq / a.Hkv);
@@ -39,7 +38,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
   const int sub = lane / LPK, li = lane % LPK;
   const int count = bp.count[b];
   const bool bank_full = (a.M > 0 && count == a.M);
-  const int free_slot = bank_full ? a.meta[sid].free_slot : -1;
 
   int P, NB, TL;
   if (a.to_prefix) { P = bp.prefix_len[b] + 1; NB = 0; TL = 0; }
@@ -55,6 +53,12 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
   const bf16* bv = a.bank_v + hoff * a.slots * D + li * 8;
   const bf16* tk = a.tail_k + hoff * a.maxT * D + li * 8;
   const bf16* tv = a.tail_v + hoff * a.maxT * D + li * 8;
+
+  pdl_wait();
+  pdl_launch_dependents();
+  // the slot being refilled holds no carrier: its key is fetched like any other (the row exists)
+  // and masked when the scores are formed, so this load delays nothing
+  const int hole = bank_full ? P + a.meta[sid].free_slot : -1;
 
   // this lane's 8 dims of the query (bf16 hi + lo pair), pre-scaled into the log2 domain
   float q[8];
@@ -90,7 +94,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
         if (v < P) { kp = pk + (size_t)v * D; vp = pv + (size_t)v * D; }
         else if (v < P + NB) {
           const int slot = v - P;
-          act[u] = slot != free_slot;                    // the slot being refilled holds no carrier
           kp = bk + (size_t)slot * D; vp = bv + (size_t)slot * D;
         } else { kp = tk + (size_t)(v - P - NB) * D; vp = tv + (size_t)(v - P - NB) * D; }
       }
@@ -110,7 +113,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
       }
 #pragma unroll
       for (int off = LPK / 2; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
-      s[u] = act[u] ? d : -INFINITY;
+      s[u] = (act[u] && base + u * kStride != hole) ? d : -INFINITY;
       mx = fmaxf(mx, s[u]);
     }
     if (mx > -INFINITY) {
