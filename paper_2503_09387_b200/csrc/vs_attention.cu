@@ -21,7 +21,7 @@ constexpr int kBatch = 8;     // keys a lane group loads before computing
 // same K/V rows from L2; spreading them over CTAs keeps every SM's instruction stream short,
 // which is what bounds this kernel (a few hundred keys of 256 bytes each).
 template <int D>
-__global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, BatchParams bp) {
+__global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs a, BatchParams bp) {
   constexpr int LPK = D / 8;            // lanes that share one key row (16 bytes each)
   constexpr int KPW = 32 / LPK;         // lane groups (keys in parallel) per warp
   __shared__ float st_m[kDecWarps];
@@ -54,11 +54,37 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
   const bf16* tk = a.tail_k + hoff * a.maxT * D + li * 8;
   const bf16* tv = a.tail_v + hoff * a.maxT * D + li * 8;
 
+  // Only the step's own token (the last key) was written by the kernel just before this one; every
+  // other key, and the bank's metadata, date from earlier steps, whose kernels had completed before
+  // that kernel let this one start.  So the first pass of K/V rows is fetched before the wait.
+  // The slot being refilled holds no carrier: its key is fetched like any other (the row exists)
+  // and masked when the scores are formed.
+  const int hole = bank_full ? P + a.meta[sid].free_slot : -1;
+  const int own_v = Lv - 1;
+  constexpr int kStride = kDecWarps * KPW;
+  // late == false: every key of the pass but the step's own; late == true: the step's own only
+  auto load_pass = [&](int wbase, uint4 (&kr)[kBatch], uint4 (&vr)[kBatch], bool late) {
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int v = wbase + sub + u * kStride;
+      if (v < end && ((v == own_v) == late)) {
+        const bf16* kp; const bf16* vp;
+        if (v < P) { kp = pk + (size_t)v * D; vp = pv + (size_t)v * D; }
+        else if (v < P + NB) { kp = bk + (size_t)(v - P) * D; vp = bv + (size_t)(v - P) * D; }
+        else { kp = tk + (size_t)(v - P - NB) * D; vp = tv + (size_t)(v - P - NB) * D; }
+        kr[u] = *reinterpret_cast<const uint4*>(kp);
+        vr[u] = *reinterpret_cast<const uint4*>(vp);
+      } else if (!late) {
+        kr[u] = make_uint4(0, 0, 0, 0); vr[u] = make_uint4(0, 0, 0, 0);
+      }
+    }
+  };
+  const int wbase0 = begin + warp * KPW;                 // keys are dealt to (warp, lane group) round-robin
+  uint4 kr0[kBatch], vr0[kBatch];
+  load_pass(wbase0, kr0, vr0, false);
+
   pdl_wait();
   pdl_launch_dependents();
-  // the slot being refilled holds no carrier: its key is fetched like any other (the row exists)
-  // and masked when the scores are formed, so this load delays nothing
-  const int hole = bank_full ? P + a.meta[sid].free_slot : -1;
 
   // this lane's 8 dims of the query (bf16 hi + lo pair), pre-scaled into the log2 domain
   float q[8];
@@ -79,31 +105,12 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
 #pragma unroll
   for (int i = 0; i < 8; ++i) o[i] = 0.f;
 
-  // keys of this CTA are dealt to (warp, lane group) round-robin, kBatch at a time
-  constexpr int kStride = kDecWarps * KPW;
-  for (int wbase = begin + warp * KPW; wbase < end; wbase += kBatch * kStride) {   // uniform over the warp
-    const int base = wbase + sub;
-    uint4 kr[kBatch], vr[kBatch];
-    bool act[kBatch];
-#pragma unroll
-    for (int u = 0; u < kBatch; ++u) {
-      const int v = base + u * kStride;
-      act[u] = v < end;
-      const bf16* kp = pk; const bf16* vp = pv;
-      if (act[u]) {
-        if (v < P) { kp = pk + (size_t)v * D; vp = pv + (size_t)v * D; }
-        else if (v < P + NB) {
-          const int slot = v - P;
-          kp = bk + (size_t)slot * D; vp = bv + (size_t)slot * D;
-        } else { kp = tk + (size_t)(v - P - NB) * D; vp = tv + (size_t)(v - P - NB) * D; }
-      }
-      kr[u] = act[u] ? *reinterpret_cast<const uint4*>(kp) : make_uint4(0, 0, 0, 0);
-      vr[u] = act[u] ? *reinterpret_cast<const uint4*>(vp) : make_uint4(0, 0, 0, 0);
-    }
+  auto compute_pass = [&](int wbase, const uint4 (&kr)[kBatch], const uint4 (&vr)[kBatch]) {
     float s[kBatch];
     float mx = m;
 #pragma unroll
     for (int u = 0; u < kBatch; ++u) {
+      const int v = wbase + sub + u * kStride;
       const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kr[u]);
       float d = 0.f;
 #pragma unroll
@@ -113,7 +120,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
       }
 #pragma unroll
       for (int off = LPK / 2; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
-      s[u] = (act[u] && base + u * kStride != hole) ? d : -INFINITY;
+      s[u] = (v < end && v != hole) ? d : -INFINITY;
       mx = fmaxf(mx, s[u]);
     }
     if (mx > -INFINITY) {
@@ -135,6 +142,16 @@ __global__ void __launch_bounds__(kDecThreads) decode_attn_kernel(DecodeArgs a, 
         }
       }
     }
+  };
+  if (wbase0 < end) {                                    // uniform over the warp
+    load_pass(wbase0, kr0, vr0, true);
+    compute_pass(wbase0, kr0, vr0);
+  }
+  for (int wbase = wbase0 + kBatch * kStride; wbase < end; wbase += kBatch * kStride) {
+    uint4 kr[kBatch], vr[kBatch];
+    load_pass(wbase, kr, vr, false);
+    load_pass(wbase, kr, vr, true);
+    compute_pass(wbase, kr, vr);
   }
 
   // lane groups of a warp merge by shuffles (they own the same dims of different keys)

@@ -20,7 +20,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kRowsPerCta = 32;     // 16 rotation pairs
-constexpr int kU = 4;               // 16-byte chunks per W row in one batch of loads
+constexpr int kU = 2;               // 16-byte chunks per W row in one batch of loads (two batches in flight)
 
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
@@ -34,7 +34,7 @@ __device__ __forceinline__ float dot8(const uint4& w, const uint4& x, float acc)
 }
 
 template <int R>   // token rows held (1, 2 or 4)
-__global__ void __launch_bounds__(kThreads) qkv_gemv_kernel(const bf16* __restrict__ W, const bf16* __restrict__ x,
+__global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __restrict__ W, const bf16* __restrict__ x,
                                                             ProjectionOut o, BatchParams bp, int rows, int d) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   uint4* xs = reinterpret_cast<uint4*>(smem_raw);                       // [R][d / 8]
