@@ -19,6 +19,7 @@
 #include <type_traits>
 
 #include "vs_common.cuh"
+#include "vs_bank_update.cuh"
 
 namespace vs {
 
@@ -199,6 +200,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   float* max_x = reinterpret_cast<float*>(gbase + L::kMax);
 
   const int tid = threadIdx.x, warp = tid >> 5;
+  // ---- bank update CTAs (frame steps): the first a.bank_blocks of each stream.  What they read --
+  // carrier embeddings, the bank's order and metadata -- was complete before the kernel ahead of
+  // this one let it start, and nothing else in this launch touches what they write.
+  if ((int)blockIdx.x < a.bank_blocks) {
+    if (blockIdx.y == 0) bank_update_block(a.bank, bp, (int)blockIdx.z, (int)blockIdx.x);
+    return;
+  }
   // ---- set-up that needs nothing from earlier kernels: barriers, tensor memory ------------------
   if (tid == 0) {
     mbar_init(bar_s0, 1); mbar_init(bar_s0 + 8, 1);
@@ -217,7 +225,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   }
   // (the key axis below is laid out from the kernel's parameters alone, so it too comes before the wait)
   const int b = blockIdx.z, hkv = blockIdx.y;
-  const int r0 = blockIdx.x * kTok;
+  const int r0 = ((int)blockIdx.x - a.bank_blocks) * kTok;
   const int rps = bp.rows_per_stream;
   const int sid = bp.stream_id[b];
   const int G = a.Hq / a.Hkv;
@@ -256,7 +264,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
 
   pdl_wait();                       // earlier kernels of the stream have completed
   pdl_launch_dependents();
-  if (bank_full) hole = bank_begin + a.meta[sid].free_slot;      // the slot being refilled holds no carrier
+  if (bank_full) hole = bank_begin + a.free_slot[sid * a.free_slot_stride];      // the slot being refilled holds no carrier
 
   tc_fence_before();
   __syncthreads();
@@ -559,7 +567,7 @@ cudaError_t prefill_attention_tc_init() {
 }
 
 cudaError_t launch_prefill_attention_tc(const AttnArgs& a, const BatchParams& bp, int* status, cudaStream_t st) {
-  dim3 grid((bp.rows_per_stream + kTok - 1) / kTok, a.Hkv, bp.n_active);
+  dim3 grid((bp.rows_per_stream + kTok - 1) / kTok + a.bank_blocks, a.Hkv, bp.n_active);
   if (a.D == 128) return launch_pdl(prefill_attn_tc_kernel<128>, grid, dim3(kAttnThreads), (size_t)Smem<128>::kTotal, st, a, bp, status);
   if (a.D == 64) return launch_pdl(prefill_attn_tc_kernel<64>, grid, dim3(kAttnThreads), (size_t)Smem<64>::kTotal, st, a, bp, status);
   return cudaErrorInvalidValue;

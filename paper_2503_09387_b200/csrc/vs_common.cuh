@@ -72,6 +72,7 @@ struct Layout {
   size_t scores;                // f64   [S][slots]
   size_t inv_freq;              // f64   [D/2]
   size_t status;                // int32 [8]
+  size_t step_slot;             // int32 [S]  free slot as the running frame step found it
   size_t tickets;               // int32 [S*Hq]  split-KV decode: CTAs finished per (stream, query head)
   size_t gemm_flags;            // int32 [GEMM_XCHG_CTAS]  projection K split: partials delivered per slice owner
   size_t persistent_end;
@@ -119,6 +120,7 @@ struct PoolArgs {
   bf16* x;                       // [n_active][N+1][d]
   bf16* emb;                     // [S][slots][d]
   const StreamMeta* meta;        // [S]
+  int32_t* step_slot;            // [S] copy of meta.free_slot for the rest of the step
   const double* inv_freq;        // [D/2]
   float2* rope;                  // [n_active][N+1][D/2]
   int N, d, D, slots, M, agg_mode;
@@ -147,7 +149,8 @@ struct ProjectionOut {
   bf16* vf;                      // [rows][Hkv*D]
   bf16* bank_k; bf16* bank_v;    // layer base [S][Hkv][slots][D]
   bf16* text_k; bf16* text_v;    // layer base [S][Hkv][text_cap][D]: prefix or tail
-  const StreamMeta* meta;
+  const int32_t* free_slot;      // free slot of stream s at free_slot[s * free_slot_stride]
+  int free_slot_stride;
   int Hq, Hkv, D, slots, text_cap, M;
   int mode;                      // 0 frame step (carrier row -> bank), 1 text -> prefix, 2 text -> tail
 };
@@ -170,6 +173,13 @@ bool qkv_gemv_supported(const ProjectionOut& o, int rows, int d);
 cudaError_t launch_qkv_gemv(const bf16* W, const bf16* x, const ProjectionOut& o, const BatchParams& bp, int rows, int E_out,
                             int d, cudaStream_t st);
 
+struct BankUpdateArgs {
+  const bf16* emb;               // [S][slots][d]
+  StreamMeta* meta;
+  const int32_t* step_slot;      // [S] the slot the incoming carrier was written to
+  int32_t* order; int32_t* slot_frame; int64_t* slot_pos; int32_t* evict_log; double* scores;
+  int d, slots, M, policy, log_cap;
+};
 struct AttnSegment {
   const bf16* k; const bf16* v;
   long long stream_stride;       // elements between streams (by stream id, or by batch slot when by_batch)
@@ -187,9 +197,13 @@ struct AttnArgs {
   int out_fp32;
   const bf16* h_in;              // residual input [rows][d] or null
   bf16* h_out;                   // residual output or null
-  const StreamMeta* meta;
+  const int32_t* free_slot;      // free slot of stream s at free_slot[s * free_slot_stride]
+  int free_slot_stride;
   int Hq, Hkv, D, slots, M;
   float scale_log2e;
+  // frame steps, last layer: the first bank_blocks CTAs of every stream do the bank update
+  BankUpdateArgs bank;
+  int bank_blocks;
 };
 cudaError_t launch_prefill_attention_tc(const AttnArgs& a, const BatchParams& bp, int* status, cudaStream_t st);
 cudaError_t prefill_attention_tc_init();
@@ -212,13 +226,6 @@ struct DecodeArgs {
 };
 cudaError_t launch_decode_attention(const DecodeArgs& a, const BatchParams& bp, cudaStream_t st);
 
-struct BankUpdateArgs {
-  const bf16* emb;               // [S][slots][d]
-  StreamMeta* meta;
-  int32_t* order; int32_t* slot_frame; int64_t* slot_pos; int32_t* evict_log; double* scores;
-  int d, slots, M, policy, log_cap;
-};
-cudaError_t launch_bank_update(const BankUpdateArgs& a, const BatchParams& bp, bool any_full, cudaStream_t st);
 
 cudaError_t launch_poison(void* p, size_t bytes, cudaStream_t st);
 cudaError_t launch_reset(StreamMeta* meta, int32_t* slot_frame, int slots, const BatchParams& bp, cudaStream_t st);

@@ -409,7 +409,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
           bf16* dst = nullptr;
           if (p.o.mode == 0) {
             if (tt == rps - 1 && p.o.M > 0) {
-              const int slot = p.o.meta[sid].free_slot;
+              const int slot = p.o.free_slot[sid * p.o.free_slot_stride];
               dst = (is_k ? p.o.bank_k : p.o.bank_v) + (((size_t)sid * p.o.Hkv + hkv) * p.o.slots + slot) * D + k0;
             }
           } else {

@@ -74,6 +74,7 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.scores = take((size_t)D.S * D.slots * 8);
   Lo.inv_freq = take((size_t)(D.D / 2) * 8);
   Lo.status = take(8 * 4);
+  Lo.step_slot = take((size_t)D.S * 4);
   Lo.tickets = take((size_t)D.S * D.Hq * 4);
   Lo.gemm_flags = take((size_t)GEMM_XCHG_CTAS * 4);
   Lo.persistent_end = off;
@@ -325,12 +326,20 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
   const int rows = n_active * (N + 1);
   StreamMeta* meta = h->at<StreamMeta>(lo.meta);
 
+  BankUpdateArgs ba;
+  ba.emb = h->at<bf16>(lo.emb); ba.meta = meta; ba.step_slot = h->at<int32_t>(lo.step_slot);
+  ba.order = h->at<int32_t>(lo.order); ba.slot_frame = h->at<int32_t>(lo.slot_frame);
+  ba.slot_pos = h->at<int64_t>(lo.slot_pos); ba.evict_log = h->at<int32_t>(lo.evict_log);
+  ba.scores = h->at<double>(lo.scores);
+  ba.d = D.d; ba.slots = D.slots; ba.M = D.M; ba.policy = D.evict_policy; ba.log_cap = D.log_cap;
+
   PoolArgs pa;
   pa.hidden = static_cast<const bf16*>(hidden);
   pa.carrier_override = static_cast<const bf16*>(carrier_override);
   pa.x = h->at<bf16>(lo.hbuf[0]);
   pa.emb = h->at<bf16>(lo.emb);
   pa.meta = meta;
+  pa.step_slot = h->at<int32_t>(lo.step_slot);
   pa.inv_freq = h->at<double>(lo.inv_freq);
   pa.rope = h->at<float2>(lo.rope);
   pa.N = N; pa.d = D.d; pa.D = D.D; pa.slots = D.slots; pa.M = D.M; pa.agg_mode = D.agg_mode;
@@ -355,7 +364,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     fa.bank_k = h->at<bf16>(lo.bank_k) + (size_t)l * layer_stride_bank(D);
     fa.bank_v = h->at<bf16>(lo.bank_v) + (size_t)l * layer_stride_bank(D);
     fa.text_k = nullptr; fa.text_v = nullptr;
-    fa.meta = meta;
+    fa.free_slot = h->at<int32_t>(lo.step_slot); fa.free_slot_stride = 1;
     fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D; fa.slots = D.slots; fa.text_cap = 0; fa.mode = 0; fa.M = D.M;
     rc = run_projection(h, l, src, rows, fa, bp, st);
     if (rc != VS_OK) return rc;
@@ -374,20 +383,14 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     aa.out_fp32 = D.out_fp32;
     aa.h_in = D.residual ? h_in : nullptr;
     aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
-    aa.meta = meta;
+    aa.free_slot = h->at<int32_t>(lo.step_slot); aa.free_slot_stride = 1;
+    if (last) { aa.bank = ba; aa.bank_blocks = any_full ? (D.M + 7) / 8 : 1; }
     aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
     aa.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
     VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, bp, h->at<int>(lo.status), st));
     if (D.residual) cur ^= 1;
   }
 
-  BankUpdateArgs ba;
-  ba.emb = h->at<bf16>(lo.emb); ba.meta = meta;
-  ba.order = h->at<int32_t>(lo.order); ba.slot_frame = h->at<int32_t>(lo.slot_frame);
-  ba.slot_pos = h->at<int64_t>(lo.slot_pos); ba.evict_log = h->at<int32_t>(lo.evict_log);
-  ba.scores = h->at<double>(lo.scores);
-  ba.d = D.d; ba.slots = D.slots; ba.M = D.M; ba.policy = D.evict_policy; ba.log_cap = D.log_cap;
-  VS_LAUNCH(h, st, KC_COMMIT, launch_bank_update(ba, bp, any_full, st));
 
   for (int i = 0; i < n_active; ++i) {
     HostStream& s = h->hs[stream_ids[i]];
@@ -468,7 +471,7 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
     fa.bank_k = bk; fa.bank_v = bv;
     fa.text_k = to_prefix ? pk : tk; fa.text_v = to_prefix ? pv : tv;
-    fa.meta = meta;
+    fa.free_slot = &meta->free_slot; fa.free_slot_stride = (int)(sizeof(StreamMeta) / sizeof(int32_t));
     fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D; fa.slots = D.slots;
     fa.text_cap = to_prefix ? D.maxP : D.maxT; fa.mode = to_prefix ? 1 : 2; fa.M = D.M;
     rc = run_projection(h, l, src, rows, fa, bp, st);
@@ -511,7 +514,7 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       aa.out_fp32 = D.out_fp32;
       aa.h_in = D.residual ? h_in : nullptr;
       aa.h_out = h_out;
-      aa.meta = meta;
+      aa.free_slot = &meta->free_slot; aa.free_slot_stride = (int)(sizeof(StreamMeta) / sizeof(int32_t));
       aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
       aa.scale_log2e = scale_log2e;
       VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, bp, h->at<int>(lo.status), st));

@@ -93,6 +93,9 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, i
     if (a.M > 0) {
       const int slot = a.meta[sid].free_slot;
       a.emb[((size_t)sid * a.slots + slot) * d + c] = cv;
+      // the step's other kernels take the slot from this copy: the bank update, which moves
+      // meta.free_slot on, runs beside the last attention kernel
+      if (blockIdx.x == 0 && threadIdx.x == 0) a.step_slot[sid] = slot;
     }
   }
 }
@@ -162,143 +165,6 @@ __global__ void __launch_bounds__(256) rms_stats_kernel(const bf16* __restrict__
 cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* row_scale, int rows, int d, float eps,
                              cudaStream_t st) {
   return launch_pdl(rms_stats_kernel, dim3(rows), dim3(256), 0, st, h, gain, hg, row_scale, d, eps);
-}
-
-// ------------------------------------------------------------------------------------------
-// Bank update (Section 3.3, memory mechanism): evict-if-full, then append.  One launch per
-// frame step, grid = (blocks, n_active).
-// Bank not full: block 0 appends; the other blocks exit.
-// Bank full: one warp per temporal index j scores cos(e_j, e_other) -- e_other is the incoming
-// carrier (policy 0) or the next carrier in temporal order (policy 1).  Dot products are
-// accumulated in fp64 in a fixed order -- lane p sums elements k = p (mod 32) in ascending k,
-// then a butterfly 16, 8, 4, 2, 1 -- so that the score, and with it the argmax, is
-// reproducible bit for bit; products of two bf16 values are exact in fp64, so fused and
-// unfused accumulation agree.  The last block of a stream to finish picks the victim (largest
-// score, oldest on ties), closes the gap in the temporal order and appends.
-// ------------------------------------------------------------------------------------------
-__device__ __forceinline__ double warp_tree_sum(double v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = __dadd_rn(v, __shfl_xor_sync(0xffffffffu, v, o));
-  return v;
-}
-
-__global__ void __launch_bounds__(256) bank_update_kernel(BankUpdateArgs a, BatchParams bp) {
-  pdl_wait();
-  pdl_launch_dependents();
-  const int b = blockIdx.y;
-  const int sid = bp.stream_id[b];
-  StreamMeta* meta = a.meta + sid;
-  if (a.M == 0) {
-    if (blockIdx.x == 0 && threadIdx.x == 0) { meta->frames_seen += 1; meta->last_victim_frame = -1; }
-    return;
-  }
-  int32_t* order = a.order + (size_t)sid * a.slots;
-  int32_t* slot_frame = a.slot_frame + (size_t)sid * a.slots;
-  int64_t* slot_pos = a.slot_pos + (size_t)sid * a.slots;
-  const int count = bp.count[b];
-  const int incoming = meta->free_slot;
-  const int64_t carrier_pos = bp.pos_base[b] + bp.rows_per_stream - 1;
-  if (count < a.M) {
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-      order[count] = incoming;
-      slot_frame[incoming] = (int32_t)bp.frame_id[b];
-      slot_pos[incoming] = carrier_pos;
-      meta->count = count + 1;
-      meta->free_slot = count + 1;          // slots fill in order until the bank is full
-      meta->last_victim_frame = -1;
-      meta->frames_seen += 1;
-    }
-    return;
-  }
-  // ---- bank full: score, then the last block commits --------------------------------------
-  double* scores = a.scores + (size_t)sid * a.slots;
-  const int lane = threadIdx.x & 31;
-  const int n_score_blocks = (a.M + 7) / 8;
-  if ((int)blockIdx.x >= n_score_blocks) return;
-  const int j = blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (j < count && a.policy != 2) {
-    const int sa = order[j];
-    const int sb = (a.policy == 1 && j + 1 < count) ? order[j + 1] : incoming;
-    const bf16* va = a.emb + ((size_t)sid * a.slots + sa) * a.d;
-    const bf16* vb = a.emb + ((size_t)sid * a.slots + sb) * a.d;
-    double dot = 0.0, na = 0.0, nb = 0.0;
-    for (int k = lane; k < a.d; k += 32) {
-      const double x = (double)__bfloat162float(va[k]);
-      const double y = (double)__bfloat162float(vb[k]);
-      dot = __dadd_rn(dot, __dmul_rn(x, y));
-      na = __dadd_rn(na, __dmul_rn(x, x));
-      nb = __dadd_rn(nb, __dmul_rn(y, y));
-    }
-    dot = warp_tree_sum(dot); na = warp_tree_sum(na); nb = warp_tree_sum(nb);
-    if (lane == 0) {
-      double s = 0.0;
-      if (na != 0.0 && nb != 0.0) s = __ddiv_rn(dot, __dmul_rn(__dsqrt_rn(na), __dsqrt_rn(nb)));
-      scores[j] = s;
-    }
-  }
-  __shared__ int is_last;
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) is_last = (atomicAdd(&meta->score_ticket, 1) == n_score_blocks - 1);
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-  __shared__ double best_s[256];
-  __shared__ int best_j[256];
-  double bs = -2.0; int bj = 0x7fffffff;
-  if (a.policy != 2) {
-    for (int i = threadIdx.x; i < count; i += blockDim.x) {
-      const double s = __ldcg(scores + i);
-      if (s > bs) { bs = s; bj = i; }                 // ascending i: first maximum kept
-    }
-  }
-  best_s[threadIdx.x] = bs; best_j[threadIdx.x] = bj;
-  __syncthreads();
-  for (int o = 128; o > 0; o >>= 1) {
-    if ((int)threadIdx.x < o) {
-      const double s2 = best_s[threadIdx.x + o]; const int j2 = best_j[threadIdx.x + o];
-      if (s2 > best_s[threadIdx.x] || (s2 == best_s[threadIdx.x] && j2 < best_j[threadIdx.x])) {
-        best_s[threadIdx.x] = s2; best_j[threadIdx.x] = j2;
-      }
-    }
-    __syncthreads();
-  }
-  const int v = (a.policy == 2) ? 0 : best_j[0];
-  const int victim_slot = order[v];
-  const int victim_frame = slot_frame[victim_slot];
-  __syncthreads();
-  // close the gap in the temporal order, one block-wide chunk at a time in ascending
-  // order: a chunk reads [base+1, base+256] before anything at or above base is written
-  for (int base = v; base < count - 1; base += blockDim.x) {
-    const int jj = base + threadIdx.x;
-    const int32_t next = (jj < count - 1) ? order[jj + 1] : 0;
-    __syncthreads();
-    if (jj < count - 1) order[jj] = next;
-    __syncthreads();
-  }
-  if (threadIdx.x == 0) {
-    order[count - 1] = incoming;
-    slot_frame[victim_slot] = -1;
-    slot_frame[incoming] = (int32_t)bp.frame_id[b];
-    slot_pos[incoming] = carrier_pos;
-    if (a.log_cap > 0) {
-      int32_t* e = a.evict_log + ((size_t)sid * a.log_cap + (meta->log_count % a.log_cap)) * 2;
-      e[0] = (int32_t)bp.frame_id[b];
-      e[1] = victim_frame;
-    }
-    meta->log_count += 1;
-    meta->evictions += 1;
-    meta->last_victim_frame = victim_frame;
-    meta->free_slot = victim_slot;
-    meta->victim_logical = -1;
-    meta->frames_seen += 1;
-    meta->score_ticket = 0;
-  }
-}
-
-cudaError_t launch_bank_update(const BankUpdateArgs& a, const BatchParams& bp, bool any_full, cudaStream_t st) {
-  dim3 grid(any_full ? (a.M + 7) / 8 : 1, bp.n_active);
-  return launch_pdl(bank_update_kernel, grid, dim3(256), 0, st, a, bp);
 }
 
 __global__ void poison_kernel(uint32_t* p, size_t n) {
