@@ -9,7 +9,8 @@ time is taken with CUDA events around the three phases; `value` = frames / frame
 
 Extra legs (same process, same workload):
   e2e          -- the same step with HOST (pinned) inputs: per-call H2D copy of the hidden
-                  states and D2H copy of the output inside the timed region.
+                  states and D2H copy of the output inside the timed region (copies on their
+                  own streams, double-buffered, so they overlap the kernels).
   roofline     -- the dominant kernel's average launch duration from CUDA events recorded
                   around every launch (vs_profile_enable) in one extra pass of the step.
   cpu_baseline -- the CPU oracle, as it stands, on a bounded sample of the same workload.
@@ -357,20 +358,41 @@ def run_ours(args, w):
         }
 
     # ---- end to end: host inputs, H2D + D2H inside the timed region ---------------------------
+    # Three streams, two buffers each way: the copy of frame t+1 to the device and the copy of
+    # frame t-1's output back overlap the kernels of frame t, as a caller that streams video would
+    # arrange it (the library only sees the stream it is given).
     pin_frames = torch.from_numpy(frames_host.view(np.int16)).pin_memory()
-    pin_out = torch.empty((N + 1, HD), dtype=torch.float32).pin_memory()
-    dev_in = torch.empty((N, d), dtype=torch.int16, device=dev)
-    p_dev_in = C.c_void_p(dev_in.data_ptr())
+    pin_out = [torch.empty((N + 1, HD), dtype=torch.float32).pin_memory() for _ in range(2)]
+    dev_in = [torch.empty((N, d), dtype=torch.int16, device=dev) for _ in range(2)]
+    dev_out = [torch.empty((N + 1, HD), dtype=torch.float32, device=dev) for _ in range(2)]
+    p_dev_in = [C.c_void_p(t_.data_ptr()) for t_ in dev_in]
+    p_dev_out = [C.c_void_p(t_.data_ptr()) for t_ in dev_out]
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    ev_in = [torch.cuda.Event() for _ in range(2)]      # frame landed in dev_in[k]
+    ev_done = [torch.cuda.Event() for _ in range(2)]    # kernels of the frame using buffers k finished
+    ev_out = [torch.cuda.Event() for _ in range(2)]     # dev_out[k] copied back
 
     def e2e_step():
         ck(lib.vs_reset_stream(h, ids, 1, sptr))
         if w.prefix_len:
             ck(lib.vs_decode_step(h, ids, 1, p_prefix, w.prefix_len, p_out_prefix, sptr))
         for t in range(w.n_frames):
-            dev_in.copy_(pin_frames[t], non_blocking=True)
-            ck(lib.vs_frame_prefill(h, ids, 1, p_dev_in, N, None, p_out_frame, sptr))
-            pin_out.copy_(out_frame, non_blocking=True)
-        stream.synchronize()
+            k = t & 1
+            with torch.cuda.stream(s_in):
+                if t >= 2:
+                    s_in.wait_event(ev_done[k])          # dev_in[k] is free again
+                dev_in[k].copy_(pin_frames[t], non_blocking=True)
+                ev_in[k].record(s_in)
+            stream.wait_event(ev_in[k])
+            if t >= 2:
+                stream.wait_event(ev_out[k])             # dev_out[k] is free again
+            ck(lib.vs_frame_prefill(h, ids, 1, p_dev_in[k], N, None, p_dev_out[k], sptr))
+            ev_done[k].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_done[k])
+                pin_out[k].copy_(dev_out[k], non_blocking=True)
+                ev_out[k].record(s_out)
+        stream.synchronize(); s_in.synchronize(); s_out.synchronize()
 
     e2e_step()
     barrier()
@@ -387,7 +409,8 @@ def run_ours(args, w):
                          "h2d_bytes_per_step": int(w.n_frames * N * d * 2),
                          "d2h_bytes_per_step": int(w.n_frames * (N + 1) * HD * 4),
                          "note": "frames phase only; per frame: pinned H2D of the hidden states, "
-                                 "vs_frame_prefill, D2H of the fp32 output; wall clock incl. launch cost"}
+                                 "vs_frame_prefill, D2H of the fp32 output, the copies on streams of their own "
+                                 "(two buffers each way); wall clock incl. launch cost"}
         if not args.no_cpu_baseline and world == 1:
             n_frames, n_decode = w.n_frames, w.decode_tokens
             fps_cpu, tps_cpu, secs = time_oracle_sample(w, n_frames, n_decode)
