@@ -35,6 +35,9 @@ if ROOT not in sys.path:
 from paper_2503_09387_b200 import synth  # noqa: E402
 
 
+GEMM_FRAME_DRAM_BYTES = 34365184 + 12288   # ncu: read + write of one 170-row projection launch
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -317,7 +320,11 @@ def run_ours(args, w):
         if dom == "qkv_gemm":
             ach = proj_flops / (kernels[dom]["avg_us"] * 1e-6) / 1e12
             roof = {"kernel": dom, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
-                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None,
+                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
+                    # dram__bytes_read.sum + dram__bytes_write.sum of one frame launch of this kernel
+                    # (cold cache, so the weights come from DRAM), from the ncu capture summarised in
+                    # profiles/qkv_gemm_frame_170rows.md; only quoted for the shape that was captured
+                    "traffic": GEMM_FRAME_DRAM_BYTES if (N, d, w.e_out) == (169, 3584, 4608) else None,
                     "peak_source": peaks["source"] + " (sustained bf16; kernel timed inside the step)",
                     "avg_launch_us": kernels[dom]["avg_us"]}
         else:
