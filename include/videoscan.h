@@ -19,6 +19,10 @@
  *  - A handle is not thread safe.  Distinct handles are independent.
  *  - Device-side waits are bounded; if one ever expires the kernel records
  *    VS_ERR_DEVICE_TIMEOUT in a device status word that vs_bank_state reports.
+ *    A handle that has reported it holds unspecified state: destroy it.
+ *  - The projection of a step whose K split spans several thread blocks lets those
+ *    blocks wait for one another, which needs all of them on the GPU at once: a
+ *    handle expects the whole GPU (no other work sharing its SMs while a step runs).
  */
 #ifndef VIDEOSCAN_H_
 #define VIDEOSCAN_H_
