@@ -16,13 +16,16 @@
  *    cudaStream_t passed as void*; NULL is the default stream) and return without
  *    synchronising.  vs_bank_state synchronises that stream.  All calls on one handle
  *    must use the same CUDA stream (or be ordered by the caller).
- *  - A handle is not thread safe.  Distinct handles are independent.
+ *  - A handle is not thread safe.  Distinct handles share no state.
  *  - Device-side waits are bounded; if one ever expires the kernel records
  *    VS_ERR_DEVICE_TIMEOUT in a device status word that vs_bank_state reports.
  *    A handle that has reported it holds unspecified state: destroy it.
  *  - The projection of a step whose K split spans several thread blocks lets those
  *    blocks wait for one another, which needs all of them on the GPU at once: a
- *    handle expects the whole GPU (no other work sharing its SMs while a step runs).
+ *    handle expects the whole GPU while a step runs.  In particular the steps of two
+ *    handles on one GPU must not overlap (same stream, or ordered by events): two such
+ *    projections holding half the SMs each would wait for blocks that cannot start,
+ *    and both would end with VS_ERR_DEVICE_TIMEOUT.
  */
 #ifndef VIDEOSCAN_H_
 #define VIDEOSCAN_H_
