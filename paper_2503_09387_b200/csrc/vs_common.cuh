@@ -141,6 +141,9 @@ cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* r
 struct ProjectionOut {
   const bf16* bias;              // [E_out] or null
   const float* row_scale;        // [rows] RMSNorm scale applied to the accumulated row, or null
+  int norm_inline;               // matrix-vector kernel only: it computes the RMSNorm scale (and h * gain) itself
+  const bf16* norm_gain;         // [d] or null
+  float norm_eps;
   const float2* rope;            // [rows][D/2] (cos, sin); null: the kernel derives them from inv_freq (few rows only)
   const double* inv_freq;        // [D/2]
   bf16* q;                       // [rows][Hq*D]  rotated query, leading bf16 part
@@ -170,6 +173,7 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
 cudaError_t qkv_gemm_init();     // opt-in shared memory attribute, once per process/device
 // Projection of one to four rows of a text step as a matrix-vector product (no RoPE table needed).
 bool qkv_gemv_supported(const ProjectionOut& o, int rows, int d);
+cudaError_t qkv_gemv_init();     // opt-in shared memory attribute, once per process/device
 cudaError_t launch_qkv_gemv(const bf16* W, const bf16* x, const ProjectionOut& o, const BatchParams& bp, int rows, int E_out,
                             int d, cudaStream_t st);
 

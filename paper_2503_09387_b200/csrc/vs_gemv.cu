@@ -1,17 +1,21 @@
 // QKV projection of a text step of one to four token rows (Eq. 1 with a handful of rows:
 // decode, Section 3.3's answer tokens).  With so few rows the projection is a matrix-vector
-// product bound by reading W once, not a tensor-core contraction: every CTA streams 32 rows of
-// W ([E_out, d] bf16, row-major) with 16-byte loads, each warp owning four rows and each lane a
-// 16-byte column of them, fp32 accumulation, a shuffle reduction per row.
+// product bound by reading W once, not a tensor-core contraction.  Every CTA owns 32 rows of
+// W ([E_out, d] bf16, row-major) and streams them through a ring of shared-memory stages filled
+// by 16-byte asynchronous copies (a stage = 256 elements of all 32 rows, 16 KiB; eight stages,
+// so up to 112 KiB per SM are in flight whatever the registers hold); each warp then reads four
+// rows back, a lane one 16-byte column of them, fp32 accumulation, a shuffle reduction per row.
 //
 // A CTA's 32 rows are 16 rotation pairs (k, k + D/2) of one head, so the epilogue has both
 // elements of a pair at hand: RMSNorm row scale, bias, RoPE (the angle in fp64 from the token's
 // position, as the table kernel computes it), bf16 rounding, the query's hi + lo pair, and the
-// write of K/V rows to the prefix or to the turn's tail.
+// write of K/V rows to the prefix or to the turn's tail.  RMSNorm is done here too (every CTA
+// holds the token rows, so each works out the row scale and, with a gain vector, bf16(h * gain)
+// itself): such a step launches no statistics kernel.
 //
-// W never changes while the stream handle lives, so the first batch of W loads and the rotation
-// angles are issued before the wait on the stream's earlier kernels; the token rows are read
-// after it.
+// W never changes while the stream handle lives, so the ring is filled and the rotation angles
+// are worked out before the wait on the stream's earlier kernels; the token rows are read after
+// it.
 #include "vs_common.cuh"
 
 namespace vs {
@@ -20,7 +24,9 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kRowsPerCta = 32;     // 16 rotation pairs
-constexpr int kU = 2;               // 16-byte chunks per W row in one batch of loads (two batches in flight)
+constexpr int kStageElems = 256;    // K elements of every row in one stage
+constexpr int kStageBytes = kRowsPerCta * kStageElems * 2;   // 16 KiB
+constexpr int kStages = 8;
 
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
@@ -32,41 +38,54 @@ __device__ __forceinline__ float dot8(const uint4& w, const uint4& x, float acc)
   acc = fmaf(bf_lo(w.w), bf_lo(x.w), acc); acc = fmaf(bf_hi(w.w), bf_hi(x.w), acc);
   return acc;
 }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 template <int R>   // token rows held (1, 2 or 4)
 __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __restrict__ W, const bf16* __restrict__ x,
                                                             ProjectionOut o, BatchParams bp, int rows, int d) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  uint4* xs = reinterpret_cast<uint4*>(smem_raw);                       // [R][d / 8]
-  float* ys = reinterpret_cast<float*>(smem_raw + (size_t)R * d * 2);   // [R][32]
+  // carve: ring [kStages][32 rows][512 B] | token rows [R][d] bf16 | results [R][32] | row scales [R] | partial sums [R][8]
+  uint4* xs = reinterpret_cast<uint4*>(smem_raw + kStages * kStageBytes);
+  float* ys = reinterpret_cast<float*>(smem_raw + kStages * kStageBytes + (size_t)R * d * 2);
+  float* rs = ys + R * kRowsPerCta;
+  float* red = rs + R;
+  const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int D = o.D, half = D >> 1;
   const int blocks_per_head = half / 16;
   const int hs = (int)blockIdx.x / blocks_per_head;                     // head slot: Q heads, K heads, V heads
   const int pb = (int)blockIdx.x - hs * blocks_per_head;
-  const int n_chunks = d >> 8;                                          // 16-byte chunks per lane and row
+  const int n_stage_total = d / kStageElems;
   const int chunks_per_row = d >> 3;
 
-  // the warp's four rows of W: local row lr -> pair lr & 15, second element of the pair if lr >= 16
-  const uint4* wrow[4];
+  // copies of a stage: thread t moves the 16-byte chunks t, t + 256, ... of the stage's 1024;
+  // chunk index -> (local row lr = idx / 32, column idx % 32); lr -> pair lr & 15, second element
+  // of the pair if lr >= 16
+  const bf16* csrc[4];
+  uint32_t cdst[4];
 #pragma unroll
-  for (int rr = 0; rr < 4; ++rr) {
-    const int lr = warp * 4 + rr;
+  for (int q = 0; q < 4; ++q) {
+    const int idx = tid + kThreads * q;
+    const int lr = idx >> 5, c = idx & 31;
     const int f = hs * D + pb * 16 + (lr & 15) + (lr >> 4) * half;
-    wrow[rr] = reinterpret_cast<const uint4*>(W + (size_t)f * d) + lane;
+    csrc[q] = W + (size_t)f * d + c * 8;
+    cdst[q] = (uint32_t)(lr * (kStageElems * 2) + c * 16);
   }
-  auto load_batch = [&](uint4 (&buf)[4][kU], int i0) {
+  auto issue_stage = [&](int i) {
+    if (i < n_stage_total) {
+      const uint32_t slot = ring + (uint32_t)(i % kStages) * kStageBytes;
 #pragma unroll
-    for (int u = 0; u < kU; ++u) {
-      const int i = i0 + u;
-#pragma unroll
-      for (int rr = 0; rr < 4; ++rr)
-        buf[rr][u] = (i < n_chunks) ? __ldg(wrow[rr] + i * 32) : make_uint4(0u, 0u, 0u, 0u);
+      for (int q = 0; q < 4; ++q) cp_async16(slot + cdst[q], csrc[q] + (size_t)i * kStageElems);
     }
+    cp_async_commit();                                                  // one group per stage, empty or not
   };
-  uint4 bufA[4][kU], bufB[4][kU];
-  load_batch(bufA, 0);                                                  // W is constant: no need to wait for it
+  for (int i = 0; i < kStages - 1; ++i) issue_stage(i);                 // W is constant: no need to wait for it
 
   // finishing threads: (token row r, pair p); the rotation depends on the parameters alone
   const int fr = tid >> 4, fp = tid & 15;
@@ -87,37 +106,73 @@ __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __res
   pdl_wait();                       // earlier kernels of the stream have completed
   pdl_launch_dependents();
 
-  for (int idx = tid; idx < R * chunks_per_row; idx += kThreads) {
-    const int r = idx / chunks_per_row;
-    xs[idx] = (r < rows) ? reinterpret_cast<const uint4*>(x)[idx] : make_uint4(0u, 0u, 0u, 0u);
+  // token rows -> shared memory; with RMSNorm: sum of squares of the raw row, and the row times
+  // the gain vector (rounded to bf16, as the statistics kernel stores it) in place of the row
+  {
+    float ss[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) ss[r] = 0.f;
+    for (int c = tid; c < chunks_per_row; c += kThreads) {
+      uint4 g4 = make_uint4(0u, 0u, 0u, 0u);
+      if (o.norm_inline && o.norm_gain != nullptr) g4 = reinterpret_cast<const uint4*>(o.norm_gain)[c];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        uint4 v = (r < rows) ? reinterpret_cast<const uint4*>(x)[r * chunks_per_row + c] : make_uint4(0u, 0u, 0u, 0u);
+        if (o.norm_inline) {
+          const uint32_t* vw = reinterpret_cast<const uint32_t*>(&v);
+          const uint32_t* gw = reinterpret_cast<const uint32_t*>(&g4);
+          uint32_t ow[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float a0 = bf_lo(vw[k]), a1 = bf_hi(vw[k]);
+            ss[r] += a0 * a0 + a1 * a1;
+            const __nv_bfloat162 p = __floats2bfloat162_rn(a0 * bf_lo(gw[k]), a1 * bf_hi(gw[k]));
+            ow[k] = *reinterpret_cast<const uint32_t*>(&p);
+          }
+          if (o.norm_gain != nullptr) v = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+        }
+        xs[r * chunks_per_row + c] = v;
+      }
+    }
+    if (o.norm_inline) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        float v = ss[r];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+        if (lane == 0) red[r * 8 + warp] = v;
+      }
+    }
   }
   __syncthreads();
+  if (o.norm_inline && tid < R) {
+    float tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) tot += red[tid * 8 + i];
+    rs[tid] = rsqrtf(tot / (float)d + o.norm_eps);
+  }
 
   float acc[4][R];
 #pragma unroll
   for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
     for (int r = 0; r < R; ++r) acc[rr][r] = 0.f;
-  auto consume = [&](const uint4 (&buf)[4][kU], int i0) {
+  for (int i = 0; i < n_stage_total; ++i) {
+    cp_async_wait<kStages - 2>();   // this thread's copies of stage i have landed
+    __syncthreads();                // everyone's have, and everyone is done with stage i - 1
+    issue_stage(i + kStages - 1);   // into the slot stage i - 1 occupied
+    const uint4* slot = reinterpret_cast<const uint4*>(smem_raw + (size_t)(i % kStages) * kStageBytes);
+    uint4 xv[R];
 #pragma unroll
-    for (int u = 0; u < kU; ++u) {
-      const int i = i0 + u;
-      if (i < n_chunks) {
+    for (int r = 0; r < R; ++r) xv[r] = xs[r * chunks_per_row + i * 32 + lane];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-          const uint4 xv = xs[r * chunks_per_row + i * 32 + lane];
+    for (int rr = 0; rr < 4; ++rr) {
+      const uint4 wv = slot[(warp * 4 + rr) * 32 + lane];
 #pragma unroll
-          for (int rr = 0; rr < 4; ++rr) acc[rr][r] = dot8(buf[rr][u], xv, acc[rr][r]);
-        }
-      }
+      for (int r = 0; r < R; ++r) acc[rr][r] = dot8(wv, xv[r], acc[rr][r]);
     }
-  };
-  for (int i0 = 0; i0 < n_chunks; i0 += 2 * kU) {
-    load_batch(bufB, i0 + kU);
-    consume(bufA, i0);
-    load_batch(bufA, i0 + 2 * kU);
-    consume(bufB, i0 + kU);
   }
+  cp_async_wait<0>();
 #pragma unroll
   for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
@@ -133,7 +188,8 @@ __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __res
     const int row = fr;
     float x1 = ys[row * kRowsPerCta + fp], x2 = ys[row * kRowsPerCta + 16 + fp];
     const int f1 = hs * D + k0, f2 = f1 + half;
-    const float rsc = (o.row_scale != nullptr) ? o.row_scale[row] : 1.f;   // RMSNorm's row scale commutes with the projection
+    // RMSNorm's row scale commutes with the projection
+    const float rsc = o.norm_inline ? rs[row] : ((o.row_scale != nullptr) ? o.row_scale[row] : 1.f);
     const float b1 = (o.bias != nullptr) ? __bfloat162float(o.bias[f1]) : 0.f;
     const float b2 = (o.bias != nullptr) ? __bfloat162float(o.bias[f2]) : 0.f;
     x1 = fmaf(x1, rsc, b1); x2 = fmaf(x2, rsc, b2);
@@ -164,10 +220,21 @@ __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __res
 
 }  // namespace
 
+static size_t gemv_smem_bytes(int R, int d) {
+  return (size_t)kStages * kStageBytes + (size_t)R * d * 2 + (size_t)R * kRowsPerCta * 4 + (size_t)R * 4 + (size_t)R * 8 * 4;
+}
+
 bool qkv_gemv_supported(const ProjectionOut& o, int rows, int d) {
   if (rows < 1 || rows > 4 || o.mode == 0) return false;                // text steps only
   if ((d & 255) != 0 || (o.D != 64 && o.D != 128)) return false;
-  return (size_t)4 * d * 2 + 4 * kRowsPerCta * 4 <= 48 * 1024;          // fits the default dynamic shared memory
+  return gemv_smem_bytes(4, d) <= 200 * 1024;
+}
+
+cudaError_t qkv_gemv_init() {
+  cudaError_t e = cudaFuncSetAttribute(qkv_gemv_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(qkv_gemv_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(qkv_gemv_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  return e;
 }
 
 cudaError_t launch_qkv_gemv(const bf16* W, const bf16* x, const ProjectionOut& o, const BatchParams& bp, int rows, int E_out,
@@ -175,7 +242,7 @@ cudaError_t launch_qkv_gemv(const bf16* W, const bf16* x, const ProjectionOut& o
   if (!qkv_gemv_supported(o, rows, d) || o.inv_freq == nullptr) return cudaErrorInvalidValue;
   const dim3 grid((E_out / o.D) * ((o.D / 2) / 16));
   const int R = rows == 1 ? 1 : (rows == 2 ? 2 : 4);
-  const size_t smem = (size_t)R * d * 2 + (size_t)R * kRowsPerCta * 4;
+  const size_t smem = gemv_smem_bytes(R, d);
   if (R == 1) return launch_pdl(qkv_gemv_kernel<1>, grid, dim3(kThreads), smem, st, W, x, o, bp, rows, d);
   if (R == 2) return launch_pdl(qkv_gemv_kernel<2>, grid, dim3(kThreads), smem, st, W, x, o, bp, rows, d);
   return launch_pdl(qkv_gemv_kernel<4>, grid, dim3(kThreads), smem, st, W, x, o, bp, rows, d);

@@ -271,7 +271,7 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights, void* work
   h->tm_w.resize(D.L);
   for (int l = 0; l < D.L; ++l)
     if (encode_2d(h, &h->tm_w[l], h->w[l], (uint64_t)D.d, (uint64_t)D.E_out, GEMM_BLOCK_M) != VS_OK) return fail(VS_ERR_CUDA);
-  if (qkv_gemm_init() != cudaSuccess || prefill_attention_tc_init() != cudaSuccess) return fail(VS_ERR_CUDA);
+  if (qkv_gemm_init() != cudaSuccess || qkv_gemv_init() != cudaSuccess || prefill_attention_tc_init() != cudaSuccess) return fail(VS_ERR_CUDA);
   // clear the whole workspace, then write the non-zero initial metadata
   if (cudaMemset(h->ws, 0, lo.total) != cudaSuccess) return fail(VS_ERR_CUDA);
   if (cudaMemset(h->ws + lo.slot_frame, 0xFF, (size_t)D.S * D.slots * 4) != cudaSuccess) return fail(VS_ERR_CUDA);
@@ -358,6 +358,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     ProjectionOut fa;
     fa.bias = h->bias[l];
     fa.row_scale = D.use_rmsnorm ? h->at<float>(lo.row_scale) : nullptr;
+    fa.norm_inline = 0; fa.norm_gain = nullptr; fa.norm_eps = 0.f;
     fa.rope = h->at<float2>(lo.rope);
     fa.inv_freq = h->at<double>(lo.inv_freq);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
@@ -451,7 +452,12 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
   int next_buf = 0;
   for (int l = 0; l < D.L; ++l) {
     const bf16* src = h_in;
-    if (D.use_rmsnorm) {
+    // a step the matrix-vector kernel takes needs no statistics launch: that kernel normalises itself
+    ProjectionOut probe;
+    std::memset(&probe, 0, sizeof(probe));
+    probe.mode = 1; probe.D = D.D;
+    const bool by_gemv = rope_inline && qkv_gemv_supported(probe, rows, D.d) && (reinterpret_cast<uintptr_t>(h_in) & 15u) == 0;
+    if (D.use_rmsnorm && !by_gemv) {
       VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_scale),
                                                     rows, D.d, D.rms_eps, st));
       if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
@@ -465,7 +471,8 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
 
     ProjectionOut fa;
     fa.bias = h->bias[l];
-    fa.row_scale = D.use_rmsnorm ? h->at<float>(lo.row_scale) : nullptr;
+    fa.row_scale = (D.use_rmsnorm && !by_gemv) ? h->at<float>(lo.row_scale) : nullptr;
+    fa.norm_inline = (D.use_rmsnorm && by_gemv) ? 1 : 0; fa.norm_gain = h->gain[l]; fa.norm_eps = D.rms_eps;
     fa.rope = rope_inline ? nullptr : h->at<float2>(lo.rope);
     fa.inv_freq = h->at<double>(lo.inv_freq);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
