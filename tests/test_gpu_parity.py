@@ -48,6 +48,21 @@ def test_odd_shapes_and_policies(N, P, M, policy):
     p.close()
 
 
+def test_width_that_is_no_multiple_of_256():
+    """d_model = 320 (five 64-wide K blocks): few-row text steps cannot take the matrix-vector
+    kernel (it moves 256 elements of a row per stage) and fall back to the tensor-core projection
+    with the rotation derived in the kernel."""
+    w = synth.workload("tiny", d_model=320, n_q_heads=4, n_kv_heads=2, head_dim=64, tokens_per_frame=21,
+                       prefix_len=3, n_frames=6, bank_capacity=3, question_len=2, decode_tokens=3, seed=31)
+    p = Pair(w, max_text=8)
+    p.gpu.profile_read()
+    run_stream(p, w)
+    launches = p.gpu.profile_read()
+    assert launches["qkv_gemv"][2] == 0 and launches["rope_table"][2] == 0
+    assert launches["qkv_gemm"][2] == 1 + 6 + 1 + 3
+    p.close()
+
+
 def test_bias_last_token_aggregation_and_carrier_override():
     w = synth.workload("tiny", seed=5, n_frames=6)
     p = Pair(w, with_bias=True, agg_mode=1)
