@@ -81,6 +81,8 @@ typedef struct {
   int32_t out_dtype;             /* element type of `out`: 0 = bf16, 1 = fp32.  Attention outputs reach
                                     |y| > 4 on LLaVA-Video-shaped inputs, where bf16 storage alone
                                     rounds by up to 1.6e-2; fp32 keeps the fp32-accumulated value    */
+  int32_t max_chunk_frames;      /* most frames one vs_frame_prefill_chunk call may bring (0 or 1:
+                                    that call is not used); sizes the per-step scratch              */
 } vs_config;
 
 /* DEVICE pointers to bf16 weights, one entry per layer.  The arrays of pointers themselves
@@ -136,6 +138,17 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights,
 int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
                      const void* hidden, int32_t N, const void* carrier_override,
                      void* out, void* cuda_stream);
+
+/* F consecutive frames of ONE stream in one call -- the offline form of the prefilling phase
+ * (Section 3.3; the paper's offline benchmarks of Section 4 feed whole videos).  The result is
+ * that of F vs_frame_prefill calls in a row: each frame attends over [prefix | the bank as the
+ * frames before it left it | own frame], evictions included, because the eviction rule looks
+ * only at carrier embeddings, which are all known once the frames are pooled.  Per layer the
+ * Q/K/V projection of all F*(N+1) rows is one GEMM; the attention runs frame by frame.
+ * hidden: DEVICE bf16 [F][N][d_model];  out: DEVICE [F][N+1][Hq*D] of `out_dtype`, or NULL.
+ * Errors: as vs_frame_prefill; VS_ERR_CAPACITY also if F > max_chunk_frames. */
+int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, int32_t F, int32_t N,
+                           void* out, void* cuda_stream);
 
 /* T text tokens per listed stream -- the decoding phase of Section 3.3 (T = 1) and the
  * text part of prefilling (T > 1).  Token i attends to [prefix | bank | tail tokens up to

@@ -26,7 +26,7 @@ VS_ERR_DEVICE_TIMEOUT = -5
 VS_ERR_UNSUPPORTED = -6
 VS_MAX_BATCH = 64
 
-EXPORTS = ["vs_workspace_bytes", "vs_create_stream", "vs_frame_prefill", "vs_decode_step",
+EXPORTS = ["vs_workspace_bytes", "vs_create_stream", "vs_frame_prefill", "vs_frame_prefill_chunk", "vs_decode_step",
            "vs_end_turn", "vs_bank_state", "vs_last_step_kv", "vs_poison_scratch",
            "vs_destroy_stream", "vs_status_string", "vs_reset_stream", "vs_profile_enable",
            "vs_profile_read", "vs_kernel_class_name", "vs_evict_choose_static"]
@@ -40,7 +40,8 @@ class VsConfig(C.Structure):
         "max_prefix", "max_text", "max_step_tokens", "bank_capacity", "n_streams", "agg_mode",
         "evict_policy", "use_rmsnorm", "residual")] + [
         ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("device", C.c_int32),
-        ("evict_log_capacity", C.c_int32), ("out_dtype", C.c_int32)]
+        ("evict_log_capacity", C.c_int32), ("out_dtype", C.c_int32),
+        ("max_chunk_frames", C.c_int32)]
 
 
 class VsWeights(C.Structure):
@@ -80,6 +81,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.vs_workspace_bytes.argtypes = [C.POINTER(VsConfig), C.POINTER(C.c_size_t)]
     lib.vs_create_stream.argtypes = [C.POINTER(VsConfig), C.POINTER(VsWeights), vp, C.c_size_t, C.POINTER(vp)]
     lib.vs_frame_prefill.argtypes = [vp, i32p, i32, vp, i32, vp, vp, vp]
+    lib.vs_frame_prefill_chunk.argtypes = [vp, i32, vp, i32, i32, vp, vp]
     lib.vs_decode_step.argtypes = [vp, i32p, i32, vp, i32, vp, vp]
     lib.vs_end_turn.argtypes = [vp, i32p, i32]
     lib.vs_bank_state.argtypes = [vp, i32, C.POINTER(VsBankInfo), i32p, C.POINTER(C.c_int64), i32p,
@@ -144,6 +146,12 @@ def vs_frame_prefill(handle: int, stream_ids: Sequence[int], hidden_ptr: int, N:
     ids, n = _ids(stream_ids)
     _check(load_library().vs_frame_prefill(handle, ids, n, hidden_ptr, N, carrier_override_ptr or None,
                                            out_ptr or None, cuda_stream or None), "vs_frame_prefill")
+
+
+def vs_frame_prefill_chunk(handle: int, stream_id: int, hidden_ptr: int, F: int, N: int,
+                           out_ptr: Optional[int] = None, cuda_stream: Optional[int] = None) -> None:
+    _check(load_library().vs_frame_prefill_chunk(handle, stream_id, hidden_ptr, F, N, out_ptr or None,
+                                                 cuda_stream or None), "vs_frame_prefill_chunk")
 
 
 def vs_decode_step(handle: int, stream_ids: Sequence[int], hidden_ptr: int, T: int, out_ptr: int,
@@ -283,6 +291,16 @@ class StreamBatch:
                          out.data_ptr() if out is not None else None, self._stream())
         return out
 
+    def frame_prefill_chunk(self, stream_id, hidden, out=None, want_out=True):
+        """hidden: [F][N][d] of one stream."""
+        F, N = hidden.shape[0], hidden.shape[1]
+        assert hidden.is_contiguous() and hidden.numel() == F * N * self.cfg.d_model
+        if out is None and want_out:
+            out = self.torch.empty((F, N + 1, self.out_width), dtype=self.out_torch_dtype, device=self.device)
+        vs_frame_prefill_chunk(self.handle, stream_id, hidden.data_ptr(), F, N,
+                               out.data_ptr() if out is not None else None, self._stream())
+        return out
+
     def decode_step(self, stream_ids, hidden, out=None):
         n = len(stream_ids)
         T = hidden.shape[-2]
@@ -328,7 +346,7 @@ class StreamBatch:
 def make_config(n_layers, d_model, n_q_heads, n_kv_heads, head_dim, max_tokens_per_frame, max_prefix,
                 max_text, bank_capacity, n_streams=1, max_step_tokens=64, agg_mode=0, evict_policy=0,
                 use_rmsnorm=0, residual=0, rope_theta=1.0e6, rms_eps=1.0e-6, device=0,
-                evict_log_capacity=4096, out_dtype=1) -> VsConfig:
+                evict_log_capacity=4096, out_dtype=1, max_chunk_frames=1) -> VsConfig:
     return VsConfig(n_layers, d_model, n_q_heads, n_kv_heads, head_dim, max_tokens_per_frame, max_prefix,
                     max_text, max_step_tokens, bank_capacity, n_streams, agg_mode, evict_policy, use_rmsnorm,
-                    residual, rope_theta, rms_eps, device, evict_log_capacity, out_dtype)
+                    residual, rope_theta, rms_eps, device, evict_log_capacity, out_dtype, max_chunk_frames)

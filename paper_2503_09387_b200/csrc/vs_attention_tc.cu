@@ -204,7 +204,25 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   // carrier embeddings, the bank's order and metadata -- was complete before the kernel ahead of
   // this one let it start, and nothing else in this launch touches what they write.
   if ((int)blockIdx.x < a.bank_blocks) {
-    if (blockIdx.y == 0) bank_update_block(a.bank, bp, (int)blockIdx.z, (int)blockIdx.x);
+    if (blockIdx.y == 0) {
+      if (a.copy_k == nullptr) {
+        bank_update_block(a.bank, bp, (int)blockIdx.z, (int)blockIdx.x);
+      } else {
+        // chunk of frames: this frame's carrier K/V row goes into the slot its bank update chose.
+        // The row is the projection's (the kernel ahead), hence the wait; nothing in this launch
+        // reads that slot (it is the hole of this frame's key axis).
+        pdl_wait();
+        const int sid = bp.stream_id[blockIdx.z];
+        const int slot = *a.copy_slot;
+        const int per_head = D / 8;                                   // 16-byte chunks of one head's row
+        for (int i = tid; i < a.Hkv * per_head; i += kAttnThreads) {
+          const int hk = i / per_head, c = i - hk * per_head;
+          const size_t dst = (((size_t)sid * a.Hkv + hk) * a.slots + slot) * D + c * 8;
+          *reinterpret_cast<uint4*>(a.copy_dst_k + dst) = *reinterpret_cast<const uint4*>(a.copy_k + hk * D + c * 8);
+          *reinterpret_cast<uint4*>(a.copy_dst_v + dst) = *reinterpret_cast<const uint4*>(a.copy_v + hk * D + c * 8);
+        }
+      }
+    }
     return;
   }
   // ---- set-up that needs nothing from earlier kernels: barriers, tensor memory ------------------

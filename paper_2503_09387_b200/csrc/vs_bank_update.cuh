@@ -38,9 +38,21 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
   int32_t* slot_frame = a.slot_frame + (size_t)sid * a.slots;
   int64_t* slot_pos = a.slot_pos + (size_t)sid * a.slots;
   const int count = bp.count[b];
-  const int incoming = a.step_slot[sid];
+  const int incoming = (a.incoming_emb != nullptr) ? meta->free_slot : a.step_slot[sid];
+  // chunked prefill: the incoming embedding is read from where it is parked and moved into its slot
+  // by whoever commits
+  const bf16* emb_in = (a.incoming_emb != nullptr) ? a.incoming_emb + (size_t)b * a.d
+                                                   : a.emb + ((size_t)sid * a.slots + incoming) * a.d;
+  auto adopt = [&]() {      // all threads of the committing block
+    if (a.incoming_emb != nullptr) {
+      bf16* dst = const_cast<bf16*>(a.emb) + ((size_t)sid * a.slots + incoming) * a.d;
+      for (int k = tid; k < a.d; k += blockDim.x) dst[k] = emb_in[k];
+      if (tid == 0) a.record_slot[b] = incoming;
+    }
+  };
   const int64_t carrier_pos = bp.pos_base[b] + bp.rows_per_stream - 1;
   if (count < a.M) {
+    if (block == 0) adopt();
     if (block == 0 && tid == 0) {
       order[count] = incoming;
       slot_frame[incoming] = (int32_t)bp.frame_id[b];
@@ -62,7 +74,7 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
     const int sa = order[j];
     const int sb = (a.policy == 1 && j + 1 < count) ? order[j + 1] : incoming;
     const bf16* va = a.emb + ((size_t)sid * a.slots + sa) * a.d;
-    const bf16* vb = a.emb + ((size_t)sid * a.slots + sb) * a.d;
+    const bf16* vb = (sb == incoming) ? emb_in : a.emb + ((size_t)sid * a.slots + sb) * a.d;
     double dot = 0.0, na = 0.0, nb = 0.0;
     for (int k = lane; k < a.d; k += 32) {
       const double x = (double)__bfloat162float(va[k]);
@@ -105,6 +117,7 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
     }
     __syncthreads();
   }
+  adopt();
   const int v = (a.policy == 2) ? 0 : best_j[0];
   const int victim_slot = order[v];
   const int victim_frame = slot_frame[victim_slot];

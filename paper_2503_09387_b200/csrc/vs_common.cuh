@@ -43,7 +43,7 @@ struct BatchParams {
 // ---- shapes ----------------------------------------------------------------------------
 struct Dims {
   int L, d, Hq, Hkv, D, G, E_out;
-  int maxN, maxP, maxT, maxStepT, M, slots, S;   // maxP / maxT: allocated rows (>= 1)
+  int maxN, maxP, maxT, maxStepT, M, slots, S, maxChunk;   // maxP / maxT: allocated rows (>= 1)
   int capP, capT;                                // caller's prefix / tail capacities
   int rows_per_stream_max, R_max;
   int log_cap;
@@ -73,6 +73,7 @@ struct Layout {
   size_t inv_freq;              // f64   [D/2]
   size_t status;                // int32 [8]
   size_t step_slot;             // int32 [S]  free slot as the running frame step found it
+  size_t chunk_slot;            // int32 [VS_MAX_BATCH]  chunked prefill: slot each frame's carrier went to
   size_t tickets;               // int32 [S*Hq]  split-KV decode: CTAs finished per (stream, query head)
   size_t gemm_flags;            // int32 [GEMM_XCHG_CTAS]  projection K split: partials delivered per slice owner
   size_t persistent_end;
@@ -86,6 +87,7 @@ struct Layout {
   size_t rope;                  // float2 [R_max][D/2]
   size_t obuf;                  // f32  [R_max][Hq*D] (holds bf16 or fp32 rows)
   size_t dec_part;              // f32  [DEC_SPLIT_MAX][S][Hq][D+2]
+  size_t emb_stage;             // bf16 [max_chunk][d]  chunked prefill: carrier embeddings before they have a slot
   size_t gemm_xchg;             // f32  [GEMM_XCHG_CTAS][256][128]  projection K split: partial tiles
   size_t scratch_begin, scratch_end;
   size_t total;
@@ -121,6 +123,8 @@ struct PoolArgs {
   bf16* emb;                     // [S][slots][d]
   const StreamMeta* meta;        // [S]
   int32_t* step_slot;            // [S] copy of meta.free_slot for the rest of the step
+  bf16* emb_stage;               // chunked prefill: [n_active][d] carrier embeddings parked here instead of the
+                                 // bank (their slots are only known as the bank updates run); else null
   const double* inv_freq;        // [D/2]
   float2* rope;                  // [n_active][N+1][D/2]
   int N, d, D, slots, M, agg_mode;
@@ -155,7 +159,8 @@ struct ProjectionOut {
   const int32_t* free_slot;      // free slot of stream s at free_slot[s * free_slot_stride]
   int free_slot_stride;
   int Hq, Hkv, D, slots, text_cap, M;
-  int mode;                      // 0 frame step (carrier row -> bank), 1 text -> prefix, 2 text -> tail
+  int mode;                      // 0 frame step (carrier row -> bank), 1 text -> prefix, 2 text -> tail,
+                                 // 3 chunk of frames (nothing kept: the attention launches copy the carrier rows)
 };
 
 struct GemmArgs {
@@ -181,6 +186,10 @@ struct BankUpdateArgs {
   const bf16* emb;               // [S][slots][d]
   StreamMeta* meta;
   const int32_t* step_slot;      // [S] the slot the incoming carrier was written to
+  // chunked prefill: the incoming carrier's embedding is still parked at `incoming_emb`; the slot
+  // is meta.free_slot, recorded in *record_slot, and the embedding moves into the bank here
+  const bf16* incoming_emb;
+  int32_t* record_slot;
   int32_t* order; int32_t* slot_frame; int64_t* slot_pos; int32_t* evict_log; double* scores;
   int d, slots, M, policy, log_cap;
 };
@@ -208,7 +217,14 @@ struct AttnArgs {
   // frame steps, last layer: the first bank_blocks CTAs of every stream do the bank update
   BankUpdateArgs bank;
   int bank_blocks;
+  // chunked prefill instead: one spare CTA copies the frame's carrier K/V row (Hkv*D each) into
+  // slot *copy_slot of this layer's bank
+  const bf16* copy_k; const bf16* copy_v;
+  bf16* copy_dst_k; bf16* copy_dst_v;   // this layer's bank [S][Hkv][slots][D]
+  const int32_t* copy_slot;
 };
+// chunked prefill: the bank update of one frame as a launch of its own (it precedes the projection)
+cudaError_t launch_bank_update(const BankUpdateArgs& a, const BatchParams& bp, bool full, cudaStream_t st);
 cudaError_t launch_prefill_attention_tc(const AttnArgs& a, const BatchParams& bp, int* status, cudaStream_t st);
 cudaError_t prefill_attention_tc_init();
 

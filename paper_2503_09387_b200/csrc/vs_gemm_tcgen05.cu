@@ -412,7 +412,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
               const int slot = p.o.free_slot[sid * p.o.free_slot_stride];
               dst = (is_k ? p.o.bank_k : p.o.bank_v) + (((size_t)sid * p.o.Hkv + hkv) * p.o.slots + slot) * D + k0;
             }
-          } else {
+          } else if (p.o.mode != 3) {
             const int tb = (p.o.mode == 1) ? bp.prefix_len[b] : bp.text_len[b];
             dst = (is_k ? p.o.text_k : p.o.text_v) + (((size_t)sid * p.o.Hkv + hkv) * p.o.text_cap + tb + tt) * D + k0;
           }

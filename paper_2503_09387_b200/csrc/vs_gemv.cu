@@ -225,7 +225,7 @@ static size_t gemv_smem_bytes(int R, int d) {
 }
 
 bool qkv_gemv_supported(const ProjectionOut& o, int rows, int d) {
-  if (rows < 1 || rows > 4 || o.mode == 0) return false;                // text steps only
+  if (rows < 1 || rows > 4 || (o.mode != 1 && o.mode != 2)) return false;   // text steps only
   if ((d & 255) != 0 || (o.D != 64 && o.D != 128)) return false;
   return gemv_smem_bytes(4, d) <= 200 * 1024;
 }

@@ -34,6 +34,7 @@ int fill_dims(const vs_config* c, Dims& D) {
   if (c->max_tokens_per_frame < 1 || c->max_prefix < 0 || c->max_text < 0 || c->bank_capacity < 0) return VS_ERR_INVALID_ARG;
   if (c->max_step_tokens < 1 || c->evict_log_capacity < 0) return VS_ERR_INVALID_ARG;
   if (c->out_dtype < 0 || c->out_dtype > 1) return VS_ERR_INVALID_ARG;
+  if (c->max_chunk_frames < 0 || c->max_chunk_frames > VS_MAX_BATCH) return VS_ERR_INVALID_ARG;
   if (c->agg_mode < 0 || c->agg_mode > 1 || c->evict_policy < 0 || c->evict_policy > 2) return VS_ERR_INVALID_ARG;
   if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f)) return VS_ERR_INVALID_ARG;
   if (c->d_model % 64 != 0) return VS_ERR_UNSUPPORTED;
@@ -49,7 +50,9 @@ int fill_dims(const vs_config* c, Dims& D) {
   D.capP = c->max_prefix; D.capT = c->max_text;
   D.M = c->bank_capacity; D.slots = D.M + 1; D.S = c->n_streams;
   D.rows_per_stream_max = (D.maxN + 1 > D.maxStepT) ? D.maxN + 1 : D.maxStepT;
+  D.maxChunk = c->max_chunk_frames > 1 ? c->max_chunk_frames : 1;
   D.R_max = D.rows_per_stream_max * D.S;
+  if (D.maxChunk * (D.maxN + 1) > D.R_max) D.R_max = D.maxChunk * (D.maxN + 1);
   D.log_cap = c->evict_log_capacity;
   D.agg_mode = c->agg_mode; D.evict_policy = c->evict_policy; D.use_rmsnorm = c->use_rmsnorm ? 1 : 0;
   D.residual = c->residual ? 1 : 0; D.out_fp32 = c->out_dtype == 1 ? 1 : 0; D.rope_theta = c->rope_theta; D.rms_eps = c->rms_eps;
@@ -75,6 +78,7 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.inv_freq = take((size_t)(D.D / 2) * 8);
   Lo.status = take(8 * 4);
   Lo.step_slot = take((size_t)D.S * 4);
+  Lo.chunk_slot = take((size_t)VS_MAX_BATCH * 4);
   Lo.tickets = take((size_t)D.S * D.Hq * 4);
   Lo.gemm_flags = take((size_t)GEMM_XCHG_CTAS * 4);
   Lo.persistent_end = off;
@@ -90,6 +94,7 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.rope = take((size_t)D.R_max * (D.D / 2) * 8);
   Lo.obuf = take((size_t)D.R_max * D.Hq * D.D * 4);
   Lo.dec_part = take((size_t)DEC_SPLIT_MAX * D.S * D.Hq * (D.D + 2) * 4);
+  Lo.emb_stage = take((size_t)D.maxChunk * D.d * 2);
   Lo.gemm_xchg = take((size_t)GEMM_XCHG_CTAS * 256 * GEMM_BLOCK_M * 4);
   Lo.scratch_end = off;
   Lo.total = off;
@@ -332,6 +337,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
   ba.slot_pos = h->at<int64_t>(lo.slot_pos); ba.evict_log = h->at<int32_t>(lo.evict_log);
   ba.scores = h->at<double>(lo.scores);
   ba.d = D.d; ba.slots = D.slots; ba.M = D.M; ba.policy = D.evict_policy; ba.log_cap = D.log_cap;
+  ba.incoming_emb = nullptr; ba.record_slot = nullptr;
 
   PoolArgs pa;
   pa.hidden = static_cast<const bf16*>(hidden);
@@ -340,6 +346,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
   pa.emb = h->at<bf16>(lo.emb);
   pa.meta = meta;
   pa.step_slot = h->at<int32_t>(lo.step_slot);
+  pa.emb_stage = nullptr;
   pa.inv_freq = h->at<double>(lo.inv_freq);
   pa.rope = h->at<float2>(lo.rope);
   pa.N = N; pa.d = D.d; pa.D = D.D; pa.slots = D.slots; pa.M = D.M; pa.agg_mode = D.agg_mode;
@@ -398,6 +405,143 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     s.next_pos += N + 1;
     s.frames_seen += 1;
   }
+  h->last_stream = st;
+  h->last_rows = rows;
+  return VS_OK;
+}
+
+int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, int32_t F, int32_t N, void* out,
+                           void* cuda_stream) {
+  int rc = check_ids(h, &stream_id, 1);
+  if (rc != VS_OK) return rc;
+  if (hidden == nullptr || N < 1 || F < 1) return VS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(hidden) & 15u) != 0) return VS_ERR_INVALID_ARG;
+  const Dims& D = h->dm;
+  const Layout& lo = h->lo;
+  if (N > D.maxN || F > D.maxChunk) return VS_ERR_CAPACITY;
+  HostStream& hs = h->hs[stream_id];
+  if (hs.text_len != 0) return VS_ERR_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  VS_CK(cudaSetDevice(h->device));
+
+  // the F frames as F batch entries of the same stream, each with the bank count and the
+  // positions it would find as a step of its own
+  BatchParams bp;
+  std::memset(&bp, 0, sizeof(bp));
+  bp.n_active = F;
+  bp.rows_per_stream = N + 1;
+  for (int j = 0; j < F; ++j) {
+    const int64_t seen = hs.frames_seen + j;
+    bp.stream_id[j] = stream_id;
+    bp.count[j] = (int32_t)(seen < D.M ? seen : D.M);
+    bp.prefix_len[j] = (int32_t)hs.prefix_len;
+    bp.text_len[j] = 0;
+    bp.pos_base[j] = hs.next_pos + (int64_t)j * (N + 1);
+    bp.frame_id[j] = seen;
+  }
+  auto one_frame = [&](int j) {
+    BatchParams b1;
+    std::memset(&b1, 0, sizeof(b1));
+    b1.n_active = 1; b1.rows_per_stream = N + 1;
+    b1.stream_id[0] = bp.stream_id[j]; b1.count[0] = bp.count[j]; b1.prefix_len[0] = bp.prefix_len[j];
+    b1.pos_base[0] = bp.pos_base[j]; b1.frame_id[0] = bp.frame_id[j];
+    return b1;
+  };
+  const int rows = F * (N + 1);
+  StreamMeta* meta = h->at<StreamMeta>(lo.meta);
+  int32_t* chunk_slot = h->at<int32_t>(lo.chunk_slot);
+
+  // 1. carriers of all frames (Section 3.3: C = mean of the frame's tokens), parked until they have a slot
+  PoolArgs pa;
+  pa.hidden = static_cast<const bf16*>(hidden);
+  pa.carrier_override = nullptr;
+  pa.x = h->at<bf16>(lo.hbuf[0]);
+  pa.emb = h->at<bf16>(lo.emb);
+  pa.meta = meta;
+  pa.step_slot = h->at<int32_t>(lo.step_slot);
+  pa.emb_stage = h->at<bf16>(lo.emb_stage);
+  pa.inv_freq = h->at<double>(lo.inv_freq);
+  pa.rope = h->at<float2>(lo.rope);
+  pa.N = N; pa.d = D.d; pa.D = D.D; pa.slots = D.slots; pa.M = D.M; pa.agg_mode = D.agg_mode;
+  VS_LAUNCH(h, st, KC_POOL, launch_pool(pa, bp, st));
+
+  // 2. the bank updates, frame by frame (Section 3.3, memory mechanism): they read embeddings only,
+  //    so they can all run before any attention; each records the slot its carrier took
+  for (int j = 0; j < F; ++j) {
+    BankUpdateArgs ba;
+    ba.emb = h->at<bf16>(lo.emb); ba.meta = meta; ba.step_slot = h->at<int32_t>(lo.step_slot);
+    ba.order = h->at<int32_t>(lo.order); ba.slot_frame = h->at<int32_t>(lo.slot_frame);
+    ba.slot_pos = h->at<int64_t>(lo.slot_pos); ba.evict_log = h->at<int32_t>(lo.evict_log);
+    ba.scores = h->at<double>(lo.scores);
+    ba.d = D.d; ba.slots = D.slots; ba.M = D.M; ba.policy = D.evict_policy; ba.log_cap = D.log_cap;
+    ba.incoming_emb = h->at<bf16>(lo.emb_stage) + (size_t)j * D.d;
+    ba.record_slot = chunk_slot + j;
+    const BatchParams b1 = one_frame(j);
+    VS_LAUNCH(h, st, KC_COMMIT, launch_bank_update(ba, b1, D.M > 0 && b1.count[0] == D.M, st));
+  }
+
+  // 3. layer by layer: one projection over all F * (N + 1) rows, then the attention frame by frame
+  //    (frame j reads the bank as frames 0 .. j-1 left it; its own carrier row is copied in beside it)
+  char* out_bytes = static_cast<char*>(out ? out : h->at<void>(lo.obuf));
+  const size_t out_row_bytes = (size_t)D.Hq * D.D * (D.out_fp32 ? 4 : 2);
+  int cur = 0;
+  for (int l = 0; l < D.L; ++l) {
+    const bf16* h_in = h->at<bf16>(lo.hbuf[cur]);
+    const bf16* src = h_in;
+    if (D.use_rmsnorm) {
+      VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_scale),
+                                                    rows, D.d, D.rms_eps, st));
+      if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
+    }
+    ProjectionOut fa;
+    std::memset(&fa, 0, sizeof(fa));
+    fa.bias = h->bias[l];
+    fa.row_scale = D.use_rmsnorm ? h->at<float>(lo.row_scale) : nullptr;
+    fa.rope = h->at<float2>(lo.rope);
+    fa.inv_freq = h->at<double>(lo.inv_freq);
+    fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
+    fa.bank_k = h->at<bf16>(lo.bank_k) + (size_t)l * layer_stride_bank(D);
+    fa.bank_v = h->at<bf16>(lo.bank_v) + (size_t)l * layer_stride_bank(D);
+    fa.free_slot = chunk_slot; fa.free_slot_stride = 0;
+    fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D; fa.slots = D.slots; fa.text_cap = 0; fa.mode = 3; fa.M = D.M;
+    rc = run_projection(h, l, src, rows, fa, bp, st);
+    if (rc != VS_OK) return rc;
+
+    const bool last = (l == D.L - 1);
+    char* layer_out = last ? out_bytes : static_cast<char*>(h->at<void>(lo.obuf));
+    for (int j = 0; j < F; ++j) {
+      const size_t r0 = (size_t)j * (N + 1);
+      AttnArgs aa;
+      std::memset(&aa, 0, sizeof(aa));
+      aa.q = fa.q + r0 * D.Hq * D.D; aa.q_lo = fa.q_lo + r0 * D.Hq * D.D;
+      aa.seg[0] = {h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D),
+                   h->at<bf16>(lo.prefix_v) + (size_t)l * layer_stride_prefix(D),
+                   (long long)D.Hkv * D.maxP * D.D, (long long)D.maxP * D.D, (long long)D.D, 0, 0};
+      aa.seg[1] = {fa.bank_k, fa.bank_v, (long long)D.Hkv * D.slots * D.D, (long long)D.slots * D.D, (long long)D.D, 1, 0};
+      aa.seg[2] = {fa.kf + r0 * D.Hkv * D.D, fa.vf + r0 * D.Hkv * D.D, (long long)(N + 1) * D.Hkv * D.D, (long long)D.D,
+                   (long long)D.Hkv * D.D, 3, 1};
+      aa.n_seg = 3;
+      aa.out = layer_out + r0 * out_row_bytes;
+      aa.out_fp32 = D.out_fp32;
+      aa.h_in = D.residual ? h_in + r0 * D.d : nullptr;
+      aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) + r0 * D.d : nullptr;
+      aa.free_slot = chunk_slot + j; aa.free_slot_stride = 0;
+      if (D.M > 0) {
+        aa.bank_blocks = 1;
+        aa.copy_k = fa.kf + (r0 + N) * D.Hkv * D.D; aa.copy_v = fa.vf + (r0 + N) * D.Hkv * D.D;
+        aa.copy_dst_k = fa.bank_k; aa.copy_dst_v = fa.bank_v;
+        aa.copy_slot = chunk_slot + j;
+      }
+      aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
+      aa.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
+      const BatchParams b1 = one_frame(j);
+      VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, b1, h->at<int>(lo.status), st));
+    }
+    if (D.residual) cur ^= 1;
+  }
+
+  hs.next_pos += (int64_t)F * (N + 1);
+  hs.frames_seen += F;
   h->last_stream = st;
   h->last_rows = rows;
   return VS_OK;

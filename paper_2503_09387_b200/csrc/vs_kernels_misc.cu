@@ -2,6 +2,7 @@
 //   carrier aggregation (Section 3.3: C = (1/N) sum_i E_i), RoPE table, RMSNorm, eviction
 //   scoring and bank commit (Section 3.3, memory mechanism).
 #include "vs_common.cuh"
+#include "vs_bank_update.cuh"
 
 namespace vs {
 
@@ -90,7 +91,9 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, i
       cv = f64_to_bf16_rne(t / (double)N);
     }
     a.x[(size_t)b * (N + 1) * d + (size_t)N * d + c] = cv;   // carrier = last token of the frame
-    if (a.M > 0) {
+    if (a.emb_stage != nullptr) {
+      a.emb_stage[(size_t)b * d + c] = cv;          // chunk of frames: the slot is not known yet
+    } else if (a.M > 0) {
       const int slot = a.meta[sid].free_slot;
       a.emb[((size_t)sid * a.slots + slot) * d + c] = cv;
       // the step's other kernels take the slot from this copy: the bank update, which moves
@@ -165,6 +168,18 @@ __global__ void __launch_bounds__(256) rms_stats_kernel(const bf16* __restrict__
 cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* row_scale, int rows, int d, float eps,
                              cudaStream_t st) {
   return launch_pdl(rms_stats_kernel, dim3(rows), dim3(256), 0, st, h, gain, hg, row_scale, d, eps);
+}
+
+// The bank update of one frame as a launch of its own (chunked prefill).
+__global__ void __launch_bounds__(256) bank_update_kernel(BankUpdateArgs a, BatchParams bp) {
+  pdl_wait();
+  pdl_launch_dependents();
+  bank_update_block(a, bp, (int)blockIdx.y, (int)blockIdx.x);
+}
+
+cudaError_t launch_bank_update(const BankUpdateArgs& a, const BatchParams& bp, bool full, cudaStream_t st) {
+  dim3 grid(full ? (a.M + 7) / 8 : 1, bp.n_active);
+  return launch_pdl(bank_update_kernel, grid, dim3(256), 0, st, a, bp);
 }
 
 __global__ void poison_kernel(uint32_t* p, size_t n) {

@@ -65,7 +65,7 @@ class Pair:
     def __init__(self, w: synth.Workload, n_streams: Optional[int] = None, max_step_tokens: int = 64,
                  evict_policy: int = 0, agg_mode: int = 0, with_bias: bool = False, with_gain: bool = False,
                  max_tokens_per_frame: Optional[int] = None, max_prefix: Optional[int] = None,
-                 max_text: Optional[int] = None, out_dtype: int = 1):
+                 max_text: Optional[int] = None, out_dtype: int = 1, max_chunk_frames: int = 1):
         self.w = w
         S = n_streams or w.n_streams
         self.S = S
@@ -82,7 +82,7 @@ class Pair:
             max_text if max_text is not None else max(w.question_len + w.decode_tokens, 1),
             w.bank_capacity, n_streams=S, max_step_tokens=max_step_tokens, agg_mode=agg_mode,
             evict_policy=evict_policy, use_rmsnorm=w.use_rmsnorm, residual=w.residual,
-            rope_theta=w.rope_theta, rms_eps=w.rms_eps, out_dtype=out_dtype)
+            rope_theta=w.rope_theta, rms_eps=w.rms_eps, out_dtype=out_dtype, max_chunk_frames=max_chunk_frames)
         self.gpu = binding.StreamBatch(self.cfg, [to_dev(b) for b in wbits],
                                        [to_dev(b) for b in bbits] if bbits else None,
                                        [to_dev(b) for b in gbits] if gbits else None)
@@ -123,6 +123,16 @@ class Pair:
             want = self.ora[sid].frame_step(synth.bf16_bits_to_f64(bits[i]), carrier_override=o, mode=mode)
             if mode == "full":
                 self._note(assert_close(got[i], want, f"{what} stream {sid}"))
+        return got
+
+    def frame_chunk(self, sid: int, bits: List[np.ndarray], what: str = "chunk"):
+        """bits[j]: [N, d], consecutive frames of stream sid in one vs_frame_prefill_chunk call; the
+        oracle takes them as streaming steps, one at a time."""
+        out = self.gpu.frame_prefill_chunk(sid, to_dev(np.stack(bits)))
+        got = to_f64(out)
+        for j, b in enumerate(bits):
+            want = self.ora[sid].frame_step(synth.bf16_bits_to_f64(b), mode="full")
+            self._note(assert_close(got[j], want, f"{what} frame {j} of the chunk"))
         return got
 
     def check_bank(self, sid: int = 0, layer: Optional[int] = 0, kv: bool = True):

@@ -142,6 +142,50 @@ def test_text_steps_of_one_to_four_rows():
     p.close()
 
 
+@pytest.mark.parametrize("policy", [0, 1, 2])
+def test_chunked_prefill_equals_streaming_steps(policy):
+    """Several frames per call (the offline form) against the oracle's one-frame steps: chunks of
+    1, 3, 5 and 4 frames with evictions inside the chunks, then streaming frames and a turn of text
+    on the same stream; two layers with RMSNorm gain and residual."""
+    w = synth.workload("deep", n_layers=2, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64,
+                       tokens_per_frame=19, n_frames=16, bank_capacity=4, prefix_len=5, question_len=3,
+                       decode_tokens=2, frame_model="iid", seed=41 + policy)
+    p = Pair(w, with_gain=True, evict_policy=policy, max_chunk_frames=5)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    t = 0
+    for F in (1, 3, 5, 4):
+        p.frame_chunk(0, [w.frame_hidden(t + j) for j in range(F)], f"chunk at frame {t}")
+        t += F
+        for layer in range(2):
+            p.check_bank(0, layer=layer)
+    assert p.ora[0].evictions == 13 - 4
+    for _ in range(3):
+        p.frame([0], [w.frame_hidden(t)], f"streaming frame {t}")
+        t += 1
+    p.check_bank(0, layer=1)
+    p.text([0], [w.question_hidden()], "question")
+    for i in range(2):
+        p.text([0], [w.decode_hidden(i)], f"decode {i}")
+    with pytest.raises(binding.VsError) as e:           # more frames than the handle was sized for
+        p.gpu.frame_prefill_chunk(0, to_dev(np.stack([w.frame_hidden(0)] * 6)))
+    assert e.value.code in (binding.VS_ERR_CAPACITY, binding.VS_ERR_STATE)
+    p.close()
+
+
+def test_chunked_prefill_qwen_shape():
+    """One layer at the Qwen2-7B shape, 8 frames per call, 24 frames: the projection of a chunk is a
+    1360-row GEMM (six token tiles, no K split)."""
+    w = synth.workload("layer", n_frames=24, bank_capacity=16)
+    p = Pair(w, max_chunk_frames=8)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    shared = w.frame_shared()
+    for t in range(0, 24, 8):
+        p.frame_chunk(0, [w.frame_hidden(t + j, shared=shared) for j in range(8)], f"chunk at frame {t}")
+        p.check_bank(0)
+    assert p.ora[0].evictions == 8
+    p.close()
+
+
 def test_scratch_holds_no_state_between_steps():
     """Section 3.3: visual tokens are discarded after prefill.  Overwriting every per-step
     scratch region with NaN between steps must not change any later output."""

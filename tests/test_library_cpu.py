@@ -33,7 +33,7 @@ def test_status_strings(lib):
 
 
 def test_struct_layout_matches_header():
-    assert C.sizeof(binding.VsConfig) == 20 * 4
+    assert C.sizeof(binding.VsConfig) == 21 * 4
     assert C.sizeof(binding.VsBankInfo) == 4 + 4 + 5 * 8 + 4 + 4 + 8 + 8
 
 
