@@ -169,6 +169,7 @@ struct GemmArgs {
   ProjectionOut out;
   int rows, E_out, d;
   int tile_n, n_tiles, ksplit;   // ksplit = CTAs per output tile along K: 1, 2 or 4
+  int m_sub;                     // 1: 128 weight rows per CTA; 2: 256 (two accumulators), only without a K split
   float* xchg;                   // [m_tiles*n_tiles][ksplit][tile_n][128] fp32, needed when ksplit > 1
   int* flags;                    // [m_tiles*n_tiles][ksplit], zero between launches
   int n_sms;

@@ -118,6 +118,7 @@ struct KernelParams {
   ProjectionOut o;
   int* status;
   int rows, E_out, tile_n, kblocks, stages, tmem_cols, ksplit;
+  int acc_stride;               // TMEM columns between the accumulators
   uint32_t data_bytes;          // shared memory ahead of the barriers: max(pipeline stages, own fp32 slice)
   float* xchg;                  // [group][rank][tile_n][128] partial tiles of the K split
   int* flags;                   // [group][rank] peers that have delivered their part of slice `rank`
@@ -129,7 +130,8 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
   return v;
 }
 
-template <bool kOwnRope>   // true: no RoPE table, every finishing thread derives the rotation of its one row
+template <bool kOwnRope, int kMSub>   // kOwnRope: no RoPE table, every finishing thread derives the rotation of its one
+                                      // row; kMSub: 128-row weight sub-tiles (accumulators) per CTA
 __global__ void __launch_bounds__(kMaxThreads, 1)
 qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, KernelParams p,
                 BatchParams bp) {
@@ -139,7 +141,8 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   // tmem slot | abort
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t stage_b_bytes = (uint32_t)p.tile_n * 128u;
-  const uint32_t stage_bytes = kStageABytes + stage_b_bytes;
+  const uint32_t stage_a_bytes = (uint32_t)kMSub * kStageABytes;
+  const uint32_t stage_bytes = stage_a_bytes + stage_b_bytes;
   const uint32_t bar_base = base + p.data_bytes;
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
   uint8_t* ctl = gen_base + p.data_bytes + 16 * p.stages;
@@ -152,7 +155,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int epi_warps = ((int)blockDim.x >> 5) - 2;   // 4, 8 or 16
   const int tok_lanes = 2 * epi_warps;                // token rows finished side by side
-  const int m0 = blockIdx.x * GEMM_BLOCK_M;
+  const int m0 = blockIdx.x * GEMM_BLOCK_M * kMSub;
   const int n0 = blockIdx.y * p.tile_n;
   const int kb0 = blockIdx.z * p.kblocks;      // blockIdx.z = rank in the K split
 
@@ -187,8 +190,10 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
         mbar_arrive_expect_tx(full_bar(s), stage_bytes);
         const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
         const int kx = (kb0 + kb) * GEMM_BLOCK_K;
-        tma_load_2d(a_dst, &tm_w, kx, m0, full_bar(s));
-        tma_load_2d(a_dst + kStageABytes, &tm_x, kx, n0, full_bar(s));
+#pragma unroll
+        for (int ms = 0; ms < kMSub; ++ms)
+          tma_load_2d(a_dst + (uint32_t)ms * kStageABytes, &tm_w, kx, m0 + ms * GEMM_BLOCK_M, full_bar(s));
+        tma_load_2d(a_dst + stage_a_bytes, &tm_x, kx, n0, full_bar(s));
         issued = kb + 1;
       }
       if (*abort_flag) {
@@ -212,12 +217,14 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
         if (!ok) break;
         tcgen05_fence_after();
         const uint32_t a_addr = base + (uint32_t)s * stage_bytes;
-        const uint32_t b_addr = a_addr + kStageABytes;
+        const uint32_t b_addr = a_addr + stage_a_bytes;
 #pragma unroll
         for (int k = 0; k < GEMM_BLOCK_K / 16; ++k) {
           // 16 bf16 = 32 bytes further along K inside the 128-byte swizzle row
-          umma_bf16(tmem_acc, make_smem_desc(a_addr + 32u * k), make_smem_desc(b_addr + 32u * k), idesc,
-                    (uint32_t)((kb | k) != 0));
+#pragma unroll
+          for (int ms = 0; ms < kMSub; ++ms)
+            umma_bf16(tmem_acc + (uint32_t)(ms * p.acc_stride), make_smem_desc(a_addr + (uint32_t)ms * kStageABytes + 32u * k),
+                      make_smem_desc(b_addr + 32u * k), idesc, (uint32_t)((kb | k) != 0));
         }
         umma_commit(empty_bar(s));          // frees the stage once these MMAs have read it
       }
@@ -266,6 +273,11 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   }
   tcgen05_fence_after();
 
+  // one pass per 128-row weight sub-tile (its own accumulator); the staging memory is shared
+#pragma unroll 1
+  for (int ms = 0; ms < kMSub; ++ms) {
+  const int m0e = m0 + ms * GEMM_BLOCK_M;
+  const uint32_t tmem_sub = tmem_acc + (uint32_t)(ms * p.acc_stride);
   float* part_local = reinterpret_cast<float*>(gen_base);      // [token - t_begin][128 features]
   if (warp >= 2 && acc_ok) {
     // warp w may touch TMEM lanes 32*(w%4) .. +31 (lane = feature)
@@ -275,7 +287,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
     for (int c = 16 * ((warp - 2) >> 2); c < p.tile_n; c += 16 * (epi_warps >> 2)) {
       if (n0 + c >= p.rows) break;                             // uniform across the warp
       uint32_t r[16];
-      tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, r);
+      tmem_ld16(tmem_sub + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, r);
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
@@ -316,17 +328,17 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
     const int p0 = (te & 15) * 4;                  // first of 4 rotation pairs inside the 128-feature tile
     const int hl = p0 / half, k0 = p0 - hl * half; // local head, index inside the half head
     const int f1 = hl * D + k0, f2 = f1 + half;
-    const int hs = (m0 + f1) / D;                  // head slot: Q heads, then K heads, then V heads
+    const int hs = (m0e + f1) / D;                  // head slot: Q heads, then K heads, then V heads
     const bool rotate = hs < p.o.Hq + p.o.Hkv;
     const float* far = p.xchg + (size_t)group * p.ksplit * p.tile_n * GEMM_BLOCK_M;
     const size_t far_stride = (size_t)p.tile_n * GEMM_BLOCK_M;
-    if (m0 + f2 + 3 < p.E_out) {
+    if (m0e + f2 + 3 < p.E_out) {
       float bb1[4] = {0.f, 0.f, 0.f, 0.f}, bb2[4] = {0.f, 0.f, 0.f, 0.f};
       if (p.o.bias != nullptr) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          bb1[i] = __bfloat162float(p.o.bias[m0 + f1 + i]);
-          bb2[i] = __bfloat162float(p.o.bias[m0 + f2 + i]);
+          bb1[i] = __bfloat162float(p.o.bias[m0e + f1 + i]);
+          bb2[i] = __bfloat162float(p.o.bias[m0e + f2 + i]);
         }
       }
       const int rps = bp.rows_per_stream;
@@ -431,6 +443,8 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
       }
     }
   }
+  if (ms + 1 < kMSub) { tcgen05_fence_before(); __syncthreads(); tcgen05_fence_after(); }   // rows finished before the staging memory is reused
+  }
 
   __syncthreads();
   if (warp == 1) {
@@ -445,9 +459,10 @@ constexpr int kMaxDynSmem = 227 * 1024;
 }  // namespace
 
 cudaError_t qkv_gemm_init() {
-  cudaError_t e = cudaFuncSetAttribute(qkv_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(qkv_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+  cudaError_t e = cudaFuncSetAttribute(qkv_gemm_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(qkv_gemm_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(qkv_gemm_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+  return e;
 }
 
 cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream_t st) {
@@ -461,11 +476,12 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   const int total_kb = a.d / GEMM_BLOCK_K;
   if (a.ksplit < 1 || a.ksplit > KSPLIT_MAX || (a.ksplit & (a.ksplit - 1)) || total_kb % a.ksplit != 0) return cudaErrorInvalidValue;
   if (a.tile_n < 16 || a.tile_n > 256 || (a.tile_n & 15)) return cudaErrorInvalidValue;
+  if (a.m_sub != 1 && !(a.m_sub == 2 && a.ksplit == 1 && a.E_out % (2 * GEMM_BLOCK_M) == 0)) return cudaErrorInvalidValue;
   if (128 % a.out.D != 0) return cudaErrorInvalidValue;
   p.kblocks = total_kb / a.ksplit;
   p.xchg = a.xchg;
   p.flags = a.flags;
-  const int stage_bytes = kStageABytes + a.tile_n * 128;
+  const int stage_bytes = a.m_sub * kStageABytes + a.tile_n * 128;
   int stages = (kMaxDynSmem - 2048) / stage_bytes;
   if (stages > 8) stages = 8;
   if (stages > p.kblocks) stages = p.kblocks;
@@ -473,7 +489,8 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   p.stages = stages;
   int cols = 32;
   while (cols < a.tile_n) cols <<= 1;
-  p.tmem_cols = cols;
+  p.acc_stride = cols;
+  p.tmem_cols = cols * a.m_sub;            // a power of two, at most 512
   size_t data = (size_t)stages * stage_bytes;
   const size_t own = (size_t)(a.tile_n / a.ksplit) * GEMM_BLOCK_M * 4;
   if (own > data) data = (own + 1023) / 1024 * 1024;
@@ -485,14 +502,14 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   const int threads = 64 + 32 * (slice_rows <= 8 ? 4 : kMaxEpiWarps);
   // without a RoPE table every finishing thread must have at most one row
   if (a.out.rope == nullptr && (a.out.inv_freq == nullptr || slice_rows > 2 * (threads / 32 - 2))) return cudaErrorInvalidValue;
-  const dim3 grid((a.E_out + GEMM_BLOCK_M - 1) / GEMM_BLOCK_M, a.n_tiles, a.ksplit);
+  const dim3 grid((a.E_out + GEMM_BLOCK_M * a.m_sub - 1) / (GEMM_BLOCK_M * a.m_sub), a.n_tiles, a.ksplit);
   if (a.ksplit > 1) {
     // the CTAs of a K split wait for one another: the whole grid has to be resident at once
     if (a.xchg == nullptr || a.flags == nullptr) return cudaErrorInvalidValue;
     int per_sm = 0;
     cudaError_t e = (a.out.rope == nullptr)
-        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, qkv_gemm_kernel<true>, threads, smem)
-        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, qkv_gemm_kernel<false>, threads, smem);
+        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, qkv_gemm_kernel<true, 1>, threads, smem)
+        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, qkv_gemm_kernel<false, 1>, threads, smem);
     if (e != cudaSuccess) return e;
     if ((long long)grid.x * grid.y * grid.z > (long long)per_sm * a.n_sms) return cudaErrorInvalidValue;
   }
@@ -506,8 +523,12 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (a.out.rope == nullptr) return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<true>, a.tm_w, a.tm_x, p, bp);
-  return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<false>, a.tm_w, a.tm_x, p, bp);
+  if (a.out.rope == nullptr) {
+    if (a.m_sub != 1) return cudaErrorInvalidValue;
+    return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<true, 1>, a.tm_w, a.tm_x, p, bp);
+  }
+  if (a.m_sub == 2) return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<false, 2>, a.tm_w, a.tm_x, p, bp);
+  return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<false, 1>, a.tm_w, a.tm_x, p, bp);
 }
 
 }  // namespace vs

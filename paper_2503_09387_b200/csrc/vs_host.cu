@@ -139,17 +139,31 @@ int encode_2d(vs_stream* h, CUtensorMap* tm, const void* base, uint64_t inner, u
   return r == CUDA_SUCCESS ? VS_OK : VS_ERR_CUDA;
 }
 
-void choose_tiles(const Dims& D, int n_sms, int rows, int& tile_n, int& n_tiles, int& ksplit) {
-  n_tiles = (rows + 255) / 256;
-  const int per = (rows + n_tiles - 1) / n_tiles;
-  tile_n = (per + 15) / 16 * 16;
-  const int m_tiles = (D.E_out + GEMM_BLOCK_M - 1) / GEMM_BLOCK_M;
+// Token tiling of the projection.  Every CTA re-reads its weight rows and its token columns from
+// L2, (rows_w + tile_n) * (d / ksplit) * 2 bytes, and that traffic bounds the main loop.  The
+// choice minimises waves * ((rows_w + tile_n) / ksplit + the cost of summing a K split, about 40
+// row-equivalents) over 128- or 256-row weight tiles, the number of token tiles and the K split.
+// A K split needs the whole grid resident at once (its CTAs wait for one another), one CTA per SM.
+void choose_tiles(const Dims& D, int n_sms, int rows, int& tile_n, int& n_tiles, int& ksplit, int& m_sub) {
   const int total_kb = D.d / GEMM_BLOCK_K;
-  const int resident = n_sms < GEMM_XCHG_CTAS ? n_sms : GEMM_XCHG_CTAS;   // one CTA per SM
-  ksplit = 1;                                  // CTAs per output tile along K: 1, 2 or 4
-  for (int ks = 1; ks <= KSPLIT_MAX; ks *= 2) {
-    if (total_kb % ks != 0) continue;
-    if (m_tiles * n_tiles * ks <= resident) ksplit = ks;
+  const int resident = n_sms < GEMM_XCHG_CTAS ? n_sms : GEMM_XCHG_CTAS;
+  const int nt_min = (rows + 255) / 256;
+  long long best = -1;
+  m_sub = 1; ksplit = 1; n_tiles = nt_min; tile_n = ((rows + nt_min - 1) / nt_min + 15) / 16 * 16;
+  for (int sub = 1; sub <= 2; ++sub) {
+    if (sub == 2 && D.E_out % (2 * GEMM_BLOCK_M) != 0) continue;
+    const int mt = (D.E_out + GEMM_BLOCK_M * sub - 1) / (GEMM_BLOCK_M * sub);
+    for (int nt = nt_min; nt <= nt_min + 32; ++nt) {
+      const int tn = ((rows + nt - 1) / nt + 15) / 16 * 16;
+      if ((long long)(nt - 1) * tn >= rows && nt > nt_min) continue;      // an empty last tile
+      if (tn < 64 && nt > nt_min) break;
+      for (int ks = 1; ks <= KSPLIT_MAX; ks *= 2) {
+        if (ks > 1 && (sub != 1 || total_kb % ks != 0 || mt * nt * ks > resident)) continue;
+        const long long waves = ((long long)mt * nt * ks + n_sms - 1) / n_sms;
+        const long long cost = waves * ((GEMM_BLOCK_M * sub + tn) * 4 / ks + (ks > 1 ? 160 : 0));   // in quarter rows
+        if (best < 0 || cost < best) { best = cost; m_sub = sub; n_tiles = nt; tile_n = tn; ksplit = ks; }
+      }
+    }
   }
 }
 
@@ -193,7 +207,7 @@ int run_projection(vs_stream* h, int l, const bf16* src, int rows, const Project
     return VS_OK;
   }
   GemmArgs g;
-  choose_tiles(D, h->n_sms, rows, g.tile_n, g.n_tiles, g.ksplit);
+  choose_tiles(D, h->n_sms, rows, g.tile_n, g.n_tiles, g.ksplit, g.m_sub);
   g.xchg = h->at<float>(h->lo.gemm_xchg);
   g.flags = h->at<int>(h->lo.gemm_flags);
   g.n_sms = h->n_sms;
