@@ -95,10 +95,17 @@ struct Layout {
 
 // ---- programmatic dependent launch ------------------------------------------------------
 // Every kernel of a step is launched with programmatic stream serialisation: it may be
-// scheduled while its predecessor in the stream is still running, does its set-up (barriers,
-// tensor memory, descriptor prefetch), and only then waits for the predecessor to have
-// completed and flushed.  No kernel touches global memory before pdl_wait(), and every kernel
-// calls it, so completion is transitive along the stream.
+// scheduled while its predecessor in the stream is still running.  The rules that keep this
+// safe:
+//  * a CTA lets the dependents start (pdl_launch_dependents) only after its own pdl_wait, or by
+//    exiting; so when a kernel starts, every kernel older than its predecessor has completed and
+//    flushed, and completion is transitive along the stream;
+//  * before its pdl_wait a kernel may do set-up (barriers, tensor memory, descriptor prefetch,
+//    arithmetic on its parameters) and may READ what neither its predecessor nor it writes: the
+//    weights, K/V rows and bank metadata of earlier steps;
+//  * everything the predecessor writes is read, and everything any earlier kernel may still read
+//    is written, only after pdl_wait.  CTAs that need nothing from the predecessor (the bank
+//    update beside the attention) skip the wait.
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

@@ -4,19 +4,26 @@
 //
 // Orientation.  A frame brings only N + 1 (<= 256) token rows but E_out = (Hq + 2 Hkv) D
 // output features (4608 at the Qwen2-7B shape), so the *features* take the MMA's M axis
-// (128 weight rows per CTA, read K-major straight from the caller's [E_out, d] matrix) and
-// the *tokens* take the MMA's N axis (any multiple of 16 up to 256: 170 tokens cost 176
-// columns, 3.5 % padding instead of 33 % with 128-row token tiles).  The reduction dimension
-// d is split over `ksplit` CTAs so that m_tiles * n_tiles * ksplit fills the 148 SMs.  The
-// tile's tokens are cut into ksplit slices and CTA r finishes slice r: every CTA stores the
-// other slices of its fp32 partial accumulator to an exchange buffer in global memory (it
-// stays in L2), counts itself in on the owners' flags, and the owner of a slice, once its
-// flag shows ksplit - 1 arrivals, adds the peers' partials to its own.  All CTAs of the grid
-// are resident at once (the launch checks it), so the wait on the flag ends; it is bounded
-// like every other wait.  The same epilogue adds the bias, applies RoPE (a 128-row tile holds whole heads, so both elements of a rotation pair are at
-// hand), writes Q as a bf16 hi + lo pair and K, V as bf16, and persists what the method keeps:
-// the carrier row's K/V goes straight into the bank's free slot (Section 3.2: only the
-// carrier keeps its K/V), text rows are appended to the prefix or to the turn's tail.
+// (128 weight rows per accumulator, read K-major straight from the caller's [E_out, d] matrix)
+// and the *tokens* take the MMA's N axis (any multiple of 16 up to 256: 170 tokens cost 176
+// columns, 3.5 % padding instead of 33 % with 128-row token tiles).
+//
+// Few rows (a frame, a short text step): the reduction dimension d is split over `ksplit` CTAs
+// so that m_tiles * n_tiles * ksplit fills the 148 SMs.  The tile's tokens are cut into ksplit
+// slices and CTA r finishes slice r: every CTA stores the other slices of its fp32 partial
+// accumulator to an exchange buffer in global memory (it stays in L2), counts itself in on the
+// owners' flags, and the owner of a slice, once its flag shows ksplit - 1 arrivals, adds the
+// peers' partials to its own.  All CTAs of the grid are resident at once (the launch checks
+// it), so the wait on the flag ends; it is bounded like every other wait.
+// Many rows (a chunk of frames, a batch of streams): no K split; a CTA may hold two 128-row
+// weight sub-tiles (two accumulators, 256 x tile_n outputs), which halves the token columns it
+// re-reads from L2 per output.
+//
+// The epilogue adds the bias, applies RoPE (a 128-row tile holds whole heads, so both elements
+// of a rotation pair are at hand), writes Q as a bf16 hi + lo pair and K, V as bf16, and
+// persists what the method keeps: the carrier row's K/V goes straight into the bank's free slot
+// (Section 3.2: only the carrier keeps its K/V), text rows are appended to the prefix or to the
+// turn's tail.
 //
 // Per CTA: 6 or 18 warps.  Warp 0 lane 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer
 // (lane 0), warps 2.. = epilogue, 4 or 16 of them (tcgen05.ld of the 32-lane quarter that
