@@ -140,7 +140,8 @@ struct Smem {
   static constexpr int kV = kK + 2 * kKStage;             // [stage] V tile
   static constexpr int kMax = kV + 2 * kKVBytes;          // float [2][2][128]: row maxima exchange
   static constexpr int kCtl = kMax + 2048;                // barriers, tmem slot, abort flag
-  static constexpr int kTotal = kCtl + 128 + 1024;        // + alignment slack
+  static constexpr int kExcl = kCtl + 128;                // chunk of frames: bitmap of masked bank-axis keys, per-tile flags
+  static constexpr int kTotal = kExcl + ATTN_EXCL_BITS / 8 + 128 + 1024;   // + alignment slack
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -198,31 +199,15 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + L::kCtl + 72);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + L::kCtl + 76);
   float* max_x = reinterpret_cast<float*>(gbase + L::kMax);
+  uint32_t* excl = reinterpret_cast<uint32_t*>(gbase + L::kExcl);                      // [ATTN_EXCL_BITS / 32]
+  uint8_t* tile_excl = gbase + L::kExcl + ATTN_EXCL_BITS / 8;                          // [128]
 
   const int tid = threadIdx.x, warp = tid >> 5;
   // ---- bank update CTAs (frame steps): the first a.bank_blocks of each stream.  What they read --
   // carrier embeddings, the bank's order and metadata -- was complete before the kernel ahead of
   // this one let it start, and nothing else in this launch touches what they write.
   if ((int)blockIdx.x < a.bank_blocks) {
-    if (blockIdx.y == 0) {
-      if (a.copy_k == nullptr) {
-        bank_update_block(a.bank, bp, (int)blockIdx.z, (int)blockIdx.x);
-      } else {
-        // chunk of frames: this frame's carrier K/V row goes into the slot its bank update chose.
-        // The row is the projection's (the kernel ahead), hence the wait; nothing in this launch
-        // reads that slot (it is the hole of this frame's key axis).
-        pdl_wait();
-        const int sid = bp.stream_id[blockIdx.z];
-        const int slot = *a.copy_slot;
-        const int per_head = D / 8;                                   // 16-byte chunks of one head's row
-        for (int i = tid; i < a.Hkv * per_head; i += kAttnThreads) {
-          const int hk = i / per_head, c = i - hk * per_head;
-          const size_t dst = (((size_t)sid * a.Hkv + hk) * a.slots + slot) * D + c * 8;
-          *reinterpret_cast<uint4*>(a.copy_dst_k + dst) = *reinterpret_cast<const uint4*>(a.copy_k + hk * D + c * 8);
-          *reinterpret_cast<uint4*>(a.copy_dst_v + dst) = *reinterpret_cast<const uint4*>(a.copy_v + hk * D + c * 8);
-        }
-      }
-    }
+    if (blockIdx.y == 0) bank_update_block(a.bank, bp, (int)blockIdx.z, (int)blockIdx.x);
     return;
   }
   // ---- set-up that needs nothing from earlier kernels: barriers, tensor memory ------------------
@@ -247,7 +232,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
   const int rps = bp.rows_per_stream;
   const int sid = bp.stream_id[b];
   const int G = a.Hq / a.Hkv;
-  const int count = bp.count[b];
+  const int count = a.chunk_mode ? a.chunk_count0 : bp.count[b];
   const bool bank_full = (a.M > 0 && count == a.M);
 
   // ---- the virtual key axis: segments end to end ----------------------------------------------
@@ -270,6 +255,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
         bank_begin = total;
       }
       else if (sg.kind == 2) len = bp.text_len[b];
+      else if (sg.kind == 4) len = (a.M == 0) ? 0 : b;   // carriers of the chunk's frames before this one
       else { len = min(rps, r0 + kTok); causal_start = total; }  // later keys are visible to no row of this tile
       const long long off = (long long)(sg.by_batch ? b : sid) * sg.stream_stride + (long long)hkv * sg.head_stride -
                             (long long)total * sg.row_stride;
@@ -282,7 +268,28 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
 
   pdl_wait();                       // earlier kernels of the stream have completed
   pdl_launch_dependents();
-  if (bank_full) hole = bank_begin + a.free_slot[sid * a.free_slot_stride];      // the slot being refilled holds no carrier
+  if (bank_full && !a.chunk_mode) hole = bank_begin + a.free_slot[sid * a.free_slot_stride];   // the slot being refilled holds no carrier
+  // chunk of frames in one launch: bank-axis keys this frame must not see, as a bitmap
+  const int excl_range = (a.chunk_mode && a.M > 0) ? (bank_full ? a.M + 1 : count) + b : 0;   // bank slots, then earlier frames' carriers
+  if (a.chunk_mode) {
+    for (int i = tid; i < ATTN_EXCL_BITS / 32; i += kAttnThreads) excl[i] = 0u;
+    if (tid < 128) tile_excl[tid] = 0;
+    __syncthreads();
+    if (tid < b) {
+      const int v = a.chunk_victim[tid];
+      if (v >= 0 && v < excl_range) {
+        atomicOr(&excl[v >> 5], 1u << (v & 31));
+        const int ti_ = (bank_begin + v) / kKeys;
+        if (ti_ < 128) tile_excl[ti_] = 1;
+      }
+    }
+    if (tid == kAttnThreads - 1 && bank_full) {        // the slot that was free when the chunk began
+      const int v = a.free_slot[0];
+      atomicOr(&excl[v >> 5], 1u << (v & 31));
+      const int ti_ = (bank_begin + v) / kKeys;
+      if (ti_ < 128) tile_excl[ti_] = 1;
+    }
+  }
 
   tc_fence_before();
   __syncthreads();
@@ -462,14 +469,23 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
       // a tile needs masking at the ragged end of the key axis, around the bank's free slot and
       // on the causal diagonal (uniform over the CTA)
       const bool need_mask = ((ti + 1) * kKeys > min(total, causal_start + r0 + 1)) ||
-                             (hole >= ti * kKeys && hole < (ti + 1) * kKeys);
+                             (hole >= ti * kKeys && hole < (ti + 1) * kKeys) || (a.chunk_mode && (ti >= 128 || tile_excl[ti]));
       float mx = -INFINITY;
       float sc[KH];
       if (ok) {
         tmem_ld32(tmem_s + lane_base + KH * half, sc);
         tmem_ld32(tmem_s + lane_base + KH * half + 32, sc + 32);
         tmem_ld_wait();
-        if (need_mask) {
+        if (need_mask && a.chunk_mode) {
+          const int nvis = lim - v0, e0 = v0 - bank_begin;          // e0: this thread's first key on the bank axis
+#pragma unroll
+          for (int j = 0; j < KH; ++j) {
+            const int e = e0 + j;
+            const bool out = (unsigned)e < (unsigned)excl_range && ((excl[e >> 5] >> (e & 31)) & 1u);
+            sc[j] = (j < nvis && !out) ? sc[j] : -INFINITY;
+            mx = fmaxf(mx, sc[j]);
+          }
+        } else if (need_mask) {
           const int nvis = lim - v0, hj = hole - v0;
 #pragma unroll
           for (int j = 0; j < KH; ++j) {

@@ -47,7 +47,7 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
     if (a.incoming_emb != nullptr) {
       bf16* dst = const_cast<bf16*>(a.emb) + ((size_t)sid * a.slots + incoming) * a.d;
       for (int k = tid; k < a.d; k += blockDim.x) dst[k] = emb_in[k];
-      if (tid == 0) a.record_slot[b] = incoming;
+      if (tid == 0) { a.record_slot[b] = incoming; a.record_victim[b] = -1; }
     }
   };
   const int64_t carrier_pos = bp.pos_base[b] + bp.rows_per_stream - 1;
@@ -144,6 +144,9 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
     meta->log_count += 1;
     meta->evictions += 1;
     meta->last_victim_frame = victim_frame;
+    if (a.incoming_emb != nullptr)
+      a.record_victim[b] = (victim_frame >= a.chunk_first_frame) ? a.chunk_l1 + (int)(victim_frame - a.chunk_first_frame)
+                                                                 : victim_slot;
     meta->free_slot = victim_slot;
     meta->victim_logical = -1;
     meta->frames_seen += 1;

@@ -74,6 +74,7 @@ struct Layout {
   size_t status;                // int32 [8]
   size_t step_slot;             // int32 [S]  free slot as the running frame step found it
   size_t chunk_slot;            // int32 [VS_MAX_BATCH]  chunked prefill: slot each frame's carrier went to
+  size_t chunk_victim;          // int32 [VS_MAX_BATCH]  ... and whom its bank update evicted (index on the bank axis)
   size_t tickets;               // int32 [S*Hq]  split-KV decode: CTAs finished per (stream, query head)
   size_t gemm_flags;            // int32 [GEMM_XCHG_CTAS]  projection K split: partials delivered per slice owner
   size_t persistent_end;
@@ -167,7 +168,7 @@ struct ProjectionOut {
   int free_slot_stride;
   int Hq, Hkv, D, slots, text_cap, M;
   int mode;                      // 0 frame step (carrier row -> bank), 1 text -> prefix, 2 text -> tail,
-                                 // 3 chunk of frames (nothing kept: the attention launches copy the carrier rows)
+                                 // 3 chunk of frames (nothing kept here: a commit kernel copies the carrier rows)
 };
 
 struct GemmArgs {
@@ -198,6 +199,12 @@ struct BankUpdateArgs {
   // is meta.free_slot, recorded in *record_slot, and the embedding moves into the bank here
   const bf16* incoming_emb;
   int32_t* record_slot;
+  // ... and whom the update evicted, as an index on the chunk's bank axis: the slot for a carrier
+  // that was in the bank before the chunk, chunk_l1 + i for the carrier of the chunk's frame i,
+  // -1 for nobody
+  int32_t* record_victim;
+  long long chunk_first_frame;
+  int chunk_l1;                  // bank slots on the key axis of the chunk's frames
   int32_t* order; int32_t* slot_frame; int64_t* slot_pos; int32_t* evict_log; double* scores;
   int d, slots, M, policy, log_cap;
 };
@@ -206,7 +213,8 @@ struct AttnSegment {
   long long stream_stride;       // elements between streams (by stream id, or by batch slot when by_batch)
   long long head_stride;         // elements between KV heads
   long long row_stride;          // elements between keys
-  int kind;                      // 0 prefix, 1 bank, 2 tail (earlier tokens of the turn), 3 this step's rows (causal)
+  int kind;                      // 0 prefix, 1 bank, 2 tail (earlier tokens of the turn), 3 this step's rows (causal),
+                                 // 4 carriers of the chunk's earlier frames (entry b sees b of them)
   int by_batch;
 };
 struct AttnArgs {
@@ -225,14 +233,24 @@ struct AttnArgs {
   // frame steps, last layer: the first bank_blocks CTAs of every stream do the bank update
   BankUpdateArgs bank;
   int bank_blocks;
-  // chunked prefill instead: one spare CTA copies the frame's carrier K/V row (Hkv*D each) into
-  // slot *copy_slot of this layer's bank
-  const bf16* copy_k; const bf16* copy_v;
-  bf16* copy_dst_k; bf16* copy_dst_v;   // this layer's bank [S][Hkv][slots][D]
-  const int32_t* copy_slot;
+  // chunk of frames in ONE launch (entry b = frame b): the bank segment is the bank as it was
+  // before the chunk (chunk_count0 carriers) for every frame; what frame b must not see -- the slot
+  // that was free, and whoever the updates of frames 0 .. b-1 evicted (chunk_victim) -- is masked
+  int chunk_mode, chunk_count0;
+  const int32_t* chunk_victim;
 };
 // chunked prefill: the bank update of one frame as a launch of its own (it precedes the projection)
 cudaError_t launch_bank_update(const BankUpdateArgs& a, const BatchParams& bp, bool full, cudaStream_t st);
+// chunked prefill, after a layer's attention: the K/V rows of the chunk's carriers that are still in
+// the bank go to their slots
+struct ChunkKvCommitArgs {
+  const bf16* kf; const bf16* vf;          // step K/V [F][N+1][Hkv*D]
+  bf16* bank_k; bf16* bank_v;              // this layer's bank [S][Hkv][slots][D]
+  const int32_t* chunk_slot; const int32_t* chunk_victim;
+  int F, N, Hkv, D, slots, sid, l1;
+};
+cudaError_t launch_chunk_kv_commit(const ChunkKvCommitArgs& a, cudaStream_t st);
+constexpr int ATTN_EXCL_BITS = 8192;   // most (bank slots + chunk frames) the one-launch chunk attention can mask
 cudaError_t launch_prefill_attention_tc(const AttnArgs& a, const BatchParams& bp, int* status, cudaStream_t st);
 cudaError_t prefill_attention_tc_init();
 

@@ -79,6 +79,7 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.status = take(8 * 4);
   Lo.step_slot = take((size_t)D.S * 4);
   Lo.chunk_slot = take((size_t)VS_MAX_BATCH * 4);
+  Lo.chunk_victim = take((size_t)VS_MAX_BATCH * 4);
   Lo.tickets = take((size_t)D.S * D.Hq * 4);
   Lo.gemm_flags = take((size_t)GEMM_XCHG_CTAS * 4);
   Lo.persistent_end = off;
@@ -351,7 +352,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
   ba.slot_pos = h->at<int64_t>(lo.slot_pos); ba.evict_log = h->at<int32_t>(lo.evict_log);
   ba.scores = h->at<double>(lo.scores);
   ba.d = D.d; ba.slots = D.slots; ba.M = D.M; ba.policy = D.evict_policy; ba.log_cap = D.log_cap;
-  ba.incoming_emb = nullptr; ba.record_slot = nullptr;
+  ba.incoming_emb = nullptr; ba.record_slot = nullptr; ba.record_victim = nullptr; ba.chunk_first_frame = 0; ba.chunk_l1 = 0;
 
   PoolArgs pa;
   pa.hidden = static_cast<const bf16*>(hidden);
@@ -464,6 +465,12 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
   const int rows = F * (N + 1);
   StreamMeta* meta = h->at<StreamMeta>(lo.meta);
   int32_t* chunk_slot = h->at<int32_t>(lo.chunk_slot);
+  int32_t* chunk_victim = h->at<int32_t>(lo.chunk_victim);
+  // the bank as every frame of the chunk finds it on its key axis: the carriers that were there
+  // before the chunk (all M + 1 slots once the bank is full)
+  const int count0 = bp.count[0];
+  const int l1 = (D.M > 0 && count0 == D.M) ? D.M + 1 : count0;
+  if (l1 + F > ATTN_EXCL_BITS) return VS_ERR_CAPACITY;   // the attention launch's mask of hidden bank keys
 
   // 1. carriers of all frames (Section 3.3: C = mean of the frame's tokens), parked until they have a slot
   PoolArgs pa;
@@ -490,12 +497,15 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
     ba.d = D.d; ba.slots = D.slots; ba.M = D.M; ba.policy = D.evict_policy; ba.log_cap = D.log_cap;
     ba.incoming_emb = h->at<bf16>(lo.emb_stage) + (size_t)j * D.d;
     ba.record_slot = chunk_slot + j;
+    ba.record_victim = chunk_victim + j;
+    ba.chunk_first_frame = bp.frame_id[0];
+    ba.chunk_l1 = l1;
     const BatchParams b1 = one_frame(j);
     VS_LAUNCH(h, st, KC_COMMIT, launch_bank_update(ba, b1, D.M > 0 && b1.count[0] == D.M, st));
   }
 
-  // 3. layer by layer: one projection over all F * (N + 1) rows, then the attention frame by frame
-  //    (frame j reads the bank as frames 0 .. j-1 left it; its own carrier row is copied in beside it)
+  // 3. layer by layer: one projection over all F * (N + 1) rows, one attention launch over all
+  //    frames, then the K/V rows of the chunk's surviving carriers go into their bank slots
   char* out_bytes = static_cast<char*>(out ? out : h->at<void>(lo.obuf));
   const size_t out_row_bytes = (size_t)D.Hq * D.D * (D.out_fp32 ? 4 : 2);
   int cur = 0;
@@ -523,33 +533,36 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
 
     const bool last = (l == D.L - 1);
     char* layer_out = last ? out_bytes : static_cast<char*>(h->at<void>(lo.obuf));
-    for (int j = 0; j < F; ++j) {
-      const size_t r0 = (size_t)j * (N + 1);
+    {
+      // every frame is a batch entry; frame b sees the bank of before the chunk minus what the
+      // updates of frames 0 .. b-1 evicted, plus the carriers of those frames (from the step's K/V)
       AttnArgs aa;
       std::memset(&aa, 0, sizeof(aa));
-      aa.q = fa.q + r0 * D.Hq * D.D; aa.q_lo = fa.q_lo + r0 * D.Hq * D.D;
+      aa.q = fa.q; aa.q_lo = fa.q_lo;
       aa.seg[0] = {h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D),
                    h->at<bf16>(lo.prefix_v) + (size_t)l * layer_stride_prefix(D),
                    (long long)D.Hkv * D.maxP * D.D, (long long)D.maxP * D.D, (long long)D.D, 0, 0};
       aa.seg[1] = {fa.bank_k, fa.bank_v, (long long)D.Hkv * D.slots * D.D, (long long)D.slots * D.D, (long long)D.D, 1, 0};
-      aa.seg[2] = {fa.kf + r0 * D.Hkv * D.D, fa.vf + r0 * D.Hkv * D.D, (long long)(N + 1) * D.Hkv * D.D, (long long)D.D,
-                   (long long)D.Hkv * D.D, 3, 1};
-      aa.n_seg = 3;
-      aa.out = layer_out + r0 * out_row_bytes;
+      aa.seg[2] = {fa.kf + (size_t)N * D.Hkv * D.D, fa.vf + (size_t)N * D.Hkv * D.D, 0, (long long)D.D,
+                   (long long)(N + 1) * D.Hkv * D.D, 4, 0};
+      aa.seg[3] = {fa.kf, fa.vf, (long long)(N + 1) * D.Hkv * D.D, (long long)D.D, (long long)D.Hkv * D.D, 3, 1};
+      aa.n_seg = 4;
+      aa.out = layer_out;
       aa.out_fp32 = D.out_fp32;
-      aa.h_in = D.residual ? h_in + r0 * D.d : nullptr;
-      aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) + r0 * D.d : nullptr;
-      aa.free_slot = chunk_slot + j; aa.free_slot_stride = 0;
-      if (D.M > 0) {
-        aa.bank_blocks = 1;
-        aa.copy_k = fa.kf + (r0 + N) * D.Hkv * D.D; aa.copy_v = fa.vf + (r0 + N) * D.Hkv * D.D;
-        aa.copy_dst_k = fa.bank_k; aa.copy_dst_v = fa.bank_v;
-        aa.copy_slot = chunk_slot + j;
-      }
+      aa.h_in = D.residual ? h_in : nullptr;
+      aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
+      aa.free_slot = chunk_slot; aa.free_slot_stride = 0;
+      aa.chunk_mode = 1; aa.chunk_count0 = count0; aa.chunk_victim = chunk_victim;
       aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
       aa.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
-      const BatchParams b1 = one_frame(j);
-      VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, b1, h->at<int>(lo.status), st));
+      VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, bp, h->at<int>(lo.status), st));
+      if (D.M > 0) {
+        ChunkKvCommitArgs ca;
+        ca.kf = fa.kf; ca.vf = fa.vf; ca.bank_k = fa.bank_k; ca.bank_v = fa.bank_v;
+        ca.chunk_slot = chunk_slot; ca.chunk_victim = chunk_victim;
+        ca.F = F; ca.N = N; ca.Hkv = D.Hkv; ca.D = D.D; ca.slots = D.slots; ca.sid = stream_id; ca.l1 = l1;
+        VS_LAUNCH(h, st, KC_OTHER, launch_chunk_kv_commit(ca, st));
+      }
     }
     if (D.residual) cur ^= 1;
   }

@@ -182,6 +182,29 @@ cudaError_t launch_bank_update(const BankUpdateArgs& a, const BatchParams& bp, b
   return launch_pdl(bank_update_kernel, grid, dim3(256), 0, st, a, bp);
 }
 
+// grid = F CTAs of 128 threads: CTA i copies the carrier row of the chunk's frame i unless a later
+// update of the chunk evicted that carrier (its slot then belongs to someone else).
+__global__ void __launch_bounds__(128) chunk_kv_commit_kernel(ChunkKvCommitArgs a) {
+  pdl_wait();                       // the attention launch has finished reading the bank
+  pdl_launch_dependents();
+  const int i = blockIdx.x;
+  for (int u = i + 1; u < a.F; ++u)
+    if (a.chunk_victim[u] == a.l1 + i) return;
+  const int slot = a.chunk_slot[i];
+  const int per_head = a.D / 8;                                       // 16-byte chunks of one head's row
+  const size_t src = ((size_t)i * (a.N + 1) + a.N) * a.Hkv * a.D;
+  for (int c = threadIdx.x; c < a.Hkv * per_head; c += blockDim.x) {
+    const int hk = c / per_head, cc = c - hk * per_head;
+    const size_t dst = (((size_t)a.sid * a.Hkv + hk) * a.slots + slot) * a.D + cc * 8;
+    *reinterpret_cast<uint4*>(a.bank_k + dst) = *reinterpret_cast<const uint4*>(a.kf + src + hk * a.D + cc * 8);
+    *reinterpret_cast<uint4*>(a.bank_v + dst) = *reinterpret_cast<const uint4*>(a.vf + src + hk * a.D + cc * 8);
+  }
+}
+
+cudaError_t launch_chunk_kv_commit(const ChunkKvCommitArgs& a, cudaStream_t st) {
+  return launch_pdl(chunk_kv_commit_kernel, dim3(a.F), dim3(128), 0, st, a);
+}
+
 __global__ void poison_kernel(uint32_t* p, size_t n) {
   pdl_wait();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)

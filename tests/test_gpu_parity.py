@@ -172,6 +172,20 @@ def test_chunked_prefill_equals_streaming_steps(policy):
     p.close()
 
 
+@pytest.mark.parametrize("M", [0, 1, 2])
+def test_chunked_prefill_with_tiny_banks(M):
+    """Bank capacities 0, 1 and 2: every frame of a chunk but the first few evicts, often a carrier
+    that entered the bank earlier in the same chunk."""
+    w = synth.workload("tiny", n_frames=11, bank_capacity=M, tokens_per_frame=9, prefix_len=2, seed=61 + M)
+    p = Pair(w, max_chunk_frames=6)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    p.frame_chunk(0, [w.frame_hidden(j) for j in range(6)], "first chunk")
+    p.check_bank(0)
+    p.frame_chunk(0, [w.frame_hidden(6 + j) for j in range(5)], "second chunk")
+    p.check_bank(0)
+    p.close()
+
+
 def test_chunked_prefill_qwen_shape():
     """One layer at the Qwen2-7B shape, 8 frames per call, 24 frames: the projection of a chunk is a
     1360-row GEMM (six token tiles, no K split)."""
