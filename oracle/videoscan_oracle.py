@@ -401,6 +401,35 @@ class OracleStream:
             self.text_len += T
         return out
 
+    def carriers_only_forward(self) -> np.ndarray:
+        """The bank's carriers as ordinary tokens, one per frame (Section 3.4, stage 1: the visual
+        input is the semantic carrier tokens only; Section 4.3, inference without KV reuse): the
+        stored carrier *embeddings*, in temporal order, go through the layers after the prompt
+        prefix, each seeing the prefix and the carriers up to itself.  The stored K/V are not
+        used and nothing changes.  Carrier i of this compact sequence sits at position
+        prefix_len + i.  Returns the last layer's outputs [count, Hq*D]."""
+        cfg = self.cfg
+        T = len(self.bank)
+        if T == 0:
+            return np.zeros((0, cfg.n_q_heads * cfg.head_dim))
+        h = np.stack([np.asarray(e.emb, dtype=np.float64) for e in self.bank])
+        ang = rope_angles([self.prefix_len + i for i in range(T)], cfg.head_dim, cfg.rope_theta)
+        out = None
+        for l in range(cfg.n_layers):
+            Q, K, V = self._project(self._layer_input(h, l), l)
+            Q = apply_rope(Q, ang)
+            K = round_to_bf16(apply_rope(K, ang))
+            V = round_to_bf16(V)
+            P = self.prefix_K[l].shape[0]
+            Kall = np.concatenate([self.prefix_K[l], K], axis=0)
+            Vall = np.concatenate([self.prefix_V[l], V], axis=0)
+            vis = np.ones((T, P + T), dtype=bool)
+            vis[:, P:] = np.tril(np.ones((T, T), dtype=bool))
+            out = attention_rows(Q, Kall, Vall, vis).reshape(T, -1)
+            if cfg.residual:
+                h = round_to_bf16(h + out)
+        return out
+
     def end_turn(self) -> None:
         """Drop the question/answer tail; prefix and bank stay, frame positions do not move."""
         Hkv, D = self.cfg.n_kv_heads, self.cfg.head_dim

@@ -471,3 +471,62 @@ def test_decode_sees_only_prefix_bank_and_text():
     assert Kall.shape[0] == 8 + 4 + 1
     want = vo.attention_rows(Q, Kall, Vall, np.ones((1, 13), dtype=bool)).reshape(1, -1)
     assert np.max(np.abs(got - want)) < 1e-12
+
+
+# ------------------------------------------------------------- carriers as ordinary tokens
+def test_carriers_only_forward_is_a_text_prefill_of_the_stored_embeddings():
+    # special case that reduces to a routine pinned above: on a stream that has seen no frame,
+    # feeding the bank's embeddings as text right after the same prompt is the same computation
+    # (same positions prefix_len + i, same causal context), whatever the bank's K/V hold
+    w = synth.workload("tiny", n_layers=2, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64,
+                       use_rmsnorm=1, residual=1)
+    cfg = vo.OracleConfig(2, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, w.bank_capacity,
+                          use_rmsnorm=1, residual=1)
+    Ws = [synth.bf16_bits_to_f64(w.weight(l)) for l in range(2)]
+    st = vo.OracleStream(cfg, Ws)
+    st.text_step(synth.bf16_bits_to_f64(w.prefix_hidden()))
+    for t in range(7):                                   # capacity 4: evictions reorder the bank
+        st.frame_step(synth.bf16_bits_to_f64(w.frame_hidden(t)))
+    before = (st.next_pos, st.frames_seen, st.evictions, [e.frame_id for e in st.bank])
+    got = st.carriers_only_forward()
+    assert (st.next_pos, st.frames_seen, st.evictions, [e.frame_id for e in st.bank]) == before
+    assert got.shape == (4, w.n_q_heads * w.head_dim)
+    ref = vo.OracleStream(cfg, Ws)
+    ref.text_step(synth.bf16_bits_to_f64(w.prefix_hidden()))
+    want = ref.text_step(np.stack([e.emb for e in st.bank]))
+    assert np.max(np.abs(got - want)) < 1e-12
+    assert vo.OracleStream(cfg, Ws).carriers_only_forward().shape == (0, w.n_q_heads * w.head_dim)
+
+
+def test_carriers_only_forward_brute_force_one_layer():
+    # written out independently: complex rotation for RoPE, explicit loops for the softmax
+    rng = _rng(77)
+    d, Hq, Hkv, D, P, theta = 64, 2, 1, 32, 3, 1e4
+    cfg = vo.OracleConfig(1, d, Hq, Hkv, D, 5, rope_theta=theta)
+    W = _bf16_vals(rng, ((Hq + 2 * Hkv) * D, d), 0.1)
+    st = vo.OracleStream(cfg, [W])
+    Xp = _bf16_vals(rng, (P, d))
+    st.text_step(Xp)
+    for t in range(4):
+        st.frame_step(_bf16_vals(rng, (6, d)))
+    got = st.carriers_only_forward()
+    C = np.stack([e.emb for e in st.bank])               # [4, d]
+    X = np.concatenate([Xp, C])                          # the compact sequence: prompt, then one token per frame
+    T = X.shape[0]
+    Y = X @ W.T
+    def rot(v, pos):                                     # v: [D]; pairs (i, i + D/2) as complex numbers
+        z = v[:D // 2] + 1j * v[D // 2:]
+        z = z * np.exp(1j * pos * theta ** (-2.0 * np.arange(D // 2) / D))
+        return np.concatenate([z.real, z.imag])
+    out = np.zeros((4, Hq * D))
+    for hq in range(Hq):
+        hk = hq // (Hq // Hkv)
+        Kr = np.stack([vo.round_to_bf16(rot(Y[t, (Hq + hk) * D:(Hq + hk + 1) * D], t)) for t in range(T)])
+        Vr = np.stack([vo.round_to_bf16(Y[t, (Hq + Hkv + hk) * D:(Hq + Hkv + hk + 1) * D]) for t in range(T)])
+        for i in range(4):
+            t = P + i
+            q = rot(Y[t, hq * D:(hq + 1) * D], t)
+            s = np.array([q @ Kr[u] / math.sqrt(D) for u in range(t + 1)])
+            p = np.exp(s - s.max()); p /= p.sum()
+            out[i, hq * D:(hq + 1) * D] = sum(p[u] * Vr[u] for u in range(t + 1))
+    assert np.max(np.abs(got - out)) < 1e-12
