@@ -150,6 +150,15 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
 int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, int32_t F, int32_t N,
                            void* out, void* cuda_stream);
 
+/* The bank's carriers as ordinary tokens, without their stored K/V (Section 3.4, stage 1: the
+ * visual input is the semantic carrier tokens only; Section 4.3, inference without KV reuse):
+ * the stored carrier embeddings of ONE stream, in temporal order, one token per frame at
+ * positions prefix_len + i, go through the layers, each attending over the prompt prefix and the
+ * carriers up to itself.  Reads the bank, changes nothing.
+ * out: DEVICE [count][Hq*D] of `out_dtype` (count = carriers in the bank; vs_bank_state tells).
+ * count = 0 is not an error: nothing is launched. */
+int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_stream);
+
 /* T text tokens per listed stream -- the decoding phase of Section 3.3 (T = 1) and the
  * text part of prefilling (T > 1).  Token i attends to [prefix | bank | tail tokens up to
  * itself]; no visual-token K/V exists any more.  Before a stream's first frame the tokens

@@ -26,7 +26,7 @@ VS_ERR_DEVICE_TIMEOUT = -5
 VS_ERR_UNSUPPORTED = -6
 VS_MAX_BATCH = 64
 
-EXPORTS = ["vs_workspace_bytes", "vs_create_stream", "vs_frame_prefill", "vs_frame_prefill_chunk", "vs_decode_step",
+EXPORTS = ["vs_workspace_bytes", "vs_create_stream", "vs_frame_prefill", "vs_frame_prefill_chunk", "vs_bank_forward", "vs_decode_step",
            "vs_end_turn", "vs_bank_state", "vs_last_step_kv", "vs_poison_scratch",
            "vs_destroy_stream", "vs_status_string", "vs_reset_stream", "vs_profile_enable",
            "vs_profile_read", "vs_kernel_class_name", "vs_evict_choose_static"]
@@ -82,6 +82,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.vs_create_stream.argtypes = [C.POINTER(VsConfig), C.POINTER(VsWeights), vp, C.c_size_t, C.POINTER(vp)]
     lib.vs_frame_prefill.argtypes = [vp, i32p, i32, vp, i32, vp, vp, vp]
     lib.vs_frame_prefill_chunk.argtypes = [vp, i32, vp, i32, i32, vp, vp]
+    lib.vs_bank_forward.argtypes = [vp, i32, vp, vp]
     lib.vs_decode_step.argtypes = [vp, i32p, i32, vp, i32, vp, vp]
     lib.vs_end_turn.argtypes = [vp, i32p, i32]
     lib.vs_bank_state.argtypes = [vp, i32, C.POINTER(VsBankInfo), i32p, C.POINTER(C.c_int64), i32p,
@@ -146,6 +147,10 @@ def vs_frame_prefill(handle: int, stream_ids: Sequence[int], hidden_ptr: int, N:
     ids, n = _ids(stream_ids)
     _check(load_library().vs_frame_prefill(handle, ids, n, hidden_ptr, N, carrier_override_ptr or None,
                                            out_ptr or None, cuda_stream or None), "vs_frame_prefill")
+
+
+def vs_bank_forward(handle: int, stream_id: int, out_ptr: int, cuda_stream: Optional[int] = None) -> None:
+    _check(load_library().vs_bank_forward(handle, stream_id, out_ptr, cuda_stream or None), "vs_bank_forward")
 
 
 def vs_frame_prefill_chunk(handle: int, stream_id: int, hidden_ptr: int, F: int, N: int,
@@ -299,6 +304,12 @@ class StreamBatch:
             out = self.torch.empty((F, N + 1, self.out_width), dtype=self.out_torch_dtype, device=self.device)
         vs_frame_prefill_chunk(self.handle, stream_id, hidden.data_ptr(), F, N,
                                out.data_ptr() if out is not None else None, self._stream())
+        return out
+
+    def bank_forward(self, stream_id, count):
+        """Carriers-only forward of one stream's bank; `count` = carriers in it."""
+        out = self.torch.empty((count, self.out_width), dtype=self.out_torch_dtype, device=self.device)
+        vs_bank_forward(self.handle, stream_id, out.data_ptr(), self._stream())
         return out
 
     def decode_step(self, stream_ids, hidden, out=None):

@@ -273,6 +273,9 @@ struct DecodeArgs {
 cudaError_t launch_decode_attention(const DecodeArgs& a, const BatchParams& bp, cudaStream_t st);
 
 
+// rows i < count of x = emb[sid][order[i]]: the bank's carrier embeddings in temporal order
+cudaError_t launch_gather_carriers(const bf16* emb, const int32_t* order, bf16* x, int sid, int slots, int d, int count,
+                                   cudaStream_t st);
 cudaError_t launch_poison(void* p, size_t bytes, cudaStream_t st);
 cudaError_t launch_reset(StreamMeta* meta, int32_t* slot_frame, int slots, const BatchParams& bp, cudaStream_t st);
 

@@ -53,6 +53,7 @@ int fill_dims(const vs_config* c, Dims& D) {
   D.maxChunk = c->max_chunk_frames > 1 ? c->max_chunk_frames : 1;
   D.R_max = D.rows_per_stream_max * D.S;
   if (D.maxChunk * (D.maxN + 1) > D.R_max) D.R_max = D.maxChunk * (D.maxN + 1);
+  if (D.M > D.R_max) D.R_max = D.M;               // vs_bank_forward runs the whole bank as one step
   D.log_cap = c->evict_log_capacity;
   D.agg_mode = c->agg_mode; D.evict_policy = c->evict_policy; D.use_rmsnorm = c->use_rmsnorm ? 1 : 0;
   D.residual = c->residual ? 1 : 0; D.out_fp32 = c->out_dtype == 1 ? 1 : 0; D.rope_theta = c->rope_theta; D.rms_eps = c->rms_eps;
@@ -569,6 +570,78 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
 
   hs.next_pos += (int64_t)F * (N + 1);
   hs.frames_seen += F;
+  h->last_stream = st;
+  h->last_rows = rows;
+  return VS_OK;
+}
+
+int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_stream) {
+  int rc = check_ids(h, &stream_id, 1);
+  if (rc != VS_OK) return rc;
+  const Dims& D = h->dm;
+  const Layout& lo = h->lo;
+  if ((D.d & 7) != 0) return VS_ERR_UNSUPPORTED;
+  const HostStream& hs = h->hs[stream_id];
+  const int count = (int)(hs.frames_seen < D.M ? hs.frames_seen : D.M);
+  if (count == 0) return VS_OK;
+  if (out == nullptr) return VS_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  VS_CK(cudaSetDevice(h->device));
+
+  // one text-like step of `count` rows right after the prompt; nothing is kept
+  BatchParams bp;
+  std::memset(&bp, 0, sizeof(bp));
+  bp.n_active = 1;
+  bp.rows_per_stream = count;
+  bp.stream_id[0] = stream_id;
+  bp.prefix_len[0] = (int32_t)hs.prefix_len;
+  bp.pos_base[0] = hs.prefix_len;
+  const int rows = count;
+  VS_LAUNCH(h, st, KC_OTHER, launch_gather_carriers(h->at<bf16>(lo.emb), h->at<int32_t>(lo.order), h->at<bf16>(lo.hbuf[0]),
+                                                    stream_id, D.slots, D.d, count, st));
+  RopeArgs ra;
+  ra.inv_freq = h->at<double>(lo.inv_freq); ra.rope = h->at<float2>(lo.rope); ra.D = D.D;
+  VS_LAUNCH(h, st, KC_ROPE, launch_rope_table(ra, bp, st));
+
+  int cur = 0;
+  for (int l = 0; l < D.L; ++l) {
+    const bf16* h_in = h->at<bf16>(lo.hbuf[cur]);
+    const bf16* src = h_in;
+    if (D.use_rmsnorm) {
+      VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_scale),
+                                                    rows, D.d, D.rms_eps, st));
+      if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
+    }
+    ProjectionOut fa;
+    std::memset(&fa, 0, sizeof(fa));
+    fa.bias = h->bias[l];
+    fa.row_scale = D.use_rmsnorm ? h->at<float>(lo.row_scale) : nullptr;
+    fa.rope = h->at<float2>(lo.rope);
+    fa.inv_freq = h->at<double>(lo.inv_freq);
+    fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
+    fa.free_slot = h->at<int32_t>(lo.step_slot); fa.free_slot_stride = 0;
+    fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D; fa.slots = D.slots; fa.text_cap = 0; fa.mode = 3; fa.M = D.M;
+    rc = run_projection(h, l, src, rows, fa, bp, st);
+    if (rc != VS_OK) return rc;
+
+    AttnArgs aa;
+    std::memset(&aa, 0, sizeof(aa));
+    aa.q = fa.q; aa.q_lo = fa.q_lo;
+    aa.seg[0] = {h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D),
+                 h->at<bf16>(lo.prefix_v) + (size_t)l * layer_stride_prefix(D),
+                 (long long)D.Hkv * D.maxP * D.D, (long long)D.maxP * D.D, (long long)D.D, 0, 0};
+    aa.seg[1] = {fa.kf, fa.vf, (long long)rows * D.Hkv * D.D, (long long)D.D, (long long)D.Hkv * D.D, 3, 1};
+    aa.n_seg = 2;
+    aa.out = (l == D.L - 1) ? out : h->at<void>(lo.obuf);
+    aa.out_fp32 = D.out_fp32;
+    aa.h_in = D.residual ? h_in : nullptr;
+    aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
+    aa.free_slot = h->at<int32_t>(lo.step_slot); aa.free_slot_stride = 0;
+    aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = 0;      // no bank segment on this key axis
+    aa.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
+    VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, bp, h->at<int>(lo.status), st));
+    if (D.residual) cur ^= 1;
+  }
   h->last_stream = st;
   h->last_rows = rows;
   return VS_OK;

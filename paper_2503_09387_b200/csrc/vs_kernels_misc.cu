@@ -205,6 +205,21 @@ cudaError_t launch_chunk_kv_commit(const ChunkKvCommitArgs& a, cudaStream_t st) 
   return launch_pdl(chunk_kv_commit_kernel, dim3(a.F), dim3(128), 0, st, a);
 }
 
+__global__ void __launch_bounds__(256) gather_carriers_kernel(const bf16* __restrict__ emb, const int32_t* __restrict__ order,
+                                                             bf16* __restrict__ x, int sid, int slots, int d) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int i = blockIdx.x;
+  const uint4* src = reinterpret_cast<const uint4*>(emb + ((size_t)sid * slots + order[(size_t)sid * slots + i]) * d);
+  uint4* dst = reinterpret_cast<uint4*>(x + (size_t)i * d);
+  for (int c = threadIdx.x; c < d / 8; c += blockDim.x) dst[c] = src[c];
+}
+
+cudaError_t launch_gather_carriers(const bf16* emb, const int32_t* order, bf16* x, int sid, int slots, int d, int count,
+                                   cudaStream_t st) {
+  return launch_pdl(gather_carriers_kernel, dim3(count), dim3(256), 0, st, emb, order, x, sid, slots, d);
+}
+
 __global__ void poison_kernel(uint32_t* p, size_t n) {
   pdl_wait();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)

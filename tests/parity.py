@@ -135,6 +135,14 @@ class Pair:
             self._note(assert_close(got[j], want, f"{what} frame {j} of the chunk"))
         return got
 
+    def bank_forward(self, sid: int = 0, what: str = "carriers-only forward"):
+        """vs_bank_forward against the oracle's carriers_only_forward; neither may change the stream."""
+        want = self.ora[sid].carriers_only_forward()
+        got = to_f64(self.gpu.bank_forward(sid, want.shape[0]))
+        if want.shape[0]:
+            self._note(assert_close(got, want, what))
+        return got
+
     def check_bank(self, sid: int = 0, layer: Optional[int] = 0, kv: bool = True):
         ora = self.ora[sid]
         st = self.gpu.bank_state(sid, layer=layer if kv else None, want_emb=True)

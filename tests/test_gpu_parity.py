@@ -200,6 +200,44 @@ def test_chunked_prefill_qwen_shape():
     p.close()
 
 
+def test_carriers_only_forward_small():
+    """The bank's embeddings as one token per frame (no stored K/V used): empty bank, a partly
+    filled one, a full one whose temporal order differs from its slot order after evictions; two
+    layers with RMSNorm gain, bias and residual.  The stream goes on unchanged afterwards."""
+    w = synth.workload("deep", n_layers=2, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64,
+                       tokens_per_frame=11, n_frames=12, bank_capacity=5, prefix_len=4, question_len=0,
+                       decode_tokens=2, frame_model="iid", seed=71)
+    p = Pair(w, with_gain=True, with_bias=True, evict_policy=1)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    p.bank_forward(0, "empty bank")
+    for t in range(3):
+        p.frame([0], [w.frame_hidden(t)], f"frame {t}")
+    p.bank_forward(0, "three carriers")
+    for t in range(3, 12):
+        p.frame([0], [w.frame_hidden(t)], f"frame {t}")
+    st = p.check_bank(0, layer=1)
+    assert list(st["slots"]) != sorted(st["slots"])          # evictions have permuted the slots
+    p.bank_forward(0, "full bank")
+    p.bank_forward(0, "full bank again")
+    for i in range(2):
+        p.text([0], [w.decode_hidden(i)], f"decode {i}")
+    p.check_bank(0, layer=0)
+    p.close()
+
+
+def test_carriers_only_forward_qwen_shape():
+    """64 carriers at the Qwen2-7B shape: a 64-row projection (K split) and a 128-key attention."""
+    w = synth.workload("layer", n_frames=70, bank_capacity=64)
+    p = Pair(w)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    shared = w.frame_shared()
+    for t in range(70):
+        p.frame([0], [w.frame_hidden(t, shared=shared)], f"frame {t}", mode="carrier")
+    p.bank_forward(0)
+    p.check_bank(0)
+    p.close()
+
+
 def test_scratch_holds_no_state_between_steps():
     """Section 3.3: visual tokens are discarded after prefill.  Overwriting every per-step
     scratch region with NaN between steps must not change any later output."""
