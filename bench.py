@@ -193,6 +193,21 @@ def workload_config(w):
             "out_dtype": "fp32"}
 
 
+# ------------------------------------------------------------------ replicas
+def max_over_ranks(t, world):
+    """Slowest rank's value of every element of tensor `t` (in place): the job ends when it does."""
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t
+
+
+def replica_throughput(world, units_per_rank, ms):
+    """Whole-job rate of `world` independent replicas that each did `units_per_rank` in `ms`
+    (the slowest rank's time): no rank shares work with another, so the units add up."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
 # ------------------------------------------------------------------ our arm
 def run_ours(args, w):
     import ctypes as C
@@ -290,11 +305,9 @@ def run_ours(args, w):
     ms_frames = sum(e[1].elapsed_time(e[2]) for e in ev)
     ms_decode = sum(e[2].elapsed_time(e[3]) for e in ev)
     times = torch.tensor([ms_prefix, ms_frames, ms_decode], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_prefix, ms_frames, ms_decode = times.tolist()
-    fps = world * args.steps * w.n_frames / (ms_frames * 1e-3)
-    tps = world * args.steps * w.decode_tokens / (ms_decode * 1e-3) if w.decode_tokens else 0.0
+    ms_prefix, ms_frames, ms_decode = max_over_ranks(times, world).tolist()
+    fps = replica_throughput(world, args.steps * w.n_frames, ms_frames)
+    tps = replica_throughput(world, args.steps * w.decode_tokens, ms_decode) if w.decode_tokens else 0.0
 
     # ---- the same frames, CHUNK_FRAMES per call (offline form; informative, not the headline) ----
     chunk_fps = None
@@ -321,9 +334,7 @@ def run_ours(args, w):
             flush.zero_(); chunk_step(*cev[k])
         barrier()
         ms_chunk = torch.tensor([sum(a_.elapsed_time(b_) for a_, b_ in cev)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(ms_chunk, op=dist.ReduceOp.MAX)
-        chunk_fps = world * c_steps * w.n_frames / (ms_chunk.item() * 1e-3)
+        chunk_fps = replica_throughput(world, c_steps * w.n_frames, max_over_ranks(ms_chunk, world).item())
         sb.profile_read()
 
     # ---- per-kernel pass: events around every launch, one extra step ------------------------
@@ -443,10 +454,9 @@ def run_ours(args, w):
         e2e_step()
     barrier()
     e2e_s = torch.tensor([time.perf_counter() - t0], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
+    max_over_ranks(e2e_s, world)
     if rank == 0:
-        result["e2e"] = {"value": world * e_steps * w.n_frames / e2e_s.item(), "unit": "frames/s",
+        result["e2e"] = {"value": replica_throughput(world, e_steps * w.n_frames, 1e3 * e2e_s.item()), "unit": "frames/s",
                          "h2d_bytes_per_step": int(w.n_frames * N * d * 2),
                          "d2h_bytes_per_step": int(w.n_frames * (N + 1) * HD * 4),
                          "note": "frames phase only; per frame: pinned H2D of the hidden states, "
