@@ -35,7 +35,7 @@ if ROOT not in sys.path:
 from paper_2503_09387_b200 import synth  # noqa: E402
 
 
-CHUNK_FRAMES = 16                           # frames per vs_frame_prefill_chunk call in the `chunked_prefill` leg
+CHUNK_FRAMES = 8                            # frames per vs_frame_prefill_chunk call in the `chunked_prefill` leg
 GEMM_FRAME_DRAM_BYTES = 34364928 + 218368   # ncu: read + write of one 170-row projection launch
 
 
