@@ -186,6 +186,26 @@ def test_chunked_prefill_with_tiny_banks(M):
     p.close()
 
 
+def test_chunks_and_streaming_steps_interleaved_on_two_streams():
+    """One handle, two streams: stream 0 is fed in chunks, stream 1 frame by frame in between, both
+    with full banks; neither may disturb the other's bank (the chunk's bookkeeping is per call)."""
+    w = synth.workload("tiny", n_streams=2, n_frames=20, bank_capacity=3, tokens_per_frame=13, prefix_len=3, seed=83)
+    p = Pair(w, max_chunk_frames=4, evict_policy=1)
+    p.text([0, 1], [w.prefix_hidden(0), w.prefix_hidden(1)], "prefixes")
+    t0 = t1 = 0
+    for rnd in range(4):
+        p.frame_chunk(0, [w.frame_hidden(t0 + j, 0) for j in range(4)], f"stream 0 chunk {rnd}")
+        t0 += 4
+        for _ in range(3):
+            p.frame([1], [w.frame_hidden(t1, 1)], f"stream 1 frame {t1}")
+            t1 += 1
+        p.check_bank(0); p.check_bank(1)
+    p.frame([0, 1], [w.frame_hidden(t0, 0), w.frame_hidden(t1, 1)], "both streams, one step")
+    p.text([0, 1], [w.decode_hidden(0, 0), w.decode_hidden(0, 1)], "decode")
+    p.check_bank(0); p.check_bank(1)
+    p.close()
+
+
 def test_chunked_prefill_qwen_shape():
     """One layer at the Qwen2-7B shape, 8 frames per call, 24 frames: the projection of a chunk is a
     1360-row GEMM (six token tiles, no K split)."""
