@@ -111,6 +111,9 @@ struct vs_stream {
   size_t ws_bytes = 0;
   int device = 0;
   int n_sms = 0;
+  // chunked prefill: the chunk's bank updates run on a stream of their own beside the projection
+  cudaStream_t side_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   std::vector<const bf16*> w, bias, gain;
   std::vector<CUtensorMap> tm_w;
   std::vector<HostStream> hs;
@@ -312,6 +315,9 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights, void* work
 int vs_destroy_stream(vs_stream* h) {
   if (h == nullptr) return VS_ERR_INVALID_ARG;
   for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);
+  if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+  if (h->ev_join) cudaEventDestroy(h->ev_join);
+  if (h->side_stream) cudaStreamDestroy(h->side_stream);
   delete h;
   return VS_OK;
 }
@@ -488,7 +494,23 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
   VS_LAUNCH(h, st, KC_POOL, launch_pool(pa, bp, st));
 
   // 2. the bank updates, frame by frame (Section 3.3, memory mechanism): they read embeddings only,
-  //    so they can all run before any attention; each records the slot its carrier took
+  //    so they can all run before any attention; each records the slot its carrier took.  The
+  //    projection needs nothing of theirs, so they run beside it on a stream of the handle's own,
+  //    forked here and joined ahead of the first attention launch.
+  if (h->side_stream == nullptr) {
+    // highest priority: its few small CTAs must not queue behind the projection's second wave
+    int prio_low = 0, prio_high = 0;
+    VS_CK(cudaDeviceGetStreamPriorityRange(&prio_low, &prio_high));
+    VS_CK(cudaStreamCreateWithPriority(&h->side_stream, cudaStreamNonBlocking, prio_high));
+    VS_CK(cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
+    VS_CK(cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
+  }
+  const bool beside = !h->prof_on;           // the per-launch timing pass keeps everything on one stream
+  cudaStream_t bst = beside ? h->side_stream : st;
+  if (beside) {
+    VS_CK(cudaEventRecord(h->ev_fork, st));
+    VS_CK(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
+  }
   for (int j = 0; j < F; ++j) {
     BankUpdateArgs ba;
     ba.emb = h->at<bf16>(lo.emb); ba.meta = meta; ba.step_slot = h->at<int32_t>(lo.step_slot);
@@ -502,8 +524,9 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
     ba.chunk_first_frame = bp.frame_id[0];
     ba.chunk_l1 = l1;
     const BatchParams b1 = one_frame(j);
-    VS_LAUNCH(h, st, KC_COMMIT, launch_bank_update(ba, b1, D.M > 0 && b1.count[0] == D.M, st));
+    VS_LAUNCH(h, bst, KC_COMMIT, launch_bank_update(ba, b1, D.M > 0 && b1.count[0] == D.M, bst));
   }
+  if (beside) VS_CK(cudaEventRecord(h->ev_join, h->side_stream));
 
   // 3. layer by layer: one projection over all F * (N + 1) rows, one attention launch over all
   //    frames, then the K/V rows of the chunk's surviving carriers go into their bank slots
@@ -534,6 +557,7 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
 
     const bool last = (l == D.L - 1);
     char* layer_out = last ? out_bytes : static_cast<char*>(h->at<void>(lo.obuf));
+    if (l == 0 && beside) VS_CK(cudaStreamWaitEvent(st, h->ev_join, 0));
     {
       // every frame is a batch entry; frame b sees the bank of before the chunk minus what the
       // updates of frames 0 .. b-1 evicted, plus the carriers of those frames (from the step's K/V)

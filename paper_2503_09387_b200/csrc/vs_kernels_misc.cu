@@ -171,7 +171,7 @@ cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* r
 }
 
 // The bank update of one frame as a launch of its own (chunked prefill).
-__global__ void __launch_bounds__(256) bank_update_kernel(BankUpdateArgs a, BatchParams bp) {
+__global__ void __launch_bounds__(256, 8) bank_update_kernel(BankUpdateArgs a, BatchParams bp) {   // <= 32 registers: fits beside a projection CTA
   pdl_wait();
   pdl_launch_dependents();
   bank_update_block(a, bp, (int)blockIdx.y, (int)blockIdx.x);
