@@ -146,7 +146,11 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
  * only at carrier embeddings, which are all known once the frames are pooled.  Per layer the
  * Q/K/V projection of all F*(N+1) rows is one GEMM; the attention runs frame by frame.
  * hidden: DEVICE bf16 [F][N][d_model];  out: DEVICE [F][N+1][Hq*D] of `out_dtype`, or NULL.
- * Errors: as vs_frame_prefill; VS_ERR_CAPACITY also if F > max_chunk_frames. */
+ * The chunk's bank updates are enqueued on a stream that the handle owns, forked from and joined
+ * back into `cuda_stream` by events, so that they run beside the projection; the handle's first
+ * call of this function creates that stream and its two events (no device memory).
+ * Errors: as vs_frame_prefill; VS_ERR_CAPACITY also if F > max_chunk_frames or if
+ *         bank_capacity + 1 + F > 8192. */
 int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, int32_t F, int32_t N,
                            void* out, void* cuda_stream);
 
