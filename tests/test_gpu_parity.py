@@ -206,6 +206,23 @@ def test_chunks_and_streaming_steps_interleaved_on_two_streams():
     p.close()
 
 
+def test_chunked_prefill_long_run_with_many_evictions():
+    """96 frames at the Qwen2-7B shape in chunks of 16 with a 12-carrier bank: 84 evictions, most of
+    them of carriers that entered the bank earlier in the same chunk; the projection of a chunk is
+    a 2720-row GEMM in two waves of CTAs."""
+    w = synth.workload("long", n_frames=96, bank_capacity=12, question_len=0, decode_tokens=2)
+    p = Pair(w, max_chunk_frames=16)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    shared = w.frame_shared()
+    for t in range(0, 96, 16):
+        p.frame_chunk(0, [w.frame_hidden(t + j, shared=shared) for j in range(16)], f"chunk at frame {t}")
+        p.check_bank(0)
+    assert p.ora[0].evictions == 84
+    for i in range(2):
+        p.text([0], [w.decode_hidden(i)], f"decode {i}")
+    p.close()
+
+
 def test_chunked_prefill_qwen_shape():
     """One layer at the Qwen2-7B shape, 8 frames per call, 24 frames: the projection of a chunk is a
     1360-row GEMM (six token tiles, no K split)."""
