@@ -551,31 +551,50 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(AttnAr
         stage_o[row * F4 + (((DH * half + c) >> 2) ^ (row & (F4 - 1)))] =
             make_float4(o_acc[c] * inv, o_acc[c + 1] * inv, o_acc[c + 2] * inv, o_acc[c + 3] * inv);
     }
-    softmax_barrier_and(true);
-    if (all_ok) {
-      const float4* stage_o = reinterpret_cast<const float4*>(gbase + L::kQhi);
-      const int lane = tid & 31;
-      for (int r = warp * 16; r < warp * 16 + 16; ++r) {           // 8 warps x 16 rows
+    if (!all_ok) *abort_flag = 1;
+  }
+
+  // ---- rows out: all 12 warps, a warp per row, four rows' reads ahead of their stores ---------------
+  __syncthreads();
+  if (!*abort_flag) {
+    constexpr int F4 = D / 4;
+    constexpr int kWarps = kAttnThreads / 32;
+    const float4* stage_o = reinterpret_cast<const float4*>(gbase + L::kQhi);
+    const int lane = tid & 31;
+    const int G = a.Hq / a.Hkv;
+    const int rps = bp.rows_per_stream;
+    const int b = blockIdx.z, hkv = blockIdx.y;
+    const int r0 = ((int)blockIdx.x - a.bank_blocks) * kTok;
+    for (int rb = warp; rb < kRows; rb += 4 * kWarps) {
+      float4 v[4];
+      bool valid[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int r = rb + k * kWarps;
+        valid[k] = r < kRows && (r >> 4) < G && r0 + (r & 15) < rps && lane < F4;      // row part uniform over the warp
+        if (valid[k]) v[k] = stage_o[r * F4 + (lane ^ (r & (F4 - 1)))];
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (!valid[k]) continue;
+        const int r = rb + k * kWarps;
         const int gg = r >> 4, tt = r0 + (r & 15);
-        if (gg >= G || tt >= rps) continue;                        // uniform over the warp
         const size_t obase = (((size_t)b * rps + tt) * a.Hq + (size_t)hkv * G + gg) * D;
-        for (int u = lane; u < F4; u += 32) {
-          const float4 v = stage_o[r * F4 + (u ^ (r & (F4 - 1)))];
-          if (a.out_fp32) {
-            *reinterpret_cast<float4*>(static_cast<float*>(a.out) + obase + 4 * u) = v;
-          } else {
-            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
-            uint2 w; w.x = *reinterpret_cast<uint32_t*>(&lo); w.y = *reinterpret_cast<uint32_t*>(&hi);
-            *reinterpret_cast<uint2*>(static_cast<bf16*>(a.out) + obase + 4 * u) = w;
-          }
-          if (a.h_out != nullptr) {
-            const uint2 hraw = *reinterpret_cast<const uint2*>(a.h_in + obase + 4 * u);
-            const float2 h0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hraw.x));
-            const float2 h1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hraw.y));
-            __nv_bfloat162 lo = __floats2bfloat162_rn(h0.x + v.x, h0.y + v.y), hi = __floats2bfloat162_rn(h1.x + v.z, h1.y + v.w);
-            uint2 w; w.x = *reinterpret_cast<uint32_t*>(&lo); w.y = *reinterpret_cast<uint32_t*>(&hi);
-            *reinterpret_cast<uint2*>(a.h_out + obase + 4 * u) = w;
-          }
+        const int u = lane;
+        if (a.out_fp32) {
+          *reinterpret_cast<float4*>(static_cast<float*>(a.out) + obase + 4 * u) = v[k];
+        } else {
+          __nv_bfloat162 lo = __floats2bfloat162_rn(v[k].x, v[k].y), hi = __floats2bfloat162_rn(v[k].z, v[k].w);
+          uint2 w; w.x = *reinterpret_cast<uint32_t*>(&lo); w.y = *reinterpret_cast<uint32_t*>(&hi);
+          *reinterpret_cast<uint2*>(static_cast<bf16*>(a.out) + obase + 4 * u) = w;
+        }
+        if (a.h_out != nullptr) {
+          const uint2 hraw = *reinterpret_cast<const uint2*>(a.h_in + obase + 4 * u);
+          const float2 h0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hraw.x));
+          const float2 h1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hraw.y));
+          __nv_bfloat162 lo = __floats2bfloat162_rn(h0.x + v[k].x, h0.y + v[k].y), hi = __floats2bfloat162_rn(h1.x + v[k].z, h1.y + v[k].w);
+          uint2 w; w.x = *reinterpret_cast<uint32_t*>(&lo); w.y = *reinterpret_cast<uint32_t*>(&hi);
+          *reinterpret_cast<uint2*>(a.h_out + obase + 4 * u) = w;
         }
       }
     }
