@@ -303,12 +303,14 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
         else dst_far[(size_t)t * GEMM_BLOCK_M] = __uint_as_float(r[j]);
       }
     }
-    if (p.ksplit > 1) __threadfence();                         // the stores above, before the flag below
   }
   tcgen05_fence_before();
   __syncthreads();
   if (p.ksplit > 1 && threadIdx.x == 64) {
     if (!*abort_flag) {
+      // the barrier above ordered every thread's stores before this point; one cumulative fence
+      // then orders them before the flag increments for whoever acquires a flag
+      __threadfence();
       for (int s = 0; s < p.ksplit; ++s)
         if (s != rank) atomicAdd(p.flags + group * p.ksplit + s, 1);
     }
