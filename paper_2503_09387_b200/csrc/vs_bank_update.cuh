@@ -13,6 +13,23 @@ __device__ __forceinline__ double warp_tree_sum(double v) {
   return v;
 }
 
+// cos(va, vb) over d elements by one warp: lane p sums elements k = p (mod 32) in ascending k in
+// fp64, then a butterfly 16, 8, 4, 2, 1; the result is the same in every lane
+__device__ __forceinline__ double warp_cosine(const bf16* va, const bf16* vb, int d, int lane) {
+  double dot = 0.0, na = 0.0, nb = 0.0;
+  for (int k = lane; k < d; k += 32) {
+    const double x = (double)__bfloat162float(va[k]);
+    const double y = (double)__bfloat162float(vb[k]);
+    dot = __dadd_rn(dot, __dmul_rn(x, y));
+    na = __dadd_rn(na, __dmul_rn(x, x));
+    nb = __dadd_rn(nb, __dmul_rn(y, y));
+  }
+  dot = warp_tree_sum(dot); na = warp_tree_sum(na); nb = warp_tree_sum(nb);
+  double s = 0.0;
+  if (na != 0.0 && nb != 0.0) s = __ddiv_rn(dot, __dmul_rn(__dsqrt_rn(na), __dsqrt_rn(nb)));
+  return s;
+}
+
 // Block `block` of `n_blocks` (as the host sized them: one if no listed stream's bank is full,
 // else ceil(M / 8)) working on listed stream b.  Called by every thread of the CTA; threads
 // beyond the first 256 only keep the barriers company.
@@ -68,6 +85,8 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
   double* scores = a.scores + (size_t)sid * a.slots;
   const int lane = tid & 31;
   const int n_score_blocks = (a.M + 7) / 8;
+  const bool planned = a.pre_scores != nullptr;      // one block, scores already there: no ticket
+  if (!planned) {
   if (block >= n_score_blocks) return;
   const int j = block * 8 + (tid >> 5);
   if (on && j < count && a.policy != 2) {
@@ -75,20 +94,8 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
     const int sb = (a.policy == 1 && j + 1 < count) ? order[j + 1] : incoming;
     const bf16* va = a.emb + ((size_t)sid * a.slots + sa) * a.d;
     const bf16* vb = (sb == incoming) ? emb_in : a.emb + ((size_t)sid * a.slots + sb) * a.d;
-    double dot = 0.0, na = 0.0, nb = 0.0;
-    for (int k = lane; k < a.d; k += 32) {
-      const double x = (double)__bfloat162float(va[k]);
-      const double y = (double)__bfloat162float(vb[k]);
-      dot = __dadd_rn(dot, __dmul_rn(x, y));
-      na = __dadd_rn(na, __dmul_rn(x, x));
-      nb = __dadd_rn(nb, __dmul_rn(y, y));
-    }
-    dot = warp_tree_sum(dot); na = warp_tree_sum(na); nb = warp_tree_sum(nb);
-    if (lane == 0) {
-      double s = 0.0;
-      if (na != 0.0 && nb != 0.0) s = __ddiv_rn(dot, __dmul_rn(__dsqrt_rn(na), __dsqrt_rn(nb)));
-      scores[j] = s;
-    }
+    const double s = warp_cosine(va, vb, a.d, lane);
+    if (lane == 0) scores[j] = s;
   }
   __shared__ int is_last;
   __threadfence();
@@ -97,12 +104,22 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
   __syncthreads();
   if (!is_last) return;
   __threadfence();
+  }
   __shared__ double best_s[NT];
   __shared__ int best_j[NT];
   double bs = -2.0; int bj = 0x7fffffff;
   if (on && a.policy != 2) {
     for (int i = tid; i < count; i += NT) {
-      const double s = __ldcg(scores + i);
+      double s;
+      if (planned) {
+        // the carrier at temporal index i, as an index on the chunk's bank axis
+        const int slot_i = order[i];
+        const long long fr = slot_frame[slot_i];
+        const int c = (fr >= a.chunk_first_frame) ? a.chunk_l1 + (int)(fr - a.chunk_first_frame) : slot_i;
+        s = a.pre_scores[(size_t)b * a.pre_stride + c];
+      } else {
+        s = __ldcg(scores + i);
+      }
       if (s > bs) { bs = s; bj = i; }                 // ascending i: first maximum kept
     }
   }
@@ -150,7 +167,7 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
     meta->free_slot = victim_slot;
     meta->victim_logical = -1;
     meta->frames_seen += 1;
-    meta->score_ticket = 0;
+    if (!planned) meta->score_ticket = 0;
   }
 }
 

@@ -89,6 +89,7 @@ struct Layout {
   size_t obuf;                  // f32  [R_max][Hq*D] (holds bf16 or fp32 rows)
   size_t dec_part;              // f32  [DEC_SPLIT_MAX][S][Hq][D+2]
   size_t emb_stage;             // bf16 [max_chunk][d]  chunked prefill: carrier embeddings before they have a slot
+  size_t chunk_scores;          // f64  [max_chunk][slots + max_chunk]  chunked prefill: cosines of (frame, candidate) pairs
   size_t gemm_xchg;             // f32  [GEMM_XCHG_CTAS][256][128]  projection K split: partial tiles
   size_t scratch_begin, scratch_end;
   size_t total;
@@ -205,6 +206,10 @@ struct BankUpdateArgs {
   int32_t* record_victim;
   long long chunk_first_frame;
   int chunk_l1;                  // bank slots on the key axis of the chunk's frames
+  // ... planned by ONE block for all frames in turn: the cosine of every (frame, candidate) pair was
+  // worked out beforehand, pre_scores[b * pre_stride + index on the chunk's bank axis]; else null
+  const double* pre_scores;
+  int pre_stride;
   int32_t* order; int32_t* slot_frame; int64_t* slot_pos; int32_t* evict_log; double* scores;
   int d, slots, M, policy, log_cap;
 };
@@ -241,6 +246,11 @@ struct AttnArgs {
 };
 // chunked prefill: the bank update of one frame as a launch of its own (it precedes the projection)
 cudaError_t launch_bank_update(const BankUpdateArgs& a, const BatchParams& bp, bool full, cudaStream_t st);
+// chunked prefill, policies that score against the incoming carrier only: all cosines of the chunk
+// in one launch (frame b against bank slots 0 .. l1-1 and the chunk's carriers 0 .. b-1), then the
+// F bank updates in turn by one block
+cudaError_t launch_chunk_scores(const BankUpdateArgs& a, const BatchParams& bp, const bf16* emb_stage, double* out, cudaStream_t st);
+cudaError_t launch_chunk_plan(const BankUpdateArgs& a, const BatchParams& bp, cudaStream_t st);
 // chunked prefill, after a layer's attention: the K/V rows of the chunk's carriers that are still in
 // the bank go to their slots
 struct ChunkKvCommitArgs {

@@ -97,6 +97,7 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.obuf = take((size_t)D.R_max * D.Hq * D.D * 4);
   Lo.dec_part = take((size_t)DEC_SPLIT_MAX * D.S * D.Hq * (D.D + 2) * 4);
   Lo.emb_stage = take((size_t)D.maxChunk * D.d * 2);
+  Lo.chunk_scores = take(D.maxChunk > 1 ? (size_t)D.maxChunk * (D.slots + D.maxChunk) * 8 : 8);
   Lo.gemm_xchg = take((size_t)GEMM_XCHG_CTAS * 256 * GEMM_BLOCK_M * 4);
   Lo.scratch_end = off;
   Lo.total = off;
@@ -360,6 +361,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
   ba.scores = h->at<double>(lo.scores);
   ba.d = D.d; ba.slots = D.slots; ba.M = D.M; ba.policy = D.evict_policy; ba.log_cap = D.log_cap;
   ba.incoming_emb = nullptr; ba.record_slot = nullptr; ba.record_victim = nullptr; ba.chunk_first_frame = 0; ba.chunk_l1 = 0;
+  ba.pre_scores = nullptr; ba.pre_stride = 0;
 
   PoolArgs pa;
   pa.hidden = static_cast<const bf16*>(hidden);
@@ -511,20 +513,38 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
     VS_CK(cudaEventRecord(h->ev_fork, st));
     VS_CK(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
   }
-  for (int j = 0; j < F; ++j) {
+  {
     BankUpdateArgs ba;
     ba.emb = h->at<bf16>(lo.emb); ba.meta = meta; ba.step_slot = h->at<int32_t>(lo.step_slot);
     ba.order = h->at<int32_t>(lo.order); ba.slot_frame = h->at<int32_t>(lo.slot_frame);
     ba.slot_pos = h->at<int64_t>(lo.slot_pos); ba.evict_log = h->at<int32_t>(lo.evict_log);
     ba.scores = h->at<double>(lo.scores);
     ba.d = D.d; ba.slots = D.slots; ba.M = D.M; ba.policy = D.evict_policy; ba.log_cap = D.log_cap;
-    ba.incoming_emb = h->at<bf16>(lo.emb_stage) + (size_t)j * D.d;
-    ba.record_slot = chunk_slot + j;
-    ba.record_victim = chunk_victim + j;
     ba.chunk_first_frame = bp.frame_id[0];
     ba.chunk_l1 = l1;
-    const BatchParams b1 = one_frame(j);
-    VS_LAUNCH(h, bst, KC_COMMIT, launch_bank_update(ba, b1, D.M > 0 && b1.count[0] == D.M, bst));
+    ba.pre_scores = nullptr; ba.pre_stride = 0;
+    const bool any_full = D.M > 0 && bp.count[F - 1] == D.M;
+    if (D.evict_policy != 1 && F > 1) {
+      // the updates score against their incoming carrier only (or not at all): every cosine of the
+      // chunk in one launch, then all F updates in turn by one block
+      ba.incoming_emb = h->at<bf16>(lo.emb_stage);
+      ba.record_slot = chunk_slot;
+      ba.record_victim = chunk_victim;
+      ba.pre_scores = h->at<double>(lo.chunk_scores);
+      ba.pre_stride = D.slots + D.maxChunk;
+      if (any_full && D.evict_policy == 0)
+        VS_LAUNCH(h, bst, KC_EVICT, launch_chunk_scores(ba, bp, h->at<bf16>(lo.emb_stage), h->at<double>(lo.chunk_scores), bst));
+      VS_LAUNCH(h, bst, KC_COMMIT, launch_chunk_plan(ba, bp, bst));
+    } else {
+      // adjacent-pair scoring: which pairs are adjacent depends on the updates before, one launch per frame
+      for (int j = 0; j < F; ++j) {
+        ba.incoming_emb = h->at<bf16>(lo.emb_stage) + (size_t)j * D.d;
+        ba.record_slot = chunk_slot + j;
+        ba.record_victim = chunk_victim + j;
+        const BatchParams b1 = one_frame(j);
+        VS_LAUNCH(h, bst, KC_COMMIT, launch_bank_update(ba, b1, D.M > 0 && b1.count[0] == D.M, bst));
+      }
+    }
   }
   if (beside) VS_CK(cudaEventRecord(h->ev_join, h->side_stream));
 
@@ -861,7 +881,7 @@ int vs_profile_read(vs_stream* h, double* ms, int64_t* timed, int64_t* launches)
 
 const char* vs_kernel_class_name(int32_t k) {
   static const char* names[VS_N_KERNEL_CLASSES] = {"pool", "rope_table", "rmsnorm", "qkv_gemm", "qkv_gemv",
-                                                   "prefill_attention", "decode_attention", "unused",
+                                                   "prefill_attention", "decode_attention", "chunk_scores",
                                                    "bank_update", "other"};
   return (k >= 0 && k < VS_N_KERNEL_CLASSES) ? names[k] : "?";
 }

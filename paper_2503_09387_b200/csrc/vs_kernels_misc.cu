@@ -182,6 +182,43 @@ cudaError_t launch_bank_update(const BankUpdateArgs& a, const BatchParams& bp, b
   return launch_pdl(bank_update_kernel, grid, dim3(256), 0, st, a, bp);
 }
 
+// All cosines a chunk's bank updates can need when every update scores against its incoming carrier
+// (policy 0): frame b's carrier against bank slots 0 .. l1-1 as they were before the chunk and against
+// the chunk's carriers 0 .. b-1.  grid = (ceil((l1 + F) / 8), F), one warp per pair.
+__global__ void __launch_bounds__(256, 8) chunk_scores_kernel(BankUpdateArgs a, BatchParams bp, const bf16* emb_stage,
+                                                              double* out) {
+  pdl_wait();                       // the pooled carriers are in place
+  pdl_launch_dependents();
+  const int b = blockIdx.y, lane = threadIdx.x & 31;
+  const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (c >= a.chunk_l1 + b) return;                                 // uniform over the warp
+  const int sid = bp.stream_id[b];
+  const bf16* va = (c < a.chunk_l1) ? a.emb + ((size_t)sid * a.slots + c) * a.d : emb_stage + (size_t)(c - a.chunk_l1) * a.d;
+  const double s = warp_cosine(va, emb_stage + (size_t)b * a.d, a.d, lane);
+  if (lane == 0) out[(size_t)b * a.pre_stride + c] = s;
+}
+
+cudaError_t launch_chunk_scores(const BankUpdateArgs& a, const BatchParams& bp, const bf16* emb_stage, double* out, cudaStream_t st) {
+  dim3 grid((a.chunk_l1 + bp.n_active + 7) / 8, bp.n_active);
+  return launch_pdl(chunk_scores_kernel, grid, dim3(256), 0, st, a, bp, emb_stage, out);
+}
+
+// The chunk's bank updates in turn by one block (the scores are looked up, the rest is the streaming
+// update): frame b finds the bank as frame b-1 left it.
+__global__ void __launch_bounds__(256, 8) chunk_plan_kernel(BankUpdateArgs a, BatchParams bp) {
+  pdl_wait();
+  pdl_launch_dependents();
+  for (int b = 0; b < bp.n_active; ++b) {
+    bank_update_block(a, bp, b, 0);
+    __threadfence_block();
+    __syncthreads();
+  }
+}
+
+cudaError_t launch_chunk_plan(const BankUpdateArgs& a, const BatchParams& bp, cudaStream_t st) {
+  return launch_pdl(chunk_plan_kernel, dim3(1), dim3(256), 0, st, a, bp);
+}
+
 // grid = F CTAs of 128 threads: CTA i copies the carrier row of the chunk's frame i unless a later
 // update of the chunk evicted that carrier (its slot then belongs to someone else).
 __global__ void __launch_bounds__(128) chunk_kv_commit_kernel(ChunkKvCommitArgs a) {
