@@ -12,6 +12,13 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200) and the built library")
 
 
+def pytest_sessionstart(session):
+    """The library is the only implementation: (re)build it if a source is newer than it, so that a
+    fresh checkout can run the suite (nvcc cross-compiles for sm_100a without a GPU)."""
+    from paper_2503_09387_b200 import build
+    build.build_library()
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch
