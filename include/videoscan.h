@@ -144,7 +144,8 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
  * that of F vs_frame_prefill calls in a row: each frame attends over [prefix | the bank as the
  * frames before it left it | own frame], evictions included, because the eviction rule looks
  * only at carrier embeddings, which are all known once the frames are pooled.  Per layer the
- * Q/K/V projection of all F*(N+1) rows is one GEMM; the attention runs frame by frame.
+ * Q/K/V projection of all F*(N+1) rows is one GEMM and the attention of all F frames is one launch
+ * (each frame with its own view of the bank).
  * hidden: DEVICE bf16 [F][N][d_model];  out: DEVICE [F][N+1][Hq*D] of `out_dtype`, or NULL.
  * The chunk's bank updates are enqueued on a stream that the handle owns, forked from and joined
  * back into `cuda_stream` by events, so that they run beside the projection; the handle's first
@@ -226,7 +227,8 @@ const char* vs_kernel_class_name(int32_t k);
  *   incoming  : DEVICE bf16 [d_model];
  *   policy    : as vs_config.evict_policy (0 similarity to the incoming carrier, 1 most
  *               similar adjacent pair, 2 FIFO);
- *   victim_out: DEVICE int32[1], receives the temporal index to discard (ties: oldest).
+ *   victim_out: DEVICE int32[1], receives the temporal index to discard (ties: oldest; a carrier
+ *               holding Inf or NaN has no cosine, its score counts as 0; always < count).
  * The call only enqueues work on cuda_stream.  Its scratch (count fp64 scores and one block
  * counter) lives in a static device array of the library, VS_STATIC_MAX_BANK * 8 + 256
  * bytes, which every GPU that loads the library holds until the process exits; count above

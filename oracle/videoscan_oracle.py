@@ -160,7 +160,8 @@ def _canonical_sum(prod: np.ndarray) -> np.ndarray:
 
 def canonical_dot(a: np.ndarray, b: np.ndarray) -> np.ndarray:
     """Dot product over the last axis; the products of two bf16 values are exact in fp64."""
-    return _canonical_sum(np.asarray(a, dtype=np.float64) * np.asarray(b, dtype=np.float64))
+    with np.errstate(invalid="ignore", over="ignore"):
+        return _canonical_sum(np.asarray(a, dtype=np.float64) * np.asarray(b, dtype=np.float64))
 
 
 def cosine_similarity(a: np.ndarray, b: np.ndarray) -> np.ndarray:
@@ -168,20 +169,25 @@ def cosine_similarity(a: np.ndarray, b: np.ndarray) -> np.ndarray:
     na = canonical_dot(a, a)
     nb = canonical_dot(b, b)
     den = np.sqrt(na) * np.sqrt(nb)
-    with np.errstate(divide="ignore", invalid="ignore"):
+    with np.errstate(divide="ignore", invalid="ignore", over="ignore"):
         s = dot / den
-    return np.where((na == 0.0) | (nb == 0.0), 0.0, s)
+    # the cosine is undefined for a zero vector and for a vector holding Inf or NaN: both count as 0
+    # (the paper does not say; with 0 such a carrier is never preferred over a real duplicate, and
+    # the argmax below always names a stored carrier)
+    return np.where((na == 0.0) | (nb == 0.0) | ~np.isfinite(s), 0.0, s)
 
 
 def choose_victim(bank_emb: np.ndarray, incoming: np.ndarray, policy: int = 0) -> int:
     """Index (temporal order, 0 = oldest) of the carrier to discard when the bank is full.
 
-    policy 0: the stored carrier most similar (cosine) to the incoming carrier.
-    policy 1: over the temporal sequence e_0 .. e_{M-1}, e_in, the older member of the
-              most similar ADJACENT pair (the other reading of "compares embeddings of
-              adjacent semantic carriers").
+    Section 3.3 (memory mechanism) states the rule in one sentence that can be read two ways:
+    policy 0: the stored carrier most similar (cosine) to the incoming carrier leaves -- every
+              stored carrier is older than the incoming one, which is never the victim.
+    policy 1: over the temporal sequence e_0 .. e_{M-1}, e_in, the older member of the most
+              similar pair of NEIGHBOURS leaves (the reading that takes the comparison to be
+              between carriers adjacent in time).
     policy 2: FIFO (oldest leaves); a test aid, not in the paper.
-    Ties go to the oldest carrier."""
+    Ties go to the oldest carrier; an undefined cosine (zero or non-finite vector) counts as 0."""
     if policy == 2:
         return 0
     if policy == 0:

@@ -27,6 +27,8 @@ __device__ __forceinline__ double warp_cosine(const bf16* va, const bf16* vb, in
   dot = warp_tree_sum(dot); na = warp_tree_sum(na); nb = warp_tree_sum(nb);
   double s = 0.0;
   if (na != 0.0 && nb != 0.0) s = __ddiv_rn(dot, __dmul_rn(__dsqrt_rn(na), __dsqrt_rn(nb)));
+  // a vector holding Inf or NaN has no cosine: counted as 0, like a zero vector
+  if (!(s >= -2.0 && s <= 2.0)) s = 0.0;
   return s;
 }
 
@@ -107,7 +109,7 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
   }
   __shared__ double best_s[NT];
   __shared__ int best_j[NT];
-  double bs = -2.0; int bj = 0x7fffffff;
+  double bs = -4.0; int bj = 0x7fffffff;   // every score lies in [-2, 2], so some thread takes an index < count
   if (on && a.policy != 2) {
     for (int i = tid; i < count; i += NT) {
       double s;
@@ -135,7 +137,8 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
     __syncthreads();
   }
   adopt();
-  const int v = (a.policy == 2) ? 0 : best_j[0];
+  // the index stays inside the bank whatever the scores were
+  const int v = (a.policy == 2 || (unsigned)best_j[0] >= (unsigned)count) ? 0 : best_j[0];
   const int victim_slot = order[v];
   const int victim_frame = slot_frame[victim_slot];
   __syncthreads();

@@ -47,6 +47,7 @@ evict_choose_static_kernel(const vs::bf16* __restrict__ bank, const vs::bf16* __
     if (lane == 0) {
       double s = 0.0;
       if (na != 0.0 && nb != 0.0) s = __ddiv_rn(dot, __dmul_rn(__dsqrt_rn(na), __dsqrt_rn(nb)));
+      if (!(s >= -2.0 && s <= 2.0)) s = 0.0;          // Inf or NaN in a vector: no cosine, counted as 0
       scratch->scores[j] = s;
     }
   }
@@ -59,7 +60,7 @@ evict_choose_static_kernel(const vs::bf16* __restrict__ bank, const vs::bf16* __
   __threadfence();
   __shared__ double best_s[256];
   __shared__ int best_j[256];
-  double bs = -2.0; int bj = 0x7fffffff;
+  double bs = -4.0; int bj = 0x7fffffff;              // every score lies in [-2, 2]
   for (int i = threadIdx.x; i < count; i += blockDim.x) {
     const double s = __ldcg(scratch->scores + i);
     if (s > bs) { bs = s; bj = i; }
@@ -76,7 +77,7 @@ evict_choose_static_kernel(const vs::bf16* __restrict__ bank, const vs::bf16* __
     __syncthreads();
   }
   if (threadIdx.x == 0) {
-    *victim_out = (policy == 2) ? 0 : best_j[0];
+    *victim_out = (policy == 2 || (unsigned)best_j[0] >= (unsigned)count) ? 0 : best_j[0];
     scratch->ticket = 0;
   }
 }

@@ -514,6 +514,42 @@ def test_large_bank_with_evictions_and_long_decode_context():
         p.close()
 
 
+def test_non_finite_carrier_keeps_the_bank_bookkeeping_in_range():
+    """A carrier that holds a NaN (or an Inf) has no cosine with anything: the score counts as 0 on
+    both sides, so the victim is still a stored carrier (the oldest when nothing else is preferred)
+    and the bookkeeping goes on; both eviction policies, streaming steps and a chunk."""
+    from oracle import videoscan_oracle as vo
+    for policy in (0, 1):
+        w = synth.workload("tiny", n_frames=12, bank_capacity=3, seed=17 + policy)
+        cfg = binding.make_config(1, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens_per_frame, 8, 4,
+                                  w.bank_capacity, evict_policy=policy, max_chunk_frames=4)
+        sb = binding.StreamBatch(cfg, [to_dev(w.weight(0))])
+        ora = vo.OracleStream(vo.OracleConfig(1, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, 3, evict_policy=policy),
+                              [synth.bf16_bits_to_f64(w.weight(0))])
+        for t in range(8):
+            x = w.frame_hidden(t)
+            ov = None
+            if t in (3, 6):                                  # bank full: a carrier with a NaN, later one with an Inf
+                ov = w.frame_hidden(t)[0].copy()
+                ov[5] = 0x7FC0 if t == 3 else 0x7F80
+            sb.frame_prefill([0], to_dev(x[None]), carrier_override=None if ov is None else to_dev(ov[None]), want_out=False)
+            with np.errstate(invalid="ignore"):
+                ora.frame_step(synth.bf16_bits_to_f64(x), carrier_override=None if ov is None else synth.bf16_bits_to_f64(ov),
+                               mode="meta")
+            st = sb.bank_state(0)
+            assert st["device_status"] == 0 and st["count"] == min(t + 1, 3)
+            assert list(st["frame_ids"]) == ora.bank_frame_ids()
+            assert st["last_victim_frame"] == ora.last_victim_frame
+        # a chunk of four frames over a bank that holds the non-finite carriers
+        sb.frame_prefill_chunk(0, to_dev(np.stack([w.frame_hidden(8 + j) for j in range(4)])))
+        for j in range(4):
+            ora.frame_step(synth.bf16_bits_to_f64(w.frame_hidden(8 + j)), mode="meta")
+        st = sb.bank_state(0)
+        assert st["device_status"] == 0 and list(st["frame_ids"]) == ora.bank_frame_ids()
+        assert [tuple(r) for r in st["evict_log"].tolist()] == ora.evict_log[-len(st["evict_log"]):]
+        sb.close()
+
+
 def test_argument_errors_leave_the_stream_untouched():
     w = synth.workload("tiny")
     p = Pair(w)

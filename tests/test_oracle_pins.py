@@ -184,13 +184,16 @@ def test_attention_matches_torch_sdpa_and_gqa_equals_repeated_mha():
 
 # ------------------------------------------------------------------ streaming == dense masked attention
 def _dense_reference(cfg, Ws, prefix_X, frames, texts, evict_after, norm=False, residual=False,
-                     theta=1e6, eps=1e-6):
+                     theta=1e6, eps=1e-6, gains=None, biases=None, carriers=None):
     """Textbook masked attention over the full un-pruned sequence
     [prefix | f0 tokens, c0 | f1 tokens, c1 | ... | text] with positions 0..S-1 and the
     semantic-aware mask of Section 3.4 / Fig. 3: a token sees the prefix, the carriers of
     earlier frames that are still in the bank when its own segment is processed, and the
     tokens of its own segment up to itself.  Written with explicit loops and complex
-    rotations, independently of the oracle's vectorised code."""
+    rotations, independently of the oracle's vectorised code.  Optional per-layer RMSNorm gain
+    (a multiply AFTER the division by the root mean square), per-layer bias (added to the
+    projected row BEFORE the rotation, Eq. 1 with an affine term) and caller-supplied carrier
+    tokens (they replace the mean as the frame's last token)."""
     Hq, Hkv, D = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
     G = Hq // Hkv
     toks, seg, is_carrier = [], [], []
@@ -199,7 +202,7 @@ def _dense_reference(cfg, Ws, prefix_X, frames, texts, evict_after, norm=False, 
     for t, E in enumerate(frames):
         for x in E:
             toks.append(x); seg.append(t); is_carrier.append(False)
-        toks.append(E.mean(axis=0)); seg.append(t); is_carrier.append(True)
+        toks.append(E.mean(axis=0) if carriers is None else carriers[t]); seg.append(t); is_carrier.append(True)
     TEXT = len(frames)
     for x in texts:
         toks.append(x); seg.append(TEXT); is_carrier.append(False)
@@ -221,11 +224,15 @@ def _dense_reference(cfg, Ws, prefix_X, frames, texts, evict_after, norm=False, 
         return gone is None or gone >= seg[i]
     freqs = np.array([theta ** (-2.0 * k / D) for k in range(D // 2)])
     outs = []
-    for W in Ws:
+    for li, W in enumerate(Ws):
         x = h
         if norm:
             x = h / np.sqrt((h * h).mean(axis=1, keepdims=True) + eps)
+            if gains is not None:
+                x = np.stack([row * gains[li] for row in x])
         y = x @ W.T
+        if biases is not None:
+            y = np.stack([row + biases[li] for row in y])
         Qm = y[:, :Hq * D].reshape(S, Hq, D)
         Km = y[:, Hq * D:(Hq + Hkv) * D].reshape(S, Hkv, D)
         Vm = y[:, (Hq + Hkv) * D:].reshape(S, Hkv, D)
@@ -248,8 +255,10 @@ def _dense_reference(cfg, Ws, prefix_X, frames, texts, evict_after, norm=False, 
     return outs[-1], seg
 
 
-@pytest.mark.parametrize("layers,norm,policy", [(1, False, 0), (2, True, 0), (1, False, 1)])
-def test_streaming_equals_dense_masked_attention(monkeypatch, layers, norm, policy):
+@pytest.mark.parametrize("layers,norm,policy,affine,override",
+                         [(1, False, 0, False, False), (2, True, 0, False, False), (1, False, 1, False, False),
+                          (2, True, 0, True, False), (1, False, 0, True, True), (2, True, 1, True, True)])
+def test_streaming_equals_dense_masked_attention(monkeypatch, layers, norm, policy, affine, override):
     # storage rounding is pinned on its own above; switch it off so the comparison with
     # the textbook computation is exact to fp64 rounding
     monkeypatch.setattr(vo, "round_to_bf16", lambda x: np.asarray(x, dtype=np.float64))
@@ -261,15 +270,23 @@ def test_streaming_equals_dense_masked_attention(monkeypatch, layers, norm, poli
     prefix = rng.standard_normal((P, d))
     frames = [rng.standard_normal((N, d)) for _ in range(F)]
     texts = rng.standard_normal((T, d))
-    st = vo.OracleStream(cfg, Ws)
+    E_out = (Hq + 2 * Hkv) * D
+    # affine: RMSNorm gain far from 1 and a bias as large as the projected values, so that a gain
+    # applied inside the root, or a bias added after the rotation, moves the result visibly
+    gains = [1.0 + 0.5 * rng.standard_normal(d) for _ in range(layers)] if (affine and norm) else None
+    biases = [rng.standard_normal(E_out) for _ in range(layers)] if affine else None
+    # override: the caller's carrier token replaces the mean everywhere -- as the frame's last
+    # token, as the bank's embedding (so eviction follows it) and as the source of the kept K/V
+    carriers = [rng.standard_normal(d) for _ in range(F)] if override else None
+    st = vo.OracleStream(cfg, Ws, biases, gains)
     got = [st.text_step(prefix)]
-    for E in frames:
-        got.append(st.frame_step(E))
+    for t, E in enumerate(frames):
+        got.append(st.frame_step(E, carrier_override=None if carriers is None else carriers[t]))
     got.append(st.text_step(texts[:2]))
     got.append(st.text_step(texts[2:]))
     got = np.concatenate(got, axis=0)
     # eviction trace recomputed naively from the carrier embeddings
-    embs = [E.mean(axis=0) for E in frames]
+    embs = [E.mean(axis=0) for E in frames] if carriers is None else carriers
     bank, gone = [], {}
     cos = lambda a, b: float(a @ b / (np.linalg.norm(a) * np.linalg.norm(b)))
     for t in range(F):
@@ -282,9 +299,12 @@ def test_streaming_equals_dense_masked_attention(monkeypatch, layers, norm, poli
             gone[bank.pop(int(np.argmax(s)))] = t
         bank.append(t)
     assert [(s, v) for v, s in sorted(gone.items(), key=lambda kv: kv[1])] == st.evict_log
-    want, _ = _dense_reference(cfg, Ws, prefix, frames, texts, gone, norm=norm, residual=layers > 1)
+    want, _ = _dense_reference(cfg, Ws, prefix, frames, texts, gone, norm=norm, residual=layers > 1,
+                               gains=gains, biases=biases, carriers=carriers)
     assert got.shape == want.shape
     assert np.max(np.abs(got - want)) < 1e-10
+    if override:
+        assert all(np.array_equal(e.emb, carriers[e.frame_id]) for e in st.bank)
 
 
 def test_zero_capacity_is_plain_causal_attention_per_frame(monkeypatch):
@@ -365,6 +385,15 @@ def test_eviction_hand_built_sequences():
     z = np.zeros(d)
     assert vo.choose_victim(np.stack([z, b]), b, 0) == 1         # zero norm counts as cosine 0
     assert vo.choose_victim(np.stack([z, a]), b, 0) == 0
+    # a non-finite embedding has no cosine either: it counts as 0, so a real duplicate still wins,
+    # and with nothing else to prefer the oldest leaves (the index always names a stored carrier)
+    bad = a.copy(); bad[3] = np.nan
+    inf = a.copy(); inf[0] = np.inf
+    assert vo.choose_victim(np.stack([bad, b, c]), b, 0) == 1
+    assert vo.choose_victim(np.stack([a, inf, c]), c, 0) == 2
+    assert vo.choose_victim(np.stack([a, b, c]), bad, 0) == 0    # every cosine undefined
+    assert vo.choose_victim(np.stack([a, b, c]), inf, 1) == 0    # only the pair with the incoming is undefined; rest orthogonal
+    assert vo.choose_victim(np.stack([a, a, bad]), c, 1) == 0    # pair (a, a) = 1 beats the undefined pairs
 
 
 def test_canonical_cosine_agrees_with_naive():
