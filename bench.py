@@ -36,7 +36,12 @@ from paper_2503_09387_b200 import synth  # noqa: E402
 
 
 CHUNK_FRAMES = 8                            # frames per vs_frame_prefill_chunk call in the `chunked_prefill` leg
-GEMM_FRAME_DRAM_BYTES = 34365184 + 35840    # ncu: read + write of one 170-row projection launch
+ORACLE_KIND = "oracle (numpy, BLAS threads)"
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel at the bench's
+# shape, from the ncu capture summarised under profiles/ (cold cache: the weights come from DRAM,
+# whereas inside the timed one-layer loop they are L2-resident).  None = not captured since the
+# kernel last changed.
+DOMINANT_KERNEL_TRAFFIC = {"bytes": None, "source": "no ncu capture of the current kernel"}
 
 
 def load_peaks():
@@ -178,7 +183,7 @@ def run_reference(args, w):
         "ms_per_step": 1e3 * t_total / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": workload_config(w),
-        "cpu_baseline": {"value": fps, "unit": "frames/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": fps, "unit": "frames/s", "cores": cores, "kind": ORACLE_KIND, "sample": sample},
         "e2e": {"value": fps, "unit": "frames/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
@@ -209,8 +214,86 @@ def replica_throughput(world, units_per_rank, ms):
 
 
 # ------------------------------------------------------------------ our arm
+REPEATS = 5                                 # the --steps block is timed this many times; the median block is reported
+DEEP_TIMED_FRAMES = 16                      # deep leg: the last frames of the 512-frame stream are the timed ones
+DEEP_TIMED_DECODE = 32
+
+
+def draw_parallel(fn, n):
+    """fn(i) for i < n on a thread pool (numpy releases the GIL inside the generator's array
+    operations); the draws are counter based, so the order of evaluation does not matter."""
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(max_workers=max(1, min(16, (os.cpu_count() or 2) - 1))) as ex:
+        return list(ex.map(fn, range(n)))
+
+
+class Streamer:
+    """One handle of the library fed from device-resident synthetic inputs of workload `w`."""
+
+    def __init__(self, w, dev, local, lib, binding, torch, chunk_frames=1):
+        import ctypes as C
+        self.w, self.dev, self.lib, self.C, self.torch = w, dev, lib, C, torch
+        to_dev = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).to(dev)
+        self.weights = [to_dev(b) for b in draw_parallel(w.weight, w.n_layers)]
+        shared = w.frame_shared() if w.frame_model != "iid" else None
+        self.frames_host = np.stack(draw_parallel(lambda t: w.frame_hidden(t, shared=shared), w.n_frames))
+        self.frames = to_dev(self.frames_host)                          # [F, N, d]
+        self.prefix = to_dev(w.prefix_hidden())
+        self.question = to_dev(w.question_hidden()) if w.question_len else None
+        self.dec = to_dev(np.concatenate([w.decode_hidden(i) for i in range(w.decode_tokens)]))   # [n_dec, d]
+        cfg = binding.make_config(w.n_layers, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens_per_frame,
+                                  max(w.prefix_len, 1), max(w.question_len + w.decode_tokens, 1), w.bank_capacity,
+                                  n_streams=1, max_step_tokens=max(64, w.prefix_len), use_rmsnorm=w.use_rmsnorm,
+                                  residual=w.residual, rope_theta=w.rope_theta, rms_eps=w.rms_eps, device=local,
+                                  max_chunk_frames=chunk_frames)
+        self.sb = binding.StreamBatch(cfg, self.weights)
+        N, HD = w.tokens_per_frame, w.n_q_heads * w.head_dim
+        self.N, self.HD = N, HD
+        self.out_frame = torch.empty((N + 1, HD), dtype=torch.float32, device=dev)
+        self.out_text = torch.empty((max(w.prefix_len, w.question_len, 1), HD), dtype=torch.float32, device=dev)
+        self.out_dec = torch.empty((1, HD), dtype=torch.float32, device=dev)
+        self.stream = torch.cuda.current_stream(dev)
+        self.sptr = C.c_void_p(self.stream.cuda_stream)
+        self.ids = (C.c_int32 * 1)(0)
+        self.h = C.c_void_p(self.sb.handle)
+        self.frame_ptrs = [C.c_void_p(self.frames[t].data_ptr()) for t in range(w.n_frames)]
+        self.dec_ptrs = [C.c_void_p(self.dec[i:i + 1].data_ptr()) for i in range(w.decode_tokens)]
+        self.p_out_frame, self.p_out_dec = C.c_void_p(self.out_frame.data_ptr()), C.c_void_p(self.out_dec.data_ptr())
+        self.p_out_text = C.c_void_p(self.out_text.data_ptr())
+        self.binding = binding
+
+    def ck(self, code):
+        if code != 0:
+            raise RuntimeError("library call failed: %s" % self.binding.status_string(code))
+
+    def reset(self):
+        self.ck(self.lib.vs_reset_stream(self.h, self.ids, 1, self.sptr))
+
+    def text(self, x, T):
+        self.ck(self.lib.vs_decode_step(self.h, self.ids, 1, self.C.c_void_p(x.data_ptr()), T, self.p_out_text, self.sptr))
+
+    def frames_range(self, t0, t1):
+        for t in range(t0, t1):
+            self.ck(self.lib.vs_frame_prefill(self.h, self.ids, 1, self.frame_ptrs[t], self.N, None, self.p_out_frame, self.sptr))
+
+    def decode_range(self, i0, i1):
+        for i in range(i0, i1):
+            self.ck(self.lib.vs_decode_step(self.h, self.ids, 1, self.dec_ptrs[i], 1, self.p_out_dec, self.sptr))
+
+    def end_turn(self):
+        self.ck(self.lib.vs_end_turn(self.h, self.ids, 1))
+
+
+def kernel_table(phase):
+    k = {n: {"launches": v[1], "total_ms": round(v[0], 4), "avg_us": round(1e3 * v[0] / v[1], 3)}
+         for n, v in phase.items() if v[1]}
+    tot = sum(v["total_ms"] for v in k.values())
+    for v in k.values():
+        v["share"] = round(v["total_ms"] / tot, 4) if tot else 0.0
+    return k
+
+
 def run_ours(args, w):
-    import ctypes as C
     import torch
     import torch.distributed as dist
     from paper_2503_09387_b200 import binding, build
@@ -227,54 +310,25 @@ def run_ours(args, w):
     if world > 1:
         dist.barrier()
     lib = binding.load_library()
-
-    def to_dev(bits):
-        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).to(dev)
+    C = __import__("ctypes")
 
     # ---- inputs (replicas only: every rank streams its own copy of the workload) ----------
-    weights = [to_dev(w.weight(l)) for l in range(w.n_layers)]
-    shared = w.frame_shared() if w.frame_model != "iid" else None
-    frames_host = np.stack([w.frame_hidden(t, shared=shared) for t in range(w.n_frames)])
-    frames = to_dev(frames_host)                                   # [F, N, d]
-    prefix = to_dev(w.prefix_hidden())
-    dec = to_dev(np.concatenate([w.decode_hidden(i) for i in range(w.decode_tokens)]))   # [n_dec, d]
-    cfg = binding.make_config(w.n_layers, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens_per_frame,
-                              max(w.prefix_len, 1), max(w.question_len + w.decode_tokens, 1), w.bank_capacity,
-                              n_streams=1, max_step_tokens=max(64, w.prefix_len), use_rmsnorm=w.use_rmsnorm,
-                              residual=w.residual, rope_theta=w.rope_theta, rms_eps=w.rms_eps, device=local,
-                              max_chunk_frames=CHUNK_FRAMES)
-    sb = binding.StreamBatch(cfg, weights)
-    N, d, HD = w.tokens_per_frame, w.d_model, w.n_q_heads * w.head_dim
-    out_frame = torch.empty((N + 1, HD), dtype=torch.float32, device=dev)
-    out_prefix = torch.empty((max(w.prefix_len, 1), HD), dtype=torch.float32, device=dev)
-    out_dec = torch.empty((1, HD), dtype=torch.float32, device=dev)
+    S = Streamer(w, dev, local, lib, binding, torch, chunk_frames=CHUNK_FRAMES)
+    sb, N, d, HD = S.sb, S.N, w.d_model, S.HD
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    stream = torch.cuda.current_stream(dev)
-    sptr = C.c_void_p(stream.cuda_stream)
-    ids = (C.c_int32 * 1)(0)
-    h = C.c_void_p(sb.handle)
-    frame_ptrs = [C.c_void_p(frames[t].data_ptr()) for t in range(w.n_frames)]
-    dec_ptrs = [C.c_void_p(dec[i:i + 1].data_ptr()) for i in range(w.decode_tokens)]
-    p_prefix, p_out_prefix = C.c_void_p(prefix.data_ptr()), C.c_void_p(out_prefix.data_ptr())
-    p_out_frame, p_out_dec = C.c_void_p(out_frame.data_ptr()), C.c_void_p(out_dec.data_ptr())
-
-    def ck(code):
-        if code != 0:
-            raise RuntimeError("library call failed: %s" % binding.status_string(code))
+    stream = S.stream
 
     def one_step(events=None, on_phase=None):
-        ck(lib.vs_reset_stream(h, ids, 1, sptr))
+        S.reset()
         if events: events[0].record(stream)
         if w.prefix_len:
-            ck(lib.vs_decode_step(h, ids, 1, p_prefix, w.prefix_len, p_out_prefix, sptr))
+            S.text(S.prefix, w.prefix_len)
         if events: events[1].record(stream)
         if on_phase: on_phase("prefix")
-        for t in range(w.n_frames):
-            ck(lib.vs_frame_prefill(h, ids, 1, frame_ptrs[t], N, None, p_out_frame, sptr))
+        S.frames_range(0, w.n_frames)
         if events: events[2].record(stream)
         if on_phase: on_phase("frames")
-        for i in range(w.decode_tokens):
-            ck(lib.vs_decode_step(h, ids, 1, dec_ptrs[i], 1, p_out_dec, sptr))
+        S.decode_range(0, w.decode_tokens)
         if events: events[3].record(stream)
         if on_phase: on_phase("decode")
 
@@ -289,23 +343,27 @@ def run_ours(args, w):
         one_step()
     sb.profile_read()                                   # clear launch counters
     sampler = ClockSampler(local)
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    barrier()
     sampler.start()
+    # ---- the timed region: REPEATS blocks of exactly --steps steps, each block bracketed by a
+    # barrier + synchronize; per phase the device time of a block is the sum over its steps of the
+    # CUDA-event intervals, the slowest rank's block counts, and the median block is reported
+    blocks = []
     wall0 = time.perf_counter()
-    for k in range(args.steps):
-        flush.zero_()
-        one_step(ev[k])
-    barrier()
+    for _ in range(REPEATS):
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+        barrier()
+        for k in range(args.steps):
+            flush.zero_()
+            one_step(ev[k])
+        barrier()
+        t = torch.tensor([sum(e[0].elapsed_time(e[1]) for e in ev), sum(e[1].elapsed_time(e[2]) for e in ev),
+                          sum(e[2].elapsed_time(e[3]) for e in ev)], dtype=torch.float64, device=dev)
+        blocks.append(max_over_ranks(t, world).tolist())
     wall = time.perf_counter() - wall0
-    clocks = sampler.stop()
     counts = sb.profile_read()
-    gpu_launches = sum(v[2] for v in counts.values())
-    ms_prefix = sum(e[0].elapsed_time(e[1]) for e in ev)
-    ms_frames = sum(e[1].elapsed_time(e[2]) for e in ev)
-    ms_decode = sum(e[2].elapsed_time(e[3]) for e in ev)
-    times = torch.tensor([ms_prefix, ms_frames, ms_decode], dtype=torch.float64, device=dev)
-    ms_prefix, ms_frames, ms_decode = max_over_ranks(times, world).tolist()
+    gpu_launches = sum(v[2] for v in counts.values()) // REPEATS      # of one block of --steps steps
+    blocks.sort(key=lambda b: b[1])
+    ms_prefix, ms_frames, ms_decode = blocks[len(blocks) // 2]
     fps = replica_throughput(world, args.steps * w.n_frames, ms_frames)
     tps = replica_throughput(world, args.steps * w.decode_tokens, ms_decode) if w.decode_tokens else 0.0
 
@@ -314,15 +372,15 @@ def run_ours(args, w):
     if w.n_frames % CHUNK_FRAMES == 0:
         out_chunk = torch.empty((CHUNK_FRAMES, N + 1, HD), dtype=torch.float32, device=dev)
         p_out_chunk = C.c_void_p(out_chunk.data_ptr())
-        chunk_ptrs = [C.c_void_p(frames[t].data_ptr()) for t in range(0, w.n_frames, CHUNK_FRAMES)]
+        chunk_ptrs = [C.c_void_p(S.frames[t].data_ptr()) for t in range(0, w.n_frames, CHUNK_FRAMES)]
 
         def chunk_step(e0=None, e1=None):
-            ck(lib.vs_reset_stream(h, ids, 1, sptr))
+            S.reset()
             if w.prefix_len:
-                ck(lib.vs_decode_step(h, ids, 1, p_prefix, w.prefix_len, p_out_prefix, sptr))
+                S.text(S.prefix, w.prefix_len)
             if e0: e0.record(stream)
             for cp in chunk_ptrs:
-                ck(lib.vs_frame_prefill_chunk(h, 0, cp, CHUNK_FRAMES, N, p_out_chunk, sptr))
+                S.ck(lib.vs_frame_prefill_chunk(S.h, 0, cp, CHUNK_FRAMES, N, p_out_chunk, S.sptr))
             if e1: e1.record(stream)
 
         for _ in range(3):
@@ -345,17 +403,17 @@ def run_ours(args, w):
     one_step(on_phase=lambda name: per_phase.__setitem__(name, sb.profile_read()))
     sb.profile_enable(False)
 
+    # ---- deep leg: the 28-layer stack, where the weights (925 MB per pass) come from HBM -------
+    deep = None
+    if not args.no_deep and w.name == "layer":
+        deep = run_deep_leg(args, dev, local, lib, binding, torch, flush, barrier, world)
+    clocks = sampler.stop()
+
     result = None
     if rank == 0:
         peaks = load_peaks()
-        fr = per_phase["frames"]
-        kernels = {k: {"launches": v[1], "total_ms": round(v[0], 4), "avg_us": round(1e3 * v[0] / v[1], 3)}
-                   for k, v in fr.items() if v[1]}
-        tot = sum(v["total_ms"] for v in kernels.values())
-        for v in kernels.values():
-            v["share"] = round(v["total_ms"] / tot, 4)
-        kernels_dec = {k: {"launches": v[1], "total_ms": round(v[0], 4), "avg_us": round(1e3 * v[0] / v[1], 3)}
-                       for k, v in per_phase["decode"].items() if v[1]}
+        kernels = kernel_table(per_phase["frames"])
+        kernels_dec = kernel_table(per_phase["decode"])
         dom = max(kernels, key=lambda k: kernels[k]["total_ms"])
         proj_flops, _ = frame_flops(w, 0)
         avg_bank = (min(w.n_frames, w.bank_capacity) - 1) / 2.0 if w.bank_capacity else 0.0
@@ -364,12 +422,12 @@ def run_ours(args, w):
             ach = proj_flops / (kernels[dom]["avg_us"] * 1e-6) / 1e12
             roof = {"kernel": dom, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
                     "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
-                    # dram__bytes_read.sum + dram__bytes_write.sum of one frame launch of this kernel
-                    # (cold cache, so the weights come from DRAM), from the ncu capture summarised in
-                    # profiles/qkv_gemm_frame_170rows.md; only quoted for the shape that was captured
-                    "traffic": GEMM_FRAME_DRAM_BYTES if (N, d, w.e_out) == (169, 3584, 4608) else None,
-                    "peak_source": peaks["source"] + " (sustained bf16; kernel timed inside the step)",
-                    "avg_launch_us": kernels[dom]["avg_us"]}
+                    "peak_burst": peaks["bf16_tflops"], "frac_of_burst": ach / peaks["bf16_tflops"],
+                    "traffic": DOMINANT_KERNEL_TRAFFIC.get("bytes") if (N, d, w.e_out) == (169, 3584, 4608) else None,
+                    "traffic_source": DOMINANT_KERNEL_TRAFFIC.get("source"),
+                    "peak_source": peaks["source"] + ": sustained bf16 figure (the kernel is timed inside a long step, "
+                                   "tens of thousands of launches back to back); the burst figure is quoted beside it",
+                    "flops_per_launch": proj_flops, "avg_launch_us": kernels[dom]["avg_us"]}
         else:
             # every other kernel of the frame step moves bytes: report against HBM
             rows = N + 1
@@ -379,41 +437,56 @@ def run_ours(args, w):
             ach = alg / (kernels[dom]["avg_us"] * 1e-6) / 1e9
             roof = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
-                    "avg_launch_us": kernels[dom]["avg_us"]}
+                    "bytes_per_launch": alg, "avg_launch_us": kernels[dom]["avg_us"]}
         us_frame = 1e3 * ms_frames / (args.steps * w.n_frames)
-        ideal_c = (proj_flops + attn_flops) * w.n_layers / (peaks["bf16_tflops_sustained"] * 1e12) * 1e6
-        ideal_h = frame_bytes(w, avg_bank, 4, weights_from_hbm=w.n_layers > 1) / (peaks["hbm_gbs"] * 1e9) * 1e6
+        flops_frame = (proj_flops + attn_flops) * w.n_layers
+        bytes_frame = frame_bytes(w, avg_bank, 4, weights_from_hbm=w.n_layers > 1)
+        ideal_c = flops_frame / (peaks["bf16_tflops_sustained"] * 1e12) * 1e6
+        ideal_h = bytes_frame / (peaks["hbm_gbs"] * 1e9) * 1e6
         ideal = max(ideal_c, ideal_h)
         n_keys = w.prefix_len + min(w.n_frames, w.bank_capacity) + w.decode_tokens / 2.0
         us_tok = 1e3 * ms_decode / (args.steps * max(w.decode_tokens, 1))
-        dec_ideal = decode_bytes(w, n_keys, 4) * w.n_layers / (peaks["hbm_gbs"] * 1e9) * 1e6
+        bytes_tok = decode_bytes(w, n_keys, 4)
+        dec_ideal = bytes_tok / (peaks["hbm_gbs"] * 1e9) * 1e6
         result = {
             "metric": "streamed_frames_per_s", "value": fps, "unit": "frames/s",
             "decode_tokens_per_s": tps, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": (ms_prefix + ms_frames + ms_decode) / args.steps, "higher_is_better": True,
+            "repeats": REPEATS,
+            "ms_per_step": ms_prefix / args.steps + ms_frames / args.steps + ms_decode / args.steps,
+            "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": workload_config(w),
             "phase_ms_per_step": {"prefix": ms_prefix / args.steps, "frames": ms_frames / args.steps,
                                   "decode": ms_decode / args.steps},
+            "timing": f"median of {REPEATS} blocks of {args.steps} steps; frames-phase ms of every block: "
+                      + ", ".join("%.3f" % b[1] for b in blocks),
             "wall_s": wall, "clocks": clocks, "gpu_launches": gpu_launches,
             "roofline": roof, "kernels_frame_phase": kernels, "kernels_decode_phase": kernels_dec,
+            "kernels_note": "per-launch CUDA events (one extra pass): each pair adds a few microseconds and "
+                            "serialises launches that otherwise overlap, so the shares overstate the small kernels",
             "chunked_prefill": {"frames_per_call": CHUNK_FRAMES, "value": chunk_fps, "unit": "frames/s",
                                 "note": "same frames through vs_frame_prefill_chunk (offline form); not the headline"},
             "step_roofline": {
                 "frame": {"us_per_frame": us_frame, "ideal_us": ideal, "frac": ideal / us_frame,
+                          "flops_per_frame": flops_frame, "hbm_bytes_per_frame": bytes_frame,
                           "ideal_compute_us": ideal_c, "ideal_hbm_us": ideal_h,
+                          "peak_tflops": peaks["bf16_tflops_sustained"], "peak_gbs": peaks["hbm_gbs"],
                           "note": "ideal = max(flops / sustained bf16 peak, bytes / HBM peak); single-layer "
                                   "weights are L2-resident so they are not counted as HBM bytes"},
                 "decode": {"us_per_token": us_tok, "ideal_hbm_us": dec_ideal, "frac": dec_ideal / us_tok,
+                           "bytes_per_token": bytes_tok, "peak_gbs": peaks["hbm_gbs"],
                            "note": "bytes = weights + K/V + append; the weights are L2-resident in the "
-                                   "one-layer workload, so this fraction is not a DRAM fraction"}},
+                                   "one-layer workload, so this fraction is NOT a DRAM fraction: "
+                                   "step_roofline_deep.decode is"}},
         }
+        if deep is not None:
+            result["step_roofline_deep"] = deep_rooflines(deep, peaks)
 
     # ---- end to end: host inputs, H2D + D2H inside the timed region ---------------------------
     # Three streams, two buffers each way: the copy of frame t+1 to the device and the copy of
     # frame t-1's output back overlap the kernels of frame t, as a caller that streams video would
     # arrange it (the library only sees the stream it is given).
-    pin_frames = torch.from_numpy(frames_host.view(np.int16)).pin_memory()
+    pin_frames = torch.from_numpy(S.frames_host.view(np.int16)).pin_memory()
     pin_out = [torch.empty((N + 1, HD), dtype=torch.float32).pin_memory() for _ in range(2)]
     dev_in = [torch.empty((N, d), dtype=torch.int16, device=dev) for _ in range(2)]
     dev_out = [torch.empty((N + 1, HD), dtype=torch.float32, device=dev) for _ in range(2)]
@@ -425,9 +498,9 @@ def run_ours(args, w):
     ev_out = [torch.cuda.Event() for _ in range(2)]     # dev_out[k] copied back
 
     def e2e_step():
-        ck(lib.vs_reset_stream(h, ids, 1, sptr))
+        S.reset()
         if w.prefix_len:
-            ck(lib.vs_decode_step(h, ids, 1, p_prefix, w.prefix_len, p_out_prefix, sptr))
+            S.text(S.prefix, w.prefix_len)
         for t in range(w.n_frames):
             k = t & 1
             with torch.cuda.stream(s_in):
@@ -438,7 +511,7 @@ def run_ours(args, w):
             stream.wait_event(ev_in[k])
             if t >= 2:
                 stream.wait_event(ev_out[k])             # dev_out[k] is free again
-            ck(lib.vs_frame_prefill(h, ids, 1, p_dev_in[k], N, None, p_dev_out[k], sptr))
+            S.ck(lib.vs_frame_prefill(S.h, S.ids, 1, p_dev_in[k], N, None, p_dev_out[k], S.sptr))
             ev_done[k].record(stream)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_done[k])
@@ -472,13 +545,115 @@ def run_ours(args, w):
             fps_cpu = reps / inv_f
             tps_cpu = reps / inv_t if inv_t else 0.0
             result["cpu_baseline"] = {"value": fps_cpu, "unit": "frames/s", "decode_tokens_per_s": tps_cpu,
-                                      "cores": blas_threads(), "kind": "oracle", "seconds": secs,
+                                      "cores": blas_threads(), "kind": ORACLE_KIND, "seconds": secs,
                                       "sample": f"{reps} x ({w.prefix_len}-token prefix, {n_frames} frames and "
                                                 f"{n_decode} decode tokens): the same workload, whole"}
         print(json.dumps(result))
     sb.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_deep_leg(args, dev, local, lib, binding, torch, flush, barrier, world):
+    """The 28-layer workload at its stated size, end of the stream: the bank is filled by the first
+    512 - DEEP_TIMED_FRAMES frames outside the timed region, then the last DEEP_TIMED_FRAMES frames
+    are timed (bank 496 .. 511 carriers), the 32-token question is prefilled (untimed) and
+    DEEP_TIMED_DECODE single-token steps are timed over [64-token prefix | 512 carriers | text]."""
+    wd = synth.workload("deep")
+    D = Streamer(wd, dev, local, lib, binding, torch)
+    F0 = wd.n_frames - DEEP_TIMED_FRAMES
+    n_dec = min(DEEP_TIMED_DECODE, wd.decode_tokens)
+
+    def pass_(ev=None):
+        D.reset()
+        D.text(D.prefix, wd.prefix_len)
+        D.frames_range(0, F0)
+        flush.zero_()
+        if ev: ev[0].record(D.stream)
+        D.frames_range(F0, wd.n_frames)
+        if ev: ev[1].record(D.stream)
+        D.text(D.question, wd.question_len)
+        flush.zero_()
+        if ev: ev[2].record(D.stream)
+        D.decode_range(0, n_dec)
+        if ev: ev[3].record(D.stream)
+        D.end_turn()
+
+    pass_()                                                    # warm-up (every kernel has run before)
+    D.sb.profile_read()
+    reps = []
+    for _ in range(REPEATS):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        barrier()
+        pass_(ev)
+        barrier()
+        t = torch.tensor([ev[0].elapsed_time(ev[1]), ev[2].elapsed_time(ev[3])], dtype=torch.float64, device=dev)
+        reps.append(max_over_ranks(t, world).tolist())
+    counts = D.sb.profile_read()
+    # per-kernel times of the timed parts, one extra pass with events around every launch
+    D.reset(); D.text(D.prefix, wd.prefix_len); D.frames_range(0, F0)
+    D.sb.profile_read()
+    D.sb.profile_enable(True, wd.n_layers * 4 * (DEEP_TIMED_FRAMES + n_dec + 2) + 64)
+    D.frames_range(F0, wd.n_frames)
+    k_frames = D.sb.profile_read()
+    D.text(D.question, wd.question_len)
+    D.sb.profile_read()
+    D.decode_range(0, n_dec)
+    k_dec = D.sb.profile_read()
+    D.sb.profile_enable(False)
+    D.end_turn()
+    ms_f = sorted(r[0] for r in reps)[len(reps) // 2]
+    ms_d = sorted(r[1] for r in reps)[len(reps) // 2]
+    out = dict(w=wd, ms_frames=ms_f, ms_decode=ms_d, n_frames=DEEP_TIMED_FRAMES, n_decode=n_dec, F0=F0,
+               all_ms_frames=[r[0] for r in reps], all_ms_decode=[r[1] for r in reps],
+               kernels_frames=kernel_table(k_frames), kernels_decode=kernel_table(k_dec),
+               launches=sum(v[2] for v in counts.values()) // REPEATS, world=world)
+    D.sb.close()
+    return out
+
+
+def deep_rooflines(deep, peaks):
+    wd = deep["w"]
+    L = wd.n_layers
+    n_bank = deep["F0"] + (deep["n_frames"] - 1) / 2.0                     # carriers on the key axis of a timed frame
+    proj, attn = frame_flops(wd, n_bank)
+    flops = (proj + attn) * L
+    rows = wd.tokens_per_frame + 1
+    kv_row = 2 * wd.n_kv_heads * wd.head_dim * 2                           # K + V bytes of one key, one layer
+    b_frame = (L * wd.e_out * wd.d_model * 2                               # every layer's weights
+               + L * (wd.prefix_len + n_bank) * kv_row                     # prefix + bank K/V read per layer
+               + L * kv_row + wd.d_model * 2                               # carrier K/V per layer + embedding
+               + wd.tokens_per_frame * wd.d_model * 2                      # hidden in
+               + rows * wd.n_q_heads * wd.head_dim * 4)                    # last layer's output (fp32)
+    us_frame = 1e3 * deep["ms_frames"] / deep["n_frames"]
+    ideal_c = flops / (peaks["bf16_tflops_sustained"] * 1e12) * 1e6
+    ideal_h = b_frame / (peaks["hbm_gbs"] * 1e9) * 1e6
+    n_keys = wd.prefix_len + wd.bank_capacity + wd.question_len + (deep["n_decode"] + 1) / 2.0
+    b_tok = (L * wd.e_out * wd.d_model * 2 + L * n_keys * kv_row + L * kv_row
+             + wd.d_model * 2 + wd.n_q_heads * wd.head_dim * 4)
+    us_tok = 1e3 * deep["ms_decode"] / deep["n_decode"]
+    ideal_t = b_tok / (peaks["hbm_gbs"] * 1e9) * 1e6
+    return {
+        "workload": f"deep: {L} layers (RMSNorm, residual, no MLP), d={wd.d_model}, {wd.n_q_heads}/{wd.n_kv_heads} heads x "
+                    f"{wd.head_dim}, {wd.prefix_len}-token prefix, bank {wd.bank_capacity}; frames 0..{deep['F0'] - 1} "
+                    f"of the {wd.n_frames}-frame stream fill the bank outside the timed region; timed: frames "
+                    f"{deep['F0']}..{wd.n_frames - 1}, then (after the untimed {wd.question_len}-token question) "
+                    f"{deep['n_decode']} single-token decode steps; median of {REPEATS} passes; L2 flushed before "
+                    f"each timed part (925 MB of weights per pass do not fit in L2 anyway)",
+        "frame": {"us_per_frame": us_frame, "frames_per_s": deep["world"] * 1e6 / us_frame,
+                  "us_per_layer": us_frame / L, "ideal_us": max(ideal_c, ideal_h),
+                  "frac": max(ideal_c, ideal_h) / us_frame, "ideal_compute_us": ideal_c, "ideal_hbm_us": ideal_h,
+                  "flops_per_frame": flops, "hbm_bytes_per_frame": b_frame,
+                  "peak_tflops": peaks["bf16_tflops_sustained"], "peak_gbs": peaks["hbm_gbs"],
+                  "ms_all_passes": deep["all_ms_frames"]},
+        "decode": {"us_per_token": us_tok, "tokens_per_s": deep["world"] * 1e6 / us_tok, "us_per_layer": us_tok / L,
+                   "ideal_hbm_us": ideal_t, "frac": ideal_t / us_tok,
+                   "achieved_gbs": b_tok / (us_tok * 1e-6) / 1e9, "bytes_per_token": b_tok, "peak_gbs": peaks["hbm_gbs"],
+                   "ms_all_passes": deep["all_ms_decode"],
+                   "note": "a DRAM fraction: bytes = every layer's weights + K/V of all keys + append + hidden"},
+        "kernels_frame_phase": deep["kernels_frames"], "kernels_decode_phase": deep["kernels_decode"],
+        "gpu_launches": deep["launches"],
+    }
 
 
 def main():
@@ -490,6 +665,7 @@ def main():
     ap.add_argument("--workload", default="layer")
     ap.add_argument("--frames", type=int, default=None, help="override the number of frames (exploration only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-deep", action="store_true", help="skip the 28-layer leg")
     args = ap.parse_args()
     kw = {}
     if args.frames:

@@ -63,4 +63,4 @@ def test_reference_arm_prints_on_rank_zero_only():
     assert len(lines0) == 1 and res[1][1].strip() == ""
     rec = json.loads(lines0[0])
     assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["value"] > 0
-    assert rec["cpu_baseline"]["kind"] == "oracle" and rec["e2e"]["h2d_bytes_per_step"] == 0
+    assert rec["cpu_baseline"]["kind"].startswith("oracle") and rec["e2e"]["h2d_bytes_per_step"] == 0
