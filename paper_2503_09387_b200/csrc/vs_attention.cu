@@ -5,8 +5,11 @@
 // grid = (key splits, query heads, streams), 256 threads.  A group of D/8 lanes owns one key
 // row and reads it with 128-bit loads; every lane issues the K and V loads of eight keys before
 // it uses any of them, so a warp has 16 key rows (8 KB) in flight.  Warps merge their running
-// (m, l, o) by shuffles and through shared memory; with several key splits the last CTA of a
-// (stream, query head) to finish combines the partial triples -- no CTA ever waits for another.
+// (m, l, o) by shuffles and through shared memory.  The key splits of one (stream, query head)
+// form a thread-block cluster (1, 2, 4 or 8 CTAs): every CTA leaves its partial triple in its own
+// shared memory, the cluster's hardware barrier orders them, and rank 0 reads the peers' triples
+// through distributed shared memory and writes the row -- no global scratch, no atomics, no
+// polling; the co-scheduled cluster is what guarantees that the barrier completes.
 #include "vs_common.cuh"
 
 namespace vs {
@@ -16,6 +19,21 @@ namespace {
 constexpr int kDecThreads = 256;
 constexpr int kDecWarps = kDecThreads / 32;
 constexpr int kBatch = 8;     // keys a lane group loads before computing
+constexpr int kMaxCluster = 8;  // portable cluster size: most key splits of one (stream, query head)
+
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_shared_rank(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float ld_shared_cluster_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
 
 // One CTA = one query head x one key split x one stream.  The heads of a KV group read the
 // same K/V rows from L2; spreading them over CTAs keeps every SM's instruction stream short,
@@ -27,8 +45,8 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
   __shared__ float st_m[kDecWarps];
   __shared__ float st_l[kDecWarps];
   __shared__ float st_o[kDecWarps][D];
-  __shared__ float sp_w[DEC_SPLIT_MAX];
-  __shared__ int is_last;
+  __shared__ float cta_o[D];            // this CTA's partial triple, read by rank 0 of the cluster
+  __shared__ float cta_ml[2];
 
   // what follows from the parameters alone comes before the wait on the stream's earlier kernels
   const int split = blockIdx.x, qh = blockIdx.y, b = blockIdx.z;
@@ -85,6 +103,8 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
 
   pdl_wait();
   pdl_launch_dependents();
+  // the step's own key and the query are both fresh: their loads go out together
+  if (wbase0 < end) load_pass(wbase0, kr0, vr0, true);
 
   // this lane's 8 dims of the query (bf16 hi + lo pair), pre-scaled into the log2 domain
   float q[8];
@@ -143,10 +163,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
       }
     }
   };
-  if (wbase0 < end) {                                    // uniform over the warp
-    load_pass(wbase0, kr0, vr0, true);
-    compute_pass(wbase0, kr0, vr0);
-  }
+  if (wbase0 < end) compute_pass(wbase0, kr0, vr0);      // uniform over the warp
   for (int wbase = wbase0 + kBatch * kStride; wbase < end; wbase += kBatch * kStride) {
     uint4 kr[kBatch], vr[kBatch];
     load_pass(wbase, kr, vr, false);
@@ -179,8 +196,10 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
 
   // warps -> CTA
   const bool direct = a.nsplit == 1;
-  float* part = a.partials + (((size_t)split * bp.n_active + b) * a.Hq + qh) * (D + 2);
   const size_t out_off = (size_t)b * a.Hq * D + (size_t)qh * D;
+  // the residual input is needed by whoever writes the row: fetched ahead of the cluster barrier
+  float h_res = 0.f;
+  if (a.h_out != nullptr && split == 0 && threadIdx.x < D) h_res = __bfloat162float(a.h_in[out_off + threadIdx.x]);
   if (threadIdx.x < D) {
     const int c = threadIdx.x;
     float M = -INFINITY;
@@ -197,69 +216,69 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
       const float val = (L > 0.f) ? O / L : 0.f;
       if (a.out_fp32) static_cast<float*>(a.out)[out_off + c] = val;
       else static_cast<bf16*>(a.out)[out_off + c] = __float2bfloat16_rn(val);
-      if (a.h_out != nullptr) a.h_out[out_off + c] = __float2bfloat16_rn(__bfloat162float(a.h_in[out_off + c]) + val);
+      if (a.h_out != nullptr) a.h_out[out_off + c] = __float2bfloat16_rn(h_res + val);
     } else {
-      part[c] = O;
-      if (c == 0) { part[D] = M; part[D + 1] = L; }
+      cta_o[c] = O;
+      if (c == 0) { cta_ml[0] = M; cta_ml[1] = L; }
     }
   }
   if (direct) return;
 
-  // last CTA of this (stream, query head) combines the splits
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) is_last = (atomicAdd(a.tickets + sid * a.Hq + qh, 1) == a.nsplit - 1);
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-  if (threadIdx.x == 0) {
-    float ms[DEC_SPLIT_MAX], ls[DEC_SPLIT_MAX];
+  // the cluster's CTAs (the key splits of this stream and query head) meet; rank 0 combines
+  cluster_sync();
+  if (split == 0 && threadIdx.x < D) {
+    const int c = threadIdx.x;
+    const uint32_t ml_addr = static_cast<uint32_t>(__cvta_generic_to_shared(cta_ml));
+    const uint32_t o_addr = static_cast<uint32_t>(__cvta_generic_to_shared(cta_o + c));
+    float ms[kMaxCluster], ls[kMaxCluster], os[kMaxCluster];
+#pragma unroll
+    for (int r = 0; r < kMaxCluster; ++r) {
+      if (r < a.nsplit) {
+        const uint32_t rml = map_shared_rank(ml_addr, (uint32_t)r);
+        ms[r] = ld_shared_cluster_f32(rml);
+        ls[r] = ld_shared_cluster_f32(rml + 4);
+        os[r] = ld_shared_cluster_f32(map_shared_rank(o_addr, (uint32_t)r));
+      }
+    }
     float M = -INFINITY;
 #pragma unroll
-    for (int s2 = 0; s2 < DEC_SPLIT_MAX; ++s2) {
-      if (s2 < a.nsplit) {
-        const float* pp = a.partials + (((size_t)s2 * bp.n_active + b) * a.Hq + qh) * (D + 2);
-        ms[s2] = __ldcg(pp + D); ls[s2] = __ldcg(pp + D + 1);
-        M = fmaxf(M, ms[s2]);
+    for (int r = 0; r < kMaxCluster; ++r) if (r < a.nsplit) M = fmaxf(M, ms[r]);
+    float L = 0.f, val = 0.f;
+#pragma unroll
+    for (int r = 0; r < kMaxCluster; ++r) {
+      if (r < a.nsplit) {
+        const float wt = (ms[r] == -INFINITY) ? 0.f : exp2f(ms[r] - M);
+        L = fmaf(ls[r], wt, L);
+        val = fmaf(os[r], wt, val);
       }
     }
-    float L = 0.f;
-#pragma unroll
-    for (int s2 = 0; s2 < DEC_SPLIT_MAX; ++s2) {
-      if (s2 < a.nsplit) {
-        const float wt = (ms[s2] == -INFINITY) ? 0.f : exp2f(ms[s2] - M);
-        L += ls[s2] * wt;
-        sp_w[s2] = wt;
-      }
-    }
-    const float inv = (L > 0.f) ? 1.f / L : 0.f;
-#pragma unroll
-    for (int s2 = 0; s2 < DEC_SPLIT_MAX; ++s2) if (s2 < a.nsplit) sp_w[s2] *= inv;
-  }
-  __syncthreads();
-  if (threadIdx.x < D) {
-    const int c = threadIdx.x;
-    float v[DEC_SPLIT_MAX];
-#pragma unroll
-    for (int s2 = 0; s2 < DEC_SPLIT_MAX; ++s2)
-      v[s2] = (s2 < a.nsplit) ? __ldcg(a.partials + (((size_t)s2 * bp.n_active + b) * a.Hq + qh) * (D + 2) + c) : 0.f;
-    float val = 0.f;
-#pragma unroll
-    for (int s2 = 0; s2 < DEC_SPLIT_MAX; ++s2) if (s2 < a.nsplit) val = fmaf(v[s2], sp_w[s2], val);
+    val = (L > 0.f) ? val / L : 0.f;
     if (a.out_fp32) static_cast<float*>(a.out)[out_off + c] = val;
     else static_cast<bf16*>(a.out)[out_off + c] = __float2bfloat16_rn(val);
-    if (a.h_out != nullptr) a.h_out[out_off + c] = __float2bfloat16_rn(__bfloat162float(a.h_in[out_off + c]) + val);
+    if (a.h_out != nullptr) a.h_out[out_off + c] = __float2bfloat16_rn(h_res + val);
   }
-  if (threadIdx.x == 0) a.tickets[sid * a.Hq + qh] = 0;
+  // nobody's shared memory goes away while rank 0 may still be reading it
+  cluster_sync();
 }
 
 }  // namespace
 
 cudaError_t launch_decode_attention(const DecodeArgs& a, const BatchParams& bp, cudaStream_t st) {
-  if (a.nsplit < 1 || a.nsplit > DEC_SPLIT_MAX) return cudaErrorInvalidValue;
-  dim3 grid(a.nsplit, a.Hq, bp.n_active);
-  if (a.D == 128) return launch_pdl(decode_attn_kernel<128>, grid, dim3(kDecThreads), 0, st, a, bp);
-  if (a.D == 64) return launch_pdl(decode_attn_kernel<64>, grid, dim3(kDecThreads), 0, st, a, bp);
+  if (a.nsplit != 1 && a.nsplit != 2 && a.nsplit != 4 && a.nsplit != 8) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(a.nsplit, a.Hq, bp.n_active);
+  cfg.blockDim = dim3(kDecThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;            // the key splits of a row are one cluster
+  attr[1].val.clusterDim.x = a.nsplit; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  if (a.D == 128) return cudaLaunchKernelEx(&cfg, decode_attn_kernel<128>, a, bp);
+  if (a.D == 64) return cudaLaunchKernelEx(&cfg, decode_attn_kernel<64>, a, bp);
   return cudaErrorInvalidValue;
 }
 

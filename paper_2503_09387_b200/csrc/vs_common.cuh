@@ -52,7 +52,7 @@ struct Dims {
 };
 
 constexpr int KSPLIT_MAX = 4;   // CTAs sharing one output tile of the projection along K
-constexpr int DEC_SPLIT_MAX = 16;
+constexpr int DEC_SPLIT_MAX = 8;      // key splits of the decode attention = CTAs of one cluster
 constexpr int GEMM_BLOCK_M = 128;
 constexpr int GEMM_BLOCK_K = 64;
 constexpr int GEMM_XCHG_CTAS = 160;   // most CTAs a K-split projection launches (one per SM)
@@ -75,7 +75,6 @@ struct Layout {
   size_t step_slot;             // int32 [S]  free slot as the running frame step found it
   size_t chunk_slot;            // int32 [VS_MAX_BATCH]  chunked prefill: slot each frame's carrier went to
   size_t chunk_victim;          // int32 [VS_MAX_BATCH]  ... and whom its bank update evicted (index on the bank axis)
-  size_t tickets;               // int32 [S*Hq]  split-KV decode: CTAs finished per (stream, query head)
   size_t gemm_flags;            // int32 [GEMM_XCHG_CTAS]  projection K split: partials delivered per slice owner
   size_t persistent_end;
   // per-step scratch
@@ -87,7 +86,6 @@ struct Layout {
   size_t kf, vf;                // bf16 [R_max][Hkv*D]
   size_t rope;                  // float2 [R_max][D/2]
   size_t obuf;                  // f32  [R_max][Hq*D] (holds bf16 or fp32 rows)
-  size_t dec_part;              // f32  [DEC_SPLIT_MAX][S][Hq][D+2]
   size_t emb_stage;             // bf16 [max_chunk][d]  chunked prefill: carrier embeddings before they have a slot
   size_t chunk_scores;          // f64  [max_chunk][slots + max_chunk]  chunked prefill: cosines of (frame, candidate) pairs
   size_t gemm_xchg;             // f32  [GEMM_XCHG_CTAS][256][128]  projection K split: partial tiles
@@ -112,6 +110,12 @@ struct Layout {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Asks the memory system to bring [p, p + bytes) into L2 (no destination, no completion to wait
+// for).  p 16-byte aligned, bytes a multiple of 16.  Used for weight rows: the matrices are
+// constant, so the request needs no ordering with any other kernel.
+__device__ __forceinline__ void prefetch_l2_bulk(const void* p, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
   cudaLaunchConfig_t cfg = {};
@@ -190,7 +194,8 @@ cudaError_t qkv_gemm_init();     // opt-in shared memory attribute, once per pro
 bool qkv_gemv_supported(const ProjectionOut& o, int rows, int d);
 cudaError_t qkv_gemv_init();     // opt-in shared memory attribute, once per process/device
 cudaError_t launch_qkv_gemv(const bf16* W, const bf16* x, const ProjectionOut& o, const BatchParams& bp, int rows, int E_out,
-                            int d, cudaStream_t st);
+                            int d, bool l2_ahead, cudaStream_t st);   // l2_ahead: the matrix comes from HBM (several layers): ask for
+                                                                       // all of it before the wait on the stream's earlier kernels
 
 struct BankUpdateArgs {
   const bf16* emb;               // [S][slots][d]
@@ -270,13 +275,12 @@ struct DecodeArgs {
   const bf16* prefix_k; const bf16* prefix_v;  // layer base [S][Hkv][maxP][D]
   const bf16* bank_k;   const bf16* bank_v;    // [S][Hkv][slots][D]
   const bf16* tail_k;   const bf16* tail_v;    // [S][Hkv][maxT][D]
-  float* partials;               // [nsplit][n_active][Hq][D+2]
-  int* tickets;                  // [S*Hq]
   void* out;                     // [n_active][Hq*D], bf16 or fp32
   int out_fp32;
   const bf16* h_in; bf16* h_out;
   const StreamMeta* meta;
-  int Hq, Hkv, D, slots, M, maxP, maxT, nsplit;
+  int Hq, Hkv, D, slots, M, maxP, maxT;
+  int nsplit;                    // CTAs sharing one row's keys (a cluster): 1, 2, 4 or 8
   int to_prefix;                 // 1: the keys are the prefix alone (incl. the new token)
   float scale_log2e;
 };

@@ -47,7 +47,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 
 template <int R>   // token rows held (1, 2 or 4)
 __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __restrict__ W, const bf16* __restrict__ x,
-                                                            ProjectionOut o, BatchParams bp, int rows, int d) {
+                                                            ProjectionOut o, BatchParams bp, int rows, int d, int l2_ahead) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   // carve: ring [kStages][32 rows][512 B] | token rows [R][d] bf16 | results [R][32] | row scales [R] | partial sums [R][8]
   uint4* xs = reinterpret_cast<uint4*>(smem_raw + kStages * kStageBytes);
@@ -86,6 +86,14 @@ __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __res
     cp_async_commit();                                                  // one group per stage, empty or not
   };
   for (int i = 0; i < kStages - 1; ++i) issue_stage(i);                 // W is constant: no need to wait for it
+  // what the ring cannot hold yet of this CTA's 32 rows (a contiguous piece of each row) is asked
+  // into L2 now, so that all of the layer's matrix is on its way from HBM while the kernel ahead
+  // of this one -- the attention of the layer before -- still runs
+  if (l2_ahead && tid < kRowsPerCta && n_stage_total > kStages - 1) {
+    const int f = hs * D + pb * 16 + (tid & 15) + (tid >> 4) * half;
+    prefetch_l2_bulk(W + (size_t)f * d + (size_t)(kStages - 1) * kStageElems,
+                     (uint32_t)(n_stage_total - (kStages - 1)) * kStageElems * 2);
+  }
 
   // finishing threads: (token row r, pair p); the rotation depends on the parameters alone
   const int fr = tid >> 4, fp = tid & 15;
@@ -238,14 +246,15 @@ cudaError_t qkv_gemv_init() {
 }
 
 cudaError_t launch_qkv_gemv(const bf16* W, const bf16* x, const ProjectionOut& o, const BatchParams& bp, int rows, int E_out,
-                            int d, cudaStream_t st) {
+                            int d, bool l2_ahead, cudaStream_t st) {
   if (!qkv_gemv_supported(o, rows, d) || o.inv_freq == nullptr) return cudaErrorInvalidValue;
   const dim3 grid((E_out / o.D) * ((o.D / 2) / 16));
   const int R = rows == 1 ? 1 : (rows == 2 ? 2 : 4);
   const size_t smem = gemv_smem_bytes(R, d);
-  if (R == 1) return launch_pdl(qkv_gemv_kernel<1>, grid, dim3(kThreads), smem, st, W, x, o, bp, rows, d);
-  if (R == 2) return launch_pdl(qkv_gemv_kernel<2>, grid, dim3(kThreads), smem, st, W, x, o, bp, rows, d);
-  return launch_pdl(qkv_gemv_kernel<4>, grid, dim3(kThreads), smem, st, W, x, o, bp, rows, d);
+  const int ahead = l2_ahead ? 1 : 0;
+  if (R == 1) return launch_pdl(qkv_gemv_kernel<1>, grid, dim3(kThreads), smem, st, W, x, o, bp, rows, d, ahead);
+  if (R == 2) return launch_pdl(qkv_gemv_kernel<2>, grid, dim3(kThreads), smem, st, W, x, o, bp, rows, d, ahead);
+  return launch_pdl(qkv_gemv_kernel<4>, grid, dim3(kThreads), smem, st, W, x, o, bp, rows, d, ahead);
 }
 
 }  // namespace vs

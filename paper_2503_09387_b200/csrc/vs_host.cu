@@ -81,7 +81,6 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.step_slot = take((size_t)D.S * 4);
   Lo.chunk_slot = take((size_t)VS_MAX_BATCH * 4);
   Lo.chunk_victim = take((size_t)VS_MAX_BATCH * 4);
-  Lo.tickets = take((size_t)D.S * D.Hq * 4);
   Lo.gemm_flags = take((size_t)GEMM_XCHG_CTAS * 4);
   Lo.persistent_end = off;
   Lo.scratch_begin = off;
@@ -95,7 +94,6 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.vf = take((size_t)D.R_max * D.Hkv * D.D * 2);
   Lo.rope = take((size_t)D.R_max * (D.D / 2) * 8);
   Lo.obuf = take((size_t)D.R_max * D.Hq * D.D * 4);
-  Lo.dec_part = take((size_t)DEC_SPLIT_MAX * D.S * D.Hq * (D.D + 2) * 4);
   Lo.emb_stage = take((size_t)D.maxChunk * D.d * 2);
   Lo.chunk_scores = take(D.maxChunk > 1 ? (size_t)D.maxChunk * (D.slots + D.maxChunk) * 8 : 8);
   Lo.gemm_xchg = take((size_t)GEMM_XCHG_CTAS * 256 * GEMM_BLOCK_M * 4);
@@ -209,7 +207,7 @@ int run_projection(vs_stream* h, int l, const bf16* src, int rows, const Project
   const Dims& D = h->dm;
   if (po.rope == nullptr && qkv_gemv_supported(po, rows, D.d) && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
     // a text step of a few rows: bound by reading W once, done on the CUDA cores
-    VS_LAUNCH(h, st, KC_GEMV, launch_qkv_gemv(h->w[l], src, po, bp, rows, D.E_out, D.d, st));
+    VS_LAUNCH(h, st, KC_GEMV, launch_qkv_gemv(h->w[l], src, po, bp, rows, D.E_out, D.d, D.L > 1, st));
     return VS_OK;
   }
   GemmArgs g;
@@ -778,17 +776,16 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       DecodeArgs da;
       da.q = fa.q; da.q_lo = fa.q_lo;
       da.prefix_k = pk; da.prefix_v = pv; da.bank_k = bk; da.bank_v = bv; da.tail_k = tk; da.tail_v = tv;
-      da.partials = h->at<float>(lo.dec_part);
-      da.tickets = h->at<int>(lo.tickets);
       da.out = (l == D.L - 1) ? out : h->at<void>(lo.obuf);
       da.out_fp32 = D.out_fp32;
       da.h_in = D.residual ? h_in : nullptr; da.h_out = h_out;
       da.meta = meta;
       da.Hq = D.Hq; da.Hkv = D.Hkv; da.D = D.D; da.slots = D.slots; da.M = D.M; da.maxP = D.maxP; da.maxT = D.maxT;
-      // short contexts: one CTA per (stream, KV head) writes the result directly; longer ones are
-      // split so that a CTA walks about 128 keys
-      int ns = (max_keys <= 256) ? 1 : (max_keys + 127) / 128;
-      if (ns > DEC_SPLIT_MAX) ns = DEC_SPLIT_MAX;
+      // short contexts: one CTA per (stream, query head) writes the row directly; longer ones are
+      // split over a cluster of 2, 4 or 8 CTAs (a CTA then walks about 64 to 128 keys), fewer
+      // when many streams already fill the GPU
+      int ns = (max_keys <= 96) ? 1 : (max_keys <= 192 ? 2 : (max_keys <= 448 ? 4 : 8));
+      while (ns > 1 && (long long)ns * D.Hq * n_active > 4LL * h->n_sms) ns >>= 1;
       da.nsplit = ns;
       da.to_prefix = to_prefix ? 1 : 0;
       da.scale_log2e = scale_log2e;
