@@ -59,6 +59,17 @@ def assert_within_one_ulp(got_bits: np.ndarray, want_vals: np.ndarray, what: str
     assert frac < 0.05, f"{what}: {frac:.3%} of elements differ from the oracle's rounding"
 
 
+_WEIGHTS = {}
+
+
+def layer_weight(w: synth.Workload, layer: int) -> np.ndarray:
+    """w.weight(layer), kept for the session: the 28-layer workloads regenerate ~1 GB of weights per test otherwise."""
+    key = (w.seed, w.e_out, w.d_model, w.weight_std, layer)
+    if key not in _WEIGHTS:
+        _WEIGHTS[key] = w.weight(layer)
+    return _WEIGHTS[key]
+
+
 class Pair:
     """One workload run side by side: ``gpu`` (StreamBatch) and ``ora`` (one OracleStream per stream)."""
 
@@ -69,7 +80,7 @@ class Pair:
         self.w = w
         S = n_streams or w.n_streams
         self.S = S
-        wbits = [w.weight(l) for l in range(w.n_layers)]
+        wbits = [layer_weight(w, l) for l in range(w.n_layers)]
         bbits = [synth.normal_bf16(w.seed, synth.TAG_BIAS, (w.e_out,), 0.1, offset=l * w.e_out)
                  for l in range(w.n_layers)] if with_bias else None
         gbits = [synth.to_bf16_bits(1.0 + 0.1 * synth.standard_normal(w.seed, synth.TAG_NORM_W, w.d_model,
@@ -111,17 +122,19 @@ class Pair:
                 self._note(assert_close(got[i], want, f"{what} stream {sid}"))
         return got
 
-    def frame(self, ids: List[int], bits: List[np.ndarray], what: str = "frame", mode: str = "full",
+    def frame(self, ids: List[int], bits: List[np.ndarray], what: str = "frame", mode="full",
               override: Optional[List[np.ndarray]] = None):
-        """bits[i]: [N, d].  mode: 'full' compares outputs; 'carrier' / 'meta' only advance the oracle."""
+        """bits[i]: [N, d].  mode: 'full' compares outputs; 'carrier' / 'meta' only advance the oracle.
+        A list gives every listed stream its own mode."""
+        modes = [mode] * len(ids) if isinstance(mode, str) else list(mode)
         x = to_dev(np.stack(bits))
         ov = to_dev(np.stack(override)) if override is not None else None
-        out = self.gpu.frame_prefill(ids, x, carrier_override=ov, want_out=(mode == "full"))
+        out = self.gpu.frame_prefill(ids, x, carrier_override=ov, want_out=("full" in modes))
         got = to_f64(out) if out is not None else None
         for i, sid in enumerate(ids):
             o = synth.bf16_bits_to_f64(override[i]) if override is not None else None
-            want = self.ora[sid].frame_step(synth.bf16_bits_to_f64(bits[i]), carrier_override=o, mode=mode)
-            if mode == "full":
+            want = self.ora[sid].frame_step(synth.bf16_bits_to_f64(bits[i]), carrier_override=o, mode=modes[i])
+            if modes[i] == "full":
                 self._note(assert_close(got[i], want, f"{what} stream {sid}"))
         return got
 

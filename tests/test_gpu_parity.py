@@ -388,98 +388,212 @@ def test_long_stream_full_size_sampled():
 # Chained layers.  Both sides store the residual stream in bf16.  A difference of ~2e-3 in one
 # layer's attention output flips the bf16 rounding of h + O for roughly one element in eight
 # (spacing 1.6e-2 at |h| ~ 3), i.e. it injects noise of the size of one more bf16 rounding per
-# layer, which the next layer's logits (std ~ 19 with N(0, 0.02) weights) amplify.  The
-# per-operation tolerance therefore cannot hold for the 28th layer of a free-running chain; it is
-# checked layer by layer with the oracle's own layer inputs fed to a one-layer handle (below), and
-# the free-running chain gets the depth-scaled bound max |err| <= 2e-2 * sqrt(L), rel RMS <= 2e-2.
+# layer, which the next layer's logits (std ~ 19 with N(0, 0.02) weights) amplify.  Measured, the
+# stated per-operation tolerance (max |err| <= 2e-2, rel RMS <= 1e-2) FAILS on the last layers of
+# a free-running 28-layer chain and PASSES for every layer when the layer is given the oracle's
+# own bf16 input (teacher forcing; the residual stream is a storage point on both sides).  The
+# free-running chain is held to the depth-scaled bound max |err| <= 2e-2 * sqrt(L), rel RMS
+# <= 2e-2, a second, weaker figure, and each test prints whether the stated one held.
 def chain_bounds(n_layers):
     return 2e-2 * np.sqrt(n_layers), 2e-2
 
 
-def run_chain(w, max_text):
-    """Free-running multi-layer stream on both sides; returns the oracle's per-layer record."""
+class TeacherForced:
+    """One one-layer handle per layer of a stack, each holding that layer's weights and state
+    (prefix, bank, tail).  Fed the oracle's recorded bf16 layer inputs step by step, so that every
+    layer is compared at the stated tolerance on the inputs the oracle itself saw."""
+
+    def __init__(self, w, weights_dev):
+        self.w = w
+        cfg = binding.make_config(1, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens_per_frame,
+                                  max(w.prefix_len, 1), max(w.question_len + w.decode_tokens, 1), w.bank_capacity,
+                                  use_rmsnorm=w.use_rmsnorm, residual=w.residual, rope_theta=w.rope_theta,
+                                  rms_eps=w.rms_eps)
+        self.sb = [binding.StreamBatch(cfg, [weights_dev[l]]) for l in range(w.n_layers)]
+        self.worst = [[0.0, 0.0] for _ in range(w.n_layers)]
+
+    def step(self, rec, what):
+        from oracle import videoscan_oracle as vo
+        for layer, sb in enumerate(self.sb):
+            h = vo.bf16_bits_of(rec["h"][layer])
+            if rec["kind"] == "text":
+                got = to_f64(sb.decode_step([0], to_dev(h[None])))[0]
+            else:
+                got = to_f64(sb.frame_prefill([0], to_dev(h[None, :-1]), carrier_override=to_dev(h[None, -1])))[0]
+            e = assert_close(got, rec["O"][layer], f"teacher-forced layer {layer}, {what}")
+            self.worst[layer] = [max(self.worst[layer][0], e[0]), max(self.worst[layer][1], e[1])]
+
+    def close(self):
+        for sb in self.sb:
+            sb.close()
+
+
+def run_chain(w, max_text, teacher=False, bank_layers=None):
+    """Free-running multi-layer stream on both sides (depth-scaled bound); with teacher=True every
+    layer is also run teacher-forced at the stated tolerance.  Returns (worst of the chain, whether
+    the chain met the stated tolerance, per-layer worst of the teacher-forced runs)."""
     from tests import parity
     p = Pair(w, max_text=max_text)
     p.ora[0].record = []
-    saved = (parity.MAX_ABS, parity.REL_RMS)
+    tf = TeacherForced(w, p.gpu.weights) if teacher else None
+    strict = (parity.MAX_ABS, parity.REL_RMS)
+
+    def both(fn, what):
+        parity.MAX_ABS, parity.REL_RMS = chain_bounds(w.n_layers)
+        try:
+            fn()
+        finally:
+            parity.MAX_ABS, parity.REL_RMS = strict
+        rec = p.ora[0].record.pop()
+        if tf is not None:
+            tf.step(rec, what)
+
+    both(lambda: p.text([0], [w.prefix_hidden()], "prefix"), "prefix")
+    shared = w.frame_shared()
+    for t in range(w.n_frames):
+        x = w.frame_hidden(t, shared=shared)
+        both(lambda: p.frame([0], [x], f"frame {t}"), f"frame {t}")
+    if w.question_len:
+        both(lambda: p.text([0], [w.question_hidden()], "question"), "question")
+    for i in range(w.decode_tokens):
+        both(lambda: p.text([0], [w.decode_hidden(i)], f"decode {i}"), f"decode {i}")
     parity.MAX_ABS, parity.REL_RMS = chain_bounds(w.n_layers)
     try:
-        steps = [("text", w.prefix_hidden(), None)]
-        p.text([0], [w.prefix_hidden()], "prefix")
-        shared = w.frame_shared()
-        for t in range(w.n_frames):
-            x = w.frame_hidden(t, shared=shared)
-            p.frame([0], [x], f"frame {t}")
-        if w.question_len:
-            p.text([0], [w.question_hidden()], "question")
-        for i in range(w.decode_tokens):
-            p.text([0], [w.decode_hidden(i)], f"decode {i}")
-        for layer in sorted({0, w.n_layers // 2, w.n_layers - 1}):
+        for layer in (bank_layers if bank_layers is not None else sorted({0, w.n_layers // 2, w.n_layers - 1})):
             p.check_bank(0, layer=layer)
     finally:
-        parity.MAX_ABS, parity.REL_RMS = saved
-    rec = p.ora[0].record
+        parity.MAX_ABS, parity.REL_RMS = strict
     worst = list(p.worst)
+    met = worst[0] <= strict[0] and worst[1] <= strict[1]
+    per_layer = tf.worst if tf is not None else None
+    if tf is not None:
+        tf.close()
     p.close()
-    return rec, worst
+    return worst, met, per_layer
 
 
-def teacher_forced_layer(w, layer, rec):
-    """One-layer handle holding layer `layer`'s weights, fed the oracle's inputs of that layer
-    (bf16 values: the residual stream is a storage point); outputs must meet the strict tolerance."""
-    from oracle import videoscan_oracle as vo
-    w1 = synth.workload(w.name, n_layers=1, n_frames=w.n_frames, decode_tokens=w.decode_tokens,
-                        question_len=w.question_len, tokens_per_frame=w.tokens_per_frame, d_model=w.d_model,
-                        n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
-                        bank_capacity=w.bank_capacity, prefix_len=w.prefix_len, seed=w.seed)
-    cfg = binding.make_config(1, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens_per_frame,
-                              max(w.prefix_len, 1), max(w.question_len + w.decode_tokens, 1), w.bank_capacity,
-                              use_rmsnorm=w.use_rmsnorm, residual=w.residual, rope_theta=w.rope_theta,
-                              rms_eps=w.rms_eps)
-    sb = binding.StreamBatch(cfg, [to_dev(w.weight(layer))])
-    worst = [0.0, 0.0]
-    for i, r in enumerate(rec):
-        h = vo.bf16_bits_of(r["h"][layer])
-        if r["kind"] == "text":
-            got = to_f64(sb.decode_step([0], to_dev(h[None])))[0]
-        else:
-            got = to_f64(sb.frame_prefill([0], to_dev(h[None, :-1]), carrier_override=to_dev(h[None, -1])))[0]
-        e = assert_close(got, r["O"][layer], f"layer {layer} step {i} ({r['kind']})")
-        worst = [max(worst[0], e[0]), max(worst[1], e[1])]
-    sb.close()
-    return worst
+def test_deep_stack_first_16_frames_every_layer():
+    """28 layers at the Qwen2-7B shape (RMSNorm, residual, no MLP), bank 512: the prefix, the first
+    16 frames, the 32-token question and 48 answer tokens.  Free-running chain at the depth-scaled
+    bound; ALL 28 layers teacher-forced at the stated tolerance."""
+    w = synth.workload("deep", n_frames=16, decode_tokens=48)
+    worst, met, per_layer = run_chain(w, w.question_len + w.decode_tokens, teacher=True)
+    print("deep chain, free-running: worst (max_abs, rel_rms) = %.3e %.3e; stated tolerance %s" %
+          (worst[0], worst[1], "met" if met else "NOT met (depth-scaled bound met)"))
+    print("deep, teacher-forced: worst over layers = %.3e %.3e" %
+          (max(x[0] for x in per_layer), max(x[1] for x in per_layer)))
 
 
-def test_deep_stack_full_shape_first_frames():
-    """28 layers at the Qwen2-7B shape (RMSNorm, residual, no MLP), bank 512: the first 6 frames,
-    the 32-token question and 4 decode tokens, free-running and teacher-forced per layer."""
-    w = synth.workload("deep", n_frames=6, decode_tokens=4)
-    rec, worst = run_chain(w, w.question_len + w.decode_tokens)
-    print("deep chain: worst", worst)
-    for layer in (0, 1, 13, 27):
-        print("deep layer", layer, "teacher-forced worst", teacher_forced_layer(w, layer, rec))
+def test_deep_stack_small_bank_evicts_at_depth():
+    """28 layers at the Qwen2-7B shape with a bank of 4: 8 frames (4 evictions), so the hole slot is
+    masked and refilled in every layer; bank K/V compared at layers 0, 13 and 27; then a question and
+    two answer tokens over the evicted bank."""
+    w = synth.workload("deep", n_frames=8, bank_capacity=4, question_len=8, decode_tokens=2)
+    worst, met, _ = run_chain(w, w.question_len + w.decode_tokens, bank_layers=[0, 13, 27])
+    print("deep, bank of 4: worst %.3e %.3e; stated tolerance %s" % (worst[0], worst[1], "met" if met else "NOT met"))
+
+
+def test_deep_stream_all_512_frames_bookkeeping():
+    """The 28-layer stream in full on the GPU (512 frames, bank 512): bank bookkeeping, positions and
+    carrier embeddings bit-exact against the oracle's pooling-and-eviction trace of every frame (the
+    oracle skips the layers: 512 frames x 28 layers is out of its reach), outputs finite."""
+    from concurrent.futures import ThreadPoolExecutor
+    w = synth.workload("deep")
+    p = Pair(w, max_text=1)
+    p.text([0], [w.prefix_hidden()], "prefix", compare=False)
+    shared = w.frame_shared()
+    with ThreadPoolExecutor(max_workers=8) as ex:
+        frames = ex.map(lambda t: w.frame_hidden(t, shared=shared), range(w.n_frames))
+    for t, x in enumerate(frames):
+        want_out = t % 64 == 63
+        out = p.gpu.frame_prefill([0], to_dev(x[None]), want_out=want_out)
+        p.ora[0].frame_step(synth.bf16_bits_to_f64(x), mode="meta")
+        if want_out:
+            assert torch.isfinite(out).all()
+            p.check_bank(0, kv=False)
+    st = p.check_bank(0, kv=False)
+    assert st["count"] == 512 and st["evictions"] == 0 and st["frames_seen"] == 512
+    assert st["persistent_bytes"] < st["workspace_bytes"]
+    p.close()
+
+
+def test_long_key_axis_at_the_qwen_shape():
+    """One layer at the Qwen2-7B shape with the 28-layer workload's bank of 512: 511 frames fill the
+    bank (the oracle projects their carrier rows only), then three frames in full -- 64 + 511 / 512 +
+    170 = 745 / 746 keys, six key tiles, the last two evicting -- the 32-token question and 8 answer
+    tokens (split-KV decode over 609 keys and more)."""
+    w = synth.workload("deep", n_layers=1, use_rmsnorm=0, residual=0, n_frames=514, decode_tokens=8)
+    p = Pair(w, max_text=w.question_len + w.decode_tokens)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    shared = w.frame_shared()
+    for t in range(w.n_frames):
+        full = t >= 511
+        p.frame([0], [w.frame_hidden(t, shared=shared)], f"frame {t}", mode="full" if full else "carrier")
+        if full or t % 128 == 0:
+            p.check_bank(0)
+    st = p.check_bank(0)
+    assert st["count"] == 512 and st["evictions"] == 2
+    p.text([0], [w.question_hidden()], "question")
+    for i in range(w.decode_tokens):
+        p.text([0], [w.decode_hidden(i)], f"decode {i}")
+    p.check_bank(0)
+    print("long key axis: worst", p.worst)
+    p.close()
 
 
 def test_batched_streams_full_shape():
-    """16 streams x 196 tokens at the Qwen2-7B shape, bank capacity 1024, ragged lengths (scaled to
-    [6, 24] frames so the oracle finishes in seconds), then batched single-token decode."""
-    w = synth.workload("batched", n_frames=24, min_frames=6, decode_tokens=4)
+    """16 streams x 196 tokens at the Qwen2-7B shape, bank capacity 1024, ragged lengths uniform in
+    [64, 256] as stated (2656 frames in all).  Bookkeeping, embeddings and bank K/V are checked over
+    every stream in full (the oracle projects only the carrier row of frames that are not sampled);
+    full attention parity on a seeded sample of 40 (stream, frame) pairs -- each stream's first and
+    last frame among them -- and on all 64 batched decode steps."""
+    from concurrent.futures import ThreadPoolExecutor
+    w = synth.workload("batched")
     lengths = w.stream_lengths()
+    assert min(lengths) >= 64 and max(lengths) <= 256
     p = Pair(w)
     ids = list(range(w.n_streams))
     p.text(ids, [w.prefix_hidden(s) for s in ids], "prefix")
-    shared = [w.frame_shared(s) for s in ids]
-    for t in range(max(lengths)):
-        act = [s for s in ids if lengths[s] > t]
-        full = t in (0, 5, max(lengths) - 1) or len(act) < 4
-        p.frame(act, [w.frame_hidden(t, s, shared=shared[s]) for s in act], f"frame {t}",
-                mode="full" if full else "carrier")
-    for i in range(w.decode_tokens):
-        p.text(ids, [w.decode_hidden(i, s) for s in ids], f"decode {i}")
+    rng = np.random.default_rng(5)
+    sample = {(s, 0) for s in ids[:4]} | {(s, lengths[s] - 1) for s in ids}
+    while len(sample) < 40:
+        s = int(rng.integers(0, w.n_streams))
+        sample.add((s, int(rng.integers(0, lengths[s]))))
+    with ThreadPoolExecutor(max_workers=8) as ex:
+        shared = list(ex.map(w.frame_shared, ids))
+        for t in range(max(lengths)):
+            act = [s for s in ids if lengths[s] > t]
+            xs = list(ex.map(lambda s: w.frame_hidden(t, s, shared=shared[s]), act))
+            p.frame(act, xs, f"frame {t}", mode=["full" if (s, t) in sample else "carrier" for s in act])
     for s in ids:
         st = p.check_bank(s)
         assert st["frames_seen"] == lengths[s] and st["count"] == lengths[s]
-    print("batched: lengths", lengths, "worst", p.worst)
+    for i in range(w.decode_tokens):
+        p.text(ids, [w.decode_hidden(i, s) for s in ids], f"decode {i}")
+    print("batched: lengths", lengths, "sampled", len(sample), "worst", p.worst)
+    p.close()
+
+
+def test_bf16_output_against_the_oracle_at_the_qwen_shape():
+    """out_dtype = 0 (bf16 rows, the output type of the boundary as first stated) against the oracle:
+    the rows are the fp32 result rounded once, so the error is the fp32 path's plus at most half a
+    bf16 unit of the value (2^-9 |y|).  Held to that sum; prints whether the plain 2e-2 held."""
+    from tests import parity
+    w = synth.workload("layer", n_frames=6, decode_tokens=4)
+    p = Pair(w, out_dtype=0)
+    p.text([0], [w.prefix_hidden()], "prefix", compare=False)
+    shared = w.frame_shared()
+    worst, peak = 0.0, 0.0
+    for t in range(w.n_frames):
+        x = w.frame_hidden(t, shared=shared)
+        got = to_f64(p.gpu.frame_prefill([0], to_dev(x[None])))[0]
+        want = p.ora[0].frame_step(synth.bf16_bits_to_f64(x))
+        err = np.abs(got - want)
+        assert np.all(err <= parity.MAX_ABS + np.abs(want) * 2.0 ** -9)
+        assert parity.errors(got, want)[1] <= parity.REL_RMS
+        worst, peak = max(worst, float(err.max())), max(peak, float(np.abs(want).max()))
+    print("bf16 output: worst |err| %.3e at max |y| %.2f; plain 2e-2 %s" %
+          (worst, peak, "met" if worst <= parity.MAX_ABS else "NOT met"))
     p.close()
 
 
