@@ -101,8 +101,10 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
   uint4 kr0[kBatch], vr0[kBatch];
   load_pass(wbase0, kr0, vr0, false);
 
+  VS_STAMP(bp, 5, 0);
   pdl_wait();
   pdl_launch_dependents();
+  VS_STAMP(bp, 5, 1);
   // the step's own key and the query are both fresh: their loads go out together
   if (wbase0 < end) load_pass(wbase0, kr0, vr0, true);
 
@@ -222,7 +224,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
       if (c == 0) { cta_ml[0] = M; cta_ml[1] = L; }
     }
   }
-  if (direct) return;
+  if (direct) { VS_STAMP(bp, 5, 15); return; }
 
   // the cluster's CTAs (the key splits of this stream and query head) meet; rank 0 combines
   cluster_sync();
@@ -259,6 +261,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
   }
   // nobody's shared memory goes away while rank 0 may still be reading it
   cluster_sync();
+  VS_STAMP(bp, 5, 15);
 }
 
 }  // namespace

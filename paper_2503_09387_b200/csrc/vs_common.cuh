@@ -38,6 +38,10 @@ struct BatchParams {
   int32_t text_len[VS_MAX_BATCH];      // tail length before this step
   int64_t pos_base[VS_MAX_BATCH];      // position id of the step's first token
   int64_t frame_id[VS_MAX_BATCH];      // frames_seen before this step
+#ifdef VS_TRACE
+  unsigned long long* trace;           // timeline log of a -DVS_TRACE build, or null
+  unsigned trace_seq;                  // sequence number of the launch
+#endif
 };
 
 // ---- shapes ----------------------------------------------------------------------------
@@ -80,9 +84,10 @@ struct Layout {
   // per-step scratch
   size_t hbuf[2];               // bf16 [R_max][d]  residual ping-pong; hbuf[0] holds [E; carrier]
   size_t xn;                    // bf16 [R_max][d]  layer input times the RMSNorm gain (only with a gain vector)
-  size_t row_scale;             // f32  [R_max]     RMSNorm row scales
+  size_t row_ss;                // f32  [R_max][Hkv] parts of the rows' sums of squares (RMSNorm)
   size_t q;                     // bf16 [R_max][Hq*D]
   size_t q_lo;                  // bf16 [R_max][Hq*D]  low-order half of the rotated query
+  size_t q_tiled;               // bf16 [row tiles][Hkv][hi | lo][128][D]  the pair as the tensor-core attention reads it
   size_t kf, vf;                // bf16 [R_max][Hkv*D]
   size_t rope;                  // float2 [R_max][D/2]
   size_t obuf;                  // f32  [R_max][Hq*D] (holds bf16 or fp32 rows)
@@ -92,6 +97,30 @@ struct Layout {
   size_t scratch_begin, scratch_end;
   size_t total;
 };
+
+// ---- timeline trace (only in a -DVS_TRACE build; the product build compiles none of it) ----------
+// The first and the last CTA of a launch store the global time (ns) of a few phases into fixed slots
+// of a log the host reads back -- slot = (kernel, phase, first / last CTA, launch sequence number
+// modulo VS_TRACE_RING) -- with programmatic dependent launch left as it is.  A plain store: the
+// stamping thread waits for nothing.
+#if defined(VS_TRACE) && defined(__CUDACC__)
+constexpr unsigned VS_TRACE_RING = 64;
+constexpr unsigned VS_TRACE_WORDS = 8 * 16 * 2 * VS_TRACE_RING;
+__device__ __forceinline__ void vs_stamp(const BatchParams& bp, unsigned kernel, unsigned phase, unsigned thread = 0) {
+  if (bp.trace == nullptr || threadIdx.x != thread) return;
+  const bool first = (blockIdx.x | blockIdx.y | blockIdx.z) == 0;
+  const bool last = blockIdx.x == gridDim.x - 1 && blockIdx.y == gridDim.y - 1 && blockIdx.z == gridDim.z - 1;
+  if (!first && !last) return;
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  bp.trace[(((kernel & 7u) * 16u + (phase & 15u)) * 2u + (last ? 1u : 0u)) * VS_TRACE_RING + (bp.trace_seq % VS_TRACE_RING)] = t;
+}
+#define VS_STAMP(bp, kernel, phase) vs_stamp(bp, kernel, phase)
+#define VS_STAMP_BY(bp, kernel, phase, thread) vs_stamp(bp, kernel, phase, thread)
+#else
+#define VS_STAMP(bp, kernel, phase)
+#define VS_STAMP_BY(bp, kernel, phase, thread)
+#endif
 
 // ---- programmatic dependent launch ------------------------------------------------------
 // Every kernel of a step is launched with programmatic stream serialisation: it may be
@@ -151,13 +180,16 @@ struct RopeArgs {
 };
 cudaError_t launch_rope_table(const RopeArgs& a, const BatchParams& bp, cudaStream_t st);
 
-cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* row_scale, int rows, int d,
-                             float eps, cudaStream_t st);
+// sum of squares of every row -> row_ss[row][parts] (part 0; the other parts zero); with a gain vector hg = bf16(h * gain)
+cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* row_ss, int parts, int rows, int d,
+                             cudaStream_t st);
 
 // What the projection epilogue writes (finished rows: bias, RoPE, bf16) and where rows persist.
 struct ProjectionOut {
   const bf16* bias;              // [E_out] or null
-  const float* row_scale;        // [rows] RMSNorm scale applied to the accumulated row, or null
+  const float* row_ss;           // [rows][ss_parts] parts of each row's sum of squares (RMSNorm: the accumulated row is
+                                 // scaled by 1 / sqrt(sum / d + norm_eps), the parts added in index order), or null
+  int ss_parts;
   int norm_inline;               // matrix-vector kernel only: it computes the RMSNorm scale (and h * gain) itself
   const bf16* norm_gain;         // [d] or null
   float norm_eps;
@@ -165,6 +197,8 @@ struct ProjectionOut {
   const double* inv_freq;        // [D/2]
   bf16* q;                       // [rows][Hq*D]  rotated query, leading bf16 part
   bf16* q_lo;                    // [rows][Hq*D]  bf16(query - q): the pair carries 16 mantissa bits
+  bf16* q_tiled;                 // tensor-core GEMM only, or null: the pair in the attention kernel's operand layout
+                                 // instead (see AttnArgs::q_tiled); rows_per_stream rows per batch entry
   bf16* kf;                      // [rows][Hkv*D] rotated keys of this step
   bf16* vf;                      // [rows][Hkv*D]
   bf16* bank_k; bf16* bank_v;    // layer base [S][Hkv][slots][D]
@@ -218,29 +252,44 @@ struct BankUpdateArgs {
   int32_t* order; int32_t* slot_frame; int64_t* slot_pos; int32_t* evict_log; double* scores;
   int d, slots, M, policy, log_cap;
 };
+// One segment of the attention's key axis.  Its K and V rows are reached through tensor maps with
+// dimensions {head_dim, rows, Z} and a box of {64, ATTN_KEY_BOX, 1} elements (128-byte swizzle):
+// prefix / bank / tail maps span every layer, stream and KV head on Z; the step's own rows
+// ([rows][Hkv * D]) put the KV head on Z.
+constexpr int ATTN_KEY_BOX = 64;   // key rows per bulk tensor copy; segments start on multiples of it on the key axis
 struct AttnSegment {
-  const bf16* k; const bf16* v;
-  long long stream_stride;       // elements between streams (by stream id, or by batch slot when by_batch)
-  long long head_stride;         // elements between KV heads
-  long long row_stride;          // elements between keys
+  CUtensorMap tk, tv;
   int kind;                      // 0 prefix, 1 bank, 2 tail (earlier tokens of the turn), 3 this step's rows (causal),
                                  // 4 carriers of the chunk's earlier frames (entry b sees b of them)
-  int by_batch;
+  int rows_per_batch;            // row coordinate of batch entry b's first key: b * rows_per_batch
+  int z0, z_per_stream;          // Z coordinate = z0 + stream id * z_per_stream + KV head
 };
 struct AttnArgs {
   const bf16* q;                 // [rows][Hq*D]
   const bf16* q_lo;
+  const bf16* q_tiled;           // or: the query as the projection's GEMM leaves it for this kernel, one block per
+                                 // (batch entry, 16-token row tile, KV head): [hi | lo][128 rows = g * 16 + token][D],
+                                 // 128-byte swizzled like the MMA operand, fetched by one bulk copy
   AttnSegment seg[4];
   int n_seg;
   void* out;                     // [rows][Hq*D], bf16 or fp32
   int out_fp32;
   const bf16* h_in;              // residual input [rows][d] or null
   bf16* h_out;                   // residual output or null
+  // RMSNorm of the layer that follows (needs h_out): the sum of squares of every stored residual row over this KV
+  // head's query heads -> ss_out[row][Hkv]; with a gain vector also xn_out = bf16(h_out * next_gain); or null
+  float* ss_out;
+  const bf16* next_gain;
+  bf16* xn_out;
   const int32_t* free_slot;      // free slot of stream s at free_slot[s * free_slot_stride]
   int free_slot_stride;
   int Hq, Hkv, D, slots, M;
   float scale_log2e;
-  // frame steps, last layer: the first bank_blocks CTAs of every stream do the bank update
+  // CTAs that share the key tiles of one (row tile, KV head, batch entry): a thread-block cluster of 1 .. 4
+  // whose members each take a contiguous run of key tiles and combine through distributed shared memory
+  int nsplit;
+  // frame steps, last layer: the bank update (it needs the carrier embeddings only) is done by the CTAs of one more
+  // plane of the grid (blockIdx.y == Hkv), which take its bank_blocks blocks of work in turn; 0: none
   BankUpdateArgs bank;
   int bank_blocks;
   // chunk of frames in ONE launch (entry b = frame b): the bank segment is the bank as it was
@@ -268,6 +317,8 @@ cudaError_t launch_chunk_kv_commit(const ChunkKvCommitArgs& a, cudaStream_t st);
 constexpr int ATTN_EXCL_BITS = 8192;   // most (bank slots + chunk frames) the one-launch chunk attention can mask
 cudaError_t launch_prefill_attention_tc(const AttnArgs& a, const BatchParams& bp, int* status, cudaStream_t st);
 cudaError_t prefill_attention_tc_init();
+int prefill_attention_max_clusters(int head_dim, int s);
+constexpr int ATTN_MAX_SPLIT = 2;   // clusters of 3 or 4 do not all fit on the GPU at once (one CTA per SM, clusters inside a GPC)
 
 struct DecodeArgs {
   const bf16* q;                 // [n_active][Hq*D]

@@ -125,6 +125,7 @@ struct KernelParams {
   ProjectionOut o;
   int* status;
   int rows, E_out, tile_n, kblocks, stages, tmem_cols, ksplit;
+  float inv_d;                  // 1 / d_model
   int acc_stride;               // TMEM columns between the accumulators
   uint32_t data_bytes;          // shared memory ahead of the barriers: max(pipeline stages, own fp32 slice)
   float* xchg;                  // [group][rank][tile_n][128] partial tiles of the K split
@@ -184,8 +185,10 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem_acc = *tmem_slot;
+  VS_STAMP(bp, 1, 0);
   pdl_wait();                       // earlier kernels of the stream have completed
   pdl_launch_dependents();
+  VS_STAMP(bp, 1, 1);
 
   if (warp == 0) {
     if (lane == 0) {
@@ -274,11 +277,23 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
       own_rb = make_float4(r[4], r[5], r[6], r[7]);
     }
   }
+  // RMSNorm: the row scales of this CTA's token slice, worked out while the main loop runs
+  float* rsc_s = reinterpret_cast<float*>(ctl + 64);             // [slice]
+  if (warp >= 2 && p.o.row_ss != nullptr) {
+    for (int t = threadIdx.x - 64; t < slice; t += (int)blockDim.x - 64) {
+      const int row = n0 + t_begin + t;
+      float tot = 0.f;
+      if (row < p.rows)
+        for (int i = 0; i < p.o.ss_parts; ++i) tot += p.o.row_ss[(size_t)row * p.o.ss_parts + i];
+      rsc_s[t] = rsqrtf(tot * p.inv_d + p.o.norm_eps);
+    }
+  }
   bool acc_ok = true;
   if (warp >= 2) {
     acc_ok = __all_sync(0xffffffffu, mbar_wait(tmem_full_bar, 0, abort_flag));   // warp-uniform
   }
   tcgen05_fence_after();
+  VS_STAMP_BY(bp, 1, 2, 64);          // accumulator complete
 
   // one pass per 128-row weight sub-tile (its own accumulator); the staging memory is shared
 #pragma unroll 1
@@ -377,7 +392,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
           }
         }
         // RMSNorm's row scale commutes with the projection: applied here, in fp32
-        R.rsc = (p.o.row_scale != nullptr) ? p.o.row_scale[row] : 1.f;
+        R.rsc = (p.o.row_ss != nullptr) ? rsc_s[t - t_begin] : 1.f;
       };
       auto finish_row = [&](const RowRegs& R, int it) {
         const int t = t_begin + (te >> 4) + tok_lanes * it;
@@ -408,17 +423,37 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
         if (hs < p.o.Hq) {
           // the query never leaves the step, so it is kept as a bf16 pair (hi + lo): the score
           // Q K^T then sees a 16-bit mantissa instead of 8 at the cost of a second MMA
-          const size_t qo = (size_t)row * p.o.Hq * D + (size_t)hs * D + k0;
-          *reinterpret_cast<uint2*>(p.o.q + qo) = w1;
-          *reinterpret_cast<uint2*>(p.o.q + qo + half) = w2;
           __align__(8) bf16 l1[4], l2[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             l1[i] = __float2bfloat16_rn(x1[i] - __bfloat162float(o1[i]));
             l2[i] = __float2bfloat16_rn(x2[i] - __bfloat162float(o2[i]));
           }
-          *reinterpret_cast<uint2*>(p.o.q_lo + qo) = *reinterpret_cast<const uint2*>(l1);
-          *reinterpret_cast<uint2*>(p.o.q_lo + qo + half) = *reinterpret_cast<const uint2*>(l2);
+          if (p.o.q_tiled != nullptr) {
+            // straight into the attention kernel's operand layout: one block per (batch entry, 16-token
+            // row tile, KV head) holding [hi | lo][128 rows = g * 16 + token][D], rows of 128 bytes per
+            // 64 dims with the 16-byte units XOR-ed by the row (the MMA's 128-byte swizzle)
+            const int G = p.o.Hq / p.o.Hkv;
+            const int b = row / rps, tt = row - b * rps;
+            const int n_rt = (rps + 15) >> 4;
+            const size_t tile = ((size_t)b * n_rt + (size_t)(tt >> 4)) * p.o.Hkv + (size_t)(hs / G);
+            const int r = (hs % G) * 16 + (tt & 15);
+            uint8_t* tb = reinterpret_cast<uint8_t*>(p.o.q_tiled) + tile * (size_t)(2 * 128 * D * 2);
+            const int c1 = k0 >> 3, c2 = (k0 + half) >> 3;
+            const uint32_t o_1 = (uint32_t)((c1 >> 3) * (128 * 128) + r * 128 + (((c1 & 7) ^ (r & 7)) << 4) + (k0 & 7) * 2);
+            const uint32_t o_2 = (uint32_t)((c2 >> 3) * (128 * 128) + r * 128 + (((c2 & 7) ^ (r & 7)) << 4) + (k0 & 7) * 2);
+            const uint32_t lo_off = (uint32_t)(128 * D * 2);
+            *reinterpret_cast<uint2*>(tb + o_1) = w1;
+            *reinterpret_cast<uint2*>(tb + o_2) = w2;
+            *reinterpret_cast<uint2*>(tb + lo_off + o_1) = *reinterpret_cast<const uint2*>(l1);
+            *reinterpret_cast<uint2*>(tb + lo_off + o_2) = *reinterpret_cast<const uint2*>(l2);
+          } else {
+            const size_t qo = (size_t)row * p.o.Hq * D + (size_t)hs * D + k0;
+            *reinterpret_cast<uint2*>(p.o.q + qo) = w1;
+            *reinterpret_cast<uint2*>(p.o.q + qo + half) = w2;
+            *reinterpret_cast<uint2*>(p.o.q_lo + qo) = *reinterpret_cast<const uint2*>(l1);
+            *reinterpret_cast<uint2*>(p.o.q_lo + qo + half) = *reinterpret_cast<const uint2*>(l2);
+          }
         } else {
           const bool is_k = hs < p.o.Hq + p.o.Hkv;
           const int hkv = is_k ? hs - p.o.Hq : hs - p.o.Hq - p.o.Hkv;
@@ -461,6 +496,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)p.tmem_cols) : "memory");
   }
   if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, VS_ERR_DEVICE_TIMEOUT);
+  VS_STAMP(bp, 1, 15);
 }
 
 constexpr int kMaxDynSmem = 227 * 1024;
@@ -482,6 +518,7 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   p.E_out = a.E_out;
   p.tile_n = a.tile_n;
   p.ksplit = a.ksplit;
+  p.inv_d = 1.f / (float)a.d;
   const int total_kb = a.d / GEMM_BLOCK_K;
   if (a.ksplit < 1 || a.ksplit > KSPLIT_MAX || (a.ksplit & (a.ksplit - 1)) || total_kb % a.ksplit != 0) return cudaErrorInvalidValue;
   if (a.tile_n < 16 || a.tile_n > 256 || (a.tile_n & 15)) return cudaErrorInvalidValue;
@@ -491,7 +528,7 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   p.xchg = a.xchg;
   p.flags = a.flags;
   const int stage_bytes = a.m_sub * kStageABytes + a.tile_n * 128;
-  int stages = (kMaxDynSmem - 2048) / stage_bytes;
+  int stages = (kMaxDynSmem - 3072) / stage_bytes;
   if (stages > 8) stages = 8;
   if (stages > p.kblocks) stages = p.kblocks;
   if (stages < 1) return cudaErrorInvalidValue;
@@ -504,7 +541,7 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   const size_t own = (size_t)(a.tile_n / a.ksplit) * GEMM_BLOCK_M * 4;
   if (own > data) data = (own + 1023) / 1024 * 1024;
   p.data_bytes = (uint32_t)data;
-  const size_t smem = 1024 + data + 16 * stages + 64;
+  const size_t smem = 1024 + data + 16 * stages + 64 + 1024;     // + the slice's RMSNorm row scales
   if (smem > (size_t)kMaxDynSmem) return cudaErrorInvalidValue;
   // a token slice of a few rows is finished by 4 warps; wider ones by 16, which overlap one another's latency
   const int slice_rows = a.tile_n / a.ksplit;

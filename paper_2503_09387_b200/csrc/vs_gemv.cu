@@ -111,8 +111,10 @@ __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __res
     }
   }
 
+  VS_STAMP(bp, 4, 0);
   pdl_wait();                       // earlier kernels of the stream have completed
   pdl_launch_dependents();
+  VS_STAMP(bp, 4, 1);
 
   // token rows -> shared memory; with RMSNorm: sum of squares of the raw row, and the row times
   // the gain vector (rounded to bf16, as the statistics kernel stores it) in place of the row
@@ -197,7 +199,13 @@ __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __res
     float x1 = ys[row * kRowsPerCta + fp], x2 = ys[row * kRowsPerCta + 16 + fp];
     const int f1 = hs * D + k0, f2 = f1 + half;
     // RMSNorm's row scale commutes with the projection
-    const float rsc = o.norm_inline ? rs[row] : ((o.row_scale != nullptr) ? o.row_scale[row] : 1.f);
+    float rsc = 1.f;
+    if (o.norm_inline) rsc = rs[row];
+    else if (o.row_ss != nullptr) {
+      float tot = 0.f;
+      for (int i = 0; i < o.ss_parts; ++i) tot += o.row_ss[(size_t)row * o.ss_parts + i];
+      rsc = rsqrtf(tot / (float)d + o.norm_eps);
+    }
     const float b1 = (o.bias != nullptr) ? __bfloat162float(o.bias[f1]) : 0.f;
     const float b2 = (o.bias != nullptr) ? __bfloat162float(o.bias[f2]) : 0.f;
     x1 = fmaf(x1, rsc, b1); x2 = fmaf(x2, rsc, b2);
@@ -224,6 +232,7 @@ __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __res
       dst[0] = o1; dst[half] = o2;
     }
   }
+  VS_STAMP(bp, 4, 15);
 }
 
 }  // namespace

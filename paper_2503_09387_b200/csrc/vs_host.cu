@@ -87,9 +87,12 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.hbuf[0] = take((size_t)D.R_max * D.d * 2);
   Lo.hbuf[1] = take((size_t)D.R_max * D.d * 2);
   Lo.xn = take((size_t)D.R_max * D.d * 2);
-  Lo.row_scale = take((size_t)D.R_max * 4);
+  Lo.row_ss = take((size_t)D.R_max * D.Hkv * 4);
   Lo.q = take((size_t)D.R_max * D.Hq * D.D * 2);
   Lo.q_lo = take((size_t)D.R_max * D.Hq * D.D * 2);
+  // the query in the attention kernel's operand layout: per batch entry ceil(rows / 16) row tiles, per tile and KV
+  // head a block of [hi | lo][128][D]
+  Lo.q_tiled = take(((size_t)D.R_max / 16 + (size_t)VS_MAX_BATCH + 1) * D.Hkv * 2 * 128 * D.D * 2);
   Lo.kf = take((size_t)D.R_max * D.Hkv * D.D * 2);
   Lo.vf = take((size_t)D.R_max * D.Hkv * D.D * 2);
   Lo.rope = take((size_t)D.R_max * (D.D / 2) * 8);
@@ -115,6 +118,15 @@ struct vs_stream {
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   std::vector<const bf16*> w, bias, gain;
   std::vector<CUtensorMap> tm_w;
+  // key/value tensor maps of the attention: the persistent ones span all layers, streams and KV heads
+  CUtensorMap tm_prefix_k, tm_prefix_v, tm_bank_k, tm_bank_v, tm_tail_k, tm_tail_v;
+  CUtensorMap tm_step_k, tm_step_v;          // the step's own rows [rows][Hkv * D]; re-encoded when `rows` changes
+  int step_map_rows = -1;
+  int attn_clusters[ATTN_MAX_SPLIT + 1] = {0};   // clusters of s attention CTAs that can be resident at once
+#ifdef VS_TRACE
+  unsigned long long* trace = nullptr;
+  unsigned trace_seq = 0;
+#endif
   std::vector<HostStream> hs;
   EncodeTiledFn encode = nullptr;
   cudaStream_t last_stream = nullptr;
@@ -141,6 +153,58 @@ int encode_2d(vs_stream* h, CUtensorMap* tm, const void* base, uint64_t inner, u
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? VS_OK : VS_ERR_CUDA;
+}
+
+// K or V rows for the attention kernel: dimensions {head_dim, rows, Z}, box {64, ATTN_KEY_BOX, 1}, 128-byte swizzle;
+// rows (and Z) beyond the extents read as zeros.
+int encode_kv(vs_stream* h, CUtensorMap* tm, const void* base, uint64_t head_dim, uint64_t rows, uint64_t row_stride_bytes,
+              uint64_t nz, uint64_t z_stride_bytes) {
+  cuuint64_t dims[3] = {head_dim, rows, nz};
+  cuuint64_t strides[2] = {row_stride_bytes, z_stride_bytes};
+  cuuint32_t box[3] = {64, (cuuint32_t)ATTN_KEY_BOX, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = h->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? VS_OK : VS_ERR_CUDA;
+}
+
+// the step's own K/V rows as the attention's last segment: extent = the step's rows, so that a box
+// reaching past them reads zeros, not what an earlier step left in the scratch
+int ensure_step_maps(vs_stream* h, int rows) {
+  if (h->step_map_rows == rows) return VS_OK;
+  const Dims& D = h->dm;
+  const uint64_t rs = (uint64_t)D.Hkv * D.D * 2, zs = (uint64_t)D.D * 2;
+  if (encode_kv(h, &h->tm_step_k, h->at<bf16>(h->lo.kf), D.D, rows, rs, D.Hkv, zs) != VS_OK) return VS_ERR_CUDA;
+  if (encode_kv(h, &h->tm_step_v, h->at<bf16>(h->lo.vf), D.D, rows, rs, D.Hkv, zs) != VS_OK) return VS_ERR_CUDA;
+  h->step_map_rows = rows;
+  return VS_OK;
+}
+
+// CTAs to spread the key tiles of a row tile over (one cluster): every CTA of the attention kernel takes
+// a whole SM, all clusters must be resident at once, and a split pays only while it shortens the longest
+// CTA's run of key tiles.  key_len[i]: segment lengths of the longest key axis among the listed entries.
+int attn_split(const vs_stream* h, const BatchParams& bp, const int* key_len, int n_len) {
+  int padded = 0;
+  for (int i = 0; i < n_len; ++i) padded += (key_len[i] + ATTN_KEY_BOX - 1) / ATTN_KEY_BOX * ATTN_KEY_BOX;
+  const int key_tiles = (padded + 127) / 128;
+  const long long row_ctas = (long long)((bp.rows_per_stream + 15) / 16) * h->dm.Hkv * bp.n_active;
+  int best = 1;
+  for (int s = 2; s <= ATTN_MAX_SPLIT; ++s) {
+    if (s > key_tiles || row_ctas * s > h->n_sms || h->attn_clusters[s] < row_ctas) break;
+    if ((key_tiles + s - 1) / s == (key_tiles + best - 1) / best) continue;
+    best = s;
+  }
+  return best;
+}
+
+// segments of the attention's key axis
+void seg_stored(AttnSegment& sg, const CUtensorMap& k, const CUtensorMap& v, int kind, int layer, const Dims& D) {
+  sg.tk = k; sg.tv = v; sg.kind = kind; sg.rows_per_batch = 0;
+  sg.z0 = layer * D.S * D.Hkv; sg.z_per_stream = D.Hkv;
+}
+void seg_step(AttnSegment& sg, const CUtensorMap& k, const CUtensorMap& v, int kind, int rows_per_batch) {
+  sg.tk = k; sg.tv = v; sg.kind = kind; sg.rows_per_batch = rows_per_batch; sg.z0 = 0; sg.z_per_stream = 0;
 }
 
 // Token tiling of the projection.  Every CTA re-reads its weight rows and its token columns from
@@ -180,6 +244,14 @@ int check_ids(vs_stream* h, const int32_t* ids, int32_t n) {
   }
   return VS_OK;
 }
+
+#ifdef VS_TRACE
+#define VS_BP_INIT(h, bp) do { std::memset(&(bp), 0, sizeof(bp)); (bp).trace = (h)->trace; (bp).trace_seq = (h)->trace_seq; } while (0)
+#define VS_TRACE_NEXT(h, bp) do { (bp).trace_seq = ++(h)->trace_seq; } while (0)
+#else
+#define VS_BP_INIT(h, bp) std::memset(&(bp), 0, sizeof(bp))
+#define VS_TRACE_NEXT(h, bp)
+#endif
 
 #define VS_CK(expr) do { if ((expr) != cudaSuccess) return VS_ERR_CUDA; } while (0)
 
@@ -294,7 +366,18 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights, void* work
   h->tm_w.resize(D.L);
   for (int l = 0; l < D.L; ++l)
     if (encode_2d(h, &h->tm_w[l], h->w[l], (uint64_t)D.d, (uint64_t)D.E_out, GEMM_BLOCK_M) != VS_OK) return fail(VS_ERR_CUDA);
+  {
+    const uint64_t nz = (uint64_t)D.L * D.S * D.Hkv, rb = (uint64_t)D.D * 2;
+    if (encode_kv(h, &h->tm_prefix_k, h->ws + lo.prefix_k, D.D, D.maxP, rb, nz, (uint64_t)D.maxP * rb) != VS_OK ||
+        encode_kv(h, &h->tm_prefix_v, h->ws + lo.prefix_v, D.D, D.maxP, rb, nz, (uint64_t)D.maxP * rb) != VS_OK ||
+        encode_kv(h, &h->tm_bank_k, h->ws + lo.bank_k, D.D, D.slots, rb, nz, (uint64_t)D.slots * rb) != VS_OK ||
+        encode_kv(h, &h->tm_bank_v, h->ws + lo.bank_v, D.D, D.slots, rb, nz, (uint64_t)D.slots * rb) != VS_OK ||
+        encode_kv(h, &h->tm_tail_k, h->ws + lo.tail_k, D.D, D.maxT, rb, nz, (uint64_t)D.maxT * rb) != VS_OK ||
+        encode_kv(h, &h->tm_tail_v, h->ws + lo.tail_v, D.D, D.maxT, rb, nz, (uint64_t)D.maxT * rb) != VS_OK)
+      return fail(VS_ERR_CUDA);
+  }
   if (qkv_gemm_init() != cudaSuccess || qkv_gemv_init() != cudaSuccess || prefill_attention_tc_init() != cudaSuccess) return fail(VS_ERR_CUDA);
+  for (int sp = 2; sp <= ATTN_MAX_SPLIT; ++sp) h->attn_clusters[sp] = prefill_attention_max_clusters(D.D, sp);
   // clear the whole workspace, then write the non-zero initial metadata
   if (cudaMemset(h->ws, 0, lo.total) != cudaSuccess) return fail(VS_ERR_CUDA);
   if (cudaMemset(h->ws + lo.slot_frame, 0xFF, (size_t)D.S * D.slots * 4) != cudaSuccess) return fail(VS_ERR_CUDA);
@@ -335,9 +418,10 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
   VS_CK(cudaSetDevice(h->device));
 
   BatchParams bp;
-  std::memset(&bp, 0, sizeof(bp));
+  VS_BP_INIT(h, bp);
   bp.n_active = n_active;
   bp.rows_per_stream = N + 1;
+  VS_TRACE_NEXT(h, bp);
   bool any_full = false;
   for (int i = 0; i < n_active; ++i) {
     const HostStream& s = h->hs[stream_ids[i]];
@@ -373,24 +457,28 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
   pa.rope = h->at<float2>(lo.rope);
   pa.N = N; pa.d = D.d; pa.D = D.D; pa.slots = D.slots; pa.M = D.M; pa.agg_mode = D.agg_mode;
   VS_LAUNCH(h, st, KC_POOL, launch_pool(pa, bp, st));
+  if (ensure_step_maps(h, rows) != VS_OK) return VS_ERR_CUDA;
 
   void* out_final = out ? out : h->at<void>(lo.obuf);
   int cur = 0;
   for (int l = 0; l < D.L; ++l) {
+    if (l > 0) VS_TRACE_NEXT(h, bp);
     const bf16* h_in = h->at<bf16>(lo.hbuf[cur]);
     const bf16* src = h_in;
     if (D.use_rmsnorm) {
-      VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_scale),
-                                                    rows, D.d, D.rms_eps, st));
+      // layer 0: a launch of its own; deeper layers: the attention kernel that stored h_in left the statistics
+      if (l == 0) VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_ss),
+                                                                D.Hkv, rows, D.d, st));
       if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
     }
     ProjectionOut fa;
     fa.bias = h->bias[l];
-    fa.row_scale = D.use_rmsnorm ? h->at<float>(lo.row_scale) : nullptr;
-    fa.norm_inline = 0; fa.norm_gain = nullptr; fa.norm_eps = 0.f;
+    fa.row_ss = D.use_rmsnorm ? h->at<float>(lo.row_ss) : nullptr; fa.ss_parts = D.Hkv; fa.norm_eps = D.rms_eps;
+    fa.norm_inline = 0; fa.norm_gain = nullptr;
     fa.rope = h->at<float2>(lo.rope);
     fa.inv_freq = h->at<double>(lo.inv_freq);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
+    fa.q_tiled = h->at<bf16>(lo.q_tiled);
     fa.bank_k = h->at<bf16>(lo.bank_k) + (size_t)l * layer_stride_bank(D);
     fa.bank_v = h->at<bf16>(lo.bank_v) + (size_t)l * layer_stride_bank(D);
     fa.text_k = nullptr; fa.text_v = nullptr;
@@ -401,19 +489,28 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
 
     AttnArgs aa;
     std::memset(&aa, 0, sizeof(aa));
-    aa.q = fa.q; aa.q_lo = fa.q_lo;
-    aa.seg[0] = {h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D),
-                 h->at<bf16>(lo.prefix_v) + (size_t)l * layer_stride_prefix(D),
-                 (long long)D.Hkv * D.maxP * D.D, (long long)D.maxP * D.D, (long long)D.D, 0, 0};
-    aa.seg[1] = {fa.bank_k, fa.bank_v, (long long)D.Hkv * D.slots * D.D, (long long)D.slots * D.D, (long long)D.D, 1, 0};
-    aa.seg[2] = {fa.kf, fa.vf, (long long)(N + 1) * D.Hkv * D.D, (long long)D.D, (long long)D.Hkv * D.D, 3, 1};
+    aa.q = fa.q; aa.q_lo = fa.q_lo; aa.q_tiled = fa.q_tiled;
+    seg_stored(aa.seg[0], h->tm_prefix_k, h->tm_prefix_v, 0, l, D);
+    seg_stored(aa.seg[1], h->tm_bank_k, h->tm_bank_v, 1, l, D);
+    seg_step(aa.seg[2], h->tm_step_k, h->tm_step_v, 3, N + 1);
     aa.n_seg = 3;
     const bool last = (l == D.L - 1);
-    aa.out = last ? out_final : h->at<void>(lo.obuf);
+    // a layer whose rows only feed the residual stream stores no output rows
+    aa.out = last ? out_final : (D.residual ? nullptr : h->at<void>(lo.obuf));
     aa.out_fp32 = D.out_fp32;
     aa.h_in = D.residual ? h_in : nullptr;
     aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
+    if (D.use_rmsnorm && l + 1 < D.L) { aa.ss_out = h->at<float>(lo.row_ss); aa.next_gain = h->gain[l + 1]; aa.xn_out = h->at<bf16>(lo.xn); }
     aa.free_slot = h->at<int32_t>(lo.step_slot); aa.free_slot_stride = 1;
+    {
+      int kl[3] = {0, 0, N + 1};
+      for (int i = 0; i < n_active; ++i) {
+        const int bl = D.M == 0 ? 0 : (bp.count[i] == D.M ? D.M + 1 : bp.count[i]);
+        if (bp.prefix_len[i] + bl > kl[0] + kl[1]) { kl[0] = bp.prefix_len[i]; kl[1] = bl; }
+      }
+      aa.nsplit = attn_split(h, bp, kl, 3);
+    }
+    // the bank update (Section 3.3, memory mechanism: evict if full, then append) rides in the last layer's launch
     if (last) { aa.bank = ba; aa.bank_blocks = any_full ? (D.M + 7) / 8 : 1; }
     aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
     aa.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
@@ -449,7 +546,7 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
   // the F frames as F batch entries of the same stream, each with the bank count and the
   // positions it would find as a step of its own
   BatchParams bp;
-  std::memset(&bp, 0, sizeof(bp));
+  VS_BP_INIT(h, bp);
   bp.n_active = F;
   bp.rows_per_stream = N + 1;
   for (int j = 0; j < F; ++j) {
@@ -463,7 +560,7 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
   }
   auto one_frame = [&](int j) {
     BatchParams b1;
-    std::memset(&b1, 0, sizeof(b1));
+    VS_BP_INIT(h, b1);
     b1.n_active = 1; b1.rows_per_stream = N + 1;
     b1.stream_id[0] = bp.stream_id[j]; b1.count[0] = bp.count[j]; b1.prefix_len[0] = bp.prefix_len[j];
     b1.pos_base[0] = bp.pos_base[j]; b1.frame_id[0] = bp.frame_id[j];
@@ -546,26 +643,36 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
   }
   if (beside) VS_CK(cudaEventRecord(h->ev_join, h->side_stream));
 
+  if (ensure_step_maps(h, rows) != VS_OK) return VS_ERR_CUDA;
+  // the carrier rows of the chunk's frames (row N of every frame of the step's K/V) as a segment of their own
+  CUtensorMap tm_carr_k, tm_carr_v;
+  {
+    const uint64_t rs = (uint64_t)(N + 1) * D.Hkv * D.D * 2, zs = (uint64_t)D.D * 2;
+    if (encode_kv(h, &tm_carr_k, h->at<bf16>(lo.kf) + (size_t)N * D.Hkv * D.D, D.D, F, rs, D.Hkv, zs) != VS_OK ||
+        encode_kv(h, &tm_carr_v, h->at<bf16>(lo.vf) + (size_t)N * D.Hkv * D.D, D.D, F, rs, D.Hkv, zs) != VS_OK)
+      return VS_ERR_CUDA;
+  }
   // 3. layer by layer: one projection over all F * (N + 1) rows, one attention launch over all
   //    frames, then the K/V rows of the chunk's surviving carriers go into their bank slots
   char* out_bytes = static_cast<char*>(out ? out : h->at<void>(lo.obuf));
-  const size_t out_row_bytes = (size_t)D.Hq * D.D * (D.out_fp32 ? 4 : 2);
   int cur = 0;
   for (int l = 0; l < D.L; ++l) {
     const bf16* h_in = h->at<bf16>(lo.hbuf[cur]);
     const bf16* src = h_in;
     if (D.use_rmsnorm) {
-      VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_scale),
-                                                    rows, D.d, D.rms_eps, st));
+      // layer 0: a launch of its own; deeper layers: the attention kernel that stored h_in left the statistics
+      if (l == 0) VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_ss),
+                                                                D.Hkv, rows, D.d, st));
       if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
     }
     ProjectionOut fa;
     std::memset(&fa, 0, sizeof(fa));
     fa.bias = h->bias[l];
-    fa.row_scale = D.use_rmsnorm ? h->at<float>(lo.row_scale) : nullptr;
+    fa.row_ss = D.use_rmsnorm ? h->at<float>(lo.row_ss) : nullptr; fa.ss_parts = D.Hkv; fa.norm_eps = D.rms_eps;
     fa.rope = h->at<float2>(lo.rope);
     fa.inv_freq = h->at<double>(lo.inv_freq);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
+    fa.q_tiled = h->at<bf16>(lo.q_tiled);
     fa.bank_k = h->at<bf16>(lo.bank_k) + (size_t)l * layer_stride_bank(D);
     fa.bank_v = h->at<bf16>(lo.bank_v) + (size_t)l * layer_stride_bank(D);
     fa.free_slot = chunk_slot; fa.free_slot_stride = 0;
@@ -581,21 +688,23 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
       // updates of frames 0 .. b-1 evicted, plus the carriers of those frames (from the step's K/V)
       AttnArgs aa;
       std::memset(&aa, 0, sizeof(aa));
-      aa.q = fa.q; aa.q_lo = fa.q_lo;
-      aa.seg[0] = {h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D),
-                   h->at<bf16>(lo.prefix_v) + (size_t)l * layer_stride_prefix(D),
-                   (long long)D.Hkv * D.maxP * D.D, (long long)D.maxP * D.D, (long long)D.D, 0, 0};
-      aa.seg[1] = {fa.bank_k, fa.bank_v, (long long)D.Hkv * D.slots * D.D, (long long)D.slots * D.D, (long long)D.D, 1, 0};
-      aa.seg[2] = {fa.kf + (size_t)N * D.Hkv * D.D, fa.vf + (size_t)N * D.Hkv * D.D, 0, (long long)D.D,
-                   (long long)(N + 1) * D.Hkv * D.D, 4, 0};
-      aa.seg[3] = {fa.kf, fa.vf, (long long)(N + 1) * D.Hkv * D.D, (long long)D.D, (long long)D.Hkv * D.D, 3, 1};
+      aa.q = fa.q; aa.q_lo = fa.q_lo; aa.q_tiled = fa.q_tiled;
+      seg_stored(aa.seg[0], h->tm_prefix_k, h->tm_prefix_v, 0, l, D);
+      seg_stored(aa.seg[1], h->tm_bank_k, h->tm_bank_v, 1, l, D);
+      seg_step(aa.seg[2], tm_carr_k, tm_carr_v, 4, 0);
+      seg_step(aa.seg[3], h->tm_step_k, h->tm_step_v, 3, N + 1);
       aa.n_seg = 4;
-      aa.out = layer_out;
+      aa.out = (last || !D.residual) ? layer_out : nullptr;
       aa.out_fp32 = D.out_fp32;
       aa.h_in = D.residual ? h_in : nullptr;
       aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
+    if (D.use_rmsnorm && l + 1 < D.L) { aa.ss_out = h->at<float>(lo.row_ss); aa.next_gain = h->gain[l + 1]; aa.xn_out = h->at<bf16>(lo.xn); }
       aa.free_slot = chunk_slot; aa.free_slot_stride = 0;
       aa.chunk_mode = 1; aa.chunk_count0 = count0; aa.chunk_victim = chunk_victim;
+      {
+        const int kl[4] = {bp.prefix_len[0], D.M == 0 ? 0 : l1, D.M == 0 ? 0 : F - 1, N + 1};
+        aa.nsplit = attn_split(h, bp, kl, 4);
+      }
       aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
       aa.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
       VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, bp, h->at<int>(lo.status), st));
@@ -632,7 +741,7 @@ int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_strea
 
   // one text-like step of `count` rows right after the prompt; nothing is kept
   BatchParams bp;
-  std::memset(&bp, 0, sizeof(bp));
+  VS_BP_INIT(h, bp);
   bp.n_active = 1;
   bp.rows_per_stream = count;
   bp.stream_id[0] = stream_id;
@@ -644,23 +753,26 @@ int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_strea
   RopeArgs ra;
   ra.inv_freq = h->at<double>(lo.inv_freq); ra.rope = h->at<float2>(lo.rope); ra.D = D.D;
   VS_LAUNCH(h, st, KC_ROPE, launch_rope_table(ra, bp, st));
+  if (ensure_step_maps(h, rows) != VS_OK) return VS_ERR_CUDA;
 
   int cur = 0;
   for (int l = 0; l < D.L; ++l) {
     const bf16* h_in = h->at<bf16>(lo.hbuf[cur]);
     const bf16* src = h_in;
     if (D.use_rmsnorm) {
-      VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_scale),
-                                                    rows, D.d, D.rms_eps, st));
+      // layer 0: a launch of its own; deeper layers: the attention kernel that stored h_in left the statistics
+      if (l == 0) VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_ss),
+                                                                D.Hkv, rows, D.d, st));
       if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
     }
     ProjectionOut fa;
     std::memset(&fa, 0, sizeof(fa));
     fa.bias = h->bias[l];
-    fa.row_scale = D.use_rmsnorm ? h->at<float>(lo.row_scale) : nullptr;
+    fa.row_ss = D.use_rmsnorm ? h->at<float>(lo.row_ss) : nullptr; fa.ss_parts = D.Hkv; fa.norm_eps = D.rms_eps;
     fa.rope = h->at<float2>(lo.rope);
     fa.inv_freq = h->at<double>(lo.inv_freq);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
+    fa.q_tiled = h->at<bf16>(lo.q_tiled);
     fa.free_slot = h->at<int32_t>(lo.step_slot); fa.free_slot_stride = 0;
     fa.Hq = D.Hq; fa.Hkv = D.Hkv; fa.D = D.D; fa.slots = D.slots; fa.text_cap = 0; fa.mode = 3; fa.M = D.M;
     rc = run_projection(h, l, src, rows, fa, bp, st);
@@ -668,18 +780,21 @@ int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_strea
 
     AttnArgs aa;
     std::memset(&aa, 0, sizeof(aa));
-    aa.q = fa.q; aa.q_lo = fa.q_lo;
-    aa.seg[0] = {h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D),
-                 h->at<bf16>(lo.prefix_v) + (size_t)l * layer_stride_prefix(D),
-                 (long long)D.Hkv * D.maxP * D.D, (long long)D.maxP * D.D, (long long)D.D, 0, 0};
-    aa.seg[1] = {fa.kf, fa.vf, (long long)rows * D.Hkv * D.D, (long long)D.D, (long long)D.Hkv * D.D, 3, 1};
+    aa.q = fa.q; aa.q_lo = fa.q_lo; aa.q_tiled = fa.q_tiled;
+    seg_stored(aa.seg[0], h->tm_prefix_k, h->tm_prefix_v, 0, l, D);
+    seg_step(aa.seg[1], h->tm_step_k, h->tm_step_v, 3, rows);
     aa.n_seg = 2;
-    aa.out = (l == D.L - 1) ? out : h->at<void>(lo.obuf);
+    aa.out = (l == D.L - 1) ? out : (D.residual ? nullptr : h->at<void>(lo.obuf));
     aa.out_fp32 = D.out_fp32;
     aa.h_in = D.residual ? h_in : nullptr;
     aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
+    if (D.use_rmsnorm && l + 1 < D.L) { aa.ss_out = h->at<float>(lo.row_ss); aa.next_gain = h->gain[l + 1]; aa.xn_out = h->at<bf16>(lo.xn); }
     aa.free_slot = h->at<int32_t>(lo.step_slot); aa.free_slot_stride = 0;
     aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = 0;      // no bank segment on this key axis
+    {
+      const int kl[2] = {bp.prefix_len[0], rows};
+      aa.nsplit = attn_split(h, bp, kl, 2);
+    }
     aa.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
     VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, bp, h->at<int>(lo.status), st));
     if (D.residual) cur ^= 1;
@@ -708,9 +823,10 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
   VS_CK(cudaSetDevice(h->device));
 
   BatchParams bp;
-  std::memset(&bp, 0, sizeof(bp));
+  VS_BP_INIT(h, bp);
   bp.n_active = n_active;
   bp.rows_per_stream = T;
+  VS_TRACE_NEXT(h, bp);
   int max_keys = 0;
   for (int i = 0; i < n_active; ++i) {
     const HostStream& s = h->hs[stream_ids[i]];
@@ -734,9 +850,11 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
     VS_LAUNCH(h, st, KC_ROPE, launch_rope_table(ra, bp, st));
   }
 
+  if (T > 1 && ensure_step_maps(h, rows) != VS_OK) return VS_ERR_CUDA;
   const bf16* h_in = static_cast<const bf16*>(hidden);
   int next_buf = 0;
   for (int l = 0; l < D.L; ++l) {
+    if (l > 0) VS_TRACE_NEXT(h, bp);
     const bf16* src = h_in;
     // a step the matrix-vector kernel takes needs no statistics launch: that kernel normalises itself
     ProjectionOut probe;
@@ -744,8 +862,10 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
     probe.mode = 1; probe.D = D.D;
     const bool by_gemv = rope_inline && qkv_gemv_supported(probe, rows, D.d) && (reinterpret_cast<uintptr_t>(h_in) & 15u) == 0;
     if (D.use_rmsnorm && !by_gemv) {
-      VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_scale),
-                                                    rows, D.d, D.rms_eps, st));
+      // layer 0, and every layer of a single-token step (its attention kernel leaves no statistics): a launch of
+      // its own; else the tensor-core attention that stored h_in left them
+      if (l == 0 || T == 1) VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_ss),
+                                                                          D.Hkv, rows, D.d, st));
       if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
     }
     bf16* pk = h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D);
@@ -757,11 +877,13 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
 
     ProjectionOut fa;
     fa.bias = h->bias[l];
-    fa.row_scale = (D.use_rmsnorm && !by_gemv) ? h->at<float>(lo.row_scale) : nullptr;
+    fa.row_ss = (D.use_rmsnorm && !by_gemv) ? h->at<float>(lo.row_ss) : nullptr; fa.ss_parts = D.Hkv;
     fa.norm_inline = (D.use_rmsnorm && by_gemv) ? 1 : 0; fa.norm_gain = h->gain[l]; fa.norm_eps = D.rms_eps;
     fa.rope = rope_inline ? nullptr : h->at<float2>(lo.rope);
     fa.inv_freq = h->at<double>(lo.inv_freq);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
+    // a step of several rows goes to the tensor-core attention: its GEMM leaves the query in that kernel's layout
+    fa.q_tiled = (T > 1 && !by_gemv) ? h->at<bf16>(lo.q_tiled) : nullptr;
     fa.bank_k = bk; fa.bank_v = bv;
     fa.text_k = to_prefix ? pk : tk; fa.text_v = to_prefix ? pv : tv;
     fa.free_slot = &meta->free_slot; fa.free_slot_stride = (int)(sizeof(StreamMeta) / sizeof(int32_t));
@@ -793,19 +915,29 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
     } else {
       AttnArgs aa;
       std::memset(&aa, 0, sizeof(aa));
-      aa.q = fa.q; aa.q_lo = fa.q_lo;
+      aa.q = fa.q; aa.q_lo = fa.q_lo; aa.q_tiled = fa.q_tiled;
       int ns = 0;
-      aa.seg[ns++] = {pk, pv, (long long)D.Hkv * D.maxP * D.D, (long long)D.maxP * D.D, (long long)D.D, 0, 0};
+      seg_stored(aa.seg[ns++], h->tm_prefix_k, h->tm_prefix_v, 0, l, D);
       if (!to_prefix) {
-        aa.seg[ns++] = {bk, bv, (long long)D.Hkv * D.slots * D.D, (long long)D.slots * D.D, (long long)D.D, 1, 0};
-        aa.seg[ns++] = {tk, tv, (long long)D.Hkv * D.maxT * D.D, (long long)D.maxT * D.D, (long long)D.D, 2, 0};
+        seg_stored(aa.seg[ns++], h->tm_bank_k, h->tm_bank_v, 1, l, D);
+        seg_stored(aa.seg[ns++], h->tm_tail_k, h->tm_tail_v, 2, l, D);
       }
-      aa.seg[ns++] = {fa.kf, fa.vf, (long long)T * D.Hkv * D.D, (long long)D.D, (long long)D.Hkv * D.D, 3, 1};
+      seg_step(aa.seg[ns++], h->tm_step_k, h->tm_step_v, 3, T);
       aa.n_seg = ns;
-      aa.out = (l == D.L - 1) ? out : h->at<void>(lo.obuf);
+      {
+        int kl[4] = {0, 0, 0, T};
+        for (int i = 0; i < n_active; ++i) {
+          const int bl = (to_prefix || D.M == 0) ? 0 : (bp.count[i] == D.M ? D.M + 1 : bp.count[i]);
+          const int tl = to_prefix ? 0 : bp.text_len[i];
+          if (bp.prefix_len[i] + bl + tl > kl[0] + kl[1] + kl[2]) { kl[0] = bp.prefix_len[i]; kl[1] = bl; kl[2] = tl; }
+        }
+        aa.nsplit = attn_split(h, bp, kl, 4);
+      }
+      aa.out = (l == D.L - 1) ? out : (D.residual ? nullptr : h->at<void>(lo.obuf));
       aa.out_fp32 = D.out_fp32;
       aa.h_in = D.residual ? h_in : nullptr;
       aa.h_out = h_out;
+      if (D.use_rmsnorm && l + 1 < D.L && !by_gemv) { aa.ss_out = h->at<float>(lo.row_ss); aa.next_gain = h->gain[l + 1]; aa.xn_out = h->at<bf16>(lo.xn); }
       aa.free_slot = &meta->free_slot; aa.free_slot_stride = (int)(sizeof(StreamMeta) / sizeof(int32_t));
       aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
       aa.scale_log2e = scale_log2e;
@@ -831,7 +963,7 @@ int vs_reset_stream(vs_stream* h, const int32_t* stream_ids, int32_t n_active, v
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   VS_CK(cudaSetDevice(h->device));
   BatchParams bp;
-  std::memset(&bp, 0, sizeof(bp));
+  VS_BP_INIT(h, bp);
   bp.n_active = n_active;
   for (int i = 0; i < n_active; ++i) bp.stream_id[i] = stream_ids[i];
   VS_LAUNCH(h, st, KC_OTHER, launch_reset(h->at<StreamMeta>(h->lo.meta), h->at<int32_t>(h->lo.slot_frame), D.slots, bp, st));
@@ -964,6 +1096,15 @@ int vs_last_step_kv(vs_stream* h, void* k_out, void* v_out, int32_t rows) {
   if (v_out) VS_CK(cudaMemcpy(v_out, h->ws + h->lo.vf, bytes, cudaMemcpyDeviceToHost));
   return VS_OK;
 }
+
+#ifdef VS_TRACE
+// -DVS_TRACE build only: `log` = DEVICE buffer of VS_TRACE_WORDS 64-bit words, zeroed by the caller, or NULL to stop
+int vs_trace_set(vs_stream* h, void* log) {
+  if (h == nullptr) return VS_ERR_INVALID_ARG;
+  h->trace = static_cast<unsigned long long*>(log);
+  return VS_OK;
+}
+#endif
 
 int vs_poison_scratch(vs_stream* h, void* cuda_stream) {
   if (h == nullptr) return VS_ERR_INVALID_ARG;

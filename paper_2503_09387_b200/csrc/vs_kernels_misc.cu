@@ -28,6 +28,7 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, i
   const int sid = bp.stream_id[b];
   const int N = a.N, d = a.d;
   const long long pos0 = bp.pos_base[b];
+  VS_STAMP(bp, 0, 0);
   if ((int)blockIdx.x >= pool_blocks) {
     pdl_wait();
     pdl_launch_dependents();
@@ -52,6 +53,7 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, i
   bf16* dst = a.x + (size_t)b * (N + 1) * d + ch;
   pdl_wait();
   pdl_launch_dependents();
+  VS_STAMP(bp, 0, 1);
   uint4 v[MAXR];
 #pragma unroll
   for (int i = 0; i < MAXR; ++i) {
@@ -101,6 +103,7 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, i
       if (blockIdx.x == 0 && threadIdx.x == 0) a.step_slot[sid] = slot;
     }
   }
+  VS_STAMP(bp, 0, 15);
 }
 
 cudaError_t launch_pool(const PoolArgs& a, const BatchParams& bp, cudaStream_t st) {
@@ -130,15 +133,17 @@ cudaError_t launch_rope_table(const RopeArgs& a, const BatchParams& bp, cudaStre
 }
 
 // ------------------------------------------------------------------------------------------
-// RMSNorm statistics of the layer input.  xn = h * r * gain with r = 1 / sqrt(mean(h^2) + eps).
-// The row scale r commutes with the projection, so it is applied in fp32 in the GEMM epilogue
-// and the GEMM reads the bf16 residual stream itself: no rounded copy of the normalised
-// activations exists (with a gain vector, bf16(h * gain) is written and read instead).
-// One block per row.
+// RMSNorm statistics of a layer input that no kernel of this library produced (layer 0; deeper
+// layers get theirs from the attention kernel that stores the residual rows).
+// xn = h * r * gain with r = 1 / sqrt(mean(h^2) + eps).  The row scale r commutes with the
+// projection, so the projection applies it in fp32 in its epilogue and reads the bf16 residual
+// stream itself: no rounded copy of the normalised activations exists (with a gain vector,
+// bf16(h * gain) is written and read instead).  This kernel leaves the row's sum of squares in
+// part 0 of row_ss[row][parts].  One block per row.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) rms_stats_kernel(const bf16* __restrict__ h, const bf16* __restrict__ gain,
-                                                        bf16* __restrict__ hg, float* __restrict__ row_scale,
-                                                        int d, float eps) {
+                                                        bf16* __restrict__ hg, float* __restrict__ row_ss,
+                                                        int parts, int d) {
   pdl_wait();
   pdl_launch_dependents();
   const size_t row = blockIdx.x;
@@ -161,13 +166,14 @@ __global__ void __launch_bounds__(256) rms_stats_kernel(const bf16* __restrict__
     float tot = 0.f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) tot += red[i];
-    row_scale[row] = rsqrtf(tot / (float)d + eps);
+    row_ss[row * parts] = tot;
+    for (int i = 1; i < parts; ++i) row_ss[row * parts + i] = 0.f;
   }
 }
 
-cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* row_scale, int rows, int d, float eps,
+cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* row_ss, int parts, int rows, int d,
                              cudaStream_t st) {
-  return launch_pdl(rms_stats_kernel, dim3(rows), dim3(256), 0, st, h, gain, hg, row_scale, d, eps);
+  return launch_pdl(rms_stats_kernel, dim3(rows), dim3(256), 0, st, h, gain, hg, row_ss, parts, d);
 }
 
 // The bank update of one frame as a launch of its own (chunked prefill).
