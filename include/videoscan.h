@@ -44,6 +44,8 @@ extern "C" {
 #define VS_ERR_CUDA            -4   /* a CUDA runtime or driver call failed                 */
 #define VS_ERR_DEVICE_TIMEOUT  -5   /* a bounded device-side wait expired                   */
 #define VS_ERR_UNSUPPORTED     -6   /* shape outside what the kernels are built for         */
+#define VS_ERR_BOUNDS          -7   /* checked build (-DVS_DEBUG_BOUNDS) only: a kernel tried to store outside the buffer
+                                       it was writing, or the guard words behind a workspace region were overwritten */
 
 #define VS_MAX_BATCH           64   /* most streams one call may list                       */
 #define VS_N_KERNEL_CLASSES    10   /* kernel classes reported by vs_profile_read           */
@@ -105,7 +107,7 @@ typedef struct {
   int64_t prefix_len;
   int64_t text_len;
   int32_t last_victim_frame;     /* frame id discarded by the last frame step, -1 if none            */
-  int32_t device_status;         /* 0, or VS_ERR_DEVICE_TIMEOUT                                      */
+  int32_t device_status;         /* 0, or VS_ERR_DEVICE_TIMEOUT (or VS_ERR_BOUNDS in a checked build)  */
   uint64_t persistent_bytes;     /* bytes of the workspace that hold stream state; constant          */
   uint64_t workspace_bytes;      /* whole workspace; constant for the life of the handle             */
 } vs_bank_info;

@@ -24,6 +24,7 @@ VS_ERR_CAPACITY = -3
 VS_ERR_CUDA = -4
 VS_ERR_DEVICE_TIMEOUT = -5
 VS_ERR_UNSUPPORTED = -6
+VS_ERR_BOUNDS = -7
 VS_MAX_BATCH = 64
 
 EXPORTS = ["vs_workspace_bytes", "vs_create_stream", "vs_frame_prefill", "vs_frame_prefill_chunk", "vs_bank_forward", "vs_decode_step",

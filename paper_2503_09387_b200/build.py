@@ -33,9 +33,16 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
+CHECKED_LIB_PATH = os.path.join(LIB_DIR, "libvideoscan_checked.so")
+
+
+def build_library(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """checked=True builds the same sources with -DVS_DEBUG_BOUNDS into libvideoscan_checked.so: every kernel store into
+    the workspace is checked against the region it names, and guard bytes lie behind every region."""
     os.makedirs(LIB_DIR, exist_ok=True)
-    obj_dir = os.path.join(LIB_DIR, "obj")
+    obj_dir = os.path.join(LIB_DIR, "obj_checked" if checked else "obj")
+    lib_path = CHECKED_LIB_PATH if checked else LIB_PATH
+    extra = ["-DVS_DEBUG_BOUNDS"] if checked else []
     os.makedirs(obj_dir, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
     headers.append(os.path.join(os.path.dirname(HERE), "include", "videoscan.h"))
@@ -44,7 +51,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         s = os.path.join(CSRC, src)
         o = os.path.join(obj_dir, src.replace(".cu", ".o"))
         if force or _stale(o, [s] + headers):
-            cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
+            cmd = [_nvcc()] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
             jobs.append(cmd)
     def run(cmd):
         r = subprocess.run(cmd, capture_output=True, text=True)
@@ -55,11 +62,11 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     with ThreadPoolExecutor(max_workers=4) as ex:
         list(ex.map(run, jobs))
     objs = [os.path.join(obj_dir, s.replace(".cu", ".o")) for s in SOURCES]
-    if force or jobs or _stale(LIB_PATH, objs):
-        cmd = [_nvcc(), "-shared", "-cudart", "static", "-o", LIB_PATH] + objs + ["-lpthread", "-ldl", "-lrt"]
+    if force or jobs or _stale(lib_path, objs):
+        cmd = [_nvcc(), "-shared", "-cudart", "static", "-o", lib_path] + objs + ["-lpthread", "-ldl", "-lrt"]
         run(cmd)
-    return LIB_PATH
+    return lib_path
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

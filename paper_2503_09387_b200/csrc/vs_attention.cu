@@ -218,7 +218,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
       const float val = (L > 0.f) ? O / L : 0.f;
       if (a.out_fp32) static_cast<float*>(a.out)[out_off + c] = val;
       else static_cast<bf16*>(a.out)[out_off + c] = __float2bfloat16_rn(val);
-      if (a.h_out != nullptr) a.h_out[out_off + c] = __float2bfloat16_rn(h_res + val);
+      if (a.h_out != nullptr && VS_STORE_OK(bp, a.h_out_region, a.h_out + out_off + c, 2)) a.h_out[out_off + c] = __float2bfloat16_rn(h_res + val);
     } else {
       cta_o[c] = O;
       if (c == 0) { cta_ml[0] = M; cta_ml[1] = L; }
@@ -257,7 +257,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
     val = (L > 0.f) ? val / L : 0.f;
     if (a.out_fp32) static_cast<float*>(a.out)[out_off + c] = val;
     else static_cast<bf16*>(a.out)[out_off + c] = __float2bfloat16_rn(val);
-    if (a.h_out != nullptr) a.h_out[out_off + c] = __float2bfloat16_rn(h_res + val);
+    if (a.h_out != nullptr && VS_STORE_OK(bp, a.h_out_region, a.h_out + out_off + c, 2)) a.h_out[out_off + c] = __float2bfloat16_rn(h_res + val);
   }
   // nobody's shared memory goes away while rank 0 may still be reading it
   cluster_sync();

@@ -805,7 +805,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(const 
             const float2 h1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hraw.y));
             __nv_bfloat162 lo = __floats2bfloat162_rn(h0.x + v[k].x, h0.y + v[k].y), hi = __floats2bfloat162_rn(h1.x + v[k].z, h1.y + v[k].w);
             uint2 w; w.x = *reinterpret_cast<uint32_t*>(&lo); w.y = *reinterpret_cast<uint32_t*>(&hi);
-            *reinterpret_cast<uint2*>(a.h_out + obase + 4 * u) = w;
+            if (VS_STORE_OK(bp, a.h_out_region, a.h_out + obase + 4 * u, 8)) *reinterpret_cast<uint2*>(a.h_out + obase + 4 * u) = w;
             if (a.ss_out != nullptr) {
               // RMSNorm of the next layer: its statistics are those of the rows as stored (bf16)
               const float2 s0 = __bfloat1622float2(lo), s1 = __bfloat1622float2(hi);
@@ -817,7 +817,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(const 
                 const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&graw.y));
                 __nv_bfloat162 x0 = __floats2bfloat162_rn(s0.x * g0.x, s0.y * g0.y), x1 = __floats2bfloat162_rn(s1.x * g1.x, s1.y * g1.y);
                 uint2 xw; xw.x = *reinterpret_cast<uint32_t*>(&x0); xw.y = *reinterpret_cast<uint32_t*>(&x1);
-                *reinterpret_cast<uint2*>(a.xn_out + obase + 4 * u) = xw;
+                if (VS_STORE_OK(bp, DR_XN, a.xn_out + obase + 4 * u, 8)) *reinterpret_cast<uint2*>(a.xn_out + obase + 4 * u) = xw;
               }
             }
           }
@@ -836,7 +836,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) prefill_attn_tc_kernel(const 
       if (tid < kTok && tid % nsplit == split && r0 + tid < rps) {
         float tot = 0.f;
         for (int gg = 0; gg < G; ++gg) tot += ss_stage[gg * 16 + tid];
-        a.ss_out[((size_t)b * rps + r0 + tid) * a.Hkv + hkv] = tot;
+        float* sp = a.ss_out + ((size_t)b * rps + r0 + tid) * a.Hkv + hkv;
+        if (VS_STORE_OK(bp, DR_ROW_SS, sp, 4)) *sp = tot;
       }
     }
   }

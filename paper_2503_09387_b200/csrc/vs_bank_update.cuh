@@ -65,7 +65,7 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
   auto adopt = [&]() {      // all threads of the committing block
     if (a.incoming_emb != nullptr) {
       bf16* dst = const_cast<bf16*>(a.emb) + ((size_t)sid * a.slots + incoming) * a.d;
-      for (int k = tid; k < a.d; k += blockDim.x) dst[k] = emb_in[k];
+      for (int k = tid; k < a.d; k += blockDim.x) if (VS_STORE_OK(bp, DR_EMB, dst + k, 2)) dst[k] = emb_in[k];
       if (tid == 0) { a.record_slot[b] = incoming; a.record_victim[b] = -1; }
     }
   };
@@ -73,9 +73,9 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
   if (count < a.M) {
     if (block == 0) adopt();
     if (block == 0 && tid == 0) {
-      order[count] = incoming;
-      slot_frame[incoming] = (int32_t)bp.frame_id[b];
-      slot_pos[incoming] = carrier_pos;
+      if (VS_STORE_OK(bp, DR_ORDER, order + count, 4)) order[count] = incoming;
+      if (VS_STORE_OK(bp, DR_SLOT_FRAME, slot_frame + incoming, 4)) slot_frame[incoming] = (int32_t)bp.frame_id[b];
+      if (VS_STORE_OK(bp, DR_SLOT_POS, slot_pos + incoming, 8)) slot_pos[incoming] = carrier_pos;
       meta->count = count + 1;
       meta->free_slot = count + 1;          // slots fill in order until the bank is full
       meta->last_victim_frame = -1;
@@ -97,7 +97,7 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
     const bf16* va = a.emb + ((size_t)sid * a.slots + sa) * a.d;
     const bf16* vb = (sb == incoming) ? emb_in : a.emb + ((size_t)sid * a.slots + sb) * a.d;
     const double s = warp_cosine(va, vb, a.d, lane);
-    if (lane == 0) scores[j] = s;
+    if (lane == 0 && VS_STORE_OK(bp, DR_SCORES, scores + j, 8)) scores[j] = s;
   }
   __shared__ int is_last;
   __threadfence();
@@ -148,18 +148,17 @@ __device__ __forceinline__ void bank_update_block(const BankUpdateArgs& a, const
     const int jj = base + tid;
     const int32_t next = (on && jj < count - 1) ? order[jj + 1] : 0;
     __syncthreads();
-    if (on && jj < count - 1) order[jj] = next;
+    if (on && jj < count - 1 && VS_STORE_OK(bp, DR_ORDER, order + jj, 4)) order[jj] = next;
     __syncthreads();
   }
   if (tid == 0) {
-    order[count - 1] = incoming;
-    slot_frame[victim_slot] = -1;
-    slot_frame[incoming] = (int32_t)bp.frame_id[b];
-    slot_pos[incoming] = carrier_pos;
+    if (VS_STORE_OK(bp, DR_ORDER, order + count - 1, 4)) order[count - 1] = incoming;
+    if (VS_STORE_OK(bp, DR_SLOT_FRAME, slot_frame + victim_slot, 4)) slot_frame[victim_slot] = -1;
+    if (VS_STORE_OK(bp, DR_SLOT_FRAME, slot_frame + incoming, 4)) slot_frame[incoming] = (int32_t)bp.frame_id[b];
+    if (VS_STORE_OK(bp, DR_SLOT_POS, slot_pos + incoming, 8)) slot_pos[incoming] = carrier_pos;
     if (a.log_cap > 0) {
       int32_t* e = a.evict_log + ((size_t)sid * a.log_cap + (meta->log_count % a.log_cap)) * 2;
-      e[0] = (int32_t)bp.frame_id[b];
-      e[1] = victim_frame;
+      if (VS_STORE_OK(bp, DR_EVICT_LOG, e, 8)) { e[0] = (int32_t)bp.frame_id[b]; e[1] = victim_frame; }
     }
     meta->log_count += 1;
     meta->evictions += 1;

@@ -42,7 +42,37 @@ struct BatchParams {
   unsigned long long* trace;           // timeline log of a -DVS_TRACE build, or null
   unsigned trace_seq;                  // sequence number of the launch
 #endif
+#ifdef VS_DEBUG_BOUNDS
+  struct DebugTable* dbg;              // workspace regions of a checked build
+#endif
 };
+
+// ---- checked stores (only in a -DVS_DEBUG_BOUNDS build; the product build compiles none of it) ----
+// Stand-in for a memory checker: every store of a kernel into the workspace names the region it
+// means to write; a store outside that region is skipped and the first one is recorded (region,
+// byte offset from the region's start) -- no trap.  Behind every region lie 256 guard bytes that
+// vs_bank_state verifies.  Either finding is reported as VS_ERR_BOUNDS.
+enum DbgRegion { DR_BANK_K = 0, DR_BANK_V, DR_PREFIX_K, DR_PREFIX_V, DR_TAIL_K, DR_TAIL_V, DR_EMB, DR_META, DR_ORDER,
+                 DR_SLOT_FRAME, DR_SLOT_POS, DR_EVICT_LOG, DR_SCORES, DR_STEP_SLOT, DR_CHUNK_SLOT, DR_CHUNK_VICTIM,
+                 DR_GEMM_FLAGS, DR_HBUF0, DR_HBUF1, DR_XN, DR_ROW_SS, DR_Q, DR_Q_LO, DR_Q_TILED, DR_KF, DR_VF, DR_ROPE,
+                 DR_OBUF, DR_EMB_STAGE, DR_CHUNK_SCORES, DR_GEMM_XCHG, DR_COUNT };
+struct DebugTable {
+  unsigned long long begin[DR_COUNT], end[DR_COUNT];   // device addresses
+  int bad_region;                                      // -1, or the region of the first refused store
+  long long bad_offset;
+};
+#if defined(VS_DEBUG_BOUNDS) && defined(__CUDACC__)
+__device__ __forceinline__ bool vs_store_ok(const BatchParams& bp, int region, const void* p, size_t bytes) {
+  if (bp.dbg == nullptr) return true;
+  const unsigned long long a = reinterpret_cast<unsigned long long>(p);
+  if (a >= bp.dbg->begin[region] && a + bytes <= bp.dbg->end[region]) return true;
+  if (atomicCAS(&bp.dbg->bad_region, -1, region) == -1) bp.dbg->bad_offset = (long long)(a - bp.dbg->begin[region]);
+  return false;
+}
+#define VS_STORE_OK(bp, region, p, bytes) vs_store_ok(bp, region, p, bytes)
+#else
+#define VS_STORE_OK(bp, region, p, bytes) true
+#endif
 
 // ---- shapes ----------------------------------------------------------------------------
 struct Dims {
@@ -96,6 +126,9 @@ struct Layout {
   size_t gemm_xchg;             // f32  [GEMM_XCHG_CTAS][256][128]  projection K split: partial tiles
   size_t scratch_begin, scratch_end;
   size_t total;
+  // checked build: the regions as the kernels name them, and the table the kernels read
+  size_t region_begin[DR_COUNT], region_end[DR_COUNT];
+  size_t dbg_table;
 };
 
 // ---- timeline trace (only in a -DVS_TRACE build; the product build compiles none of it) ----------
@@ -281,6 +314,7 @@ struct AttnArgs {
   float* ss_out;
   const bf16* next_gain;
   bf16* xn_out;
+  int h_out_region;              // checked build: which residual buffer h_out is (DR_HBUF0 / DR_HBUF1)
   const int32_t* free_slot;      // free slot of stream s at free_slot[s * free_slot_stride]
   int free_slot_stride;
   int Hq, Hkv, D, slots, M;
@@ -329,6 +363,7 @@ struct DecodeArgs {
   void* out;                     // [n_active][Hq*D], bf16 or fp32
   int out_fp32;
   const bf16* h_in; bf16* h_out;
+  int h_out_region;              // checked build: which residual buffer h_out is (DR_HBUF0 / DR_HBUF1)
   const StreamMeta* meta;
   int Hq, Hkv, D, slots, M, maxP, maxT;
   int nsplit;                    // CTAs sharing one row's keys (a cluster): 1, 2, 4 or 8

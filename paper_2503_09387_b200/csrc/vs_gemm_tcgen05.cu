@@ -315,7 +315,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
       for (int j = 0; j < 16; ++j) {
         const int t = c + j;
         if ((unsigned)(t - t_begin) < (unsigned)slice) dst_own[(t - t_begin) * GEMM_BLOCK_M] = __uint_as_float(r[j]);
-        else dst_far[(size_t)t * GEMM_BLOCK_M] = __uint_as_float(r[j]);
+        else if (VS_STORE_OK(bp, DR_GEMM_XCHG, dst_far + (size_t)t * GEMM_BLOCK_M, 4)) dst_far[(size_t)t * GEMM_BLOCK_M] = __uint_as_float(r[j]);
       }
     }
   }
@@ -443,23 +443,30 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
             const uint32_t o_1 = (uint32_t)((c1 >> 3) * (128 * 128) + r * 128 + (((c1 & 7) ^ (r & 7)) << 4) + (k0 & 7) * 2);
             const uint32_t o_2 = (uint32_t)((c2 >> 3) * (128 * 128) + r * 128 + (((c2 & 7) ^ (r & 7)) << 4) + (k0 & 7) * 2);
             const uint32_t lo_off = (uint32_t)(128 * D * 2);
-            *reinterpret_cast<uint2*>(tb + o_1) = w1;
-            *reinterpret_cast<uint2*>(tb + o_2) = w2;
-            *reinterpret_cast<uint2*>(tb + lo_off + o_1) = *reinterpret_cast<const uint2*>(l1);
-            *reinterpret_cast<uint2*>(tb + lo_off + o_2) = *reinterpret_cast<const uint2*>(l2);
+            if (VS_STORE_OK(bp, DR_Q_TILED, tb + o_1, 8) && VS_STORE_OK(bp, DR_Q_TILED, tb + lo_off + o_2, 8)) {
+              *reinterpret_cast<uint2*>(tb + o_1) = w1;
+              *reinterpret_cast<uint2*>(tb + o_2) = w2;
+              *reinterpret_cast<uint2*>(tb + lo_off + o_1) = *reinterpret_cast<const uint2*>(l1);
+              *reinterpret_cast<uint2*>(tb + lo_off + o_2) = *reinterpret_cast<const uint2*>(l2);
+            }
           } else {
             const size_t qo = (size_t)row * p.o.Hq * D + (size_t)hs * D + k0;
-            *reinterpret_cast<uint2*>(p.o.q + qo) = w1;
-            *reinterpret_cast<uint2*>(p.o.q + qo + half) = w2;
-            *reinterpret_cast<uint2*>(p.o.q_lo + qo) = *reinterpret_cast<const uint2*>(l1);
-            *reinterpret_cast<uint2*>(p.o.q_lo + qo + half) = *reinterpret_cast<const uint2*>(l2);
+            if (VS_STORE_OK(bp, DR_Q, p.o.q + qo, 8) && VS_STORE_OK(bp, DR_Q, p.o.q + qo + half, 8) &&
+                VS_STORE_OK(bp, DR_Q_LO, p.o.q_lo + qo, 8) && VS_STORE_OK(bp, DR_Q_LO, p.o.q_lo + qo + half, 8)) {
+              *reinterpret_cast<uint2*>(p.o.q + qo) = w1;
+              *reinterpret_cast<uint2*>(p.o.q + qo + half) = w2;
+              *reinterpret_cast<uint2*>(p.o.q_lo + qo) = *reinterpret_cast<const uint2*>(l1);
+              *reinterpret_cast<uint2*>(p.o.q_lo + qo + half) = *reinterpret_cast<const uint2*>(l2);
+            }
           }
         } else {
           const bool is_k = hs < p.o.Hq + p.o.Hkv;
           const int hkv = is_k ? hs - p.o.Hq : hs - p.o.Hq - p.o.Hkv;
           bf16* f = (is_k ? p.o.kf : p.o.vf) + (size_t)row * p.o.Hkv * D + (size_t)hkv * D + k0;
-          *reinterpret_cast<uint2*>(f) = w1;
-          *reinterpret_cast<uint2*>(f + half) = w2;
+          if (VS_STORE_OK(bp, is_k ? DR_KF : DR_VF, f, 8) && VS_STORE_OK(bp, is_k ? DR_KF : DR_VF, f + half, 8)) {
+            *reinterpret_cast<uint2*>(f) = w1;
+            *reinterpret_cast<uint2*>(f + half) = w2;
+          }
           const int b = row / rps, tt = row - b * rps;
           const int sid = bp.stream_id[b];
           bf16* dst = nullptr;
@@ -472,7 +479,10 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
             const int tb = (p.o.mode == 1) ? bp.prefix_len[b] : bp.text_len[b];
             dst = (is_k ? p.o.text_k : p.o.text_v) + (((size_t)sid * p.o.Hkv + hkv) * p.o.text_cap + tb + tt) * D + k0;
           }
-          if (dst != nullptr) {
+          // (the carrier row goes to the bank, text rows to the prefix or the tail)
+          const int dreg = (p.o.mode == 0) ? (is_k ? DR_BANK_K : DR_BANK_V)
+                                           : (p.o.mode == 1 ? (is_k ? DR_PREFIX_K : DR_PREFIX_V) : (is_k ? DR_TAIL_K : DR_TAIL_V));
+          if (dst != nullptr && VS_STORE_OK(bp, dreg, dst, 8) && VS_STORE_OK(bp, dreg, dst + half, 8)) {
             *reinterpret_cast<uint2*>(dst) = w1;
             *reinterpret_cast<uint2*>(dst + half) = w2;
           }

@@ -218,18 +218,22 @@ __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __res
     if (hs < o.Hq) {
       // the query stays inside the step: kept as a bf16 pair (hi + lo)
       const size_t qo = (size_t)row * o.Hq * D + (size_t)hs * D + k0;
-      o.q[qo] = o1; o.q[qo + half] = o2;
-      o.q_lo[qo] = __float2bfloat16_rn(x1 - __bfloat162float(o1));
-      o.q_lo[qo + half] = __float2bfloat16_rn(x2 - __bfloat162float(o2));
+      if (VS_STORE_OK(bp, DR_Q, o.q + qo, 2) && VS_STORE_OK(bp, DR_Q, o.q + qo + half, 2) &&
+          VS_STORE_OK(bp, DR_Q_LO, o.q_lo + qo, 2) && VS_STORE_OK(bp, DR_Q_LO, o.q_lo + qo + half, 2)) {
+        o.q[qo] = o1; o.q[qo + half] = o2;
+        o.q_lo[qo] = __float2bfloat16_rn(x1 - __bfloat162float(o1));
+        o.q_lo[qo + half] = __float2bfloat16_rn(x2 - __bfloat162float(o2));
+      }
     } else {
       const bool is_k = hs < o.Hq + o.Hkv;
       const int hkv = is_k ? hs - o.Hq : hs - o.Hq - o.Hkv;
       bf16* f = (is_k ? o.kf : o.vf) + (size_t)row * o.Hkv * D + (size_t)hkv * D + k0;
-      f[0] = o1; f[half] = o2;
+      if (VS_STORE_OK(bp, is_k ? DR_KF : DR_VF, f, 2) && VS_STORE_OK(bp, is_k ? DR_KF : DR_VF, f + half, 2)) { f[0] = o1; f[half] = o2; }
       const int sid = bp.stream_id[fb];
       const int tb = (o.mode == 1) ? bp.prefix_len[fb] : bp.text_len[fb];
       bf16* dst = (is_k ? o.text_k : o.text_v) + (((size_t)sid * o.Hkv + hkv) * o.text_cap + tb + ftt) * D + k0;
-      dst[0] = o1; dst[half] = o2;
+      const int dreg = (o.mode == 1) ? (is_k ? DR_PREFIX_K : DR_PREFIX_V) : (is_k ? DR_TAIL_K : DR_TAIL_V);
+      if (VS_STORE_OK(bp, dreg, dst, 2) && VS_STORE_OK(bp, dreg, dst + half, 2)) { dst[0] = o1; dst[half] = o2; }
     }
   }
   VS_STAMP(bp, 4, 15);

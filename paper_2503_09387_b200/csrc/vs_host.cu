@@ -60,46 +60,58 @@ int fill_dims(const vs_config* c, Dims& D) {
   return VS_OK;
 }
 
+// Checked build: 256 guard bytes behind every region (vs_bank_state verifies them).
+#ifdef VS_DEBUG_BOUNDS
+constexpr size_t kGuardBytes = 256;
+#else
+constexpr size_t kGuardBytes = 0;
+#endif
+constexpr unsigned char kGuardByte = 0xC5;
+
 void fill_layout(const Dims& D, Layout& Lo) {
   size_t off = 0;
-  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  size_t last_bytes = 0;
+  auto take = [&](size_t bytes) { size_t o = off; last_bytes = bytes; off = align_up(off + bytes, 256) + kGuardBytes; return o; };
+  for (int r = 0; r < DR_COUNT; ++r) { Lo.region_begin[r] = 0; Lo.region_end[r] = 0; }
+  auto reg = [&](int r, size_t o) { Lo.region_begin[r] = o; Lo.region_end[r] = o + last_bytes; return o; };
   const size_t kv_bank = (size_t)D.L * D.S * D.Hkv * D.slots * D.D * 2;
   const size_t kv_pre = (size_t)D.L * D.S * D.Hkv * D.maxP * D.D * 2;
   const size_t kv_tail = (size_t)D.L * D.S * D.Hkv * D.maxT * D.D * 2;
-  Lo.bank_k = take(kv_bank); Lo.bank_v = take(kv_bank);
-  Lo.prefix_k = take(kv_pre); Lo.prefix_v = take(kv_pre);
-  Lo.tail_k = take(kv_tail); Lo.tail_v = take(kv_tail);
-  Lo.emb = take((size_t)D.S * D.slots * D.d * 2);
-  Lo.meta = take((size_t)D.S * sizeof(StreamMeta));
-  Lo.order = take((size_t)D.S * D.slots * 4);
-  Lo.slot_frame = take((size_t)D.S * D.slots * 4);
-  Lo.slot_pos = take((size_t)D.S * D.slots * 8);
-  Lo.evict_log = take((size_t)D.S * (D.log_cap > 0 ? D.log_cap : 1) * 8);
-  Lo.scores = take((size_t)D.S * D.slots * 8);
+  Lo.bank_k = reg(DR_BANK_K, take(kv_bank)); Lo.bank_v = reg(DR_BANK_V, take(kv_bank));
+  Lo.prefix_k = reg(DR_PREFIX_K, take(kv_pre)); Lo.prefix_v = reg(DR_PREFIX_V, take(kv_pre));
+  Lo.tail_k = reg(DR_TAIL_K, take(kv_tail)); Lo.tail_v = reg(DR_TAIL_V, take(kv_tail));
+  Lo.emb = reg(DR_EMB, take((size_t)D.S * D.slots * D.d * 2));
+  Lo.meta = reg(DR_META, take((size_t)D.S * sizeof(StreamMeta)));
+  Lo.order = reg(DR_ORDER, take((size_t)D.S * D.slots * 4));
+  Lo.slot_frame = reg(DR_SLOT_FRAME, take((size_t)D.S * D.slots * 4));
+  Lo.slot_pos = reg(DR_SLOT_POS, take((size_t)D.S * D.slots * 8));
+  Lo.evict_log = reg(DR_EVICT_LOG, take((size_t)D.S * (D.log_cap > 0 ? D.log_cap : 1) * 8));
+  Lo.scores = reg(DR_SCORES, take((size_t)D.S * D.slots * 8));
   Lo.inv_freq = take((size_t)(D.D / 2) * 8);
   Lo.status = take(8 * 4);
-  Lo.step_slot = take((size_t)D.S * 4);
-  Lo.chunk_slot = take((size_t)VS_MAX_BATCH * 4);
-  Lo.chunk_victim = take((size_t)VS_MAX_BATCH * 4);
-  Lo.gemm_flags = take((size_t)GEMM_XCHG_CTAS * 4);
+  Lo.step_slot = reg(DR_STEP_SLOT, take((size_t)D.S * 4));
+  Lo.chunk_slot = reg(DR_CHUNK_SLOT, take((size_t)VS_MAX_BATCH * 4));
+  Lo.chunk_victim = reg(DR_CHUNK_VICTIM, take((size_t)VS_MAX_BATCH * 4));
+  Lo.gemm_flags = reg(DR_GEMM_FLAGS, take((size_t)GEMM_XCHG_CTAS * 4));
+  Lo.dbg_table = take(sizeof(DebugTable));
   Lo.persistent_end = off;
   Lo.scratch_begin = off;
-  Lo.hbuf[0] = take((size_t)D.R_max * D.d * 2);
-  Lo.hbuf[1] = take((size_t)D.R_max * D.d * 2);
-  Lo.xn = take((size_t)D.R_max * D.d * 2);
-  Lo.row_ss = take((size_t)D.R_max * D.Hkv * 4);
-  Lo.q = take((size_t)D.R_max * D.Hq * D.D * 2);
-  Lo.q_lo = take((size_t)D.R_max * D.Hq * D.D * 2);
+  Lo.hbuf[0] = reg(DR_HBUF0, take((size_t)D.R_max * D.d * 2));
+  Lo.hbuf[1] = reg(DR_HBUF1, take((size_t)D.R_max * D.d * 2));
+  Lo.xn = reg(DR_XN, take((size_t)D.R_max * D.d * 2));
+  Lo.row_ss = reg(DR_ROW_SS, take((size_t)D.R_max * D.Hkv * 4));
+  Lo.q = reg(DR_Q, take((size_t)D.R_max * D.Hq * D.D * 2));
+  Lo.q_lo = reg(DR_Q_LO, take((size_t)D.R_max * D.Hq * D.D * 2));
   // the query in the attention kernel's operand layout: per batch entry ceil(rows / 16) row tiles, per tile and KV
   // head a block of [hi | lo][128][D]
-  Lo.q_tiled = take(((size_t)D.R_max / 16 + (size_t)VS_MAX_BATCH + 1) * D.Hkv * 2 * 128 * D.D * 2);
-  Lo.kf = take((size_t)D.R_max * D.Hkv * D.D * 2);
-  Lo.vf = take((size_t)D.R_max * D.Hkv * D.D * 2);
-  Lo.rope = take((size_t)D.R_max * (D.D / 2) * 8);
-  Lo.obuf = take((size_t)D.R_max * D.Hq * D.D * 4);
-  Lo.emb_stage = take((size_t)D.maxChunk * D.d * 2);
-  Lo.chunk_scores = take(D.maxChunk > 1 ? (size_t)D.maxChunk * (D.slots + D.maxChunk) * 8 : 8);
-  Lo.gemm_xchg = take((size_t)GEMM_XCHG_CTAS * 256 * GEMM_BLOCK_M * 4);
+  Lo.q_tiled = reg(DR_Q_TILED, take(((size_t)D.R_max / 16 + (size_t)VS_MAX_BATCH + 1) * D.Hkv * 2 * 128 * D.D * 2));
+  Lo.kf = reg(DR_KF, take((size_t)D.R_max * D.Hkv * D.D * 2));
+  Lo.vf = reg(DR_VF, take((size_t)D.R_max * D.Hkv * D.D * 2));
+  Lo.rope = reg(DR_ROPE, take((size_t)D.R_max * (D.D / 2) * 8));
+  Lo.obuf = reg(DR_OBUF, take((size_t)D.R_max * D.Hq * D.D * 4));
+  Lo.emb_stage = reg(DR_EMB_STAGE, take((size_t)D.maxChunk * D.d * 2));
+  Lo.chunk_scores = reg(DR_CHUNK_SCORES, take(D.maxChunk > 1 ? (size_t)D.maxChunk * (D.slots + D.maxChunk) * 8 : 8));
+  Lo.gemm_xchg = reg(DR_GEMM_XCHG, take((size_t)GEMM_XCHG_CTAS * 256 * GEMM_BLOCK_M * 4));
   Lo.scratch_end = off;
   Lo.total = off;
 }
@@ -245,7 +257,10 @@ int check_ids(vs_stream* h, const int32_t* ids, int32_t n) {
   return VS_OK;
 }
 
-#ifdef VS_TRACE
+#if defined(VS_DEBUG_BOUNDS)
+#define VS_BP_INIT(h, bp) do { std::memset(&(bp), 0, sizeof(bp)); (bp).dbg = (h)->at<DebugTable>((h)->lo.dbg_table); } while (0)
+#define VS_TRACE_NEXT(h, bp)
+#elif defined(VS_TRACE)
 #define VS_BP_INIT(h, bp) do { std::memset(&(bp), 0, sizeof(bp)); (bp).trace = (h)->trace; (bp).trace_seq = (h)->trace_seq; } while (0)
 #define VS_TRACE_NEXT(h, bp) do { (bp).trace_seq = ++(h)->trace_seq; } while (0)
 #else
@@ -313,6 +328,7 @@ const char* vs_status_string(int status) {
     case VS_ERR_CUDA: return "CUDA call failed";
     case VS_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
     case VS_ERR_UNSUPPORTED: return "unsupported shape";
+    case VS_ERR_BOUNDS: return "store outside a workspace region (checked build)";
     default: return "unknown status";
   }
 }
@@ -389,6 +405,20 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights, void* work
   for (int k = 0; k < D.D / 2; ++k) inv[k] = std::pow((double)D.rope_theta, -2.0 * (double)k / (double)D.D);
   if (cudaMemcpy(h->ws + lo.inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice) != cudaSuccess)
     return fail(VS_ERR_CUDA);
+#ifdef VS_DEBUG_BOUNDS
+  {
+    DebugTable t;
+    std::memset(&t, 0, sizeof(t));
+    for (int r = 0; r < DR_COUNT; ++r) {
+      t.begin[r] = reinterpret_cast<unsigned long long>(h->ws + lo.region_begin[r]);
+      t.end[r] = reinterpret_cast<unsigned long long>(h->ws + lo.region_end[r]);
+      if (lo.region_end[r] > lo.region_begin[r] &&
+          cudaMemset(h->ws + align_up(lo.region_end[r], 256), kGuardByte, kGuardBytes) != cudaSuccess) return fail(VS_ERR_CUDA);
+    }
+    t.bad_region = -1;
+    if (cudaMemcpy(h->ws + lo.dbg_table, &t, sizeof(t), cudaMemcpyHostToDevice) != cudaSuccess) return fail(VS_ERR_CUDA);
+  }
+#endif
   if (cudaDeviceSynchronize() != cudaSuccess) return fail(VS_ERR_CUDA);
   *out = h;
   return VS_OK;
@@ -500,6 +530,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     aa.out_fp32 = D.out_fp32;
     aa.h_in = D.residual ? h_in : nullptr;
     aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
+    aa.h_out_region = (cur ^ 1) ? DR_HBUF1 : DR_HBUF0;
     if (D.use_rmsnorm && l + 1 < D.L) { aa.ss_out = h->at<float>(lo.row_ss); aa.next_gain = h->gain[l + 1]; aa.xn_out = h->at<bf16>(lo.xn); }
     aa.free_slot = h->at<int32_t>(lo.step_slot); aa.free_slot_stride = 1;
     {
@@ -698,6 +729,7 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
       aa.out_fp32 = D.out_fp32;
       aa.h_in = D.residual ? h_in : nullptr;
       aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
+    aa.h_out_region = (cur ^ 1) ? DR_HBUF1 : DR_HBUF0;
     if (D.use_rmsnorm && l + 1 < D.L) { aa.ss_out = h->at<float>(lo.row_ss); aa.next_gain = h->gain[l + 1]; aa.xn_out = h->at<bf16>(lo.xn); }
       aa.free_slot = chunk_slot; aa.free_slot_stride = 0;
       aa.chunk_mode = 1; aa.chunk_count0 = count0; aa.chunk_victim = chunk_victim;
@@ -788,6 +820,7 @@ int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_strea
     aa.out_fp32 = D.out_fp32;
     aa.h_in = D.residual ? h_in : nullptr;
     aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
+    aa.h_out_region = (cur ^ 1) ? DR_HBUF1 : DR_HBUF0;
     if (D.use_rmsnorm && l + 1 < D.L) { aa.ss_out = h->at<float>(lo.row_ss); aa.next_gain = h->gain[l + 1]; aa.xn_out = h->at<bf16>(lo.xn); }
     aa.free_slot = h->at<int32_t>(lo.step_slot); aa.free_slot_stride = 0;
     aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = 0;      // no bank segment on this key axis
@@ -893,6 +926,7 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
     if (rc != VS_OK) return rc;
 
     bf16* h_out = D.residual ? h->at<bf16>(lo.hbuf[next_buf]) : nullptr;
+    const int h_out_region = next_buf ? DR_HBUF1 : DR_HBUF0;
     const float scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
     if (T == 1) {
       DecodeArgs da;
@@ -900,7 +934,7 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       da.prefix_k = pk; da.prefix_v = pv; da.bank_k = bk; da.bank_v = bv; da.tail_k = tk; da.tail_v = tv;
       da.out = (l == D.L - 1) ? out : h->at<void>(lo.obuf);
       da.out_fp32 = D.out_fp32;
-      da.h_in = D.residual ? h_in : nullptr; da.h_out = h_out;
+      da.h_in = D.residual ? h_in : nullptr; da.h_out = h_out; da.h_out_region = h_out_region;
       da.meta = meta;
       da.Hq = D.Hq; da.Hkv = D.Hkv; da.D = D.D; da.slots = D.slots; da.M = D.M; da.maxP = D.maxP; da.maxT = D.maxT;
       // short contexts: one CTA per (stream, query head) writes the row directly; longer ones are
@@ -936,7 +970,7 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       aa.out = (l == D.L - 1) ? out : (D.residual ? nullptr : h->at<void>(lo.obuf));
       aa.out_fp32 = D.out_fp32;
       aa.h_in = D.residual ? h_in : nullptr;
-      aa.h_out = h_out;
+      aa.h_out = h_out; aa.h_out_region = h_out_region;
       if (D.use_rmsnorm && l + 1 < D.L && !by_gemv) { aa.ss_out = h->at<float>(lo.row_ss); aa.next_gain = h->gain[l + 1]; aa.xn_out = h->at<bf16>(lo.xn); }
       aa.free_slot = &meta->free_slot; aa.free_slot_stride = (int)(sizeof(StreamMeta) / sizeof(int32_t));
       aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
@@ -1040,6 +1074,22 @@ int vs_bank_state(vs_stream* h, int32_t stream_id, vs_bank_info* info, int32_t* 
   VS_CK(cudaMemcpy(order.data(), h->ws + lo.order + (size_t)stream_id * D.slots * 4, (size_t)D.slots * 4, cudaMemcpyDeviceToHost));
   VS_CK(cudaMemcpy(sframe.data(), h->ws + lo.slot_frame + (size_t)stream_id * D.slots * 4, (size_t)D.slots * 4, cudaMemcpyDeviceToHost));
   VS_CK(cudaMemcpy(spos.data(), h->ws + lo.slot_pos + (size_t)stream_id * D.slots * 8, (size_t)D.slots * 8, cudaMemcpyDeviceToHost));
+#ifdef VS_DEBUG_BOUNDS
+  {
+    // a refused store, or guard bytes behind a region that no longer hold their pattern
+    DebugTable t;
+    VS_CK(cudaMemcpy(&t, h->ws + lo.dbg_table, sizeof(t), cudaMemcpyDeviceToHost));
+    bool bad = t.bad_region != -1;
+    unsigned char guard[256];
+    for (int r = 0; r < DR_COUNT && !bad; ++r) {
+      if (lo.region_end[r] <= lo.region_begin[r]) continue;
+      VS_CK(cudaMemcpy(guard, h->ws + align_up(lo.region_end[r], 256), kGuardBytes, cudaMemcpyDeviceToHost));
+      for (size_t i = 0; i < kGuardBytes; ++i) if (guard[i] != kGuardByte) { bad = true; std::fprintf(stderr, "videoscan: guard bytes behind workspace region %d overwritten\n", r); break; }
+    }
+    if (t.bad_region != -1) std::fprintf(stderr, "videoscan: store outside workspace region %d refused (offset %lld)\n", t.bad_region, t.bad_offset);
+    if (bad && status[0] == 0) status[0] = VS_ERR_BOUNDS;
+  }
+#endif
   const HostStream& s = h->hs[stream_id];
   if (info != nullptr) {
     info->count = m.count; info->capacity = D.M;
@@ -1112,6 +1162,11 @@ int vs_poison_scratch(vs_stream* h, void* cuda_stream) {
   VS_LAUNCH(h, static_cast<cudaStream_t>(cuda_stream), KC_OTHER,
             launch_poison(h->ws + h->lo.scratch_begin, h->lo.scratch_end - h->lo.scratch_begin,
                           static_cast<cudaStream_t>(cuda_stream)));
+#ifdef VS_DEBUG_BOUNDS
+  for (int r = 0; r < DR_COUNT; ++r)
+    if (h->lo.region_end[r] > h->lo.region_begin[r] && h->lo.region_begin[r] >= h->lo.scratch_begin)
+      VS_CK(cudaMemsetAsync(h->ws + align_up(h->lo.region_end[r], 256), kGuardByte, kGuardBytes, static_cast<cudaStream_t>(cuda_stream)));
+#endif
   h->last_stream = static_cast<cudaStream_t>(cuda_stream);
   return VS_OK;
 }

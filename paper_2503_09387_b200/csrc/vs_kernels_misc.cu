@@ -40,7 +40,8 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, i
       const double ang = (double)(pos0 + r) * a.inv_freq[k];
       double s, c;
       sincos(ang, &s, &c);
-      a.rope[((size_t)b * (N + 1) + r) * half + k] = make_float2((float)c, (float)s);
+      float2* rp = a.rope + ((size_t)b * (N + 1) + r) * half + k;
+      if (VS_STORE_OK(bp, DR_ROPE, rp, 8)) *rp = make_float2((float)c, (float)s);
     }
     return;
   }
@@ -67,7 +68,7 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, i
   for (int i = 0; i < MAXR; ++i) {
     const int r = grp + i * RG;
     if (r < N) {
-      *reinterpret_cast<uint4*>(dst + (size_t)r * d) = v[i];
+      if (VS_STORE_OK(bp, DR_HBUF0, dst + (size_t)r * d, 16)) *reinterpret_cast<uint4*>(dst + (size_t)r * d) = v[i];
       const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&v[i]);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -92,12 +93,14 @@ __global__ void __launch_bounds__(256) pool_kernel(PoolArgs a, BatchParams bp, i
       for (int g = 0; g < RG; ++g) t += red[g][threadIdx.x];
       cv = f64_to_bf16_rne(t / (double)N);
     }
-    a.x[(size_t)b * (N + 1) * d + (size_t)N * d + c] = cv;   // carrier = last token of the frame
+    bf16* xc = a.x + (size_t)b * (N + 1) * d + (size_t)N * d + c;
+    if (VS_STORE_OK(bp, DR_HBUF0, xc, 2)) *xc = cv;   // carrier = last token of the frame
     if (a.emb_stage != nullptr) {
-      a.emb_stage[(size_t)b * d + c] = cv;          // chunk of frames: the slot is not known yet
+      if (VS_STORE_OK(bp, DR_EMB_STAGE, a.emb_stage + (size_t)b * d + c, 2)) a.emb_stage[(size_t)b * d + c] = cv;          // chunk of frames: the slot is not known yet
     } else if (a.M > 0) {
       const int slot = a.meta[sid].free_slot;
-      a.emb[((size_t)sid * a.slots + slot) * d + c] = cv;
+      bf16* ep = a.emb + ((size_t)sid * a.slots + slot) * d + c;
+      if (VS_STORE_OK(bp, DR_EMB, ep, 2)) *ep = cv;
       // the step's other kernels take the slot from this copy: the bank update, which moves
       // meta.free_slot on, runs beside the last attention kernel
       if (blockIdx.x == 0 && threadIdx.x == 0) a.step_slot[sid] = slot;
