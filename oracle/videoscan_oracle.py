@@ -31,6 +31,11 @@ fp64.  Values are rounded to bf16 only where the method stores them: the carrier
 embedding, K/V entering bank / prefix / text tail, and the residual stream between
 layers.
 
+Optional rest of the decoder block (the backbone of Section 4.1 is a Qwen2 decoder): with
+``BlockWeights`` a layer is  h1 = h + A W_o^T,  h2 = h1 + (SiLU(n W_gate^T) * (n W_up^T)) W_down^T
+with A the attention rows and n = RMSNorm(h1); storage points (bf16) are A, h1, the gated
+activation and h2, and a step then returns the last layer's h2 instead of its attention rows.
+
 Parity pins (tests/test_oracle_*.py): closed forms for the pooling, softmax row sums,
 GQA == MHA with repeated heads, brute-force dense masked attention over the un-pruned
 sequence, textbook causal attention for M = 0 and one-frame streams, RoPE identities,
@@ -220,6 +225,22 @@ class OracleConfig:
 
 
 @dataclasses.dataclass
+class BlockWeights:
+    """The rest of one decoder layer (Qwen2 block, Section 4.1 names the backbone): output
+    projection and SwiGLU MLP.  All "out x in", bf16-valued fp64."""
+    w_o: np.ndarray                 # [d, Hq*D]
+    w_gate: np.ndarray              # [I, d]
+    w_up: np.ndarray                # [I, d]
+    w_down: np.ndarray              # [d, I]
+    norm2_w: Optional[np.ndarray] = None   # [d] gain of the post-attention RMSNorm, or None (unit gain)
+
+
+def silu(x: np.ndarray) -> np.ndarray:
+    """SiLU(x) = x * sigmoid(x) = x / (1 + exp(-x))."""
+    return x / (1.0 + np.exp(-x))
+
+
+@dataclasses.dataclass
 class BankEntry:
     frame_id: int
     pos: int
@@ -233,8 +254,12 @@ class OracleStream:
 
     def __init__(self, cfg: OracleConfig, w_qkv: List[np.ndarray],
                  b_qkv: Optional[List[Optional[np.ndarray]]] = None,
-                 norm_w: Optional[List[Optional[np.ndarray]]] = None):
+                 norm_w: Optional[List[Optional[np.ndarray]]] = None,
+                 blocks: Optional[List[BlockWeights]] = None):
         self.cfg = cfg
+        self.blocks = blocks            # None: attention sub-block only (the five workloads)
+        if blocks is not None and not cfg.residual:
+            raise ValueError("the full decoder block needs the residual stream")
         L = cfg.n_layers
         self.w = [np.asarray(w, dtype=np.float64) for w in w_qkv]       # [E_out, d]
         self.b = b_qkv if b_qkv is not None else [None] * L
@@ -275,6 +300,22 @@ class OracleStream:
         K = y[:, nq:nq + nk].reshape(rows, cfg.n_kv_heads, cfg.head_dim)
         V = y[:, nq + nk:].reshape(rows, cfg.n_kv_heads, cfg.head_dim)
         return Q, K, V
+
+    def _rest_of_block(self, h: np.ndarray, O: np.ndarray, layer: int) -> np.ndarray:
+        """h (layer input, bf16-valued) and the layer's attention rows O -> the layer's output h2."""
+        blk = self.blocks[layer]
+        A = round_to_bf16(O)                                   # the attention rows are a stored tensor
+        h1 = round_to_bf16(h + A @ np.asarray(blk.w_o, dtype=np.float64).T)
+        n = h1
+        if self.cfg.use_rmsnorm:
+            ms = np.mean(h1 * h1, axis=1, keepdims=True)
+            n = h1 / np.sqrt(ms + self.cfg.rms_eps)
+            if blk.norm2_w is not None:
+                n = n * np.asarray(blk.norm2_w, dtype=np.float64)[None, :]
+        g = n @ np.asarray(blk.w_gate, dtype=np.float64).T
+        u = n @ np.asarray(blk.w_up, dtype=np.float64).T
+        act = round_to_bf16(silu(g) * u)
+        return round_to_bf16(h1 + act @ np.asarray(blk.w_down, dtype=np.float64).T)
 
     def _bank_kv(self, layer: int):
         Hkv, D = self.cfg.n_kv_heads, self.cfg.head_dim
@@ -328,8 +369,12 @@ class OracleStream:
                 cV[l] = round_to_bf16(V[N])
                 out = O
                 rec["O"].append(O)
-                if cfg.residual:
+                if self.blocks is not None:
+                    h = self._rest_of_block(h, O, l)
+                    out = h
+                elif cfg.residual:
                     h = round_to_bf16(h + O)
+                rec.setdefault("h_out", []).append(h)
             if self.record is not None:
                 self.record.append(rec)
         elif mode == "carrier":
@@ -397,8 +442,12 @@ class OracleStream:
                 self.tail_V[l] = np.concatenate([self.tail_V[l], V], axis=0)
             out = O
             rec["O"].append(O)
-            if cfg.residual:
+            if self.blocks is not None:
+                h = self._rest_of_block(h, O, l)
+                out = h
+            elif cfg.residual:
                 h = round_to_bf16(h + O)
+            rec.setdefault("h_out", []).append(h)
         if self.record is not None:
             self.record.append(rec)
         if to_prefix:
@@ -415,6 +464,8 @@ class OracleStream:
         used and nothing changes.  Carrier i of this compact sequence sits at position
         prefix_len + i.  Returns the last layer's outputs [count, Hq*D]."""
         cfg = self.cfg
+        if self.blocks is not None:
+            raise NotImplementedError("carriers-only forward is defined for the attention sub-block")
         T = len(self.bank)
         if T == 0:
             return np.zeros((0, cfg.n_q_heads * cfg.head_dim))

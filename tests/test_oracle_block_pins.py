@@ -1,0 +1,120 @@
+"""CPU pins of the oracle's optional rest of the decoder block (output projection + SwiGLU MLP; the
+backbone of Section 4.1 is a Qwen2 decoder).  The paper prints no numbers for it; the pins are closed
+forms, special cases that reduce to the attention-only oracle, and a library restatement in torch
+(fp64 F.linear / F.silu) -- chosen so that a transposed weight, SiLU on the wrong branch, a missing
+residual or a norm taken of the wrong tensor fails one of them."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import videoscan_oracle as vo
+
+
+def _bf(x):
+    return vo.round_to_bf16(np.asarray(x, dtype=np.float64))
+
+
+def _setup(seed=0, L=2, d=32, Hq=4, Hkv=2, D=8, inter=48, norm=True, gain=True):
+    rng = np.random.default_rng(seed)
+    cfg = vo.OracleConfig(L, d, Hq, Hkv, D, bank_capacity=2, use_rmsnorm=1 if norm else 0, residual=1)
+    Ws = [_bf(rng.normal(0, 0.2, ((Hq + 2 * Hkv) * D, d))) for _ in range(L)]
+    gains = [_bf(1 + 0.1 * rng.normal(size=d)) for _ in range(L)] if gain else None
+    blocks = [vo.BlockWeights(_bf(rng.normal(0, 0.2, (d, Hq * D))), _bf(rng.normal(0, 0.2, (inter, d))),
+                              _bf(rng.normal(0, 0.2, (inter, d))), _bf(rng.normal(0, 0.2, (d, inter))),
+                              _bf(1 + 0.1 * rng.normal(size=d)) if gain else None) for _ in range(L)]
+    return rng, cfg, Ws, gains, blocks
+
+
+def _run(cfg, Ws, gains, blocks, rng_seed=1, frames=4, N=5):
+    rng = np.random.default_rng(rng_seed)
+    st = vo.OracleStream(cfg, Ws, None, gains, blocks)
+    st.record = []
+    outs = [st.text_step(_bf(rng.normal(size=(3, cfg.d_model))))]
+    for _ in range(frames):
+        outs.append(st.frame_step(_bf(rng.normal(size=(N, cfg.d_model)))))
+    outs.append(st.text_step(_bf(rng.normal(size=(2, cfg.d_model)))))
+    outs.append(st.text_step(_bf(rng.normal(size=(1, cfg.d_model)))))
+    return st, outs
+
+
+def test_silu_closed_forms():
+    assert vo.silu(np.array([0.0]))[0] == 0.0
+    assert abs(vo.silu(np.array([1.0]))[0] - 1.0 / (1.0 + math.exp(-1.0))) < 1e-15
+    assert abs(vo.silu(np.array([-1.0]))[0] + 1.0 / (1.0 + math.e)) < 1e-15
+    x = np.linspace(-6, 6, 101)
+    assert np.allclose(vo.silu(x) - vo.silu(-x), x, atol=1e-14)            # x sigma(x) - (-x) sigma(-x) = x
+    assert np.allclose(vo.silu(x), torch.nn.functional.silu(torch.from_numpy(x)).numpy(), atol=1e-15)
+
+
+def test_identity_output_projection_and_silent_mlp_reduce_to_the_attention_residual():
+    """W_o = I and W_down = 0: the layer's output is bf16(h + bf16(O)), O being the attention rows the
+    attention-only procedure computes on the same layer input."""
+    _, cfg, Ws, gains, blocks = _setup(L=1)
+    blocks[0].w_o = np.eye(cfg.d_model)
+    blocks[0].w_down = np.zeros_like(blocks[0].w_down)
+    st, outs = _run(cfg, Ws, gains, blocks)
+    for rec, out in zip(st.record, outs):
+        want = _bf(rec["h"][0] + _bf(rec["O"][0]))
+        assert np.array_equal(out, want)
+
+
+def test_zero_gate_makes_the_mlp_add_nothing():
+    _, cfg, Ws, gains, blocks = _setup(L=2)
+    for b in blocks:
+        b.w_gate = np.zeros_like(b.w_gate)                                     # SiLU(0) = 0
+    st, outs = _run(cfg, Ws, gains, blocks)
+    for rec in st.record:
+        for l in range(cfg.n_layers):
+            h1 = _bf(rec["h"][l] + _bf(rec["O"][l]) @ blocks[l].w_o.T)
+            assert np.array_equal(rec["h_out"][l], h1)
+            if l + 1 < cfg.n_layers:
+                assert np.array_equal(rec["h"][l + 1], h1)                      # and it is the next layer's input
+
+
+@pytest.mark.parametrize("norm,gain", [(True, True), (True, False), (False, False)])
+def test_block_matches_a_torch_restatement(norm, gain):
+    """Every recorded layer: torch fp64 linear / silu on the recorded layer input and attention rows."""
+    _, cfg, Ws, gains, blocks = _setup(seed=3, L=2, norm=norm, gain=gain)
+    st, outs = _run(cfg, Ws, gains, blocks, rng_seed=5)
+    F = torch.nn.functional
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(np.asarray(a, dtype=np.float64)))
+    for rec, out in zip(st.record, outs):
+        for l in range(cfg.n_layers):
+            b = blocks[l]
+            h = t(rec["h"][l])
+            a = t(_bf(rec["O"][l]))
+            h1 = t(_bf((h + F.linear(a, t(b.w_o))).numpy()))
+            n = h1
+            if norm:
+                n = h1 * torch.rsqrt((h1 * h1).mean(dim=1, keepdim=True) + cfg.rms_eps)
+                if gain:
+                    n = n * t(b.norm2_w)
+            act = t(_bf((F.silu(F.linear(n, t(b.w_gate))) * F.linear(n, t(b.w_up))).numpy()))
+            h2 = _bf((h1 + F.linear(act, t(b.w_down))).numpy())
+            assert np.allclose(rec["h_out"][l], h2, atol=1e-12, rtol=0)
+            # bf16 roundings of nearly equal fp64 values agree except on exact ties: demand equality on 99.9 %
+            assert np.mean(rec["h_out"][l] == h2) > 0.999
+        assert np.array_equal(out, rec["h_out"][-1])                           # a step returns the last layer's output
+
+
+def test_attention_only_streams_are_untouched_by_the_option():
+    _, cfg, Ws, gains, blocks = _setup(seed=4, L=2)
+    st_a, outs_a = _run(cfg, Ws, gains, None)
+    st_b = vo.OracleStream(cfg, Ws, None, gains)                               # blocks defaulted
+    rng = np.random.default_rng(1)
+    out0 = st_b.text_step(_bf(rng.normal(size=(3, cfg.d_model))))
+    assert np.array_equal(out0, outs_a[0]) and out0.shape[1] == cfg.n_q_heads * cfg.head_dim
+
+
+def test_bank_keeps_attention_keys_of_the_block_stream():
+    """The bank's K/V of a deeper layer come from that layer's input, which now carries the MLP: a stream with
+    blocks and one without differ in layer 1's bank K/V but not in layer 0's (same frames, same layer-0 input)."""
+    _, cfg, Ws, gains, blocks = _setup(seed=6, L=2)
+    st_a, _ = _run(cfg, Ws, gains, blocks)
+    st_b, _ = _run(cfg, Ws, gains, None)
+    assert len(st_a.bank) == len(st_b.bank) == 2
+    for ea, eb in zip(st_a.bank, st_b.bank):
+        assert ea.frame_id == eb.frame_id and np.array_equal(ea.emb, eb.emb)
+        assert np.array_equal(ea.K[0], eb.K[0]) and not np.array_equal(ea.K[1], eb.K[1])
