@@ -85,6 +85,10 @@ typedef struct {
                                     rounds by up to 1.6e-2; fp32 keeps the fp32-accumulated value    */
   int32_t max_chunk_frames;      /* most frames one vs_frame_prefill_chunk call may bring (0 or 1:
                                     that call is not used); sizes the per-step scratch              */
+  int32_t d_ff;                  /* 0: attention sub-block only.  > 0: width of the SwiGLU MLP of the full
+                                    decoder block (Section 4.1: the backbone is a Qwen2 decoder); a multiple
+                                    of 64; needs residual = 1, d_model a multiple of 128 and the four block
+                                    weight arrays of vs_weights                                         */
 } vs_config;
 
 /* DEVICE pointers to bf16 weights, one entry per layer.  The arrays of pointers themselves
@@ -95,6 +99,14 @@ typedef struct {
                                     16-byte aligned                                                  */
   const void* const* b_qkv;      /* [n_layers] each [E_out], or NULL (whole array or any entry)      */
   const void* const* norm_w;     /* [n_layers] each [d_model] RMSNorm gain, or NULL = all ones       */
+  /* the rest of the decoder block, read only when d_ff > 0 (all "out x in", row-major, 16-byte aligned):
+   *   h1 = h + A W_o^T (A: the layer's attention rows),  h2 = h1 + (SiLU(n W_gate^T) * (n W_up^T)) W_down^T,
+   *   n = RMSNorm(h1) when use_rmsnorm.  A step's `out` then receives the last layer's h2 ([..][d_model]). */
+  const void* const* w_o;        /* [n_layers] each [d_model, Hq*D]                                  */
+  const void* const* w_gate;     /* [n_layers] each [d_ff, d_model]                                  */
+  const void* const* w_up;       /* [n_layers] each [d_ff, d_model]                                  */
+  const void* const* w_down;     /* [n_layers] each [d_model, d_ff]                                  */
+  const void* const* norm2_w;    /* [n_layers] each [d_model] gain of the post-attention RMSNorm, or NULL */
 } vs_weights;
 
 /* Filled by vs_bank_state (HOST). */

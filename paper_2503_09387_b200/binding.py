@@ -42,12 +42,13 @@ class VsConfig(C.Structure):
         "evict_policy", "use_rmsnorm", "residual")] + [
         ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("device", C.c_int32),
         ("evict_log_capacity", C.c_int32), ("out_dtype", C.c_int32),
-        ("max_chunk_frames", C.c_int32)]
+        ("max_chunk_frames", C.c_int32), ("d_ff", C.c_int32)]
 
 
 class VsWeights(C.Structure):
     _fields_ = [("w_qkv", C.POINTER(C.c_void_p)), ("b_qkv", C.POINTER(C.c_void_p)),
-                ("norm_w", C.POINTER(C.c_void_p))]
+                ("norm_w", C.POINTER(C.c_void_p)), ("w_o", C.POINTER(C.c_void_p)), ("w_gate", C.POINTER(C.c_void_p)),
+                ("w_up", C.POINTER(C.c_void_p)), ("w_down", C.POINTER(C.c_void_p)), ("norm2_w", C.POINTER(C.c_void_p))]
 
 
 class VsBankInfo(C.Structure):
@@ -129,14 +130,15 @@ def vs_workspace_bytes(cfg: VsConfig) -> int:
 
 
 def vs_create_stream(cfg: VsConfig, w_ptrs: List[int], b_ptrs: Optional[List[Optional[int]]],
-                     g_ptrs: Optional[List[Optional[int]]], workspace_ptr: int, workspace_bytes: int) -> int:
+                     g_ptrs: Optional[List[Optional[int]]], workspace_ptr: int, workspace_bytes: int,
+                     block_ptrs: Optional[dict] = None) -> int:
+    """block_ptrs (full decoder block, cfg.d_ff > 0): {"w_o", "w_gate", "w_up", "w_down": [L pointers], "norm2_w": [L] or None}."""
     L = cfg.n_layers
-    w = (C.c_void_p * L)(*w_ptrs)
-    b = (C.c_void_p * L)(*[p or None for p in b_ptrs]) if b_ptrs is not None else None
-    g = (C.c_void_p * L)(*[p or None for p in g_ptrs]) if g_ptrs is not None else None
-    ws = VsWeights(C.cast(w, C.POINTER(C.c_void_p)),
-                   C.cast(b, C.POINTER(C.c_void_p)) if b is not None else None,
-                   C.cast(g, C.POINTER(C.c_void_p)) if g is not None else None)
+    arr = lambda ptrs: C.cast((C.c_void_p * L)(*[p or None for p in ptrs]), C.POINTER(C.c_void_p)) if ptrs is not None else None
+    keep = [arr(w_ptrs), arr(b_ptrs), arr(g_ptrs)]
+    for name in ("w_o", "w_gate", "w_up", "w_down", "norm2_w"):
+        keep.append(arr(block_ptrs.get(name)) if block_ptrs else None)
+    ws = VsWeights(*keep)
     handle = C.c_void_p(None)
     _check(load_library().vs_create_stream(C.byref(cfg), C.byref(ws), workspace_ptr, workspace_bytes,
                                            C.byref(handle)), "vs_create_stream")
@@ -262,7 +264,8 @@ class StreamBatch:
     [E_out, d_model] per layer.  All methods take / return torch CUDA tensors and only enqueue
     work on the current torch stream."""
 
-    def __init__(self, cfg: VsConfig, weights, biases=None, norm_weights=None):
+    def __init__(self, cfg: VsConfig, weights, biases=None, norm_weights=None, block=None):
+        # block (cfg.d_ff > 0): {"w_o", "w_gate", "w_up", "w_down": [L device tensors], "norm2_w": [L] or None}
         import torch
         self.torch = torch
         self.cfg = cfg
@@ -270,6 +273,7 @@ class StreamBatch:
         self.weights = [w.contiguous() for w in weights]
         self.biases = biases
         self.norm_weights = norm_weights
+        self.block = block
         nbytes = vs_workspace_bytes(cfg)
         self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
         base = self.workspace.data_ptr()
@@ -279,7 +283,9 @@ class StreamBatch:
             cfg, [w.data_ptr() for w in self.weights],
             [b.data_ptr() if b is not None else None for b in biases] if biases is not None else None,
             [g.data_ptr() if g is not None else None for g in norm_weights] if norm_weights is not None else None,
-            self._ws_ptr, nbytes)
+            self._ws_ptr, nbytes,
+            {k: ([t.data_ptr() if t is not None else None for t in v] if v is not None else None) for k, v in block.items()}
+            if block else None)
         self.out_width = cfg.n_q_heads * cfg.head_dim
         self.out_torch_dtype = torch.float32 if cfg.out_dtype == 1 else torch.bfloat16
 
@@ -358,7 +364,7 @@ class StreamBatch:
 def make_config(n_layers, d_model, n_q_heads, n_kv_heads, head_dim, max_tokens_per_frame, max_prefix,
                 max_text, bank_capacity, n_streams=1, max_step_tokens=64, agg_mode=0, evict_policy=0,
                 use_rmsnorm=0, residual=0, rope_theta=1.0e6, rms_eps=1.0e-6, device=0,
-                evict_log_capacity=4096, out_dtype=1, max_chunk_frames=1) -> VsConfig:
+                evict_log_capacity=4096, out_dtype=1, max_chunk_frames=1, d_ff=0) -> VsConfig:
     return VsConfig(n_layers, d_model, n_q_heads, n_kv_heads, head_dim, max_tokens_per_frame, max_prefix,
                     max_text, max_step_tokens, bank_capacity, n_streams, agg_mode, evict_policy, use_rmsnorm,
-                    residual, rope_theta, rms_eps, device, evict_log_capacity, out_dtype, max_chunk_frames)
+                    residual, rope_theta, rms_eps, device, evict_log_capacity, out_dtype, max_chunk_frames, d_ff)

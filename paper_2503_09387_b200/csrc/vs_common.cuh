@@ -55,7 +55,7 @@ struct BatchParams {
 enum DbgRegion { DR_BANK_K = 0, DR_BANK_V, DR_PREFIX_K, DR_PREFIX_V, DR_TAIL_K, DR_TAIL_V, DR_EMB, DR_META, DR_ORDER,
                  DR_SLOT_FRAME, DR_SLOT_POS, DR_EVICT_LOG, DR_SCORES, DR_STEP_SLOT, DR_CHUNK_SLOT, DR_CHUNK_VICTIM,
                  DR_GEMM_FLAGS, DR_HBUF0, DR_HBUF1, DR_XN, DR_ROW_SS, DR_Q, DR_Q_LO, DR_Q_TILED, DR_KF, DR_VF, DR_ROPE,
-                 DR_OBUF, DR_EMB_STAGE, DR_CHUNK_SCORES, DR_GEMM_XCHG, DR_COUNT };
+                 DR_OBUF, DR_EMB_STAGE, DR_CHUNK_SCORES, DR_GEMM_XCHG, DR_ACT, DR_COUNT };
 struct DebugTable {
   unsigned long long begin[DR_COUNT], end[DR_COUNT];   // device addresses
   int bad_region;                                      // -1, or the region of the first refused store
@@ -77,6 +77,8 @@ __device__ __forceinline__ bool vs_store_ok(const BatchParams& bp, int region, c
 // ---- shapes ----------------------------------------------------------------------------
 struct Dims {
   int L, d, Hq, Hkv, D, G, E_out;
+  int d_ff;                                      // 0, or the SwiGLU width of the full decoder block
+  int ss_parts;                                  // parts a row's sum of squares comes in: Hkv (from the attention kernel) or d / 128
   int maxN, maxP, maxT, maxStepT, M, slots, S, maxChunk;   // maxP / maxT: allocated rows (>= 1)
   int capP, capT;                                // caller's prefix / tail capacities
   int rows_per_stream_max, R_max;
@@ -114,7 +116,9 @@ struct Layout {
   // per-step scratch
   size_t hbuf[2];               // bf16 [R_max][d]  residual ping-pong; hbuf[0] holds [E; carrier]
   size_t xn;                    // bf16 [R_max][d]  layer input times the RMSNorm gain (only with a gain vector)
-  size_t row_ss;                // f32  [R_max][Hkv] parts of the rows' sums of squares (RMSNorm)
+  size_t row_ss;                // f32  [2][R_max][ss_parts] parts of the rows' sums of squares (RMSNorm; second half: the
+                                //      post-attention norm of the full decoder block)
+  size_t act;                   // bf16 [R_max][d_ff]  gated activation of the full decoder block
   size_t q;                     // bf16 [R_max][Hq*D]
   size_t q_lo;                  // bf16 [R_max][Hq*D]  low-order half of the rotated query
   size_t q_tiled;               // bf16 [row tiles][Hkv][hi | lo][128][D]  the pair as the tensor-core attention reads it
@@ -240,10 +244,20 @@ struct ProjectionOut {
   int free_slot_stride;
   int Hq, Hkv, D, slots, text_cap, M;
   int mode;                      // 0 frame step (carrier row -> bank), 1 text -> prefix, 2 text -> tail,
-                                 // 3 chunk of frames (nothing kept here: a commit kernel copies the carrier rows)
+                                 // 3 chunk of frames (nothing kept here: a commit kernel copies the carrier rows),
+                                 // 4 plain linear layer + residual, 5 SwiGLU gate/up pair (the rest of the decoder block)
+  // modes 4 and 5: lin_out[row][E] = bf16(acc * row scale + lin_res[row][E]) (mode 4, E = E_out), or
+  // lin_out[row][E_out / 2] = bf16(SiLU(gate) * up) (mode 5: every 128-row weight tile is 64 gate rows, then 64 up rows)
+  bf16* lin_out; const bf16* lin_res;
+  int lin_out_region;            // checked build: the workspace region lin_out lies in
+  void* final_out; int final_fp32;   // mode 4: the rows also go here (the step's output), or null
+  float* ss_out;                 // mode 4: sum of squares of the stored rows, one part per 128-feature tile:
+  int ss_out_parts;              //   ss_out[row][ss_out_parts], this launch's tile m at part m; or null
+  const bf16* next_gain; bf16* xn_out;   // mode 4 with ss_out: xn_out = bf16(stored row * next_gain), or null
 };
 
 struct GemmArgs {
+  CUtensorMap tm_w2;             // mode 5: the up matrix (tm_w is then the gate matrix, both with boxes of 64 rows)
   CUtensorMap tm_w;              // [E_out, d] bf16, box 64 x 128, 128-byte swizzle
   CUtensorMap tm_x;              // [rows, d] bf16, box 64 x tile_n, 128-byte swizzle
   ProjectionOut out;

@@ -141,8 +141,8 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
 template <bool kOwnRope, int kMSub>   // kOwnRope: no RoPE table, every finishing thread derives the rotation of its one
                                       // row; kMSub: 128-row weight sub-tiles (accumulators) per CTA
 __global__ void __launch_bounds__(kMaxThreads, 1)
-qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, KernelParams p,
-                BatchParams bp) {
+qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
+                const __grid_constant__ CUtensorMap tm_w2, KernelParams p, BatchParams bp) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // carve: [stages][A 16 KiB | B tile_n*128] (later reused for this CTA's own token slice of
   // the fp32 partial tile, [token][128 features]) | full[stages] | empty[stages] | tmem_full |
@@ -201,8 +201,16 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
         const uint32_t a_dst = base + (uint32_t)s * stage_bytes;
         const int kx = (kb0 + kb) * GEMM_BLOCK_K;
 #pragma unroll
-        for (int ms = 0; ms < kMSub; ++ms)
-          tma_load_2d(a_dst + (uint32_t)ms * kStageABytes, &tm_w, kx, m0 + ms * GEMM_BLOCK_M, full_bar(s));
+        for (int ms = 0; ms < kMSub; ++ms) {
+          if (p.o.mode == 5) {
+            // a 128-row tile = 64 rows of the gate matrix, then the same 64 rows of the up matrix
+            const int r64 = (m0 + ms * GEMM_BLOCK_M) >> 1;
+            tma_load_2d(a_dst + (uint32_t)ms * kStageABytes, &tm_w, kx, r64, full_bar(s));
+            tma_load_2d(a_dst + (uint32_t)ms * kStageABytes + kStageABytes / 2, &tm_w2, kx, r64, full_bar(s));
+          } else {
+            tma_load_2d(a_dst + (uint32_t)ms * kStageABytes, &tm_w, kx, m0 + ms * GEMM_BLOCK_M, full_bar(s));
+          }
+        }
         tma_load_2d(a_dst + stage_a_bytes, &tm_x, kx, n0, full_bar(s));
         issued = kb + 1;
       }
@@ -353,7 +361,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
     const int hl = p0 / half, k0 = p0 - hl * half; // local head, index inside the half head
     const int f1 = hl * D + k0, f2 = f1 + half;
     const int hs = (m0e + f1) / D;                  // head slot: Q heads, then K heads, then V heads
-    const bool rotate = hs < p.o.Hq + p.o.Hkv;
+    const bool rotate = p.o.mode < 4 && hs < p.o.Hq + p.o.Hkv;
     const float* far = p.xchg + (size_t)group * p.ksplit * p.tile_n * GEMM_BLOCK_M;
     const size_t far_stride = (size_t)p.tile_n * GEMM_BLOCK_M;
     if (m0e + f2 + 3 < p.E_out) {
@@ -415,6 +423,70 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
             const float y2 = x2[i] * cs[i] + x1[i] * sn[i];
             x1[i] = y1; x2[i] = y2;
           }
+        }
+        if (p.o.mode == 5) {
+          // SwiGLU: features f1.. are gate rows, f2 = f1 + 64.. the matching up rows
+          __align__(8) bf16 av[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) av[i] = __float2bfloat16_rn(x1[i] / (1.f + __expf(-x1[i])) * x2[i]);
+          bf16* dst = p.o.lin_out + (size_t)row * (p.E_out >> 1) + (m0e >> 1) + f1;
+          if (VS_STORE_OK(bp, p.o.lin_out_region, dst, 8)) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(av);
+          return;
+        }
+        if (p.o.mode == 4) {
+          // linear layer + residual; the rows as stored (bf16) also give the next RMSNorm its statistics
+          const size_t c1 = (size_t)row * p.E_out + m0e + f1, c2 = (size_t)row * p.E_out + m0e + f2;
+          if (p.o.lin_res != nullptr) {
+            const uint2 r1 = *reinterpret_cast<const uint2*>(p.o.lin_res + c1), r2 = *reinterpret_cast<const uint2*>(p.o.lin_res + c2);
+            const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&r1.x)), a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&r1.y));
+            const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&r2.x)), b1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&r2.y));
+            x1[0] += a0.x; x1[1] += a0.y; x1[2] += a1.x; x1[3] += a1.y;
+            x2[0] += b0.x; x2[1] += b0.y; x2[2] += b1.x; x2[3] += b1.y;
+          }
+          __align__(8) bf16 s1[4], s2[4];
+          float ss = 0.f;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            s1[i] = __float2bfloat16_rn(x1[i]); s2[i] = __float2bfloat16_rn(x2[i]);
+            const float u1 = __bfloat162float(s1[i]), u2 = __bfloat162float(s2[i]);
+            ss += u1 * u1 + u2 * u2;
+          }
+          if (VS_STORE_OK(bp, p.o.lin_out_region, p.o.lin_out + c1, 8) && VS_STORE_OK(bp, p.o.lin_out_region, p.o.lin_out + c2, 8)) {
+            *reinterpret_cast<uint2*>(p.o.lin_out + c1) = *reinterpret_cast<const uint2*>(s1);
+            *reinterpret_cast<uint2*>(p.o.lin_out + c2) = *reinterpret_cast<const uint2*>(s2);
+          }
+          if (p.o.final_out != nullptr) {
+            if (p.o.final_fp32) {
+              float* fo = static_cast<float*>(p.o.final_out);
+              *reinterpret_cast<float4*>(fo + c1) = make_float4(__bfloat162float(s1[0]), __bfloat162float(s1[1]), __bfloat162float(s1[2]), __bfloat162float(s1[3]));
+              *reinterpret_cast<float4*>(fo + c2) = make_float4(__bfloat162float(s2[0]), __bfloat162float(s2[1]), __bfloat162float(s2[2]), __bfloat162float(s2[3]));
+            } else {
+              bf16* fo = static_cast<bf16*>(p.o.final_out);
+              *reinterpret_cast<uint2*>(fo + c1) = *reinterpret_cast<const uint2*>(s1);
+              *reinterpret_cast<uint2*>(fo + c2) = *reinterpret_cast<const uint2*>(s2);
+            }
+          }
+          if (p.o.ss_out != nullptr) {
+            if (p.o.next_gain != nullptr) {
+              __align__(8) bf16 g1[4], g2[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                g1[i] = __float2bfloat16_rn(__bfloat162float(s1[i]) * __bfloat162float(p.o.next_gain[m0e + f1 + i]));
+                g2[i] = __float2bfloat16_rn(__bfloat162float(s2[i]) * __bfloat162float(p.o.next_gain[m0e + f2 + i]));
+              }
+              if (VS_STORE_OK(bp, DR_XN, p.o.xn_out + c1, 8) && VS_STORE_OK(bp, DR_XN, p.o.xn_out + c2, 8)) {
+                *reinterpret_cast<uint2*>(p.o.xn_out + c1) = *reinterpret_cast<const uint2*>(g1);
+                *reinterpret_cast<uint2*>(p.o.xn_out + c2) = *reinterpret_cast<const uint2*>(g2);
+              }
+            }
+            // the 16 threads that share the row (a half warp) add their parts in a fixed order
+            const unsigned hm = 0xFFFFu << (threadIdx.x & 16u);
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(hm, ss, o);
+            float* sp = p.o.ss_out + (size_t)row * p.o.ss_out_parts + m0e / GEMM_BLOCK_M;
+            if ((te & 15) == 0 && VS_STORE_OK(bp, DR_ROW_SS, sp, 4)) *sp = ss;
+          }
+          return;
         }
         __align__(8) bf16 o1[4], o2[4];
 #pragma unroll
@@ -581,10 +653,10 @@ cudaError_t launch_qkv_gemm(const GemmArgs& a, const BatchParams& bp, cudaStream
   cfg.numAttrs = 1;
   if (a.out.rope == nullptr) {
     if (a.m_sub != 1) return cudaErrorInvalidValue;
-    return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<true, 1>, a.tm_w, a.tm_x, p, bp);
+    return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<true, 1>, a.tm_w, a.tm_x, a.tm_w2, p, bp);
   }
-  if (a.m_sub == 2) return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<false, 2>, a.tm_w, a.tm_x, p, bp);
-  return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<false, 1>, a.tm_w, a.tm_x, p, bp);
+  if (a.m_sub == 2) return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<false, 2>, a.tm_w, a.tm_x, a.tm_w2, p, bp);
+  return cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<false, 1>, a.tm_w, a.tm_x, a.tm_w2, p, bp);
 }
 
 }  // namespace vs

@@ -57,6 +57,11 @@ int fill_dims(const vs_config* c, Dims& D) {
   D.log_cap = c->evict_log_capacity;
   D.agg_mode = c->agg_mode; D.evict_policy = c->evict_policy; D.use_rmsnorm = c->use_rmsnorm ? 1 : 0;
   D.residual = c->residual ? 1 : 0; D.out_fp32 = c->out_dtype == 1 ? 1 : 0; D.rope_theta = c->rope_theta; D.rms_eps = c->rms_eps;
+  D.d_ff = c->d_ff;
+  if (c->d_ff < 0) return VS_ERR_INVALID_ARG;
+  if (c->d_ff > 0 && (!c->residual || c->n_q_heads * c->head_dim != c->d_model)) return VS_ERR_INVALID_ARG;
+  if (c->d_ff > 0 && (c->d_ff % 64 != 0 || c->d_model % 128 != 0)) return VS_ERR_UNSUPPORTED;
+  D.ss_parts = D.d_ff > 0 ? D.d / 128 : D.Hkv;
   return VS_OK;
 }
 
@@ -99,7 +104,8 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.hbuf[0] = reg(DR_HBUF0, take((size_t)D.R_max * D.d * 2));
   Lo.hbuf[1] = reg(DR_HBUF1, take((size_t)D.R_max * D.d * 2));
   Lo.xn = reg(DR_XN, take((size_t)D.R_max * D.d * 2));
-  Lo.row_ss = reg(DR_ROW_SS, take((size_t)D.R_max * D.Hkv * 4));
+  Lo.row_ss = reg(DR_ROW_SS, take((size_t)2 * D.R_max * D.ss_parts * 4));
+  Lo.act = reg(DR_ACT, take(D.d_ff > 0 ? (size_t)D.R_max * D.d_ff * 2 : 256));
   Lo.q = reg(DR_Q, take((size_t)D.R_max * D.Hq * D.D * 2));
   Lo.q_lo = reg(DR_Q_LO, take((size_t)D.R_max * D.Hq * D.D * 2));
   // the query in the attention kernel's operand layout: per batch entry ceil(rows / 16) row tiles, per tile and KV
@@ -129,6 +135,8 @@ struct vs_stream {
   cudaStream_t side_stream = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   std::vector<const bf16*> w, bias, gain;
+  std::vector<const bf16*> gain2;                                  // full decoder block: post-attention RMSNorm gains
+  std::vector<CUtensorMap> tm_wo, tm_gate, tm_up, tm_down;         // ... and its weight matrices
   std::vector<CUtensorMap> tm_w;
   // key/value tensor maps of the attention: the persistent ones span all layers, streams and KV heads
   CUtensorMap tm_prefix_k, tm_prefix_v, tm_bank_k, tm_bank_v, tm_tail_k, tm_tail_v;
@@ -224,15 +232,15 @@ void seg_step(AttnSegment& sg, const CUtensorMap& k, const CUtensorMap& v, int k
 // choice minimises waves * ((rows_w + tile_n) / ksplit + the cost of summing a K split, about 40
 // row-equivalents) over 128- or 256-row weight tiles, the number of token tiles and the K split.
 // A K split needs the whole grid resident at once (its CTAs wait for one another), one CTA per SM.
-void choose_tiles(const Dims& D, int n_sms, int rows, int& tile_n, int& n_tiles, int& ksplit, int& m_sub) {
-  const int total_kb = D.d / GEMM_BLOCK_K;
+void choose_tiles(int K, int E, int n_sms, int rows, int& tile_n, int& n_tiles, int& ksplit, int& m_sub) {
+  const int total_kb = K / GEMM_BLOCK_K;
   const int resident = n_sms < GEMM_XCHG_CTAS ? n_sms : GEMM_XCHG_CTAS;
   const int nt_min = (rows + 255) / 256;
   long long best = -1;
   m_sub = 1; ksplit = 1; n_tiles = nt_min; tile_n = ((rows + nt_min - 1) / nt_min + 15) / 16 * 16;
   for (int sub = 1; sub <= 2; ++sub) {
-    if (sub == 2 && D.E_out % (2 * GEMM_BLOCK_M) != 0) continue;
-    const int mt = (D.E_out + GEMM_BLOCK_M * sub - 1) / (GEMM_BLOCK_M * sub);
+    if (sub == 2 && E % (2 * GEMM_BLOCK_M) != 0) continue;
+    const int mt = (E + GEMM_BLOCK_M * sub - 1) / (GEMM_BLOCK_M * sub);
     for (int nt = nt_min; nt <= nt_min + 32; ++nt) {
       const int tn = ((rows + nt - 1) / nt + 15) / 16 * 16;
       if ((long long)(nt - 1) * tn >= rows && nt > nt_min) continue;      // an empty last tile
@@ -298,17 +306,72 @@ int run_projection(vs_stream* h, int l, const bf16* src, int rows, const Project
     return VS_OK;
   }
   GemmArgs g;
-  choose_tiles(D, h->n_sms, rows, g.tile_n, g.n_tiles, g.ksplit, g.m_sub);
+  choose_tiles(D.d, D.E_out, h->n_sms, rows, g.tile_n, g.n_tiles, g.ksplit, g.m_sub);
   g.xchg = h->at<float>(h->lo.gemm_xchg);
   g.flags = h->at<int>(h->lo.gemm_flags);
   g.n_sms = h->n_sms;
-  g.tm_w = h->tm_w[l];
+  g.tm_w = h->tm_w[l]; g.tm_w2 = h->tm_w[l];
   if (encode_2d(h, &g.tm_x, src, (uint64_t)D.d, (uint64_t)rows, (uint32_t)g.tile_n) != VS_OK) return VS_ERR_CUDA;
   g.out = po;
   g.rows = rows; g.E_out = D.E_out; g.d = D.d;
   g.status = h->at<int>(h->lo.status);
   VS_LAUNCH(h, st, KC_GEMM, launch_qkv_gemm(g, bp, st));
   return VS_OK;
+}
+
+// One linear layer of the rest of the decoder block on the tensor cores: rows x K times W[E][K]^T, finished as
+// `po` says (mode 4: + residual; mode 5: SwiGLU of a gate / up pair, E = 2 * d_ff).
+int run_linear(vs_stream* h, const CUtensorMap& tm_w, const CUtensorMap& tm_w2, const bf16* src, int rows, int K, int E,
+               ProjectionOut po, const BatchParams& bp, cudaStream_t st) {
+  GemmArgs g;
+  choose_tiles(K, E, h->n_sms, rows, g.tile_n, g.n_tiles, g.ksplit, g.m_sub);
+  g.xchg = h->at<float>(h->lo.gemm_xchg);
+  g.flags = h->at<int>(h->lo.gemm_flags);
+  g.n_sms = h->n_sms;
+  g.tm_w = tm_w; g.tm_w2 = tm_w2;
+  if (encode_2d(h, &g.tm_x, src, (uint64_t)K, (uint64_t)rows, (uint32_t)g.tile_n) != VS_OK) return VS_ERR_CUDA;
+  po.rope = h->at<float2>(h->lo.rope);      // (not read: nothing is rotated; selects the kernel variant that takes a table)
+  po.inv_freq = h->at<double>(h->lo.inv_freq);
+  po.Hq = 0; po.Hkv = 0; po.D = 128; po.slots = 0; po.text_cap = 0; po.M = 0; po.norm_inline = 0;
+  g.out = po;
+  g.rows = rows; g.E_out = E; g.d = K;
+  g.status = h->at<int>(h->lo.status);
+  VS_LAUNCH(h, st, KC_GEMM, launch_qkv_gemm(g, bp, st));
+  return VS_OK;
+}
+
+// The rest of decoder layer l (Section 4.1: Qwen2 backbone) after its attention: a_rows = the attention rows (bf16,
+// [rows][d]), h_in = the layer's input.  h1 = h_in + A W_o^T -> hbuf[1]; act = SiLU(n W_gate^T) * (n W_up^T);
+// h2 = h1 + act W_down^T -> hbuf[0] (and `final_out` on the last layer).  Each stored tensor leaves its RMSNorm
+// statistics (and, with a gain vector, its gained copy) for the projection that reads it next.
+int run_block_rest(vs_stream* h, int l, int rows, const bf16* h_in, const bf16* a_rows, void* final_out, const BatchParams& bp,
+                   cudaStream_t st) {
+  const Dims& D = h->dm;
+  const Layout& lo = h->lo;
+  bf16* h1 = h->at<bf16>(lo.hbuf[1]);
+  bf16* h2 = h->at<bf16>(lo.hbuf[0]);
+  float* ss1 = h->at<float>(lo.row_ss);
+  float* ss2 = ss1 + (size_t)D.R_max * D.ss_parts;
+  ProjectionOut po;
+  std::memset(&po, 0, sizeof(po));
+  // W_o
+  po.mode = 4; po.lin_out = h1; po.lin_res = h_in; po.lin_out_region = DR_HBUF1;
+  if (D.use_rmsnorm) { po.ss_out = ss2; po.ss_out_parts = D.ss_parts; po.next_gain = h->gain2[l]; po.xn_out = h->at<bf16>(lo.xn); }
+  int rc = run_linear(h, h->tm_wo[l], h->tm_wo[l], a_rows, rows, D.d, D.d, po, bp, st);
+  if (rc != VS_OK) return rc;
+  // gate and up with the SwiGLU epilogue
+  std::memset(&po, 0, sizeof(po));
+  po.mode = 5; po.lin_out = h->at<bf16>(lo.act); po.lin_out_region = DR_ACT;
+  if (D.use_rmsnorm) { po.row_ss = ss2; po.ss_parts = D.ss_parts; po.norm_eps = D.rms_eps; }
+  const bf16* n_src = (D.use_rmsnorm && h->gain2[l] != nullptr) ? h->at<bf16>(lo.xn) : h1;
+  rc = run_linear(h, h->tm_gate[l], h->tm_up[l], n_src, rows, D.d, 2 * D.d_ff, po, bp, st);
+  if (rc != VS_OK) return rc;
+  // W_down
+  std::memset(&po, 0, sizeof(po));
+  po.mode = 4; po.lin_out = h2; po.lin_res = h1; po.lin_out_region = DR_HBUF0;
+  po.final_out = final_out; po.final_fp32 = D.out_fp32;
+  if (D.use_rmsnorm && l + 1 < D.L) { po.ss_out = ss1; po.ss_out_parts = D.ss_parts; po.next_gain = h->gain[l + 1]; po.xn_out = h->at<bf16>(lo.xn); }
+  return run_linear(h, h->tm_down[l], h->tm_down[l], h->at<bf16>(lo.act), rows, D.d_ff, D.d, po, bp, st);
 }
 
 size_t layer_stride_bank(const Dims& D) { return (size_t)D.S * D.Hkv * D.slots * D.D; }
@@ -391,6 +454,20 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights, void* work
         encode_kv(h, &h->tm_tail_k, h->ws + lo.tail_k, D.D, D.maxT, rb, nz, (uint64_t)D.maxT * rb) != VS_OK ||
         encode_kv(h, &h->tm_tail_v, h->ws + lo.tail_v, D.D, D.maxT, rb, nz, (uint64_t)D.maxT * rb) != VS_OK)
       return fail(VS_ERR_CUDA);
+  }
+  if (D.d_ff > 0) {
+    if (weights->w_o == nullptr || weights->w_gate == nullptr || weights->w_up == nullptr || weights->w_down == nullptr) return fail(VS_ERR_INVALID_ARG);
+    h->tm_wo.resize(D.L); h->tm_gate.resize(D.L); h->tm_up.resize(D.L); h->tm_down.resize(D.L);
+    for (int l = 0; l < D.L; ++l) {
+      const void* ptrs[4] = {weights->w_o[l], weights->w_gate[l], weights->w_up[l], weights->w_down[l]};
+      for (const void* q : ptrs) if (q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15u) != 0) return fail(VS_ERR_INVALID_ARG);
+      h->gain2.push_back(weights->norm2_w ? static_cast<const bf16*>(weights->norm2_w[l]) : nullptr);
+      if (encode_2d(h, &h->tm_wo[l], ptrs[0], (uint64_t)D.d, (uint64_t)D.d, GEMM_BLOCK_M) != VS_OK ||
+          encode_2d(h, &h->tm_gate[l], ptrs[1], (uint64_t)D.d, (uint64_t)D.d_ff, GEMM_BLOCK_M / 2) != VS_OK ||
+          encode_2d(h, &h->tm_up[l], ptrs[2], (uint64_t)D.d, (uint64_t)D.d_ff, GEMM_BLOCK_M / 2) != VS_OK ||
+          encode_2d(h, &h->tm_down[l], ptrs[3], (uint64_t)D.d_ff, (uint64_t)D.d, GEMM_BLOCK_M) != VS_OK)
+        return fail(VS_ERR_CUDA);
+    }
   }
   if (qkv_gemm_init() != cudaSuccess || qkv_gemv_init() != cudaSuccess || prefill_attention_tc_init() != cudaSuccess) return fail(VS_ERR_CUDA);
   for (int sp = 2; sp <= ATTN_MAX_SPLIT; ++sp) h->attn_clusters[sp] = prefill_attention_max_clusters(D.D, sp);
@@ -498,12 +575,12 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     if (D.use_rmsnorm) {
       // layer 0: a launch of its own; deeper layers: the attention kernel that stored h_in left the statistics
       if (l == 0) VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_ss),
-                                                                D.Hkv, rows, D.d, st));
+                                                                D.ss_parts, rows, D.d, st));
       if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
     }
     ProjectionOut fa;
     fa.bias = h->bias[l];
-    fa.row_ss = D.use_rmsnorm ? h->at<float>(lo.row_ss) : nullptr; fa.ss_parts = D.Hkv; fa.norm_eps = D.rms_eps;
+    fa.row_ss = D.use_rmsnorm ? h->at<float>(lo.row_ss) : nullptr; fa.ss_parts = D.ss_parts; fa.norm_eps = D.rms_eps;
     fa.norm_inline = 0; fa.norm_gain = nullptr;
     fa.rope = h->at<float2>(lo.rope);
     fa.inv_freq = h->at<double>(lo.inv_freq);
@@ -532,6 +609,11 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
     aa.h_out_region = (cur ^ 1) ? DR_HBUF1 : DR_HBUF0;
     if (D.use_rmsnorm && l + 1 < D.L) { aa.ss_out = h->at<float>(lo.row_ss); aa.next_gain = h->gain[l + 1]; aa.xn_out = h->at<bf16>(lo.xn); }
+    if (D.d_ff > 0) {
+      // full decoder block: the attention rows (bf16) feed the output projection; the residual comes there
+      aa.out = h->at<void>(lo.obuf); aa.out_fp32 = 0;
+      aa.h_in = nullptr; aa.h_out = nullptr; aa.ss_out = nullptr; aa.next_gain = nullptr; aa.xn_out = nullptr;
+    }
     aa.free_slot = h->at<int32_t>(lo.step_slot); aa.free_slot_stride = 1;
     {
       int kl[3] = {0, 0, N + 1};
@@ -546,9 +628,12 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active, 
     aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
     aa.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
     VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, bp, h->at<int>(lo.status), st));
-    if (D.residual) cur ^= 1;
+    if (D.d_ff > 0) {
+      // h2 lands in hbuf[0] again: the layer input of every layer is hbuf[0]
+      rc = run_block_rest(h, l, rows, h_in, h->at<bf16>(lo.obuf), last ? out_final : nullptr, bp, st);
+      if (rc != VS_OK) return rc;
+    } else if (D.residual) cur ^= 1;
   }
-
 
   for (int i = 0; i < n_active; ++i) {
     HostStream& s = h->hs[stream_ids[i]];
@@ -569,6 +654,7 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
   const Dims& D = h->dm;
   const Layout& lo = h->lo;
   if (N > D.maxN || F > D.maxChunk) return VS_ERR_CAPACITY;
+  if (D.d_ff > 0) return VS_ERR_UNSUPPORTED;       // the full decoder block is built for streaming and text steps
   HostStream& hs = h->hs[stream_id];
   if (hs.text_len != 0) return VS_ERR_STATE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -693,13 +779,13 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
     if (D.use_rmsnorm) {
       // layer 0: a launch of its own; deeper layers: the attention kernel that stored h_in left the statistics
       if (l == 0) VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_ss),
-                                                                D.Hkv, rows, D.d, st));
+                                                                D.ss_parts, rows, D.d, st));
       if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
     }
     ProjectionOut fa;
     std::memset(&fa, 0, sizeof(fa));
     fa.bias = h->bias[l];
-    fa.row_ss = D.use_rmsnorm ? h->at<float>(lo.row_ss) : nullptr; fa.ss_parts = D.Hkv; fa.norm_eps = D.rms_eps;
+    fa.row_ss = D.use_rmsnorm ? h->at<float>(lo.row_ss) : nullptr; fa.ss_parts = D.ss_parts; fa.norm_eps = D.rms_eps;
     fa.rope = h->at<float2>(lo.rope);
     fa.inv_freq = h->at<double>(lo.inv_freq);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
@@ -763,7 +849,7 @@ int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_strea
   if (rc != VS_OK) return rc;
   const Dims& D = h->dm;
   const Layout& lo = h->lo;
-  if ((D.d & 7) != 0) return VS_ERR_UNSUPPORTED;
+  if ((D.d & 7) != 0 || D.d_ff > 0) return VS_ERR_UNSUPPORTED;
   const HostStream& hs = h->hs[stream_id];
   const int count = (int)(hs.frames_seen < D.M ? hs.frames_seen : D.M);
   if (count == 0) return VS_OK;
@@ -794,13 +880,13 @@ int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_strea
     if (D.use_rmsnorm) {
       // layer 0: a launch of its own; deeper layers: the attention kernel that stored h_in left the statistics
       if (l == 0) VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_ss),
-                                                                D.Hkv, rows, D.d, st));
+                                                                D.ss_parts, rows, D.d, st));
       if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
     }
     ProjectionOut fa;
     std::memset(&fa, 0, sizeof(fa));
     fa.bias = h->bias[l];
-    fa.row_ss = D.use_rmsnorm ? h->at<float>(lo.row_ss) : nullptr; fa.ss_parts = D.Hkv; fa.norm_eps = D.rms_eps;
+    fa.row_ss = D.use_rmsnorm ? h->at<float>(lo.row_ss) : nullptr; fa.ss_parts = D.ss_parts; fa.norm_eps = D.rms_eps;
     fa.rope = h->at<float2>(lo.rope);
     fa.inv_freq = h->at<double>(lo.inv_freq);
     fa.q = h->at<bf16>(lo.q); fa.q_lo = h->at<bf16>(lo.q_lo); fa.kf = h->at<bf16>(lo.kf); fa.vf = h->at<bf16>(lo.vf);
@@ -897,8 +983,8 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
     if (D.use_rmsnorm && !by_gemv) {
       // layer 0, and every layer of a single-token step (its attention kernel leaves no statistics): a launch of
       // its own; else the tensor-core attention that stored h_in left them
-      if (l == 0 || T == 1) VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_ss),
-                                                                          D.Hkv, rows, D.d, st));
+      if (l == 0 || (T == 1 && D.d_ff == 0)) VS_LAUNCH(h, st, KC_RMSNORM, launch_rms_stats(h_in, h->gain[l], h->at<bf16>(lo.xn), h->at<float>(lo.row_ss),
+                                                                          D.ss_parts, rows, D.d, st));
       if (h->gain[l] != nullptr) src = h->at<bf16>(lo.xn);
     }
     bf16* pk = h->at<bf16>(lo.prefix_k) + (size_t)l * layer_stride_prefix(D);
@@ -910,7 +996,7 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
 
     ProjectionOut fa;
     fa.bias = h->bias[l];
-    fa.row_ss = (D.use_rmsnorm && !by_gemv) ? h->at<float>(lo.row_ss) : nullptr; fa.ss_parts = D.Hkv;
+    fa.row_ss = (D.use_rmsnorm && !by_gemv) ? h->at<float>(lo.row_ss) : nullptr; fa.ss_parts = D.ss_parts;
     fa.norm_inline = (D.use_rmsnorm && by_gemv) ? 1 : 0; fa.norm_gain = h->gain[l]; fa.norm_eps = D.rms_eps;
     fa.rope = rope_inline ? nullptr : h->at<float2>(lo.rope);
     fa.inv_freq = h->at<double>(lo.inv_freq);
@@ -935,6 +1021,7 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       da.out = (l == D.L - 1) ? out : h->at<void>(lo.obuf);
       da.out_fp32 = D.out_fp32;
       da.h_in = D.residual ? h_in : nullptr; da.h_out = h_out; da.h_out_region = h_out_region;
+      if (D.d_ff > 0) { da.out = h->at<void>(lo.obuf); da.out_fp32 = 0; da.h_in = nullptr; da.h_out = nullptr; }
       da.meta = meta;
       da.Hq = D.Hq; da.Hkv = D.Hkv; da.D = D.D; da.slots = D.slots; da.M = D.M; da.maxP = D.maxP; da.maxT = D.maxT;
       // short contexts: one CTA per (stream, query head) writes the row directly; longer ones are
@@ -975,9 +1062,17 @@ int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active, co
       aa.free_slot = &meta->free_slot; aa.free_slot_stride = (int)(sizeof(StreamMeta) / sizeof(int32_t));
       aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = D.M;
       aa.scale_log2e = scale_log2e;
+      if (D.d_ff > 0) {
+        aa.out = h->at<void>(lo.obuf); aa.out_fp32 = 0;
+        aa.h_in = nullptr; aa.h_out = nullptr; aa.ss_out = nullptr; aa.next_gain = nullptr; aa.xn_out = nullptr;
+      }
       VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, bp, h->at<int>(lo.status), st));
     }
-    if (D.residual) { h_in = h_out; next_buf ^= 1; }
+    if (D.d_ff > 0) {
+      rc = run_block_rest(h, l, rows, h_in, h->at<bf16>(lo.obuf), (l == D.L - 1) ? out : nullptr, bp, st);
+      if (rc != VS_OK) return rc;
+      h_in = h->at<bf16>(lo.hbuf[0]);
+    } else if (D.residual) { h_in = h_out; next_buf ^= 1; }
   }
 
   for (int i = 0; i < n_active; ++i) {

@@ -53,6 +53,11 @@ TAG_SCENE_CUT = 7
 TAG_LENGTHS = 8
 TAG_BIAS = 9
 TAG_NORM_W = 10
+TAG_W_O = 11
+TAG_W_GATE = 12
+TAG_W_UP = 13
+TAG_W_DOWN = 14
+TAG_NORM2_W = 15
 
 
 def splitmix64(x: np.ndarray) -> np.ndarray:
@@ -143,6 +148,14 @@ class Workload:
         n = self.e_out * self.d_model
         return normal_bf16(self.seed, TAG_WEIGHT, (self.e_out, self.d_model),
                            self.weight_std, offset=layer * n)
+
+    def block_weights(self, layer: int, d_ff: int) -> dict:
+        """The rest of decoder layer `layer` (output projection and SwiGLU MLP of width d_ff), bf16 bits,
+        all "out x in"; drawn like the projection weights, N(0, weight_std^2)."""
+        d = self.d_model
+        draw = lambda tag, shape: normal_bf16(self.seed, tag, shape, self.weight_std, offset=layer * shape[0] * shape[1])
+        return {"w_o": draw(TAG_W_O, (d, d)), "w_gate": draw(TAG_W_GATE, (d_ff, d)),
+                "w_up": draw(TAG_W_UP, (d_ff, d)), "w_down": draw(TAG_W_DOWN, (d, d_ff))}
 
     # ---- text-side hidden states -----------------------------------------------------
     def prefix_hidden(self, stream: int = 0) -> np.ndarray:

@@ -76,7 +76,7 @@ class Pair:
     def __init__(self, w: synth.Workload, n_streams: Optional[int] = None, max_step_tokens: int = 64,
                  evict_policy: int = 0, agg_mode: int = 0, with_bias: bool = False, with_gain: bool = False,
                  max_tokens_per_frame: Optional[int] = None, max_prefix: Optional[int] = None,
-                 max_text: Optional[int] = None, out_dtype: int = 1, max_chunk_frames: int = 1):
+                 max_text: Optional[int] = None, out_dtype: int = 1, max_chunk_frames: int = 1, d_ff: int = 0):
         self.w = w
         S = n_streams or w.n_streams
         self.S = S
@@ -93,18 +93,28 @@ class Pair:
             max_text if max_text is not None else max(w.question_len + w.decode_tokens, 1),
             w.bank_capacity, n_streams=S, max_step_tokens=max_step_tokens, agg_mode=agg_mode,
             evict_policy=evict_policy, use_rmsnorm=w.use_rmsnorm, residual=w.residual,
-            rope_theta=w.rope_theta, rms_eps=w.rms_eps, out_dtype=out_dtype, max_chunk_frames=max_chunk_frames)
+            rope_theta=w.rope_theta, rms_eps=w.rms_eps, out_dtype=out_dtype, max_chunk_frames=max_chunk_frames, d_ff=d_ff)
+        # the rest of the decoder block (output projection, SwiGLU MLP), with a gain for its norm when gains are on
+        blk = [w.block_weights(l, d_ff) for l in range(w.n_layers)] if d_ff else None
+        g2 = [synth.to_bf16_bits(1.0 + 0.1 * synth.standard_normal(w.seed, synth.TAG_NORM2_W, w.d_model, offset=l * w.d_model))
+              for l in range(w.n_layers)] if (d_ff and with_gain) else None
+        dev_block = None
+        if blk:
+            dev_block = {k: [to_dev(b[k]) for b in blk] for k in ("w_o", "w_gate", "w_up", "w_down")}
+            dev_block["norm2_w"] = [to_dev(g) for g in g2] if g2 else None
         self.gpu = binding.StreamBatch(self.cfg, [to_dev(b) for b in wbits],
                                        [to_dev(b) for b in bbits] if bbits else None,
-                                       [to_dev(b) for b in gbits] if gbits else None)
+                                       [to_dev(b) for b in gbits] if gbits else None, dev_block)
         ocfg = vo.OracleConfig(w.n_layers, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, w.bank_capacity,
                                agg_mode=agg_mode, evict_policy=evict_policy, use_rmsnorm=w.use_rmsnorm,
                                residual=w.residual, rope_theta=w.rope_theta, rms_eps=w.rms_eps)
         f64 = synth.bf16_bits_to_f64
+        oblk = [vo.BlockWeights(f64(b["w_o"]), f64(b["w_gate"]), f64(b["w_up"]), f64(b["w_down"]),
+                                f64(g2[l]) if g2 else None) for l, b in enumerate(blk)] if blk else None
         self.ora: List[vo.OracleStream] = [
             vo.OracleStream(ocfg, [f64(b) for b in wbits],
                             [f64(b) for b in bbits] if bbits else None,
-                            [f64(b) for b in gbits] if gbits else None) for _ in range(S)]
+                            [f64(b) for b in gbits] if gbits else None, oblk) for _ in range(S)]
         self.worst = [0.0, 0.0]
 
     def _note(self, e):

@@ -597,6 +597,34 @@ def test_bf16_output_against_the_oracle_at_the_qwen_shape():
     p.close()
 
 
+# ------------------------------------------------------------------ the rest of the decoder block
+def test_full_decoder_block_small():
+    """Output projection and SwiGLU MLP after every layer's attention (the Qwen2 block of the backbone,
+    Section 4.1): two layers with RMSNorm gains, frames with evictions, a question, single-token and
+    multi-token steps; a step's output is the last layer's hidden state."""
+    w = synth.workload("deep", n_layers=2, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64, tokens_per_frame=21,
+                       n_frames=6, bank_capacity=3, prefix_len=6, question_len=7, decode_tokens=3)
+    p = Pair(w, with_gain=True, d_ff=320)
+    run_stream(p, w, check_every=2)
+    for layer in range(2):
+        p.check_bank(0, layer=layer)
+    print("full block, small: worst", p.worst)
+    p.close()
+    # without RMSNorm, one layer, head_dim 128, a batch of two streams
+    w = synth.workload("batched", n_layers=1, d_model=512, n_q_heads=4, n_kv_heads=2, head_dim=128, tokens_per_frame=30,
+                       n_frames=4, min_frames=0, bank_capacity=2, prefix_len=4, decode_tokens=2, n_streams=2, residual=1)
+    p = Pair(w, d_ff=192)
+    ids = [0, 1]
+    p.text(ids, [w.prefix_hidden(s) for s in ids], "prefix")
+    for t in range(w.n_frames):
+        p.frame(ids, [w.frame_hidden(t, s) for s in ids], f"frame {t}")
+    for i in range(w.decode_tokens):
+        p.text(ids, [w.decode_hidden(i, s) for s in ids], f"decode {i}")
+    for s in ids:
+        p.check_bank(s)
+    p.close()
+
+
 # ------------------------------------------------------------------ limits and degenerate shapes
 def test_largest_frame_and_widest_group():
     """N = 255 (256-column token tile, the MMA's widest), 8 query heads per KV head (a full

@@ -27,13 +27,14 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_status_strings(lib):
     assert binding.status_string(0) == "ok"
-    for code in range(-6, 0):
+    for code in range(-7, 0):
         assert binding.status_string(code) not in ("ok", "unknown status")
     assert binding.status_string(-99) == "unknown status"
 
 
 def test_struct_layout_matches_header():
-    assert C.sizeof(binding.VsConfig) == 21 * 4
+    assert C.sizeof(binding.VsConfig) == 22 * 4
+    assert C.sizeof(binding.VsWeights) == 8 * 8
     assert C.sizeof(binding.VsBankInfo) == 4 + 4 + 5 * 8 + 4 + 4 + 8 + 8
 
 
