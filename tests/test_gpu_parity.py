@@ -5,7 +5,7 @@ import pytest
 import torch
 
 from paper_2503_09387_b200 import binding, synth
-from tests.parity import Pair, assert_close, bits_of, to_dev, to_f64
+from tests.parity import Pair, assert_close, assert_close_stored, bits_of, to_dev, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -403,13 +403,15 @@ class TeacherForced:
     (prefix, bank, tail).  Fed the oracle's recorded bf16 layer inputs step by step, so that every
     layer is compared at the stated tolerance on the inputs the oracle itself saw."""
 
-    def __init__(self, w, weights_dev):
+    def __init__(self, w, weights_dev, block_dev=None, d_ff=0):
         self.w = w
+        self.d_ff = d_ff
         cfg = binding.make_config(1, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens_per_frame,
                                   max(w.prefix_len, 1), max(w.question_len + w.decode_tokens, 1), w.bank_capacity,
                                   use_rmsnorm=w.use_rmsnorm, residual=w.residual, rope_theta=w.rope_theta,
-                                  rms_eps=w.rms_eps)
-        self.sb = [binding.StreamBatch(cfg, [weights_dev[l]]) for l in range(w.n_layers)]
+                                  rms_eps=w.rms_eps, d_ff=d_ff)
+        one = lambda l: {k: ([v[l]] if v is not None else None) for k, v in block_dev.items()} if block_dev else None
+        self.sb = [binding.StreamBatch(cfg, [weights_dev[l]], None, None, one(l)) for l in range(w.n_layers)]
         self.worst = [[0.0, 0.0] for _ in range(w.n_layers)]
 
     def step(self, rec, what):
@@ -420,7 +422,11 @@ class TeacherForced:
                 got = to_f64(sb.decode_step([0], to_dev(h[None])))[0]
             else:
                 got = to_f64(sb.frame_prefill([0], to_dev(h[None, :-1]), carrier_override=to_dev(h[None, -1])))[0]
-            e = assert_close(got, rec["O"][layer], f"teacher-forced layer {layer}, {what}")
+            if self.d_ff:      # the layer's output is its hidden state, a stored (bf16) tensor
+                e = assert_close_stored(got, rec["h_out"][layer], f"teacher-forced layer {layer}, {what}",
+                                        float(np.sqrt(1.0 + self.d_ff / self.w.d_model)))
+            else:
+                e = assert_close(got, rec["O"][layer], f"teacher-forced layer {layer}, {what}")
             self.worst[layer] = [max(self.worst[layer][0], e[0]), max(self.worst[layer][1], e[1])]
 
     def close(self):
@@ -428,14 +434,14 @@ class TeacherForced:
             sb.close()
 
 
-def run_chain(w, max_text, teacher=False, bank_layers=None):
+def run_chain(w, max_text, teacher=False, bank_layers=None, d_ff=0):
     """Free-running multi-layer stream on both sides (depth-scaled bound); with teacher=True every
     layer is also run teacher-forced at the stated tolerance.  Returns (worst of the chain, whether
     the chain met the stated tolerance, per-layer worst of the teacher-forced runs)."""
     from tests import parity
-    p = Pair(w, max_text=max_text)
+    p = Pair(w, max_text=max_text, d_ff=d_ff)
     p.ora[0].record = []
-    tf = TeacherForced(w, p.gpu.weights) if teacher else None
+    tf = TeacherForced(w, p.gpu.weights, p.gpu.block, d_ff) if teacher else None
     strict = (parity.MAX_ABS, parity.REL_RMS)
 
     def both(fn, what):
@@ -622,6 +628,28 @@ def test_full_decoder_block_small():
         p.text(ids, [w.decode_hidden(i, s) for s in ids], f"decode {i}")
     for s in ids:
         p.check_bank(s)
+    p.close()
+
+
+def test_full_decoder_block_28_layers_scaled_width():
+    """28 full decoder layers (attention, output projection, SwiGLU MLP; RMSNorm before each half) at a scaled
+    width (d_model 512, d_ff 1408): free-running at the depth-scaled bound, every layer teacher-forced at the
+    tolerance of stored tensors; 5 frames with evictions, a question, decode tokens."""
+    w = synth.workload("deep", d_model=512, n_q_heads=4, n_kv_heads=2, head_dim=128, tokens_per_frame=33, n_frames=5,
+                       bank_capacity=3, prefix_len=6, question_len=9, decode_tokens=3)
+    worst, met, per_layer = run_chain(w, w.question_len + w.decode_tokens, teacher=True, bank_layers=[0, 13, 27], d_ff=1408)
+    print("full block, 28 layers: chain worst %.3e %.3e (%s); teacher-forced worst %.3e %.3e" %
+          (worst[0], worst[1], "stated tolerance met" if met else "stated tolerance NOT met",
+           max(x[0] for x in per_layer), max(x[1] for x in per_layer)))
+
+
+def test_full_decoder_block_at_the_qwen2_7b_shape():
+    """One full decoder layer at the Qwen2-7B shape (d_model 3584, 28/4 heads x 128, d_ff 18944): prefix, three
+    frames of 169 tokens with a bank of 2 (one eviction), an 8-token question, two decode tokens."""
+    w = synth.workload("deep", n_layers=1, n_frames=3, bank_capacity=2, prefix_len=16, question_len=8, decode_tokens=2)
+    p = Pair(w, d_ff=18944, max_text=10)
+    run_stream(p, w, check_every=1)
+    print("full block, Qwen2-7B shape: worst", p.worst)
     p.close()
 
 
