@@ -41,7 +41,9 @@ ORACLE_KIND = "oracle (numpy, BLAS threads)"
 # shape, from the ncu capture summarised under profiles/ (cold cache: the weights come from DRAM,
 # whereas inside the timed one-layer loop they are L2-resident).  None = not captured since the
 # kernel last changed.
-DOMINANT_KERNEL_TRAFFIC = {"bytes": None, "source": "no ncu capture of the current kernel"}
+DOMINANT_KERNEL_TRAFFIC = {"bytes": 34.38e6 + 0.02e6,
+                           "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one cold-cache frame launch "
+                                     "(profiles/qkv_gemm_frame_170rows.md); in the timed loop the weights are L2-resident"}
 
 
 def load_peaks():
