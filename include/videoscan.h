@@ -130,8 +130,8 @@ int vs_workspace_bytes(const vs_config* cfg, size_t* out_bytes);
 /* Builds a handle over caller memory: carves `workspace` (DEVICE, >= vs_workspace_bytes,
  * 256-byte aligned) into bank, prefix, tail, metadata and per-step scratch, clears the
  * metadata (synchronously) and encodes the TMA descriptors of the weights.  Nothing is
- * allocated on the device, so memory use does not depend on stream length (the paper's
- * "stable GPU memory consumption", Section 3.3). */
+ * allocated on the device, so memory use does not depend on stream length (the constant
+ * memory footprint that Section 3.3 claims for the method holds by construction). */
 int vs_create_stream(const vs_config* cfg, const vs_weights* weights,
                      void* workspace, size_t workspace_bytes, vs_stream** out);
 
@@ -146,7 +146,9 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights,
  * carrier_override: DEVICE bf16 [n_active][d_model] used as the carrier token instead of
  *             the mean (e.g. projector(mean) computed by the caller), or NULL.
  * out:        DEVICE [n_active][N+1][Hq*D] of `out_dtype`, last layer's attention output, row N
- *             being the carrier's; may be NULL.
+ *             being the carrier's; may be NULL.  On a handle with d_ff > 0: the hidden state that
+ *             leaves the last decoder block (Hq*D == d_model there), a bf16 storage point widened
+ *             to `out_dtype`.
  * Errors: VS_ERR_STATE if a listed stream has an open text turn (call vs_end_turn first);
  *         VS_ERR_CAPACITY if N > max_tokens_per_frame. */
 int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
@@ -165,7 +167,8 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
  * back into `cuda_stream` by events, so that they run beside the projection; the handle's first
  * call of this function creates that stream and its two events (no device memory).
  * Errors: as vs_frame_prefill; VS_ERR_CAPACITY also if F > max_chunk_frames or if
- *         bank_capacity + 1 + F > 8192. */
+ *         bank_capacity + 1 + F > 8192; VS_ERR_UNSUPPORTED on a handle with d_ff > 0 (the rest of
+ *         the decoder block runs in the one-frame and text steps only). */
 int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, int32_t F, int32_t N,
                            void* out, void* cuda_stream);
 
@@ -175,7 +178,7 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
  * positions prefix_len + i, go through the layers, each attending over the prompt prefix and the
  * carriers up to itself.  Reads the bank, changes nothing.
  * out: DEVICE [count][Hq*D] of `out_dtype` (count = carriers in the bank; vs_bank_state tells).
- * count = 0 is not an error: nothing is launched. */
+ * count = 0 is not an error: nothing is launched.  VS_ERR_UNSUPPORTED on a handle with d_ff > 0. */
 int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_stream);
 
 /* T text tokens per listed stream -- the decoding phase of Section 3.3 (T = 1) and the
