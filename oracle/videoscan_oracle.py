@@ -36,6 +36,10 @@ Optional rest of the decoder block (the backbone of Section 4.1 is a Qwen2 decod
 with A the attention rows and n = RMSNorm(h1); storage points (bf16) are A, h1, the gated
 activation and h2, and a step then returns the last layer's h2 instead of its attention rows.
 
+Optional language-model head (``lm_head``): the final RMSNorm of the backbone, the vocabulary
+projection and the greedy choice of the next token -- what turns the hidden state of the last
+position into the first answer token of Section 3.3's decoding phase.
+
 Parity pins (tests/test_oracle_*.py): closed forms for the pooling, softmax row sums,
 GQA == MHA with repeated heads, brute-force dense masked attention over the un-pruned
 sequence, textbook causal attention for M = 0 and one-frame streams, RoPE identities,
@@ -238,6 +242,38 @@ class BlockWeights:
 def silu(x: np.ndarray) -> np.ndarray:
     """SiLU(x) = x * sigmoid(x) = x / (1 + exp(-x))."""
     return x / (1.0 + np.exp(-x))
+
+
+def lm_head(h: np.ndarray, w_lm: np.ndarray, gain: Optional[np.ndarray] = None, use_rmsnorm: bool = True,
+            rms_eps: float = 1e-6):
+    """Hidden states of the positions to be continued -> (logits, greedy next tokens).
+
+    Section 3.3 (decoding phase): the answer is generated token by token from the model's output at the
+    last position; the backbone of Section 4.1 (a Qwen2 decoder) ends in an RMSNorm and a vocabulary
+    projection.  h: [rows][d] (rounded to bf16 on entry: a hidden state is a stored tensor);
+    w_lm: [vocab][d] ("out x in"); gain: [d] of the final norm or None (unit gain).
+    logits[r][v] = sum_k n[r][k] * w_lm[v][k] with n = RMSNorm(h) * gain (n = h without the norm), kept in
+    fp64; token[r] = the index of the largest logit, the lowest index among equals."""
+    h = round_to_bf16(np.asarray(h, dtype=np.float64))
+    n = h
+    if use_rmsnorm:
+        ms = np.mean(h * h, axis=1, keepdims=True)
+        n = h / np.sqrt(ms + rms_eps)
+        if gain is not None:
+            n = n * np.asarray(gain, dtype=np.float64)[None, :]
+    logits = n @ np.asarray(w_lm, dtype=np.float64).T
+    tokens = np.array([greedy_token(row) for row in logits], dtype=np.int64)
+    return logits, tokens
+
+
+def greedy_token(logits_row: np.ndarray) -> int:
+    """Index of the largest value; the lowest index among equal largest values.  A NaN counts as
+    smaller than every number (a row of NaNs gives token 0)."""
+    best, best_v = 0, -math.inf
+    for i, v in enumerate(np.asarray(logits_row, dtype=np.float64)):
+        if v > best_v:                       # false for NaN
+            best, best_v = i, float(v)
+    return best
 
 
 @dataclasses.dataclass

@@ -118,3 +118,69 @@ def test_bank_keeps_attention_keys_of_the_block_stream():
     for ea, eb in zip(st_a.bank, st_b.bank):
         assert ea.frame_id == eb.frame_id and np.array_equal(ea.emb, eb.emb)
         assert np.array_equal(ea.K[0], eb.K[0]) and not np.array_equal(ea.K[1], eb.K[1])
+
+
+# ------------------------------------------------------------------ language-model head
+def test_lm_head_matches_a_library_restatement_and_scaling_laws():
+    """logits against torch (fp64 F.linear of a hand-normalised input); RMSNorm makes the logits
+    invariant to a power-of-two scaling of the hidden state (exact in bf16) up to the epsilon term;
+    without the norm they scale linearly."""
+    rng = np.random.default_rng(3)
+    d, V, R = 48, 37, 5
+    h = _bf(rng.normal(size=(R, d))); W = _bf(rng.normal(0, 0.3, (V, d))); g = _bf(1 + 0.2 * rng.normal(size=d))
+    logits, tok = vo.lm_head(h, W, g, True, 1e-6)
+    ht = torch.from_numpy(h)
+    nt = ht * torch.rsqrt((ht * ht).mean(dim=1, keepdim=True) + 1e-6) * torch.from_numpy(g)
+    want = torch.nn.functional.linear(nt, torch.from_numpy(W)).numpy()
+    np.testing.assert_allclose(logits, want, rtol=1e-12, atol=1e-12)
+    assert list(tok) == list(want.argmax(axis=1))
+    l4, _ = vo.lm_head(4.0 * h, W, g, True, 0.0)
+    l1, _ = vo.lm_head(h, W, g, True, 0.0)
+    np.testing.assert_allclose(l4, l1, rtol=1e-12, atol=1e-12)
+    p4, _ = vo.lm_head(4.0 * h, W, None, False)
+    p1, _ = vo.lm_head(h, W, None, False)
+    np.testing.assert_allclose(p4, 4.0 * p1, rtol=1e-12, atol=1e-12)
+
+
+def test_lm_head_closed_forms():
+    """One-hot vocabulary rows read single channels of the normalised state; a constant hidden row
+    normalises to +-1 per channel; the gain multiplies after the normalisation (a gain inside the
+    mean of squares, or a transposed weight, fails here)."""
+    d = 16
+    W = np.eye(d)                                   # vocab = d, row v reads channel v
+    h = np.full((1, d), 3.0)
+    logits, tok = vo.lm_head(h, W, None, True, 0.0)
+    np.testing.assert_allclose(logits, np.ones((1, d)), atol=1e-12)
+    assert tok[0] == 0                              # all equal: lowest index
+    g = np.arange(1, d + 1, dtype=np.float64)
+    logits, tok = vo.lm_head(-h, W, g, True, 0.0)
+    np.testing.assert_allclose(logits, -g[None, :], atol=1e-12)
+    assert tok[0] == 0                              # -1 is the largest of -1 .. -16
+    h2 = np.zeros((1, d)); h2[0, 5] = 2.0           # one live channel: rms = 2 / sqrt(d)
+    logits, tok = vo.lm_head(h2, W, g, True, 0.0)
+    assert tok[0] == 5 and abs(logits[0, 5] - math.sqrt(d) * 6.0) < 1e-12
+    Wr = np.zeros((3, d)); Wr[0, 1] = 1.0; Wr[1, 2] = 1.0; Wr[2, 1] = 1.0       # non-square: [vocab][d]
+    h3 = np.zeros((1, d)); h3[0, 2] = 1.0
+    assert vo.lm_head(h3, Wr, None, False)[1][0] == 1
+
+
+def test_greedy_token_ties_and_non_finite_values():
+    assert vo.greedy_token(np.array([1.0, 3.0, 3.0, 2.0])) == 1
+    assert vo.greedy_token(np.array([-math.inf, -math.inf])) == 0
+    assert vo.greedy_token(np.array([math.nan, -5.0, math.nan])) == 1
+    assert vo.greedy_token(np.array([math.nan, math.nan])) == 0
+    assert vo.greedy_token(np.array([0.0, math.inf, math.inf])) == 1
+    rng = np.random.default_rng(0)
+    for _ in range(20):
+        x = rng.integers(-3, 4, size=50).astype(np.float64)
+        assert vo.greedy_token(x) == int(np.argmax(x))          # numpy's argmax also takes the first maximum
+
+
+def test_lm_head_rounds_the_hidden_state_on_entry():
+    """The hidden state is a stored (bf16) tensor: values that differ below bf16 resolution give the
+    same logits."""
+    rng = np.random.default_rng(5)
+    h = _bf(rng.normal(size=(2, 32))); W = _bf(rng.normal(size=(9, 32)))
+    a, _ = vo.lm_head(h, W, None, True)
+    b, _ = vo.lm_head(h * (1 + 2.0 ** -12), W, None, True)
+    np.testing.assert_array_equal(a, b)
