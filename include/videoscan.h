@@ -89,6 +89,8 @@ typedef struct {
                                     decoder block (Section 4.1: the backbone is a Qwen2 decoder); a multiple
                                     of 64; needs residual = 1, d_model a multiple of 128 and the four block
                                     weight arrays of vs_weights                                         */
+  int32_t vocab;                 /* 0: no language-model head.  > 0: rows of the vocabulary projection used by
+                                    vs_lm_head; a multiple of 128; needs vs_weights.w_lm                */
 } vs_config;
 
 /* DEVICE pointers to bf16 weights, one entry per layer.  The arrays of pointers themselves
@@ -107,6 +109,9 @@ typedef struct {
   const void* const* w_up;       /* [n_layers] each [d_ff, d_model]                                  */
   const void* const* w_down;     /* [n_layers] each [d_model, d_ff]                                  */
   const void* const* norm2_w;    /* [n_layers] each [d_model] gain of the post-attention RMSNorm, or NULL */
+  /* the language-model head, read only when vocab > 0 (single DEVICE pointers, not per layer): */
+  const void* w_lm;              /* [vocab, d_model] row-major, 16-byte aligned                      */
+  const void* norm_f_w;          /* [d_model] gain of the final RMSNorm, or NULL = all ones          */
 } vs_weights;
 
 /* Filled by vs_bank_state (HOST). */
@@ -191,6 +196,21 @@ int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_strea
  * Errors: VS_ERR_CAPACITY on prefix / tail overflow or T > max_step_tokens. */
 int vs_decode_step(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
                    const void* hidden, int32_t T, void* out, void* cuda_stream);
+
+/* Language-model head -- what turns the hidden state of a last position into the next answer token in
+ * the decoding phase of Section 3.3.  The paper prints no formula for it; it is the head of the Qwen2
+ * backbone named in Section 4.1:  logits = (RMSNorm(hidden) * norm_f_w) W_lm^T  (no norm when
+ * use_rmsnorm = 0),  next_token = the index of the largest logit, the lowest index among equals, a NaN
+ * ranking below every number.
+ * hidden: DEVICE [rows][d_model] of `out_dtype` (so the rows a step wrote to `out` can be passed on as
+ *         they are); each value is rounded to bf16 on entry -- a hidden state is a stored tensor;
+ *         8-byte aligned.  rows: 1 .. 256, and no more than the handle's largest step.
+ * logits: DEVICE fp32 [rows][vocab], 16-byte aligned, the caller's; always written.
+ * next_token: DEVICE int32 [rows], or NULL.
+ * Uses the step scratch of the handle: enqueue it on the handle's stream like any other step.
+ * Errors: VS_ERR_UNSUPPORTED on a handle created with vocab = 0; VS_ERR_CAPACITY for too many rows. */
+int vs_lm_head(vs_stream* h, const void* hidden, int32_t rows, void* logits, int32_t* next_token,
+               void* cuda_stream);
 
 /* Ends a question/answer turn: the text tail is dropped, prefix and bank stay, frame
  * positions do not move.  Host-only bookkeeping. */

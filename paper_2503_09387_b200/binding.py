@@ -28,7 +28,7 @@ VS_ERR_BOUNDS = -7
 VS_MAX_BATCH = 64
 
 EXPORTS = ["vs_workspace_bytes", "vs_create_stream", "vs_frame_prefill", "vs_frame_prefill_chunk", "vs_bank_forward", "vs_decode_step",
-           "vs_end_turn", "vs_bank_state", "vs_last_step_kv", "vs_poison_scratch",
+           "vs_lm_head", "vs_end_turn", "vs_bank_state", "vs_last_step_kv", "vs_poison_scratch",
            "vs_destroy_stream", "vs_status_string", "vs_reset_stream", "vs_profile_enable",
            "vs_profile_read", "vs_kernel_class_name", "vs_evict_choose_static"]
 VS_STATIC_MAX_BANK = 4096
@@ -42,13 +42,14 @@ class VsConfig(C.Structure):
         "evict_policy", "use_rmsnorm", "residual")] + [
         ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("device", C.c_int32),
         ("evict_log_capacity", C.c_int32), ("out_dtype", C.c_int32),
-        ("max_chunk_frames", C.c_int32), ("d_ff", C.c_int32)]
+        ("max_chunk_frames", C.c_int32), ("d_ff", C.c_int32), ("vocab", C.c_int32)]
 
 
 class VsWeights(C.Structure):
     _fields_ = [("w_qkv", C.POINTER(C.c_void_p)), ("b_qkv", C.POINTER(C.c_void_p)),
                 ("norm_w", C.POINTER(C.c_void_p)), ("w_o", C.POINTER(C.c_void_p)), ("w_gate", C.POINTER(C.c_void_p)),
-                ("w_up", C.POINTER(C.c_void_p)), ("w_down", C.POINTER(C.c_void_p)), ("norm2_w", C.POINTER(C.c_void_p))]
+                ("w_up", C.POINTER(C.c_void_p)), ("w_down", C.POINTER(C.c_void_p)), ("norm2_w", C.POINTER(C.c_void_p)),
+                ("w_lm", C.c_void_p), ("norm_f_w", C.c_void_p)]
 
 
 class VsBankInfo(C.Structure):
@@ -87,6 +88,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.vs_bank_forward.argtypes = [vp, i32, vp, vp]
     lib.vs_decode_step.argtypes = [vp, i32p, i32, vp, i32, vp, vp]
     lib.vs_end_turn.argtypes = [vp, i32p, i32]
+    lib.vs_lm_head.argtypes = [vp, vp, i32, vp, vp, vp]
     lib.vs_bank_state.argtypes = [vp, i32, C.POINTER(VsBankInfo), i32p, C.POINTER(C.c_int64), i32p,
                                   i32p, i32, i32p, vp, i32, vp, vp]
     lib.vs_last_step_kv.argtypes = [vp, vp, vp, i32]
@@ -131,14 +133,15 @@ def vs_workspace_bytes(cfg: VsConfig) -> int:
 
 def vs_create_stream(cfg: VsConfig, w_ptrs: List[int], b_ptrs: Optional[List[Optional[int]]],
                      g_ptrs: Optional[List[Optional[int]]], workspace_ptr: int, workspace_bytes: int,
-                     block_ptrs: Optional[dict] = None) -> int:
-    """block_ptrs (full decoder block, cfg.d_ff > 0): {"w_o", "w_gate", "w_up", "w_down": [L pointers], "norm2_w": [L] or None}."""
+                     block_ptrs: Optional[dict] = None, lm_ptrs: Optional[Sequence[Optional[int]]] = None) -> int:
+    """block_ptrs (full decoder block, cfg.d_ff > 0): {"w_o", "w_gate", "w_up", "w_down": [L pointers], "norm2_w": [L] or None}.
+    lm_ptrs (language-model head, cfg.vocab > 0): (w_lm pointer, final-norm gain pointer or None)."""
     L = cfg.n_layers
     arr = lambda ptrs: C.cast((C.c_void_p * L)(*[p or None for p in ptrs]), C.POINTER(C.c_void_p)) if ptrs is not None else None
     keep = [arr(w_ptrs), arr(b_ptrs), arr(g_ptrs)]
     for name in ("w_o", "w_gate", "w_up", "w_down", "norm2_w"):
         keep.append(arr(block_ptrs.get(name)) if block_ptrs else None)
-    ws = VsWeights(*keep)
+    ws = VsWeights(*keep, (lm_ptrs[0] if lm_ptrs else None), (lm_ptrs[1] if lm_ptrs else None) or None)
     handle = C.c_void_p(None)
     _check(load_library().vs_create_stream(C.byref(cfg), C.byref(ws), workspace_ptr, workspace_bytes,
                                            C.byref(handle)), "vs_create_stream")
@@ -150,6 +153,12 @@ def vs_frame_prefill(handle: int, stream_ids: Sequence[int], hidden_ptr: int, N:
     ids, n = _ids(stream_ids)
     _check(load_library().vs_frame_prefill(handle, ids, n, hidden_ptr, N, carrier_override_ptr or None,
                                            out_ptr or None, cuda_stream or None), "vs_frame_prefill")
+
+
+def vs_lm_head(handle: int, hidden_ptr: int, rows: int, logits_ptr: int, next_token_ptr: Optional[int],
+               cuda_stream: Optional[int] = None) -> None:
+    _check(load_library().vs_lm_head(handle, hidden_ptr, rows, logits_ptr, next_token_ptr or None, cuda_stream or None),
+           "vs_lm_head")
 
 
 def vs_bank_forward(handle: int, stream_id: int, out_ptr: int, cuda_stream: Optional[int] = None) -> None:
@@ -264,8 +273,9 @@ class StreamBatch:
     [E_out, d_model] per layer.  All methods take / return torch CUDA tensors and only enqueue
     work on the current torch stream."""
 
-    def __init__(self, cfg: VsConfig, weights, biases=None, norm_weights=None, block=None):
+    def __init__(self, cfg: VsConfig, weights, biases=None, norm_weights=None, block=None, lm=None):
         # block (cfg.d_ff > 0): {"w_o", "w_gate", "w_up", "w_down": [L device tensors], "norm2_w": [L] or None}
+        # lm (cfg.vocab > 0): (w_lm [vocab, d_model] device tensor, final-norm gain [d_model] or None)
         import torch
         self.torch = torch
         self.cfg = cfg
@@ -274,6 +284,7 @@ class StreamBatch:
         self.biases = biases
         self.norm_weights = norm_weights
         self.block = block
+        self.lm = lm
         nbytes = vs_workspace_bytes(cfg)
         self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
         base = self.workspace.data_ptr()
@@ -285,12 +296,23 @@ class StreamBatch:
             [g.data_ptr() if g is not None else None for g in norm_weights] if norm_weights is not None else None,
             self._ws_ptr, nbytes,
             {k: ([t.data_ptr() if t is not None else None for t in v] if v is not None else None) for k, v in block.items()}
-            if block else None)
+            if block else None,
+            (lm[0].data_ptr(), lm[1].data_ptr() if lm[1] is not None else None) if lm else None)
         self.out_width = cfg.n_q_heads * cfg.head_dim
         self.out_torch_dtype = torch.float32 if cfg.out_dtype == 1 else torch.bfloat16
 
     def _stream(self) -> int:
         return self.torch.cuda.current_stream(self.device).cuda_stream
+
+    def lm_head(self, hidden, logits=None, want_token=True):
+        """hidden: [rows, d_model] of the handle's output dtype -> (logits fp32 [rows, vocab], next tokens int32 [rows] or None)."""
+        rows = hidden.shape[0]
+        assert hidden.is_contiguous() and hidden.dtype == self.out_torch_dtype and hidden.numel() == rows * self.cfg.d_model
+        if logits is None:
+            logits = self.torch.empty((rows, self.cfg.vocab), dtype=self.torch.float32, device=self.device)
+        token = self.torch.empty((rows,), dtype=self.torch.int32, device=self.device) if want_token else None
+        vs_lm_head(self.handle, hidden.data_ptr(), rows, logits.data_ptr(), token.data_ptr() if want_token else None, self._stream())
+        return logits, token
 
     def frame_prefill(self, stream_ids, hidden, carrier_override=None, out=None, want_out=True):
         n = len(stream_ids)
@@ -364,7 +386,7 @@ class StreamBatch:
 def make_config(n_layers, d_model, n_q_heads, n_kv_heads, head_dim, max_tokens_per_frame, max_prefix,
                 max_text, bank_capacity, n_streams=1, max_step_tokens=64, agg_mode=0, evict_policy=0,
                 use_rmsnorm=0, residual=0, rope_theta=1.0e6, rms_eps=1.0e-6, device=0,
-                evict_log_capacity=4096, out_dtype=1, max_chunk_frames=1, d_ff=0) -> VsConfig:
+                evict_log_capacity=4096, out_dtype=1, max_chunk_frames=1, d_ff=0, vocab=0) -> VsConfig:
     return VsConfig(n_layers, d_model, n_q_heads, n_kv_heads, head_dim, max_tokens_per_frame, max_prefix,
                     max_text, max_step_tokens, bank_capacity, n_streams, agg_mode, evict_policy, use_rmsnorm,
-                    residual, rope_theta, rms_eps, device, evict_log_capacity, out_dtype, max_chunk_frames, d_ff)
+                    residual, rope_theta, rms_eps, device, evict_log_capacity, out_dtype, max_chunk_frames, d_ff, vocab)

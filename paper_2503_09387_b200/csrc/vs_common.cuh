@@ -78,6 +78,7 @@ __device__ __forceinline__ bool vs_store_ok(const BatchParams& bp, int region, c
 struct Dims {
   int L, d, Hq, Hkv, D, G, E_out;
   int d_ff;                                      // 0, or the SwiGLU width of the full decoder block
+  int vocab;                                     // 0, or the rows of the vocabulary projection (language-model head)
   int ss_parts;                                  // parts a row's sum of squares comes in: Hkv (from the attention kernel) or d / 128
   int maxN, maxP, maxT, maxStepT, M, slots, S, maxChunk;   // maxP / maxT: allocated rows (>= 1)
   int capP, capT;                                // caller's prefix / tail capacities
@@ -220,6 +221,12 @@ cudaError_t launch_rope_table(const RopeArgs& a, const BatchParams& bp, cudaStre
 // sum of squares of every row -> row_ss[row][parts] (part 0; the other parts zero); with a gain vector hg = bf16(h * gain)
 cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* row_ss, int parts, int rows, int d,
                              cudaStream_t st);
+// Input of the language-model head: xn[row] = bf16(h[row]) (times gain, rounded again, with a gain vector), the
+// sum of squares of bf16(h[row]) in part 0 of row_ss[row][parts].  h is fp32 or bf16.
+cudaError_t launch_lm_norm(const void* h, int h_fp32, const bf16* gain, bf16* xn, float* row_ss, int parts, int rows, int d,
+                           cudaStream_t st);
+// token[row] = index of the largest of logits[row][0..vocab), the lowest index among equals, NaN below everything
+cudaError_t launch_argmax_rows(const float* logits, int32_t* token, int rows, int vocab, cudaStream_t st);
 
 // What the projection epilogue writes (finished rows: bias, RoPE, bf16) and where rows persist.
 struct ProjectionOut {
@@ -245,7 +252,8 @@ struct ProjectionOut {
   int Hq, Hkv, D, slots, text_cap, M;
   int mode;                      // 0 frame step (carrier row -> bank), 1 text -> prefix, 2 text -> tail,
                                  // 3 chunk of frames (nothing kept here: a commit kernel copies the carrier rows),
-                                 // 4 plain linear layer + residual, 5 SwiGLU gate/up pair (the rest of the decoder block)
+                                 // 4 plain linear layer + residual, 5 SwiGLU gate/up pair (the rest of the decoder block),
+                                 // 6 plain linear layer, fp32 rows to final_out[row][E_out] (the vocabulary projection)
   // modes 4 and 5: lin_out[row][E] = bf16(acc * row scale + lin_res[row][E]) (mode 4, E = E_out), or
   // lin_out[row][E_out / 2] = bf16(SiLU(gate) * up) (mode 5: every 128-row weight tile is 64 gate rows, then 64 up rows)
   bf16* lin_out; const bf16* lin_res;

@@ -433,6 +433,13 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
           if (VS_STORE_OK(bp, p.o.lin_out_region, dst, 8)) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(av);
           return;
         }
+        if (p.o.mode == 6) {
+          // plain linear layer, rows kept in fp32 (logits of the vocabulary projection); the buffer is the caller's
+          float* fo = static_cast<float*>(p.o.final_out) + (size_t)row * p.E_out + m0e;
+          *reinterpret_cast<float4*>(fo + f1) = make_float4(x1[0], x1[1], x1[2], x1[3]);
+          *reinterpret_cast<float4*>(fo + f2) = make_float4(x2[0], x2[1], x2[2], x2[3]);
+          return;
+        }
         if (p.o.mode == 4) {
           // linear layer + residual; the rows as stored (bf16) also give the next RMSNorm its statistics
           const size_t c1 = (size_t)row * p.E_out + m0e + f1, c2 = (size_t)row * p.E_out + m0e + f2;

@@ -62,6 +62,9 @@ int fill_dims(const vs_config* c, Dims& D) {
   if (c->d_ff > 0 && (!c->residual || c->n_q_heads * c->head_dim != c->d_model)) return VS_ERR_INVALID_ARG;
   if (c->d_ff > 0 && (c->d_ff % 64 != 0 || c->d_model % 128 != 0)) return VS_ERR_UNSUPPORTED;
   D.ss_parts = D.d_ff > 0 ? D.d / 128 : D.Hkv;
+  D.vocab = c->vocab;
+  if (c->vocab < 0) return VS_ERR_INVALID_ARG;
+  if (c->vocab > 0 && c->vocab % GEMM_BLOCK_M != 0) return VS_ERR_UNSUPPORTED;
   return VS_OK;
 }
 
@@ -138,6 +141,8 @@ struct vs_stream {
   std::vector<const bf16*> gain2;                                  // full decoder block: post-attention RMSNorm gains
   std::vector<CUtensorMap> tm_wo, tm_gate, tm_up, tm_down;         // ... and its weight matrices
   std::vector<CUtensorMap> tm_w;
+  CUtensorMap tm_lm;                         // language-model head: the vocabulary projection [vocab][d]
+  const bf16* gain_f = nullptr;              // ... and the gain of the final RMSNorm (null: unit gain)
   // key/value tensor maps of the attention: the persistent ones span all layers, streams and KV heads
   CUtensorMap tm_prefix_k, tm_prefix_v, tm_bank_k, tm_bank_v, tm_tail_k, tm_tail_v;
   CUtensorMap tm_step_k, tm_step_v;          // the step's own rows [rows][Hkv * D]; re-encoded when `rows` changes
@@ -468,6 +473,11 @@ int vs_create_stream(const vs_config* cfg, const vs_weights* weights, void* work
           encode_2d(h, &h->tm_down[l], ptrs[3], (uint64_t)D.d_ff, (uint64_t)D.d, GEMM_BLOCK_M) != VS_OK)
         return fail(VS_ERR_CUDA);
     }
+  }
+  if (D.vocab > 0) {
+    if (weights->w_lm == nullptr || (reinterpret_cast<uintptr_t>(weights->w_lm) & 15u) != 0) return fail(VS_ERR_INVALID_ARG);
+    h->gain_f = static_cast<const bf16*>(weights->norm_f_w);
+    if (encode_2d(h, &h->tm_lm, weights->w_lm, (uint64_t)D.d, (uint64_t)D.vocab, GEMM_BLOCK_M) != VS_OK) return fail(VS_ERR_CUDA);
   }
   if (qkv_gemm_init() != cudaSuccess || qkv_gemv_init() != cudaSuccess || prefill_attention_tc_init() != cudaSuccess) return fail(VS_ERR_CUDA);
   for (int sp = 2; sp <= ATTN_MAX_SPLIT; ++sp) h->attn_clusters[sp] = prefill_attention_max_clusters(D.D, sp);
@@ -1142,6 +1152,34 @@ const char* vs_kernel_class_name(int32_t k) {
                                                    "prefill_attention", "decode_attention", "chunk_scores",
                                                    "bank_update", "other"};
   return (k >= 0 && k < VS_N_KERNEL_CLASSES) ? names[k] : "?";
+}
+
+int vs_lm_head(vs_stream* h, const void* hidden, int32_t rows, void* logits, int32_t* next_token, void* cuda_stream) {
+  if (h == nullptr || hidden == nullptr || logits == nullptr) return VS_ERR_INVALID_ARG;
+  const Dims& D = h->dm;
+  const Layout& lo = h->lo;
+  if (D.vocab == 0) return VS_ERR_UNSUPPORTED;
+  if (rows < 1) return VS_ERR_INVALID_ARG;
+  if (rows > D.R_max || rows > 256) return VS_ERR_CAPACITY;
+  if ((reinterpret_cast<uintptr_t>(hidden) & 7u) != 0 || (reinterpret_cast<uintptr_t>(logits) & 15u) != 0) return VS_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  VS_CK(cudaSetDevice(h->device));
+  BatchParams bp;
+  VS_BP_INIT(h, bp);
+  bp.n_active = 1;
+  bp.rows_per_stream = rows;
+  VS_TRACE_NEXT(h, bp);
+  bf16* xn = h->at<bf16>(lo.xn);
+  float* ss = h->at<float>(lo.row_ss);
+  VS_LAUNCH(h, st, KC_RMSNORM, launch_lm_norm(hidden, D.out_fp32, D.use_rmsnorm ? h->gain_f : nullptr, xn, ss, D.ss_parts, rows, D.d, st));
+  ProjectionOut po;
+  std::memset(&po, 0, sizeof(po));
+  po.mode = 6; po.final_out = logits; po.final_fp32 = 1;
+  if (D.use_rmsnorm) { po.row_ss = ss; po.ss_parts = D.ss_parts; po.norm_eps = D.rms_eps; }
+  int rc = run_linear(h, h->tm_lm, h->tm_lm, xn, rows, D.d, D.vocab, po, bp, st);
+  if (rc != VS_OK) return rc;
+  if (next_token != nullptr) VS_LAUNCH(h, st, KC_OTHER, launch_argmax_rows(static_cast<const float*>(logits), next_token, rows, D.vocab, st));
+  return VS_OK;
 }
 
 int vs_end_turn(vs_stream* h, const int32_t* stream_ids, int32_t n_active) {

@@ -179,6 +179,93 @@ cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* r
   return launch_pdl(rms_stats_kernel, dim3(rows), dim3(256), 0, st, h, gain, hg, row_ss, parts, d);
 }
 
+// ------------------------------------------------------------------------------------------
+// Language-model head (Section 3.3, decoding phase: the next token comes from the output at the last
+// position; the Qwen2 backbone of Section 4.1 ends in an RMSNorm and a vocabulary projection).
+// lm_norm_kernel: the hidden rows enter as a stored (bf16) tensor whatever type they arrive in; the
+// projection reads xn and applies the row scale from the sum of squares left here.  One block per row.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) lm_norm_kernel(const void* __restrict__ h, int h_fp32, const bf16* __restrict__ gain,
+                                                      bf16* __restrict__ xn, float* __restrict__ row_ss, int parts, int d) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const size_t row = blockIdx.x;
+  float ss = 0.f;
+  for (int c = threadIdx.x * 2; c < d; c += 512) {
+    __nv_bfloat162 hv;
+    if (h_fp32) {
+      const float2 f = *reinterpret_cast<const float2*>(static_cast<const float*>(h) + row * d + c);
+      hv = __floats2bfloat162_rn(f.x, f.y);
+    } else {
+      hv = *reinterpret_cast<const __nv_bfloat162*>(static_cast<const bf16*>(h) + row * d + c);
+    }
+    const float2 v = __bfloat1622float2(hv);
+    ss += v.x * v.x + v.y * v.y;
+    if (gain != nullptr) {
+      const float2 g = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(gain + c));
+      hv = __floats2bfloat162_rn(v.x * g.x, v.y * g.y);
+    }
+    *reinterpret_cast<__nv_bfloat162*>(xn + row * d + c) = hv;
+  }
+  __shared__ float red[8];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) tot += red[i];
+    row_ss[row * parts] = tot;
+    for (int i = 1; i < parts; ++i) row_ss[row * parts + i] = 0.f;
+  }
+}
+
+cudaError_t launch_lm_norm(const void* h, int h_fp32, const bf16* gain, bf16* xn, float* row_ss, int parts, int rows, int d,
+                           cudaStream_t st) {
+  return launch_pdl(lm_norm_kernel, dim3(rows), dim3(256), 0, st, h, h_fp32, gain, xn, row_ss, parts, d);
+}
+
+// Greedy choice: one block per row.  (value, index) pairs are compared as "larger value, else
+// equal value and lower index"; a NaN is never larger, so it loses to every number, and a row
+// without any number above -inf gives token 0.
+__global__ void __launch_bounds__(1024) argmax_rows_kernel(const float* __restrict__ logits, int32_t* __restrict__ token, int vocab) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const float* src = logits + (size_t)blockIdx.x * vocab;
+  float bv = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int i = threadIdx.x; i < vocab; i += 1024) {
+    const float v = src[i];
+    if (v > bv) { bv = v; bi = i; }          // ascending i per thread: the first of equals stays
+  }
+  auto better = [](float v1, int i1, float v2, int i2) { return v1 > v2 || (v1 == v2 && i1 < i2); };
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+  }
+  __shared__ float sv[32];
+  __shared__ int si[32];
+  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    bv = sv[threadIdx.x]; bi = si[threadIdx.x];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    }
+    if (threadIdx.x == 0) token[blockIdx.x] = (bi == 0x7fffffff) ? 0 : bi;
+  }
+}
+
+cudaError_t launch_argmax_rows(const float* logits, int32_t* token, int rows, int vocab, cudaStream_t st) {
+  return launch_pdl(argmax_rows_kernel, dim3(rows), dim3(1024), 0, st, logits, token, vocab);
+}
+
 // The bank update of one frame as a launch of its own (chunked prefill).
 __global__ void __launch_bounds__(256, 8) bank_update_kernel(BankUpdateArgs a, BatchParams bp) {   // <= 32 registers: fits beside a projection CTA
   pdl_wait();

@@ -58,6 +58,8 @@ TAG_W_GATE = 12
 TAG_W_UP = 13
 TAG_W_DOWN = 14
 TAG_NORM2_W = 15
+TAG_W_LM = 16
+TAG_NORM_F_W = 17
 
 
 def splitmix64(x: np.ndarray) -> np.ndarray:
@@ -156,6 +158,10 @@ class Workload:
         draw = lambda tag, shape: normal_bf16(self.seed, tag, shape, self.weight_std, offset=layer * shape[0] * shape[1])
         return {"w_o": draw(TAG_W_O, (d, d)), "w_gate": draw(TAG_W_GATE, (d_ff, d)),
                 "w_up": draw(TAG_W_UP, (d_ff, d)), "w_down": draw(TAG_W_DOWN, (d, d_ff))}
+
+    def lm_weights(self, vocab: int) -> np.ndarray:
+        """Vocabulary projection [vocab, d_model] of the language-model head, bf16 bits, N(0, weight_std^2)."""
+        return normal_bf16(self.seed, TAG_W_LM, (vocab, self.d_model), self.weight_std)
 
     # ---- text-side hidden states -----------------------------------------------------
     def prefix_hidden(self, stream: int = 0) -> np.ndarray:

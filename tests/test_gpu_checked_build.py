@@ -98,3 +98,12 @@ def test_the_guard_check_is_alive(checked_library):
         p.gpu.bank_state(0)
     assert err.value.code == binding.VS_ERR_BOUNDS
     p.close()
+
+
+def test_lm_head_through_the_checked_build(checked_library):
+    """The language-model head writes only its own scratch (normalised rows, row statistics) and the caller's
+    logits: parity holds and no guard byte behind a region changes."""
+    from tests.test_gpu_parity import _lm_case, _check_lm
+    for (d, vocab, rows, norm, gain, od) in [(256, 384, 3, True, True, 1), (320, 1152, 16, False, False, 0)]:
+        got, gt, want, wt = _lm_case(d, vocab, rows, norm, gain, od)      # asserts device_status == 0 after the call
+        _check_lm(got, gt, want, wt, f"checked build, lm head d={d} vocab={vocab}")

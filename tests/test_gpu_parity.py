@@ -653,6 +653,111 @@ def test_full_decoder_block_at_the_qwen2_7b_shape():
     p.close()
 
 
+# ------------------------------------------------------------------ language-model head
+def _lm_case(d, vocab, rows, norm, gain, out_dtype, seed=11, chunk=16384, special=None):
+    """One vs_lm_head call against the oracle.  Returns (gpu logits, gpu tokens, oracle logits, oracle tokens)."""
+    from oracle import videoscan_oracle as vo
+    w = synth.workload("tiny", d_model=d, n_q_heads=d // 64, n_kv_heads=d // 64, head_dim=64, seed=seed)
+    cfg = binding.make_config(1, d, d // 64, d // 64, 64, 8, 4, 4, 2, use_rmsnorm=1 if norm else 0, out_dtype=out_dtype, vocab=vocab)
+    wl_bits = np.concatenate([synth.normal_bf16(w.seed, synth.TAG_W_LM, (min(chunk, vocab - r0), d), w.weight_std, offset=r0 * d)
+                              for r0 in range(0, vocab, chunk)])
+    h_bits = synth.normal_bf16(w.seed, synth.TAG_DECODE, (rows, d), 1.0)
+    if special is not None:
+        special(wl_bits, h_bits)
+    g_bits = synth.to_bf16_bits(1.0 + 0.1 * synth.bf16_bits_to_f64(synth.normal_bf16(w.seed, synth.TAG_NORM_F_W, (d,), 1.0))) if gain else None
+    sb = binding.StreamBatch(cfg, [to_dev(w.weight(0))], lm=(to_dev(wl_bits), to_dev(g_bits) if gain else None))
+    hid = to_dev(h_bits)
+    if out_dtype == 1:
+        hid = hid.float()
+    logits, tok = sb.lm_head(hid.contiguous())
+    torch.cuda.synchronize()
+    assert sb.bank_state(0)["device_status"] == 0
+    got = logits.double().cpu().numpy()
+    got_tok = tok.cpu().numpy()
+    h64 = synth.bf16_bits_to_f64(h_bits)
+    g64 = synth.bf16_bits_to_f64(g_bits) if gain else None
+    want = np.concatenate([vo.lm_head(h64, synth.bf16_bits_to_f64(wl_bits[r0:r0 + chunk]), g64, norm, w.rms_eps)[0]
+                           for r0 in range(0, vocab, chunk)], axis=1)
+    want_tok = np.array([vo.greedy_token(r) for r in want])
+    sb.close()
+    return got, got_tok, want, want_tok
+
+
+def _check_lm(got, got_tok, want, want_tok, what):
+    from oracle import videoscan_oracle as vo
+    from tests.parity import MAX_ABS
+    e = assert_close(got, want, what)
+    # the kernel's own choice is exact on the kernel's own logits (first of equals) ...
+    for r in range(got.shape[0]):
+        assert int(got_tok[r]) == vo.greedy_token(got[r]), f"{what}: row {r} token is not the first largest of the returned logits"
+        # ... and agrees with the oracle's unless the two candidates are closer than the logits' error bound
+        assert want[r, int(got_tok[r])] >= want[r, int(want_tok[r])] - 2 * MAX_ABS, f"{what}: row {r} token far from the oracle's maximum"
+    return e, int((got_tok == want_tok).sum())
+
+
+def test_lm_head_small_shapes():
+    """Final RMSNorm (with and without gain, and no norm), vocabulary projection, greedy token: fp32 and bf16
+    hidden rows, 1 .. 16 rows, vocabularies of one and of several 128-row tiles (K split and no K split)."""
+    for (d, vocab, rows, norm, gain, od) in [(256, 512, 3, True, True, 1), (256, 128, 1, True, False, 0),
+                                             (320, 1152, 16, False, False, 1), (512, 33024, 5, True, True, 0)]:
+        got, gt, want, wt = _lm_case(d, vocab, rows, norm, gain, od)
+        e, same = _check_lm(got, gt, want, wt, f"lm head d={d} vocab={vocab} rows={rows}")
+        print("lm head", (d, vocab, rows, norm, gain, od), "errors", e, "tokens equal to the oracle's:", same, "of", rows)
+
+
+def test_lm_head_ties_and_non_finite_logits():
+    """Two identical vocabulary rows in different tiles give equal logits: the lower index wins.  A hidden row
+    holding a NaN makes every logit of its row NaN: token 0, and the other rows are untouched."""
+    def dup(wl, h):
+        wl[300] = wl[5]
+        wl[700] = wl[5]
+        h[0] = wl[5]                                  # row 0 points along vocabulary row 5: its logit is the largest
+        h[2, 7] = np.uint16(0x7FC0)                   # NaN in row 2
+    from oracle import videoscan_oracle as vo
+    got, gt, want, wt = _lm_case(256, 1024, 4, False, False, 0, special=dup)
+    assert got[0, 5] == got[0, 300] == got[0, 700] and int(gt[0]) == 5 and int(wt[0]) == 5
+    assert np.isnan(got[2]).all() and int(gt[2]) == 0 and int(wt[2]) == 0
+    for r in (0, 1, 3):
+        assert_close(got[r:r + 1], want[r:r + 1], f"lm head row {r}")
+        assert int(gt[r]) == vo.greedy_token(got[r])
+
+
+def test_lm_head_at_the_qwen2_7b_shape():
+    """d_model 3584, vocabulary 152064 (1188 tiles of 128 rows, 1.09 GB of weights), final norm with gain:
+    four rows, and one row (the decode case)."""
+    for rows in (4, 1):
+        got, gt, want, wt = _lm_case(3584, 152064, rows, True, True, 1)
+        e, same = _check_lm(got, gt, want, wt, f"lm head, Qwen2-7B shape, {rows} rows")
+        print("lm head, Qwen2-7B shape, rows", rows, "errors", e, "tokens equal:", same)
+
+
+def test_lm_head_argument_errors():
+    w = synth.workload("tiny")
+    p = Pair(w)                                       # no head on this handle
+    x = torch.zeros((1, w.d_model), dtype=torch.float32, device="cuda")
+    lg = torch.zeros((1, 128), dtype=torch.float32, device="cuda")
+    with pytest.raises(binding.VsError) as ei:
+        binding.vs_lm_head(p.gpu.handle, x.data_ptr(), 1, lg.data_ptr(), None)
+    assert ei.value.code == binding.VS_ERR_UNSUPPORTED
+    p.close()
+    cfg = binding.make_config(1, 256, 4, 4, 64, 8, 4, 4, 2, vocab=100)
+    with pytest.raises(binding.VsError) as ei:
+        binding.vs_workspace_bytes(cfg)
+    assert ei.value.code == binding.VS_ERR_UNSUPPORTED          # vocabulary not a multiple of 128
+    cfg = binding.make_config(1, 256, 4, 4, 64, 8, 4, 4, 2, vocab=128)
+    wl = torch.zeros((128, 256), dtype=torch.bfloat16, device="cuda")
+    sb = binding.StreamBatch(cfg, [to_dev(synth.workload("tiny", d_model=256, n_q_heads=4, n_kv_heads=4, head_dim=64).weight(0))], lm=(wl, None))
+    x = torch.zeros((1, 256), dtype=torch.float32, device="cuda")
+    for rows, code in ((0, binding.VS_ERR_INVALID_ARG), (100000, binding.VS_ERR_CAPACITY)):
+        with pytest.raises(binding.VsError) as ei:
+            binding.vs_lm_head(sb.handle, x.data_ptr(), rows, lg.data_ptr(), None)
+        assert ei.value.code == code
+    with pytest.raises(binding.VsError) as ei:
+        binding.vs_lm_head(sb.handle, x.data_ptr(), 1, 0, None)
+    assert ei.value.code == binding.VS_ERR_INVALID_ARG
+    sb.close()
+
+
 # ------------------------------------------------------------------ limits and degenerate shapes
 def test_largest_frame_and_widest_group():
     """N = 255 (256-column token tile, the MMA's widest), 8 query heads per KV head (a full

@@ -33,8 +33,8 @@ def test_status_strings(lib):
 
 
 def test_struct_layout_matches_header():
-    assert C.sizeof(binding.VsConfig) == 22 * 4
-    assert C.sizeof(binding.VsWeights) == 8 * 8
+    assert C.sizeof(binding.VsConfig) == 23 * 4
+    assert C.sizeof(binding.VsWeights) == 10 * 8
     assert C.sizeof(binding.VsBankInfo) == 4 + 4 + 5 * 8 + 4 + 4 + 8 + 8
 
 
