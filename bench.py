@@ -409,6 +409,9 @@ def run_ours(args, w):
     deep = None
     if not args.no_deep and w.name == "layer":
         deep = run_deep_leg(args, dev, local, lib, binding, torch, flush, barrier, world)
+    block = None
+    if not args.no_block and w.name == "layer":
+        block = run_block_leg(dev, local, binding, torch, flush, barrier, world)
     clocks = sampler.stop()
 
     result = None
@@ -483,6 +486,8 @@ def run_ours(args, w):
         }
         if deep is not None:
             result["step_roofline_deep"] = deep_rooflines(deep, peaks)
+        if block is not None:
+            result["full_block_leg"] = block_rooflines(block, peaks)
 
     # ---- end to end: host inputs, H2D + D2H inside the timed region ---------------------------
     # Three streams, two buffers each way: the copy of frame t+1 to the device and the copy of
@@ -614,6 +619,102 @@ def run_deep_leg(args, dev, local, lib, binding, torch, flush, barrier, world):
     return out
 
 
+BLOCK_LAYERS, BLOCK_D_FF, BLOCK_VOCAB, BLOCK_FRAMES, BLOCK_DECODE = 2, 18944, 152064, 8, 16
+
+
+def run_block_leg(dev, local, binding, torch, flush, barrier, world):
+    """Full Qwen2-7B decoder layers (attention, output projection, SwiGLU MLP of width 18944, RMSNorm before each
+    half) and the language-model head (vocabulary 152064): BLOCK_LAYERS layers, a 64-token prefix and 8 untimed
+    frames, then 8 timed frames; then BLOCK_DECODE timed token steps, each one vs_decode_step + vs_lm_head of its
+    output row; then the head alone.  Weights are seeded N(0, 0.02^2) drawn on the device (2.1 GB)."""
+    wb = synth.workload("layer", n_layers=BLOCK_LAYERS, use_rmsnorm=1, residual=1, n_frames=2 * BLOCK_FRAMES,
+                        decode_tokens=BLOCK_DECODE)
+    g = torch.Generator(device=dev); g.manual_seed(1234 + local)
+    draw = lambda *shape: (torch.randn(shape, generator=g, device=dev, dtype=torch.float32) * wb.weight_std).to(torch.bfloat16)
+    d, L = wb.d_model, wb.n_layers
+    weights = [draw(wb.e_out, d) for _ in range(L)]
+    blockw = {"w_o": [draw(d, d) for _ in range(L)], "w_gate": [draw(BLOCK_D_FF, d) for _ in range(L)],
+              "w_up": [draw(BLOCK_D_FF, d) for _ in range(L)], "w_down": [draw(d, BLOCK_D_FF) for _ in range(L)], "norm2_w": None}
+    w_lm = draw(BLOCK_VOCAB, d)
+    cfg = binding.make_config(L, d, wb.n_q_heads, wb.n_kv_heads, wb.head_dim, wb.tokens_per_frame, wb.prefix_len,
+                              wb.decode_tokens, wb.bank_capacity, use_rmsnorm=1, residual=1, rope_theta=wb.rope_theta,
+                              rms_eps=wb.rms_eps, device=local, d_ff=BLOCK_D_FF, vocab=BLOCK_VOCAB)
+    sb = binding.StreamBatch(cfg, weights, block=blockw, lm=(w_lm, None))
+    to_dev = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).to(dev)
+    shared = wb.frame_shared() if wb.frame_model != "iid" else None
+    frames = to_dev(np.stack(draw_parallel(lambda t: wb.frame_hidden(t, shared=shared), wb.n_frames)))
+    prefix = to_dev(wb.prefix_hidden())
+    dec = to_dev(np.concatenate([wb.decode_hidden(i) for i in range(wb.decode_tokens)]))
+    out_f = torch.empty((1, wb.tokens_per_frame + 1, d), dtype=torch.float32, device=dev)
+    out_d = torch.empty((1, 1, d), dtype=torch.float32, device=dev)
+    logits = torch.empty((1, BLOCK_VOCAB), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def pass_(ev=None):
+        sb.reset([0])
+        sb.decode_step([0], prefix[None])
+        for t in range(BLOCK_FRAMES):
+            sb.frame_prefill([0], frames[t][None], out=out_f)
+        flush.zero_()
+        if ev: ev[0].record(stream)
+        for t in range(BLOCK_FRAMES, 2 * BLOCK_FRAMES):
+            sb.frame_prefill([0], frames[t][None], out=out_f)
+        if ev: ev[1].record(stream)
+        flush.zero_()
+        if ev: ev[2].record(stream)
+        for i in range(BLOCK_DECODE):
+            sb.decode_step([0], dec[i:i + 1][None], out=out_d)
+            sb.lm_head(out_d[0], logits=logits)
+        if ev: ev[3].record(stream)
+        flush.zero_()
+        if ev: ev[4].record(stream)
+        for i in range(4):
+            sb.lm_head(out_d[0], logits=logits)
+        if ev: ev[5].record(stream)
+        sb.end_turn([0])
+
+    pass_()
+    reps = []
+    for _ in range(3):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+        barrier()
+        pass_(ev)
+        barrier()
+        t = torch.tensor([ev[0].elapsed_time(ev[1]), ev[2].elapsed_time(ev[3]), ev[4].elapsed_time(ev[5])], dtype=torch.float64, device=dev)
+        reps.append(max_over_ranks(t, world).tolist())
+    assert sb.bank_state(0)["device_status"] == 0
+    sb.close()
+    med = lambda k: sorted(r[k] for r in reps)[len(reps) // 2]
+    return dict(w=wb, ms_frames=med(0), ms_tokens=med(1), ms_head=med(2), world=world)
+
+
+def block_rooflines(blk, peaks):
+    wb = blk["w"]
+    L, d, E, I, V, rows = wb.n_layers, wb.d_model, wb.e_out, BLOCK_D_FF, BLOCK_VOCAB, wb.tokens_per_frame + 1
+    w_layer = (E * d + d * d + 3 * I * d) * 2                                  # bytes of one layer's matrices
+    flops_frame = L * 2 * rows * (E * d + d * d + 3 * I * d)                   # attention's own flops left out (< 1 %)
+    us_frame = 1e3 * blk["ms_frames"] / BLOCK_FRAMES
+    us_tok = 1e3 * blk["ms_tokens"] / BLOCK_DECODE
+    us_head = 1e3 * blk["ms_head"] / 4
+    ideal_frame = max(flops_frame / (peaks["bf16_tflops_sustained"] * 1e12), L * w_layer / (peaks["hbm_gbs"] * 1e9)) * 1e6
+    b_tok = L * w_layer + V * d * 2 + V * 4
+    return {
+        "workload": f"{L} full Qwen2-7B decoder layers (d={d}, d_ff={I}) + language-model head (vocabulary {V}); "
+                    f"{BLOCK_FRAMES} timed frames of {wb.tokens_per_frame} tokens, then {BLOCK_DECODE} token steps "
+                    f"(vs_decode_step + vs_lm_head), then the head alone; median of 3 passes; L2 flushed before each part",
+        "frame": {"us_per_frame": us_frame, "us_per_layer": us_frame / L, "ideal_us": ideal_frame, "frac": ideal_frame / us_frame,
+                  "flops_per_frame": flops_frame, "weight_bytes_per_layer": w_layer,
+                  "note": "ideal = max(flops / sustained bf16 peak, weight bytes / HBM peak)"},
+        "token": {"us_per_token": us_tok, "tokens_per_s": blk["world"] * 1e6 / us_tok, "bytes_per_token": b_tok,
+                  "ideal_hbm_us": b_tok / (peaks["hbm_gbs"] * 1e9) * 1e6, "frac": b_tok / (peaks["hbm_gbs"] * 1e9) * 1e6 / us_tok,
+                  "achieved_gbs": b_tok / us_tok * 1e-3,
+                  "note": "a DRAM fraction: bytes = every layer's matrices + the vocabulary projection + the logits"},
+        "lm_head": {"us_per_call": us_head, "bytes_per_call": V * d * 2 + V * 4,
+                    "achieved_gbs": (V * d * 2 + V * 4) / us_head * 1e-3,
+                    "frac": (V * d * 2 + V * 4) / (peaks["hbm_gbs"] * 1e9) * 1e6 / us_head},
+    }
+
+
 def deep_rooflines(deep, peaks):
     wd = deep["w"]
     L = wd.n_layers
@@ -668,6 +769,7 @@ def main():
     ap.add_argument("--frames", type=int, default=None, help="override the number of frames (exploration only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-deep", action="store_true", help="skip the 28-layer leg")
+    ap.add_argument("--no-block", action="store_true", help="skip the full-decoder-block + language-model-head leg")
     args = ap.parse_args()
     kw = {}
     if args.frames:

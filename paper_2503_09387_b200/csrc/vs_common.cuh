@@ -113,6 +113,7 @@ struct Layout {
   size_t chunk_slot;            // int32 [VS_MAX_BATCH]  chunked prefill: slot each frame's carrier went to
   size_t chunk_victim;          // int32 [VS_MAX_BATCH]  ... and whom its bank update evicted (index on the bank axis)
   size_t gemm_flags;            // int32 [GEMM_XCHG_CTAS]  projection K split: partials delivered per slice owner
+  size_t lm_keys, lm_tickets;   // uint64 [256], int32 [256]  language-model head: greedy-choice keys and tickets per row
   size_t persistent_end;
   // per-step scratch
   size_t hbuf[2];               // bf16 [R_max][d]  residual ping-pong; hbuf[0] holds [E; carrier]
@@ -225,8 +226,10 @@ cudaError_t launch_rms_stats(const bf16* h, const bf16* gain, bf16* hg, float* r
 // sum of squares of bf16(h[row]) in part 0 of row_ss[row][parts].  h is fp32 or bf16.
 cudaError_t launch_lm_norm(const void* h, int h_fp32, const bf16* gain, bf16* xn, float* row_ss, int parts, int rows, int d,
                            cudaStream_t st);
-// token[row] = index of the largest of logits[row][0..vocab), the lowest index among equals, NaN below everything
-cudaError_t launch_argmax_rows(const float* logits, int32_t* token, int rows, int vocab, cudaStream_t st);
+// token[row] = index of the largest of logits[row][0..vocab), the lowest index among equals, NaN below everything.
+// keys[rows] and tickets[rows] are scratch that is zero between calls (the kernel leaves it so).
+cudaError_t launch_argmax_rows(const float* logits, int32_t* token, unsigned long long* keys, int* tickets, int rows, int vocab,
+                               cudaStream_t st);
 
 // What the projection epilogue writes (finished rows: bias, RoPE, bf16) and where rows persist.
 struct ProjectionOut {

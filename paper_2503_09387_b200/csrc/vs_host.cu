@@ -101,6 +101,8 @@ void fill_layout(const Dims& D, Layout& Lo) {
   Lo.chunk_slot = reg(DR_CHUNK_SLOT, take((size_t)VS_MAX_BATCH * 4));
   Lo.chunk_victim = reg(DR_CHUNK_VICTIM, take((size_t)VS_MAX_BATCH * 4));
   Lo.gemm_flags = reg(DR_GEMM_FLAGS, take((size_t)GEMM_XCHG_CTAS * 4));
+  Lo.lm_keys = take((size_t)256 * 8);          // language-model head: per-row argmax keys and tickets, zero between calls
+  Lo.lm_tickets = take((size_t)256 * 4);
   Lo.dbg_table = take(sizeof(DebugTable));
   Lo.persistent_end = off;
   Lo.scratch_begin = off;
@@ -1178,7 +1180,8 @@ int vs_lm_head(vs_stream* h, const void* hidden, int32_t rows, void* logits, int
   if (D.use_rmsnorm) { po.row_ss = ss; po.ss_parts = D.ss_parts; po.norm_eps = D.rms_eps; }
   int rc = run_linear(h, h->tm_lm, h->tm_lm, xn, rows, D.d, D.vocab, po, bp, st);
   if (rc != VS_OK) return rc;
-  if (next_token != nullptr) VS_LAUNCH(h, st, KC_OTHER, launch_argmax_rows(static_cast<const float*>(logits), next_token, rows, D.vocab, st));
+  if (next_token != nullptr) VS_LAUNCH(h, st, KC_OTHER, launch_argmax_rows(static_cast<const float*>(logits), next_token, h->at<unsigned long long>(lo.lm_keys),
+                                                                    h->at<int>(lo.lm_tickets), rows, D.vocab, st));
   return VS_OK;
 }
 

@@ -226,44 +226,63 @@ cudaError_t launch_lm_norm(const void* h, int h_fp32, const bf16* gain, bf16* xn
   return launch_pdl(lm_norm_kernel, dim3(rows), dim3(256), 0, st, h, h_fp32, gain, xn, row_ss, parts, d);
 }
 
-// Greedy choice: one block per row.  (value, index) pairs are compared as "larger value, else
-// equal value and lower index"; a NaN is never larger, so it loses to every number, and a row
-// without any number above -inf gives token 0.
-__global__ void __launch_bounds__(1024) argmax_rows_kernel(const float* __restrict__ logits, int32_t* __restrict__ token, int vocab) {
+// Greedy choice.  (value, index) pairs are compared as "larger value, else equal value and lower
+// index"; a NaN is never larger, so it loses to every number, and a row without any number above
+// -inf gives token 0.  grid = (slices, rows): every block reduces its slice of the row and offers
+// the result to the row's 64-bit key by atomicMax -- the key orders like the pair: the value's
+// bits mapped monotonically to an unsigned word on top, the complemented index below -- and the
+// block that arrives last (a ticket per row) turns the key back into the token and clears key and
+// ticket for the next call.
+__device__ __forceinline__ unsigned long long argmax_key(float v, int i) {
+  const uint32_t b = __float_as_uint(v);
+  const uint32_t ordered = (b & 0x80000000u) ? ~b : (b | 0x80000000u);     // ascending with v (no NaN gets here)
+  return ((unsigned long long)ordered << 32) | (uint32_t)(0x7fffffff - i);
+}
+
+__global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restrict__ logits, int32_t* __restrict__ token,
+                                                          unsigned long long* __restrict__ keys, int* __restrict__ tickets, int vocab) {
   pdl_wait();
   pdl_launch_dependents();
-  const float* src = logits + (size_t)blockIdx.x * vocab;
+  const int row = blockIdx.y;
+  const float* src = logits + (size_t)row * vocab;
+  const int per = (vocab + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int i0 = (int)blockIdx.x * per, i1 = min(vocab, i0 + per);
   float bv = -INFINITY;
   int bi = 0x7fffffff;
-  for (int i = threadIdx.x; i < vocab; i += 1024) {
+  for (int i = i0 + (int)threadIdx.x; i < i1; i += 256) {
     const float v = src[i];
     if (v > bv) { bv = v; bi = i; }          // ascending i per thread: the first of equals stays
   }
-  auto better = [](float v1, int i1, float v2, int i2) { return v1 > v2 || (v1 == v2 && i1 < i2); };
+  auto better = [](float v1, int i1_, float v2, int i2_) { return v1 > v2 || (v1 == v2 && i1_ < i2_); };
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
     const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
     if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
   }
-  __shared__ float sv[32];
-  __shared__ int si[32];
+  __shared__ float sv[8];
+  __shared__ int si[8];
   if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
   __syncthreads();
-  if (threadIdx.x < 32) {
-    bv = sv[threadIdx.x]; bi = si[threadIdx.x];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w)
+      if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; }
+    if (bi != 0x7fffffff) atomicMax(keys + row, argmax_key(bv, bi));      // a slice without a number offers nothing
+    __threadfence();
+    if (atomicAdd(tickets + row, 1) == (int)gridDim.x - 1) {
+      __threadfence();
+      const unsigned long long k = atomicExch(keys + row, 0ull);
+      token[row] = (k == 0ull) ? 0 : 0x7fffffff - (int)(uint32_t)(k & 0xffffffffull);
+      tickets[row] = 0;
     }
-    if (threadIdx.x == 0) token[blockIdx.x] = (bi == 0x7fffffff) ? 0 : bi;
   }
 }
 
-cudaError_t launch_argmax_rows(const float* logits, int32_t* token, int rows, int vocab, cudaStream_t st) {
-  return launch_pdl(argmax_rows_kernel, dim3(rows), dim3(1024), 0, st, logits, token, vocab);
+cudaError_t launch_argmax_rows(const float* logits, int32_t* token, unsigned long long* keys, int* tickets, int rows, int vocab,
+                               cudaStream_t st) {
+  int slices = (vocab + 4095) / 4096;
+  if (slices > 64) slices = 64;
+  return launch_pdl(argmax_rows_kernel, dim3(slices, rows), dim3(256), 0, st, logits, token, keys, tickets, vocab);
 }
 
 // The bank update of one frame as a launch of its own (chunked prefill).
