@@ -6,10 +6,10 @@
 // row and reads it with 128-bit loads; every lane issues the K and V loads of eight keys before
 // it uses any of them, so a warp has 16 key rows (8 KB) in flight.  Warps merge their running
 // (m, l, o) by shuffles and through shared memory.  The key splits of one (stream, query head)
-// form a thread-block cluster (1, 2, 4 or 8 CTAs): every CTA leaves its partial triple in its own
-// shared memory, the cluster's hardware barrier orders them, and rank 0 reads the peers' triples
-// through distributed shared memory and writes the row -- no global scratch, no atomics, no
-// polling; the co-scheduled cluster is what guarantees that the barrier completes.
+// form a thread-block cluster (1, 2, 4 or 8 CTAs): every CTA writes its partial triple into rank 0's
+// shared memory (distributed shared memory) and arrives at the cluster's hardware barrier; rank 0
+// alone waits there, combines and writes the row -- no global scratch, no atomics, no polling; the
+// co-scheduled cluster is what guarantees that the barrier completes.
 #include "vs_common.cuh"
 
 namespace vs {
@@ -29,11 +29,12 @@ __device__ __forceinline__ uint32_t map_shared_rank(uint32_t addr, uint32_t rank
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
   return r;
 }
-__device__ __forceinline__ float ld_shared_cluster_f32(uint32_t addr) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
-  return v;
+__device__ __forceinline__ void st_shared_cluster_f32(uint32_t addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
 // One CTA = one query head x one key split x one stream.  The heads of a KV group read the
 // same K/V rows from L2; spreading them over CTAs keeps every SM's instruction stream short,
@@ -45,8 +46,8 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
   __shared__ float st_m[kDecWarps];
   __shared__ float st_l[kDecWarps];
   __shared__ float st_o[kDecWarps][D];
-  __shared__ float cta_o[D];            // this CTA's partial triple, read by rank 0 of the cluster
-  __shared__ float cta_ml[2];
+  __shared__ float peer_o[kMaxCluster][D];     // rank 0 only: the partial triples its peers (and itself) leave here
+  __shared__ float peer_ml[kMaxCluster][2];
 
   // what follows from the parameters alone comes before the wait on the stream's earlier kernels
   const int split = blockIdx.x, qh = blockIdx.y, b = blockIdx.z;
@@ -56,6 +57,9 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
   const int sub = lane / LPK, li = lane % LPK;
   const int count = bp.count[b];
   const bool bank_full = (a.M > 0 && count == a.M);
+  // first phase of the cluster's barrier: "this CTA runs", so that nobody writes into the shared memory of a
+  // CTA that has not started; everyone arrives here and waits only just before its one remote write
+  if (a.nsplit > 1) cluster_arrive_relaxed();
 
   int P, NB, TL;
   if (a.to_prefix) { P = bp.prefix_len[b] + 1; NB = 0; TL = 0; }
@@ -202,6 +206,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
   // the residual input is needed by whoever writes the row: fetched ahead of the cluster barrier
   float h_res = 0.f;
   if (a.h_out != nullptr && split == 0 && threadIdx.x < D) h_res = __bfloat162float(a.h_in[out_off + threadIdx.x]);
+  float M_cta = -INFINITY, L_cta = 0.f, O_cta = 0.f;      // this CTA's partial triple (threads below D)
   if (threadIdx.x < D) {
     const int c = threadIdx.x;
     float M = -INFINITY;
@@ -220,38 +225,41 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
       else static_cast<bf16*>(a.out)[out_off + c] = __float2bfloat16_rn(val);
       if (a.h_out != nullptr && VS_STORE_OK(bp, a.h_out_region, a.h_out + out_off + c, 2)) a.h_out[out_off + c] = __float2bfloat16_rn(h_res + val);
     } else {
-      cta_o[c] = O;
-      if (c == 0) { cta_ml[0] = M; cta_ml[1] = L; }
+      M_cta = M; L_cta = L; O_cta = O;
     }
   }
   if (direct) { VS_STAMP(bp, 5, 15); return; }
 
-  // the cluster's CTAs (the key splits of this stream and query head) meet; rank 0 combines
-  cluster_sync();
-  if (split == 0 && threadIdx.x < D) {
+  // Every CTA of the cluster (the key splits of this stream and query head) leaves its partial triple in rank 0's
+  // shared memory and arrives at the cluster's barrier; only rank 0 waits there, then combines what it was given.
+  // The other CTAs are done: nothing of theirs is read after they exit.
+  VS_STAMP(bp, 5, 4);
+  cluster_wait_acquire();                           // phase 1 (every CTA of the cluster has started) -- long since complete
+  if (threadIdx.x < D) {
     const int c = threadIdx.x;
-    const uint32_t ml_addr = static_cast<uint32_t>(__cvta_generic_to_shared(cta_ml));
-    const uint32_t o_addr = static_cast<uint32_t>(__cvta_generic_to_shared(cta_o + c));
-    float ms[kMaxCluster], ls[kMaxCluster], os[kMaxCluster];
-#pragma unroll
-    for (int r = 0; r < kMaxCluster; ++r) {
-      if (r < a.nsplit) {
-        const uint32_t rml = map_shared_rank(ml_addr, (uint32_t)r);
-        ms[r] = ld_shared_cluster_f32(rml);
-        ls[r] = ld_shared_cluster_f32(rml + 4);
-        os[r] = ld_shared_cluster_f32(map_shared_rank(o_addr, (uint32_t)r));
-      }
+    st_shared_cluster_f32(map_shared_rank(static_cast<uint32_t>(__cvta_generic_to_shared(&peer_o[split][c])), 0u), O_cta);
+    if (c == 0) {
+      const uint32_t ml = map_shared_rank(static_cast<uint32_t>(__cvta_generic_to_shared(&peer_ml[split][0])), 0u);
+      st_shared_cluster_f32(ml, M_cta);
+      st_shared_cluster_f32(ml + 4, L_cta);
     }
+  }
+  cluster_arrive_release();                         // phase 2: "my triple is in place"
+  if (split != 0) { VS_STAMP(bp, 5, 15); return; }
+  cluster_wait_acquire();
+  VS_STAMP(bp, 5, 5);
+  if (threadIdx.x < D) {
+    const int c = threadIdx.x;
     float M = -INFINITY;
 #pragma unroll
-    for (int r = 0; r < kMaxCluster; ++r) if (r < a.nsplit) M = fmaxf(M, ms[r]);
+    for (int r = 0; r < kMaxCluster; ++r) if (r < a.nsplit) M = fmaxf(M, peer_ml[r][0]);
     float L = 0.f, val = 0.f;
 #pragma unroll
     for (int r = 0; r < kMaxCluster; ++r) {
       if (r < a.nsplit) {
-        const float wt = (ms[r] == -INFINITY) ? 0.f : exp2f(ms[r] - M);
-        L = fmaf(ls[r], wt, L);
-        val = fmaf(os[r], wt, val);
+        const float wt = (peer_ml[r][0] == -INFINITY) ? 0.f : exp2f(peer_ml[r][0] - M);
+        L = fmaf(peer_ml[r][1], wt, L);
+        val = fmaf(peer_o[r][c], wt, val);
       }
     }
     val = (L > 0.f) ? val / L : 0.f;
@@ -259,8 +267,6 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_attn_kernel(DecodeArgs 
     else static_cast<bf16*>(a.out)[out_off + c] = __float2bfloat16_rn(val);
     if (a.h_out != nullptr && VS_STORE_OK(bp, a.h_out_region, a.h_out + out_off + c, 2)) a.h_out[out_off + c] = __float2bfloat16_rn(h_res + val);
   }
-  // nobody's shared memory goes away while rank 0 may still be reading it
-  cluster_sync();
   VS_STAMP(bp, 5, 15);
 }
 
