@@ -3,8 +3,11 @@
 // product bound by reading W once, not a tensor-core contraction.  Every CTA owns 32 rows of
 // W ([E_out, d] bf16, row-major) and streams them through a ring of shared-memory stages filled
 // by 16-byte asynchronous copies (a stage = 256 elements of all 32 rows, 16 KiB; eight stages,
-// so up to 112 KiB per SM are in flight whatever the registers hold); each warp then reads four
-// rows back, a lane one 16-byte column of them, fp32 accumulation, a shuffle reduction per row.
+// so up to 112 KiB per SM are in flight whatever the registers hold).  The products are formed by
+// the warp-level tensor-core instruction (mma.sync m16n8k16, bf16 x bf16 -> fp32) with the token rows
+// as its 8-column operand: not for its arithmetic rate but for its instruction count -- unpacking
+// bf16 pairs and multiply-adding them one by one on the CUDA cores cost some 95 instructions per warp
+// and stage and made the loop issue-bound; this way it is ten.
 //
 // A CTA's 32 rows are 16 rotation pairs (k, k + D/2) of one head, so the epilogue has both
 // elements of a pair at hand: RMSNorm row scale, bias, RoPE (the angle in fp64 from the token's
@@ -31,13 +34,6 @@ constexpr int kStages = 8;
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
-__device__ __forceinline__ float dot8(const uint4& w, const uint4& x, float acc) {
-  acc = fmaf(bf_lo(w.x), bf_lo(x.x), acc); acc = fmaf(bf_hi(w.x), bf_hi(x.x), acc);
-  acc = fmaf(bf_lo(w.y), bf_lo(x.y), acc); acc = fmaf(bf_hi(w.y), bf_hi(x.y), acc);
-  acc = fmaf(bf_lo(w.z), bf_lo(x.z), acc); acc = fmaf(bf_hi(w.z), bf_hi(x.z), acc);
-  acc = fmaf(bf_lo(w.w), bf_lo(x.w), acc); acc = fmaf(bf_hi(w.w), bf_hi(x.w), acc);
-  return acc;
-}
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
@@ -49,10 +45,10 @@ template <int R>   // token rows held (1, 2 or 4)
 __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __restrict__ W, const bf16* __restrict__ x,
                                                             ProjectionOut o, BatchParams bp, int rows, int d, int l2_ahead) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  // carve: ring [kStages][32 rows][512 B] | token rows [R][d] bf16 | results [R][32] | row scales [R] | partial sums [R][8]
+  // carve: ring [kStages][32 rows][512 B] | token rows [R][d] bf16 | partial results [4][R][32] | row scales [R] | partial sums [R][8]
   uint4* xs = reinterpret_cast<uint4*>(smem_raw + kStages * kStageBytes);
-  float* ys = reinterpret_cast<float*>(smem_raw + kStages * kStageBytes + (size_t)R * d * 2);
-  float* rs = ys + R * kRowsPerCta;
+  float* ysp = reinterpret_cast<float*>(smem_raw + kStages * kStageBytes + (size_t)R * d * 2);   // [4 K quarters][R][32]
+  float* rs = ysp + 4 * R * kRowsPerCta;
   float* red = rs + R;
   const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw));
 
@@ -75,7 +71,9 @@ __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __res
     const int lr = idx >> 5, c = idx & 31;
     const int f = hs * D + pb * 16 + (lr & 15) + (lr >> 4) * half;
     csrc[q] = W + (size_t)f * d + c * 8;
-    cdst[q] = (uint32_t)(lr * (kStageElems * 2) + c * 16);
+    // rows 2j and 2j + 1 are read side by side by a quarter warp: bit 2 of the chunk index is flipped in odd
+    // rows so that the two rows' 64-byte pieces fall into different banks
+    cdst[q] = (uint32_t)(lr * (kStageElems * 2) + ((c ^ ((lr & 1) << 2)) * 16));
   }
   auto issue_stage = [&](int i) {
     if (i < n_stage_total) {
@@ -162,41 +160,61 @@ __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __res
     rs[tid] = rsqrtf(tot / (float)d + o.norm_eps);
   }
 
-  float acc[4][R];
-#pragma unroll
-  for (int rr = 0; rr < 4; ++rr)
-#pragma unroll
-    for (int r = 0; r < R; ++r) acc[rr][r] = 0.f;
+  // Warp w owns the 16-row tile w & 1 (first or second elements of the CTA's rotation pairs) and the two 32-element
+  // K blocks 2 * (w >> 1), + 1 of every stage.  Inside a block, lane (g, t) = (lane / 4, lane % 4) reads the 16 bytes
+  // k = 8t .. 8t + 7 of weight rows g and g + 8 and of token row g: the first 8 bytes feed one MMA, the last 8 the
+  // next -- a permutation of K that the weights and the tokens share, which a dot product does not see.
+  const int mt = warp & 1, kg = warp >> 1;
+  const int g = lane >> 2, t4 = lane & 3;
+  const uint32_t ring_u = ring;
+  const uint32_t a_row0 = (uint32_t)((mt * 16 + g) * (kStageElems * 2)), a_row1 = a_row0 + 8u * (kStageElems * 2);
+  const uint32_t sw0 = (uint32_t)(((mt * 16 + g) & 1) << 2);                // rows g and g + 8 have the same parity
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
   for (int i = 0; i < n_stage_total; ++i) {
     cp_async_wait<kStages - 2>();   // this thread's copies of stage i have landed
     __syncthreads();                // everyone's have, and everyone is done with stage i - 1
     issue_stage(i + kStages - 1);   // into the slot stage i - 1 occupied
-    const uint4* slot = reinterpret_cast<const uint4*>(smem_raw + (size_t)(i % kStages) * kStageBytes);
-    uint4 xv[R];
+    const uint32_t slot = ring_u + (uint32_t)(i % kStages) * kStageBytes;
 #pragma unroll
-    for (int r = 0; r < R; ++r) xv[r] = xs[r * chunks_per_row + i * 32 + lane];
-#pragma unroll
-    for (int rr = 0; rr < 4; ++rr) {
-      const uint4 wv = slot[(warp * 4 + rr) * 32 + lane];
-#pragma unroll
-      for (int r = 0; r < R; ++r) acc[rr][r] = dot8(wv, xv[r], acc[rr][r]);
+    for (int kb2 = 0; kb2 < 2; ++kb2) {
+      const int kb = kg * 2 + kb2;                                          // 32-element block inside the stage
+      const uint32_t chunk = (uint32_t)(kb * 4 + t4);
+      uint32_t a0[4], a1[4];
+      asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(a0[0]), "=r"(a0[1]), "=r"(a0[2]), "=r"(a0[3])
+                   : "r"(slot + a_row0 + ((chunk ^ sw0) << 4)));
+      asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(a1[0]), "=r"(a1[1]), "=r"(a1[2]), "=r"(a1[3])
+                   : "r"(slot + a_row1 + ((chunk ^ sw0) << 4)));
+      uint4 xv = make_uint4(0u, 0u, 0u, 0u);
+      if (g < R) xv = xs[g * chunks_per_row + i * 32 + (int)chunk];
+      asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                   : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3])
+                   : "r"(a0[0]), "r"(a1[0]), "r"(a0[1]), "r"(a1[1]), "r"(xv.x), "r"(xv.y));
+      asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                   : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3])
+                   : "r"(a0[2]), "r"(a1[2]), "r"(a0[3]), "r"(a1[3]), "r"(xv.z), "r"(xv.w));
     }
   }
   cp_async_wait<0>();
+  // accumulator: acc[0], acc[1] = (row g, tokens 2t, 2t + 1), acc[2], acc[3] = (row g + 8, same tokens);
+  // the four warps that share a row tile leave their parts side by side, the finishing threads add them
 #pragma unroll
-  for (int rr = 0; rr < 4; ++rr)
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      float v = acc[rr][r];
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-      if (lane == 0) ys[r * kRowsPerCta + warp * 4 + rr] = v;
+  for (int j = 0; j < 2; ++j) {
+    const int tok = 2 * t4 + j;
+    if (tok < R) {
+      ysp[(kg * R + tok) * kRowsPerCta + mt * 16 + g] = acc[j];
+      ysp[(kg * R + tok) * kRowsPerCta + mt * 16 + g + 8] = acc[2 + j];
     }
+  }
   __syncthreads();
 
   if (finisher) {
     const int row = fr;
-    float x1 = ys[row * kRowsPerCta + fp], x2 = ys[row * kRowsPerCta + 16 + fp];
+    float x1 = 0.f, x2 = 0.f;
+#pragma unroll
+    for (int k4 = 0; k4 < 4; ++k4) {                       // the K quarters of the stage, in a fixed order
+      x1 += ysp[(k4 * R + row) * kRowsPerCta + fp];
+      x2 += ysp[(k4 * R + row) * kRowsPerCta + 16 + fp];
+    }
     const int f1 = hs * D + k0, f2 = f1 + half;
     // RMSNorm's row scale commutes with the projection
     float rsc = 1.f;
@@ -242,7 +260,7 @@ __global__ void __launch_bounds__(kThreads, 2) qkv_gemv_kernel(const bf16* __res
 }  // namespace
 
 static size_t gemv_smem_bytes(int R, int d) {
-  return (size_t)kStages * kStageBytes + (size_t)R * d * 2 + (size_t)R * kRowsPerCta * 4 + (size_t)R * 4 + (size_t)R * 8 * 4;
+  return (size_t)kStages * kStageBytes + (size_t)R * d * 2 + (size_t)4 * R * kRowsPerCta * 4 + (size_t)R * 4 + (size_t)R * 8 * 4;
 }
 
 bool qkv_gemv_supported(const ProjectionOut& o, int rows, int d) {
