@@ -500,8 +500,6 @@ class OracleStream:
         used and nothing changes.  Carrier i of this compact sequence sits at position
         prefix_len + i.  Returns the last layer's outputs [count, Hq*D]."""
         cfg = self.cfg
-        if self.blocks is not None:
-            raise NotImplementedError("carriers-only forward is defined for the attention sub-block")
         T = len(self.bank)
         if T == 0:
             return np.zeros((0, cfg.n_q_heads * cfg.head_dim))
@@ -519,7 +517,10 @@ class OracleStream:
             vis = np.ones((T, P + T), dtype=bool)
             vis[:, P:] = np.tril(np.ones((T, T), dtype=bool))
             out = attention_rows(Q, Kall, Vall, vis).reshape(T, -1)
-            if cfg.residual:
+            if self.blocks is not None:
+                h = self._rest_of_block(h, out, l)          # full decoder layer: the result is its hidden state
+                out = h
+            elif cfg.residual:
                 h = round_to_bf16(h + out)
         return out
 

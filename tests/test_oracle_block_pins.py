@@ -184,3 +184,26 @@ def test_lm_head_rounds_the_hidden_state_on_entry():
     a, _ = vo.lm_head(h, W, None, True)
     b, _ = vo.lm_head(h * (1 + 2.0 ** -12), W, None, True)
     np.testing.assert_array_equal(a, b)
+
+
+def test_carriers_only_forward_with_the_block_is_a_text_prefill_of_the_stored_embeddings():
+    """With the full decoder block too, feeding the bank's embeddings as text right after the same prompt on a
+    stream that has seen no frame is the same computation (positions prefix_len + i, causal context), and the
+    call changes nothing of the stream."""
+    rng, cfg, Ws, gains, blocks = _setup(seed=8, L=2)
+    st, _ = _run(cfg, Ws, gains, blocks, frames=5)
+    st.end_turn()
+    before = (st.next_pos, st.frames_seen, st.evictions, [e.frame_id for e in st.bank])
+    got = st.carriers_only_forward()
+    assert (st.next_pos, st.frames_seen, st.evictions, [e.frame_id for e in st.bank]) == before
+    assert got.shape == (2, cfg.d_model)
+    ref = vo.OracleStream(cfg, Ws, None, gains, blocks)
+    r2 = np.random.default_rng(1)
+    ref.text_step(_bf(r2.normal(size=(3, cfg.d_model))))          # the same prompt _run feeds (seed 1, 3 rows)
+    want = ref.text_step(np.stack([e.emb for e in st.bank]))
+    assert np.max(np.abs(got - want)) < 1e-12
+    # and it is not the attention-only result: the block is really applied
+    plain = vo.OracleStream(cfg, Ws, None, gains, None)
+    r3 = np.random.default_rng(1)
+    plain.text_step(_bf(r3.normal(size=(3, cfg.d_model))))
+    assert np.max(np.abs(plain.text_step(np.stack([e.emb for e in st.bank])) - got)) > 1e-3
