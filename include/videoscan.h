@@ -172,8 +172,7 @@ int vs_frame_prefill(vs_stream* h, const int32_t* stream_ids, int32_t n_active,
  * back into `cuda_stream` by events, so that they run beside the projection; the handle's first
  * call of this function creates that stream and its two events (no device memory).
  * Errors: as vs_frame_prefill; VS_ERR_CAPACITY also if F > max_chunk_frames or if
- *         bank_capacity + 1 + F > 8192; VS_ERR_UNSUPPORTED on a handle with d_ff > 0 (the rest of
- *         the decoder block runs in the one-frame and text steps only). */
+ *         bank_capacity + 1 + F > 8192. */
 int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, int32_t F, int32_t N,
                            void* out, void* cuda_stream);
 
@@ -183,7 +182,7 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
  * positions prefix_len + i, go through the layers, each attending over the prompt prefix and the
  * carriers up to itself.  Reads the bank, changes nothing.
  * out: DEVICE [count][Hq*D] of `out_dtype` (count = carriers in the bank; vs_bank_state tells).
- * count = 0 is not an error: nothing is launched.  VS_ERR_UNSUPPORTED on a handle with d_ff > 0. */
+ * count = 0 is not an error: nothing is launched. */
 int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_stream);
 
 /* T text tokens per listed stream -- the decoding phase of Section 3.3 (T = 1) and the

@@ -342,6 +342,7 @@ class OracleStream:
         blk = self.blocks[layer]
         A = round_to_bf16(O)                                   # the attention rows are a stored tensor
         h1 = round_to_bf16(h + A @ np.asarray(blk.w_o, dtype=np.float64).T)
+        self.last_h1 = h1                                      # kept for inspection (the other stored tensor of the residual path)
         n = h1
         if self.cfg.use_rmsnorm:
             ms = np.mean(h1 * h1, axis=1, keepdims=True)
@@ -411,6 +412,7 @@ class OracleStream:
                 elif cfg.residual:
                     h = round_to_bf16(h + O)
                 rec.setdefault("h_out", []).append(h)
+                rec.setdefault("h1", []).append(getattr(self, "last_h1", None))
             if self.record is not None:
                 self.record.append(rec)
         elif mode == "carrier":
@@ -484,6 +486,7 @@ class OracleStream:
             elif cfg.residual:
                 h = round_to_bf16(h + O)
             rec.setdefault("h_out", []).append(h)
+            rec.setdefault("h1", []).append(getattr(self, "last_h1", None))
         if self.record is not None:
             self.record.append(rec)
         if to_prefix:

@@ -666,7 +666,6 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
   const Dims& D = h->dm;
   const Layout& lo = h->lo;
   if (N > D.maxN || F > D.maxChunk) return VS_ERR_CAPACITY;
-  if (D.d_ff > 0) return VS_ERR_UNSUPPORTED;       // the full decoder block is built for streaming and text steps
   HostStream& hs = h->hs[stream_id];
   if (hs.text_len != 0) return VS_ERR_STATE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -829,6 +828,11 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
       aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
     aa.h_out_region = (cur ^ 1) ? DR_HBUF1 : DR_HBUF0;
     if (D.use_rmsnorm && l + 1 < D.L) { aa.ss_out = h->at<float>(lo.row_ss); aa.next_gain = h->gain[l + 1]; aa.xn_out = h->at<bf16>(lo.xn); }
+      if (D.d_ff > 0) {
+        // full decoder block: the attention rows (bf16) feed the output projection; the residual comes there
+        aa.out = h->at<void>(lo.obuf); aa.out_fp32 = 0;
+        aa.h_in = nullptr; aa.h_out = nullptr; aa.ss_out = nullptr; aa.next_gain = nullptr; aa.xn_out = nullptr;
+      }
       aa.free_slot = chunk_slot; aa.free_slot_stride = 0;
       aa.chunk_mode = 1; aa.chunk_count0 = count0; aa.chunk_victim = chunk_victim;
       {
@@ -846,7 +850,11 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
         VS_LAUNCH(h, st, KC_OTHER, launch_chunk_kv_commit(ca, st));
       }
     }
-    if (D.residual) cur ^= 1;
+    if (D.d_ff > 0) {
+      // h2 lands in hbuf[0] again: the layer input of every layer is hbuf[0]
+      rc = run_block_rest(h, l, rows, h_in, h->at<bf16>(lo.obuf), (last && out != nullptr) ? out : nullptr, bp, st);
+      if (rc != VS_OK) return rc;
+    } else if (D.residual) cur ^= 1;
   }
 
   hs.next_pos += (int64_t)F * (N + 1);
@@ -861,7 +869,7 @@ int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_strea
   if (rc != VS_OK) return rc;
   const Dims& D = h->dm;
   const Layout& lo = h->lo;
-  if ((D.d & 7) != 0 || D.d_ff > 0) return VS_ERR_UNSUPPORTED;
+  if ((D.d & 7) != 0) return VS_ERR_UNSUPPORTED;
   const HostStream& hs = h->hs[stream_id];
   const int count = (int)(hs.frames_seen < D.M ? hs.frames_seen : D.M);
   if (count == 0) return VS_OK;
@@ -920,6 +928,10 @@ int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_strea
     aa.h_out = D.residual ? h->at<bf16>(lo.hbuf[cur ^ 1]) : nullptr;
     aa.h_out_region = (cur ^ 1) ? DR_HBUF1 : DR_HBUF0;
     if (D.use_rmsnorm && l + 1 < D.L) { aa.ss_out = h->at<float>(lo.row_ss); aa.next_gain = h->gain[l + 1]; aa.xn_out = h->at<bf16>(lo.xn); }
+    if (D.d_ff > 0) {
+      aa.out = h->at<void>(lo.obuf); aa.out_fp32 = 0;
+      aa.h_in = nullptr; aa.h_out = nullptr; aa.ss_out = nullptr; aa.next_gain = nullptr; aa.xn_out = nullptr;
+    }
     aa.free_slot = h->at<int32_t>(lo.step_slot); aa.free_slot_stride = 0;
     aa.Hq = D.Hq; aa.Hkv = D.Hkv; aa.D = D.D; aa.slots = D.slots; aa.M = 0;      // no bank segment on this key axis
     {
@@ -928,7 +940,10 @@ int vs_bank_forward(vs_stream* h, int32_t stream_id, void* out, void* cuda_strea
     }
     aa.scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)D.D));
     VS_LAUNCH(h, st, KC_PREFILL_ATTN, launch_prefill_attention_tc(aa, bp, h->at<int>(lo.status), st));
-    if (D.residual) cur ^= 1;
+    if (D.d_ff > 0) {
+      rc = run_block_rest(h, l, rows, h_in, h->at<bf16>(lo.obuf), (l == D.L - 1) ? out : nullptr, bp, st);
+      if (rc != VS_OK) return rc;
+    } else if (D.residual) cur ^= 1;
   }
   h->last_stream = st;
   h->last_rows = rows;

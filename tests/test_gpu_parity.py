@@ -423,7 +423,7 @@ class TeacherForced:
             else:
                 got = to_f64(sb.frame_prefill([0], to_dev(h[None, :-1]), carrier_override=to_dev(h[None, -1])))[0]
             if self.d_ff:      # the layer's output is its hidden state, a stored (bf16) tensor
-                e = assert_close_stored(got, rec["h_out"][layer], f"teacher-forced layer {layer}, {what}",
+                e = assert_close_stored(got, rec["h_out"][layer], f"teacher-forced layer {layer}, {what}", rec["h1"][layer],
                                         float(np.sqrt(1.0 + self.d_ff / self.w.d_model)))
             else:
                 e = assert_close(got, rec["O"][layer], f"teacher-forced layer {layer}, {what}")
@@ -628,6 +628,39 @@ def test_full_decoder_block_small():
         p.text(ids, [w.decode_hidden(i, s) for s in ids], f"decode {i}")
     for s in ids:
         p.check_bank(s)
+    p.close()
+
+
+def test_full_decoder_block_in_chunks_and_carriers_only_forward():
+    """The full decoder block through the other two entry points: several frames per call (equal to streaming
+    steps, evictions inside the chunk included) and the carriers-only forward of the bank's embeddings."""
+    w = synth.workload("deep", n_layers=2, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64, tokens_per_frame=21,
+                       n_frames=9, bank_capacity=3, prefix_len=6, question_len=5, decode_tokens=2)
+    p = Pair(w, with_gain=True, d_ff=320, max_chunk_frames=4)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    p.frame([0], [w.frame_hidden(0)], "frame 0")
+    p.frame_chunk(0, [w.frame_hidden(1 + j) for j in range(4)], "chunk of 4")
+    p.check_bank(0, layer=1)
+    p.bank_forward(0)
+    p.frame([0], [w.frame_hidden(5)], "frame 5")
+    p.frame_chunk(0, [w.frame_hidden(6 + j) for j in range(3)], "chunk of 3")
+    for layer in range(2):
+        p.check_bank(0, layer=layer)
+    p.bank_forward(0)
+    p.text([0], [w.question_hidden()], "question")
+    for i in range(w.decode_tokens):
+        p.text([0], [w.decode_hidden(i)], f"decode {i}")
+    p.check_bank(0)
+    print("full block, chunks and carriers-only forward: worst", p.worst)
+    p.close()
+    # one layer at the Qwen2-7B width with a small MLP: a 680-row chunk (three token tiles per GEMM)
+    w = synth.workload("deep", n_layers=1, n_frames=4, bank_capacity=2, prefix_len=16, question_len=0, decode_tokens=1)
+    p = Pair(w, d_ff=1024, max_chunk_frames=4, max_text=2)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    p.frame_chunk(0, [w.frame_hidden(j) for j in range(4)], "chunk of 4 at the Qwen width")
+    p.check_bank(0)
+    p.bank_forward(0)
+    p.text([0], [w.decode_hidden(0)], "decode")
     p.close()
 
 
