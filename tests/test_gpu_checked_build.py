@@ -107,3 +107,24 @@ def test_lm_head_through_the_checked_build(checked_library):
     for (d, vocab, rows, norm, gain, od) in [(256, 384, 3, True, True, 1), (320, 1152, 16, False, False, 0)]:
         got, gt, want, wt = _lm_case(d, vocab, rows, norm, gain, od)      # asserts device_status == 0 after the call
         _check_lm(got, gt, want, wt, f"checked build, lm head d={d} vocab={vocab}")
+
+
+def test_block_in_chunks_and_carriers_only_forward_through_the_checked_build(checked_library):
+    """The full decoder block inside a chunk of frames and inside the carriers-only forward: the GEMMs of the block
+    run on F * (N + 1) rows (several token tiles) and write the activation, both residual buffers and the gained
+    copies; no store may leave its region and no guard byte may change."""
+    w = synth.workload("deep", n_layers=2, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64, tokens_per_frame=33,
+                       n_frames=7, bank_capacity=3, prefix_len=6, question_len=5, decode_tokens=2)
+    p = Pair(w, with_gain=True, d_ff=320, max_chunk_frames=3)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    p.frame([0], [w.frame_hidden(0)], "frame 0")
+    p.frame_chunk(0, [w.frame_hidden(1 + j) for j in range(3)], "chunk of 3")
+    assert p.check_bank(0, layer=1)["device_status"] == 0
+    p.bank_forward(0)
+    p.frame_chunk(0, [w.frame_hidden(4 + j) for j in range(3)], "second chunk of 3")
+    p.bank_forward(0)
+    p.text([0], [w.question_hidden()], "question")
+    for i in range(w.decode_tokens):
+        p.text([0], [w.decode_hidden(i)], f"decode {i}")
+    assert p.check_bank(0)["device_status"] == 0
+    p.close()

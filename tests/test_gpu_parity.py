@@ -730,9 +730,10 @@ def _check_lm(got, got_tok, want, want_tok, what):
 
 def test_lm_head_small_shapes():
     """Final RMSNorm (with and without gain, and no norm), vocabulary projection, greedy token: fp32 and bf16
-    hidden rows, 1 .. 16 rows, vocabularies of one and of several 128-row tiles (K split and no K split)."""
+    hidden rows, 1 .. 64 rows (the handle's largest step), vocabularies of one and of several 128-row tiles (K split and no K split)."""
     for (d, vocab, rows, norm, gain, od) in [(256, 512, 3, True, True, 1), (256, 128, 1, True, False, 0),
-                                             (320, 1152, 16, False, False, 1), (512, 33024, 5, True, True, 0)]:
+                                             (320, 1152, 16, False, False, 1), (512, 33024, 5, True, True, 0),
+                                             (256, 640, 64, True, True, 1)]:
         got, gt, want, wt = _lm_case(d, vocab, rows, norm, gain, od)
         e, same = _check_lm(got, gt, want, wt, f"lm head d={d} vocab={vocab} rows={rows}")
         print("lm head", (d, vocab, rows, norm, gain, od), "errors", e, "tokens equal to the oracle's:", same, "of", rows)
