@@ -99,7 +99,7 @@ class Pair:
     def __init__(self, w: synth.Workload, n_streams: Optional[int] = None, max_step_tokens: int = 64,
                  evict_policy: int = 0, agg_mode: int = 0, with_bias: bool = False, with_gain: bool = False,
                  max_tokens_per_frame: Optional[int] = None, max_prefix: Optional[int] = None,
-                 max_text: Optional[int] = None, out_dtype: int = 1, max_chunk_frames: int = 1, d_ff: int = 0):
+                 max_text: Optional[int] = None, out_dtype: int = 1, max_chunk_frames: int = 1, d_ff: int = 0, vocab: int = 0):
         self.w = w
         S = n_streams or w.n_streams
         self.S = S
@@ -116,7 +116,8 @@ class Pair:
             max_text if max_text is not None else max(w.question_len + w.decode_tokens, 1),
             w.bank_capacity, n_streams=S, max_step_tokens=max_step_tokens, agg_mode=agg_mode,
             evict_policy=evict_policy, use_rmsnorm=w.use_rmsnorm, residual=w.residual,
-            rope_theta=w.rope_theta, rms_eps=w.rms_eps, out_dtype=out_dtype, max_chunk_frames=max_chunk_frames, d_ff=d_ff)
+            rope_theta=w.rope_theta, rms_eps=w.rms_eps, out_dtype=out_dtype, max_chunk_frames=max_chunk_frames, d_ff=d_ff,
+            vocab=vocab)
         # the rest of the decoder block (output projection, SwiGLU MLP), with a gain for its norm when gains are on
         blk = [w.block_weights(l, d_ff) for l in range(w.n_layers)] if d_ff else None
         g2 = [synth.to_bf16_bits(1.0 + 0.1 * synth.standard_normal(w.seed, synth.TAG_NORM2_W, w.d_model, offset=l * w.d_model))
@@ -125,9 +126,17 @@ class Pair:
         if blk:
             dev_block = {k: [to_dev(b[k]) for b in blk] for k in ("w_o", "w_gate", "w_up", "w_down")}
             dev_block["norm2_w"] = [to_dev(g) for g in g2] if g2 else None
+        # language-model head: vocabulary projection and the gain of the final norm
+        lm = None
+        if vocab:
+            lm_w = w.lm_weights(vocab)
+            lm_g = synth.to_bf16_bits(1.0 + 0.1 * synth.standard_normal(w.seed, synth.TAG_NORM_F_W, w.d_model)) if with_gain else None
+            self.lm_w64 = synth.bf16_bits_to_f64(lm_w)
+            self.lm_g64 = synth.bf16_bits_to_f64(lm_g) if lm_g is not None else None
+            lm = (to_dev(lm_w), to_dev(lm_g) if lm_g is not None else None)
         self.gpu = binding.StreamBatch(self.cfg, [to_dev(b) for b in wbits],
                                        [to_dev(b) for b in bbits] if bbits else None,
-                                       [to_dev(b) for b in gbits] if gbits else None, dev_block)
+                                       [to_dev(b) for b in gbits] if gbits else None, dev_block, lm)
         ocfg = vo.OracleConfig(w.n_layers, w.d_model, w.n_q_heads, w.n_kv_heads, w.head_dim, w.bank_capacity,
                                agg_mode=agg_mode, evict_policy=evict_policy, use_rmsnorm=w.use_rmsnorm,
                                residual=w.residual, rope_theta=w.rope_theta, rms_eps=w.rms_eps)
@@ -160,8 +169,10 @@ class Pair:
         x = to_dev(np.stack(bits))
         out = self.gpu.decode_step(ids, x)
         got = to_f64(out)
+        self.last_out, self.last_want = out, []          # device rows / the oracle's rows of this step, per listed stream
         for i, sid in enumerate(ids):
             want = self.ora[sid].text_step(synth.bf16_bits_to_f64(bits[i]))
+            self.last_want.append(want)
             if compare:
                 self._note(self.close_fn(sid, got[i], want, f"{what} stream {sid}"))
         return got

@@ -765,6 +765,33 @@ def test_lm_head_at_the_qwen2_7b_shape():
         print("lm head, Qwen2-7B shape, rows", rows, "errors", e, "tokens equal:", same)
 
 
+def test_first_answer_token_end_to_end():
+    """Section 3.3 from end to end on a small full model: prompt, frames (with evictions), question, then answer
+    steps whose output row goes through the language-model head -- logits and greedy token against the oracle's
+    (its own hidden state through its own head), the next answer token's hidden state being synthetic."""
+    from oracle import videoscan_oracle as vo
+    w = synth.workload("deep", n_layers=2, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64, tokens_per_frame=21,
+                       n_frames=5, bank_capacity=3, prefix_len=6, question_len=7, decode_tokens=3)
+    vocab = 640
+    p = Pair(w, with_gain=True, d_ff=320, vocab=vocab)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    for t in range(w.n_frames):
+        p.frame([0], [w.frame_hidden(t)], f"frame {t}")
+    last = p.text([0], [w.question_hidden()], "question")[0][-1:]          # hidden state of the question's last token
+    same = 0
+    for i in range(w.decode_tokens + 1):
+        # the oracle's own hidden state of that position through its own head
+        want_logits, want_tok = vo.lm_head(p.last_want[0][-1:], p.lm_w64, p.lm_g64, True, w.rms_eps)
+        logits, tok = p.gpu.lm_head(p.last_out[0][-1:].contiguous())
+        got = logits.double().cpu().numpy()
+        e = _check_lm(got, tok.cpu().numpy(), want_logits, want_tok, f"answer token {i}")
+        same += e[1]
+        if i < w.decode_tokens:
+            p.text([0], [w.decode_hidden(i)], f"decode {i}")
+    print("first answer tokens: equal to the oracle's:", same, "of", w.decode_tokens + 1)
+    p.close()
+
+
 def test_lm_head_argument_errors():
     w = synth.workload("tiny")
     p = Pair(w)                                       # no head on this handle
