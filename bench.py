@@ -414,6 +414,9 @@ def run_ours(args, w):
     deep = None
     if not args.no_deep and w.name == "layer":
         deep = run_deep_leg(args, dev, local, lib, binding, torch, flush, barrier, world)
+    batched = None
+    if not args.no_batched and w.name == "layer":
+        batched = run_batched_leg(dev, local, binding, torch, flush, barrier, world)
     block = None
     if not args.no_block and w.name == "layer":
         block = run_block_leg(dev, local, binding, torch, flush, barrier, world)
@@ -493,6 +496,8 @@ def run_ours(args, w):
             result["step_roofline_deep"] = deep_rooflines(deep, peaks)
         if block is not None:
             result["full_block_leg"] = block_rooflines(block, peaks)
+        if batched is not None:
+            result["batched_leg"] = batched_rooflines(batched, peaks)
 
     # ---- end to end: host inputs, H2D + D2H inside the timed region ---------------------------
     # Three streams, two buffers each way: the copy of frame t+1 to the device and the copy of
@@ -638,6 +643,81 @@ def run_deep_leg(args, dev, local, lib, binding, torch, flush, barrier, world):
 
 
 BLOCK_LAYERS, BLOCK_D_FF, BLOCK_VOCAB, BLOCK_FRAMES, BLOCK_DECODE = 2, 18944, 152064, 8, 16
+BATCHED_WARM, BATCHED_FRAMES, BATCHED_DECODE = 24, 8, 16
+
+
+def run_batched_leg(dev, local, binding, torch, flush, barrier, world):
+    """Sixteen streams per call (the 16-stream workload's shape: 196 tokens per frame, one Qwen2-7B-shaped
+    attention layer, bank capacity 1024): BATCHED_WARM untimed frame steps of all streams, then BATCHED_FRAMES timed
+    ones, then BATCHED_DECODE timed single-token steps of all streams.  Frames are seeded iid N(0, 1) rows drawn
+    on the device; weights from the workload's generator."""
+    wq = synth.workload("batched")
+    S_, N, d, HD = wq.n_streams, wq.tokens_per_frame, wq.d_model, wq.n_q_heads * wq.head_dim
+    to_dev = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).to(dev)
+    g = torch.Generator(device=dev); g.manual_seed(4321 + local)
+    n_fr = BATCHED_WARM + BATCHED_FRAMES
+    frames = torch.randn((n_fr, S_, N, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    prefix = torch.randn((S_, wq.prefix_len, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    dec = torch.randn((BATCHED_DECODE, S_, 1, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    cfg = binding.make_config(1, d, wq.n_q_heads, wq.n_kv_heads, wq.head_dim, N, wq.prefix_len, BATCHED_DECODE,
+                              wq.bank_capacity, n_streams=S_, max_step_tokens=max(64, wq.prefix_len),
+                              rope_theta=wq.rope_theta, rms_eps=wq.rms_eps, device=local)
+    sb = binding.StreamBatch(cfg, [to_dev(wq.weight(0))])
+    ids = list(range(S_))
+    out_f = torch.empty((S_, N + 1, HD), dtype=torch.float32, device=dev)
+    out_d = torch.empty((S_, 1, HD), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def pass_(ev=None):
+        sb.reset(ids)
+        sb.decode_step(ids, prefix)
+        for t in range(BATCHED_WARM):
+            sb.frame_prefill(ids, frames[t], out=out_f)
+        flush.zero_()
+        if ev: ev[0].record(stream)
+        for t in range(BATCHED_WARM, n_fr):
+            sb.frame_prefill(ids, frames[t], out=out_f)
+        if ev: ev[1].record(stream)
+        flush.zero_()
+        if ev: ev[2].record(stream)
+        for i in range(BATCHED_DECODE):
+            sb.decode_step(ids, dec[i], out=out_d)
+        if ev: ev[3].record(stream)
+        sb.end_turn(ids)
+
+    pass_()
+    reps = []
+    for _ in range(3):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        barrier()
+        pass_(ev)
+        barrier()
+        t = torch.tensor([ev[0].elapsed_time(ev[1]), ev[2].elapsed_time(ev[3])], dtype=torch.float64, device=dev)
+        reps.append(max_over_ranks(t, world).tolist())
+    assert sb.bank_state(0)["device_status"] == 0
+    sb.close()
+    med = lambda k: sorted(r[k] for r in reps)[len(reps) // 2]
+    return dict(w=wq, ms_frames=med(0), ms_decode=med(1), world=world)
+
+
+def batched_rooflines(bt, peaks):
+    wq = bt["w"]
+    S_, rows = wq.n_streams, wq.tokens_per_frame + 1
+    n_bank = BATCHED_WARM + (BATCHED_FRAMES - 1) / 2.0
+    proj, attn = frame_flops(wq, n_bank)                      # per stream (its own rows and keys)
+    flops = S_ * (proj + attn)
+    us_step = 1e3 * bt["ms_frames"] / BATCHED_FRAMES
+    ideal = flops / (peaks["bf16_tflops_sustained"] * 1e12) * 1e6
+    us_dec = 1e3 * bt["ms_decode"] / BATCHED_DECODE
+    return {
+        "workload": f"{S_} streams per call, {wq.tokens_per_frame} tokens per frame, one Qwen2-7B-shaped attention layer, "
+                    f"{wq.prefix_len}-token prefix, bank capacity {wq.bank_capacity}; {BATCHED_WARM} untimed frame steps, "
+                    f"{BATCHED_FRAMES} timed, then {BATCHED_DECODE} timed batched decode steps; median of 3 passes",
+        "frame": {"us_per_batched_step": us_step, "frames_per_s": bt["world"] * S_ * 1e6 / us_step, "ideal_us": ideal,
+                  "frac": ideal / us_step, "flops_per_step": flops, "peak_tflops": peaks["bf16_tflops_sustained"],
+                  "note": "ideal = flops / sustained bf16 peak (weights L2-resident: one layer)"},
+        "decode": {"us_per_batched_step": us_dec, "tokens_per_s": bt["world"] * S_ * 1e6 / us_dec},
+    }
 
 
 def run_block_leg(dev, local, binding, torch, flush, barrier, world):
@@ -787,6 +867,7 @@ def main():
     ap.add_argument("--frames", type=int, default=None, help="override the number of frames (exploration only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-deep", action="store_true", help="skip the 28-layer leg")
+    ap.add_argument("--no-batched", action="store_true", help="skip the 16-streams-per-call leg")
     ap.add_argument("--no-block", action="store_true", help="skip the full-decoder-block + language-model-head leg")
     args = ap.parse_args()
     kw = {}
