@@ -128,3 +128,20 @@ def test_block_in_chunks_and_carriers_only_forward_through_the_checked_build(che
         p.text([0], [w.decode_hidden(i)], f"decode {i}")
     assert p.check_bank(0)["device_status"] == 0
     p.close()
+
+
+def test_qwen_shape_through_the_checked_build(checked_library):
+    """The kernels' full-size launch shapes (K split over four CTAs, 176-column token tiles, clusters of two in the
+    attention, the matrix-vector projection and the split decode attention) with every workspace store checked:
+    one Qwen2-7B-shaped attention layer, bank of 4 so that frames evict; then one layer with RMSNorm, the decoder
+    block (d_ff 1024) and the language-model head."""
+    w = synth.workload("layer", n_frames=7, bank_capacity=4, question_len=9, decode_tokens=3)
+    p = Pair(w, max_text=12, max_chunk_frames=2)
+    _stream(p, w, 7, chunk=2)
+    p.close()
+    w = synth.workload("deep", n_layers=1, n_frames=3, bank_capacity=2, prefix_len=16, question_len=5, decode_tokens=2)
+    p = Pair(w, d_ff=1024, vocab=1024, max_text=8)
+    _stream(p, w, 3)
+    logits, tok = p.gpu.lm_head(p.last_out[0][-1:].contiguous())
+    assert p.check_bank(0)["device_status"] == 0
+    p.close()
