@@ -344,6 +344,28 @@ def test_batched_ragged_streams_small():
     p.close()
 
 
+def test_sixty_four_streams_in_one_call():
+    """The most streams a call may list (64): ragged lengths, evictions in every stream, subsets in any order,
+    batched text steps; two layers with RMSNorm so that the residual path runs at that batch size too."""
+    w = synth.workload("batched", n_layers=2, use_rmsnorm=1, residual=1, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64,
+                       tokens_per_frame=9, n_frames=7, min_frames=3, bank_capacity=2, n_streams=64, prefix_len=3, decode_tokens=2)
+    lengths = w.stream_lengths()
+    p = Pair(w)
+    ids = list(range(64))
+    p.text(ids, [w.prefix_hidden(s) for s in ids], "prefix")
+    for t in range(max(lengths)):
+        act = [s for s in ids if lengths[s] > t]
+        if t % 2:
+            act = act[::-1]                                  # the order of the listed streams is the caller's
+        p.frame(act, [w.frame_hidden(t, s) for s in act], f"frame {t}")
+    for i in range(w.decode_tokens):
+        p.text(ids, [w.decode_hidden(i, s) for s in ids], f"decode {i}")
+    for s in (0, 17, 63):
+        st = p.check_bank(s, layer=1)
+        assert st["frames_seen"] == lengths[s]
+    p.close()
+
+
 def test_one_layer_qwen_shape_full_stream():
     """The single-layer Qwen2-7B-shaped workload in full: 64-token prefix, 64 frames x 169
     tokens, bank 64 (never evicts), 32 decode tokens."""
