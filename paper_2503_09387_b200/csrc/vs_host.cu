@@ -702,7 +702,9 @@ int vs_frame_prefill_chunk(vs_stream* h, int32_t stream_id, const void* hidden, 
   // before the chunk (all M + 1 slots once the bank is full)
   const int count0 = bp.count[0];
   const int l1 = (D.M > 0 && count0 == D.M) ? D.M + 1 : count0;
-  if (l1 + F > ATTN_EXCL_BITS) return VS_ERR_CAPACITY;   // the attention launch's mask of hidden bank keys
+  // the attention launch's mask of hidden bank keys; refused on the bank's capacity, not on its fill, so that a
+  // stream does not run into the limit only once its bank is full
+  if ((D.M > 0 ? D.M + 1 : 0) + F > ATTN_EXCL_BITS) return VS_ERR_CAPACITY;
 
   // 1. carriers of all frames (Section 3.3: C = mean of the frame's tokens), parked until they have a slot
   PoolArgs pa;

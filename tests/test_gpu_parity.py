@@ -908,6 +908,41 @@ def test_non_finite_carrier_keeps_the_bank_bookkeeping_in_range():
         sb.close()
 
 
+def test_very_large_bank_and_the_chunk_limit():
+    """A bank of 2100 carriers (a key axis of 17 and more 128-key tiles in the prefill attention, split decode over
+    2100 keys): filled by frames whose layers the oracle skips, then ten full frames that evict; and the limit of
+    the chunk call's victim bitmap (bank capacity + 1 + frames per call <= 8192)."""
+    w = synth.workload("long", d_model=128, n_q_heads=2, n_kv_heads=1, head_dim=64, tokens_per_frame=3, n_frames=2110,
+                       bank_capacity=2100, prefix_len=5, question_len=4, decode_tokens=2)
+    p = Pair(w, max_text=8)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    shared = w.frame_shared()
+    for t in range(w.n_frames):
+        full = t >= 2100
+        p.frame([0], [w.frame_hidden(t, shared=shared)], f"frame {t}", mode="full" if full else "carrier")
+        if full or t % 700 == 0:
+            p.check_bank(0, kv=full)
+    st = p.check_bank(0)
+    assert st["count"] == 2100 and st["evictions"] == 10
+    p.text([0], [w.question_hidden()], "question")
+    for i in range(w.decode_tokens):
+        p.text([0], [w.decode_hidden(i)], f"decode {i}")
+    print("bank of 2100: worst", p.worst)
+    p.close()
+    for M, ok in ((8189, True), (8190, False)):
+        cfg = binding.make_config(1, 64, 1, 1, 64, 2, 2, 2, M, max_chunk_frames=2)
+        sb = binding.StreamBatch(cfg, [to_dev(synth.normal_bf16(3, synth.TAG_WEIGHT, (192, 64), 0.05))])
+        x = to_dev(synth.normal_bf16(3, synth.TAG_FRAME_NOISE, (2, 2, 64)))
+        if ok:
+            sb.frame_prefill_chunk(0, x)
+            assert sb.bank_state(0)["count"] == 2 and sb.bank_state(0)["device_status"] == 0
+        else:
+            with pytest.raises(binding.VsError) as e:
+                sb.frame_prefill_chunk(0, x)
+            assert e.value.code == binding.VS_ERR_CAPACITY
+        sb.close()
+
+
 def test_argument_errors_leave_the_stream_untouched():
     w = synth.workload("tiny")
     p = Pair(w)
