@@ -48,6 +48,27 @@ def test_odd_shapes_and_policies(N, P, M, policy):
     p.close()
 
 
+@pytest.mark.parametrize("Hq,Hkv,D,d", [(1, 1, 64, 64), (2, 2, 128, 256), (3, 1, 64, 192), (5, 1, 128, 320), (6, 2, 64, 128),
+                                         (3, 3, 64, 192)])
+def test_head_groupings(Hq, Hkv, D, d):
+    """Query heads per KV head from 1 (plain multi-head attention) to 6, both head sizes, projection widths
+    (Hq + 2 Hkv) D that are no multiple of the 128-row weight tile, d_model different from Hq D (no residual)."""
+    w = synth.workload("tiny", d_model=d, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, tokens_per_frame=18, n_frames=6,
+                       bank_capacity=3, prefix_len=5, question_len=6, decode_tokens=2, seed=7 * Hq + Hkv)
+    p = Pair(w, max_text=8, max_chunk_frames=2)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    for t in range(4):
+        p.frame([0], [w.frame_hidden(t)], f"frame {t}")
+    p.frame_chunk(0, [w.frame_hidden(4), w.frame_hidden(5)], "chunk")
+    p.check_bank(0)
+    p.bank_forward(0)
+    p.text([0], [w.question_hidden()], "question")
+    for i in range(w.decode_tokens):
+        p.text([0], [w.decode_hidden(i)], f"decode {i}")
+    p.check_bank(0)
+    p.close()
+
+
 def test_width_that_is_no_multiple_of_256():
     """d_model = 320 (five 64-wide K blocks): few-row text steps cannot take the matrix-vector
     kernel (it moves 256 elements of a row per stage) and fall back to the tensor-core projection
