@@ -707,6 +707,29 @@ def test_full_decoder_block_in_chunks_and_carriers_only_forward():
     p.close()
 
 
+@pytest.mark.parametrize("d,Hq,Hkv,D,d_ff,kw", [
+    (128, 2, 1, 64, 64, dict()),                                   # the narrowest block: one 128-feature tile, one gate/up tile
+    (256, 2, 2, 128, 448, dict(with_bias=True, with_gain=True)),   # QKV bias with the block, d_ff no multiple of 128
+    (384, 6, 2, 64, 192, dict(agg_mode=1, evict_policy=1)),        # last-token carrier, adjacent-pair eviction
+    (256, 4, 1, 64, 320, dict(evict_policy=2, with_gain=True)),
+])
+def test_full_decoder_block_variants(d, Hq, Hkv, D, d_ff, kw):
+    """One decoder layer with the options that meet the block's kernels at their edges; carrier overrides too."""
+    w = synth.workload("deep", n_layers=1, d_model=d, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, tokens_per_frame=17,
+                       n_frames=5, bank_capacity=2, prefix_len=4, question_len=5, decode_tokens=2, seed=d + d_ff)
+    p = Pair(w, d_ff=d_ff, max_text=8, **kw)
+    p.text([0], [w.prefix_hidden()], "prefix")
+    for t in range(w.n_frames):
+        ov = [synth.normal_bf16(w.seed, synth.TAG_PREFIX, (d,), 1.0, offset=1000 + t * d)] if t == 2 else None
+        p.frame([0], [w.frame_hidden(t)], f"frame {t}", override=ov)
+    p.check_bank(0)
+    p.text([0], [w.question_hidden()], "question")
+    for i in range(w.decode_tokens):
+        p.text([0], [w.decode_hidden(i)], f"decode {i}")
+    p.check_bank(0)
+    p.close()
+
+
 def test_full_decoder_block_28_layers_scaled_width():
     """28 full decoder layers (attention, output projection, SwiGLU MLP; RMSNorm before each half) at a scaled
     width (d_model 512, d_ff 1408): free-running at the depth-scaled bound, every layer teacher-forced at the
