@@ -730,6 +730,31 @@ def test_full_decoder_block_variants(d, Hq, Hkv, D, d_ff, kw):
     p.close()
 
 
+def test_full_decoder_block_text_steps_of_every_size():
+    """Text steps of 1 .. 4 rows (matrix-vector projection), 7 and 16 rows (tensor cores, rotation derived in the
+    kernel) and 40 rows (RoPE table) through one full decoder layer, on single streams and small batches."""
+    w = synth.workload("deep", n_layers=1, d_model=512, n_q_heads=4, n_kv_heads=2, head_dim=128, tokens_per_frame=23,
+                       n_frames=4, bank_capacity=3, prefix_len=3, question_len=0, decode_tokens=0, n_streams=3,
+                       frame_model="iid", seed=29)
+    p = Pair(w, with_gain=True, d_ff=704, max_prefix=8, max_text=80, max_step_tokens=40)
+    ids = [0, 1, 2]
+    draw = lambda tag, T, s: synth.normal_bf16(w.seed, synth.TAG_QUESTION, (T, w.d_model), 1.0, offset=(tag * 8 + s) * 40 * w.d_model)
+    p.text([0], [w.prefix_hidden(0)], "prefix of 3 rows")
+    p.text([1, 2], [w.prefix_hidden(1)[:1], w.prefix_hidden(2)[:1]], "two one-row prefixes")
+    p.text([1], [draw(0, 4, 1)], "prefix extended by 4 rows")
+    for t in range(4):
+        p.frame(ids, [w.frame_hidden(t, s) for s in ids], f"frame {t}")
+    p.text([0], [draw(1, 2, 0)], "2-row question")
+    p.text(ids, [draw(2, 1, s) for s in ids], "3 streams x 1 token")
+    p.text([2], [draw(3, 4, 2)], "4-row step")
+    p.text([0], [draw(6, 7, 0)], "7-row step")
+    p.text([1, 2], [draw(7, 8, s) for s in (1, 2)], "2 streams x 8 rows")
+    p.text([0], [draw(8, 40, 0)], "40-row step")
+    for s in ids:
+        p.check_bank(s)
+    p.close()
+
+
 def test_full_decoder_block_28_layers_scaled_width():
     """28 full decoder layers (attention, output projection, SwiGLU MLP; RMSNorm before each half) at a scaled
     width (d_model 512, d_ff 1408): free-running at the depth-scaled bound, every layer teacher-forced at the
