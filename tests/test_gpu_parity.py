@@ -299,23 +299,31 @@ def test_carriers_only_forward_qwen_shape():
 def test_scratch_holds_no_state_between_steps():
     """Section 3.3: visual tokens are discarded after prefill.  Overwriting every per-step
     scratch region with NaN between steps must not change any later output."""
-    w = synth.workload("tiny")
-    a, b = Pair(w), Pair(w)
-    outs = []
-    for p, poison in ((a, False), (b, True)):
-        o = [p.text([0], [w.prefix_hidden()])]
-        for t in range(w.n_frames):
-            o.append(p.frame([0], [w.frame_hidden(t)]))
-            if poison:
-                p.gpu.poison_scratch()
-        for i in range(w.decode_tokens):
-            o.append(p.text([0], [w.decode_hidden(i)]))
-            if poison:
-                p.gpu.poison_scratch()
-        outs.append(o)
-    for x, y in zip(*outs):
-        assert np.array_equal(x, y)
-    a.close(); b.close()
+    for kw in (dict(), dict(d_ff=192, vocab=256, with_gain=True)):     # attention only; full decoder layers + head
+        w = synth.workload("tiny") if not kw else synth.workload("tiny", n_layers=2, use_rmsnorm=1, residual=1, n_q_heads=4,
+                                                                 n_kv_heads=2, head_dim=64)
+        a, b = Pair(w, **kw), Pair(w, **kw)
+        outs = []
+        for p, poison in ((a, False), (b, True)):
+            o = [p.text([0], [w.prefix_hidden()])]
+            for t in range(w.n_frames):
+                o.append(p.frame([0], [w.frame_hidden(t)]))
+                if poison:
+                    p.gpu.poison_scratch()
+            for i in range(w.decode_tokens):
+                o.append(p.text([0], [w.decode_hidden(i)]))
+                if kw:
+                    row = p.last_out[0][-1:].contiguous()       # (copied out of the step's output before the poison)
+                    if poison:
+                        p.gpu.poison_scratch()
+                    logits, tok = p.gpu.lm_head(row)
+                    o.append(logits.double().cpu().numpy()); o.append(tok.cpu().numpy().astype(np.float64))
+                if poison:
+                    p.gpu.poison_scratch()
+            outs.append(o)
+        for x, y in zip(*outs):
+            assert np.array_equal(x, y)
+        a.close(); b.close()
 
 
 def test_question_prefill_decode_and_end_turn():
